@@ -1,0 +1,223 @@
+/*
+ * bsa.h -- C ABI of the B200 (sm_100a) forward of dynamic block-sparse attention.
+ *
+ * A request R = <A, M, B, x> (paper, Section 3 "Online request path" and Section 4.4) supplies a
+ * logical block mask M with geometry B = (B_Q, B_KV) and the tensor properties x (here: bf16,
+ * head dim d, layout [heads, N, d]).  The library computes masked attention (Section 2.1, Eq. 1)
+ *
+ *     O_M = softmax(Q K^T / sqrt(d) + B_M) V,   B_M = 0 on E(M), -inf elsewhere,
+ *
+ * plus the fp32 log-sum-exp of each row, touching only physical tiles that cover active blocks.
+ *
+ * All pointers named *_dev are DEVICE pointers on the current CUDA device; pointers named
+ * *_host are HOST pointers.  No function throws; every call returns a status.  `stream` is a
+ * cudaStream_t passed as void* (NULL = the legacy default stream).
+ */
+#ifndef BSA_H_
+#define BSA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define BSA_API __attribute__((visibility("default")))
+#else
+#define BSA_API
+#endif
+
+typedef struct bsa_plan bsa_plan_t; /* opaque; owned by the library */
+
+typedef enum {
+    BSA_OK = 0,
+    BSA_ERR_INVALID_ARG = 1,      /* null pointer, N <= 0, heads <= 0, ... (GPU untouched)            */
+    BSA_ERR_UNSUPPORTED = 2,      /* d not in {64,128}; B_Q/B_KV not a power of two in [16,256]      */
+    BSA_ERR_NO_ELIGIBLE_PLAN = 3, /* Algorithm 2, last line: no plan of the ranking is eligible      */
+    BSA_ERR_OOM = 4,              /* device or host allocation failed                               */
+    BSA_ERR_CUDA = 5,             /* a CUDA call failed; see bsa_last_cuda_error()                   */
+    BSA_ERR_DEVICE_TIMEOUT = 6,   /* a bounded device-side wait expired (kernel gave up, no hang)    */
+    BSA_ERR_LUT = 7               /* plan-table file missing, malformed, or for another catalog      */
+} bsa_status_t;
+
+/* Mapping of one dimension of the logical geometry onto the physical tile (Section 4.2). */
+enum { BSA_MAP_DIRECT = 0, BSA_MAP_COARSENED = 1, BSA_MAP_REFINED = 2 };
+/* Traversal order of the work queue (Section 4.3). */
+enum { BSA_ORDER_HEAD_MAJOR_LPT = 0, BSA_ORDER_GLOBAL_LPT = 1 };
+
+/* One catalog entry: a physical plan P = <g_Q, g_KV, sigma, e> (Section 4.1).  g_Q and g_KV follow
+ * from (B_Q, B_KV) and the tile shape; sigma = {order, split_tau, split_pmax, stages}; e = kernel. */
+typedef struct bsa_plan_desc {
+    int32_t plan_id;
+    int32_t T_Q, T_KV;       /* physical tile geometry                                               */
+    int32_t stages;          /* K/V ring depth (pipeline depth); 0 = as many as shared memory holds  */
+    int32_t split_tau;       /* a Q tile row with more than tau tiles is split ...                   */
+    int32_t split_pmax;      /* ... into at most pmax KV ranges (1 = never split)                    */
+    int32_t order;           /* BSA_ORDER_*                                                          */
+    int32_t kernel;          /* kernel variant id                                                    */
+    char name[48];
+} bsa_plan_desc_t;
+
+typedef struct bsa_options {
+    int32_t force_plan_id;        /* >= 0: skip the lookup and use this catalog entry (still checked for
+                                     eligibility); -1: Algorithm 2                                   */
+    int32_t reserved0;
+    int64_t max_workspace_bytes;  /* Split-K workspace the request may bind; <= 0: library default   */
+} bsa_options_t;
+
+/* Scalar mask statistics s_A(M) (Section 5.1) and what launch preparation produced. */
+typedef struct bsa_plan_info {
+    bsa_plan_desc_t plan;         /* the selected plan                                               */
+    int32_t map_q, map_kv;        /* BSA_MAP_* per dimension                                         */
+    int32_t heads, d, B_Q, B_KV;
+    int64_t N;
+    int32_t nQb, nKb, nQt, nKt;   /* logical block grid and physical tile grid per head              */
+    int32_t member_bits;          /* membership bits per tile (1 = no intra-tile mask needed)        */
+    int32_t lut_hit;              /* 1: regime found in the plan table; 0: base plan used            */
+    int32_t regime_bucket[4];     /* N, density, skew, run-coverage bucket indices used for lookup   */
+    int64_t nnz_blocks;           /* active logical blocks                                           */
+    int64_t blocks_in_runs;       /* active blocks in runs of length >= 2                            */
+    int32_t max_row_nnz;
+    int32_t reserved0;
+    double density, run_coverage, skew;
+    int64_t ntiles;               /* physical tiles                                                  */
+    int64_t nitems;               /* work items (Q tile rows x KV partitions)                        */
+    int64_t nsplit_rows;          /* Q tile rows with more than one partition                        */
+    int64_t workspace_bytes;      /* Split-K workspace owned by the plan                             */
+    int64_t covered_pairs;        /* token pairs the tiles compute, incl. masked-out ones            */
+    /* host wall time of bsa_plan_create, microseconds */
+    float us_mask_state;          /* launch of the mask-state kernels                                */
+    float us_stats_sync;          /* waiting for + copying the scalar statistics                     */
+    float us_lookup;              /* regime lookup + ranked fallback + eligibility                   */
+    float us_launch_prep;         /* CSR fill, tile mapping, task organisation (launch + allocs)    */
+    float us_total;
+    int32_t device_status;        /* 0, or BSA_ERR_DEVICE_TIMEOUT if any forward hit a bounded wait  */
+} bsa_plan_info_t;
+
+/* ---------------------------------------------------------------------------------------------
+ * bsa_plan_create -- online plan selection and launch preparation (Section 5.2, Algorithm 2).
+ *
+ * Builds the shared mask state mu(M) on the GPU (block-CSR offsets, active KV column indices and
+ * the scalar statistics), copies only the scalars to the host (the one synchronisation of the
+ * call), looks up the regime in the loaded plan table, takes the first eligible plan of its
+ * ranking (base plan on a miss), then derives that plan's metadata on the GPU: physical tile
+ * lists with membership bits (Direct / Coarsened / Refined mapping, Section 4.2), work items per Q
+ * tile row, Split-K partitions of heavy rows, longest-first order (Section 4.3).
+ *
+ *   mask_dev : uint8 [heads, ceil(N/B_Q), ceil(N/B_KV)], row-major, nonzero = active block.
+ *              Borrowed: read by kernels this call submits to `stream`; it may be freed or
+ *              overwritten by work ordered after the call on that stream (or after a stream sync).
+ *   B_Q,B_KV : logical block geometry, powers of two in [16, 256].
+ *   N        : tokens per head (N_q = N_kv = N); need not be a multiple of the block sizes.
+ *   heads    : independent (batch x head) problems.
+ *   d        : head dimension, 64 or 128.  Scale is 1/sqrt(d); attention is non-causal.
+ *   out_plan : receives the plan; the plan owns its device buffers (CSR, tile lists, work items,
+ *              Split-K workspace).  Reusable for any number of forwards with the same mask.
+ *
+ * Runs on the legacy default stream (the _ex variant takes a stream and options) and returns after
+ * the statistics copy; the remaining preparation kernels are stream-ordered before any forward
+ * submitted to the same stream.  A forward on ANOTHER stream must be ordered after the create by the caller.
+ * Errors: INVALID_ARG / UNSUPPORTED (GPU untouched), NO_ELIGIBLE_PLAN, OOM, CUDA.
+ */
+BSA_API bsa_status_t bsa_plan_create(const uint8_t* mask_dev, int B_Q, int B_KV, int64_t N, int heads, int d,
+                             bsa_plan_t** out_plan);
+BSA_API bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int B_KV, int64_t N, int heads, int d,
+                                const bsa_options_t* options /* may be NULL */, void* stream,
+                                bsa_plan_t** out_plan);
+
+/* ---------------------------------------------------------------------------------------------
+ * bsa_forward -- execute the plan's native kernels (Section 4: main attention kernel, then the
+ * Split-K reduction kernel when the plan has partitions).
+ *
+ *   Q,K,V : bf16 [heads, N, d], d contiguous, 16-byte aligned base, device memory, borrowed.
+ *   O     : bf16 [heads, N, d], written for every row; rows with no active block get 0.
+ *   LSE   : fp32 [heads, N], natural-log log-sum-exp of the scaled scores over E(M); -inf for rows
+ *           with no active block.
+ *
+ * Asynchronous on `stream`; no host synchronisation.  Forwards that share a plan must be
+ * stream-ordered (they share the Split-K workspace).  A bounded device wait that expires is
+ * recorded in the plan (see bsa_plan_get_info().device_status) -- the kernel returns, it never hangs.
+ * Errors: INVALID_ARG (null or misaligned pointers), CUDA.
+ */
+BSA_API bsa_status_t bsa_forward(const bsa_plan_t* plan, const void* Q_dev, const void* K_dev, const void* V_dev,
+                         void* O_dev, float* LSE_dev, void* stream);
+
+/* Frees the plan and every device buffer it owns.  Synchronises with the plan's create stream. */
+BSA_API bsa_status_t bsa_plan_destroy(bsa_plan_t* plan);
+
+/* ---------------------------------------------------------------------------------------------
+ * bsa_request_host -- one complete request from HOST buffers: copies mask, Q, K, V to the device,
+ * creates the plan, runs the forward, copies O and LSE back, frees everything.  Same semantics as
+ * the three calls above; used to measure end-to-end request cost including transfers.
+ *   info_out (optional) receives the plan info.
+ */
+BSA_API bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int B_KV, int64_t N, int heads, int d,
+                              const void* Q_host, const void* K_host, const void* V_host,
+                              void* O_host, float* LSE_host, const bsa_options_t* options,
+                              bsa_plan_info_t* info_out);
+
+/* ---------------------------------------------------------------------------------------------
+ * Introspection (tests, benches, the offline profiler).  These synchronise with the plan's stream.
+ */
+BSA_API bsa_status_t bsa_plan_get_info(const bsa_plan_t* plan, bsa_plan_info_t* info_out);
+
+/* Block-CSR of the shared mask state: row_ptr_host int32 [heads*nQb + 1], col_idx_host int32
+ * [nnz_blocks] (pass NULL to skip either).  Rows are (head, query block) in row-major order. */
+BSA_API bsa_status_t bsa_plan_export_csr(const bsa_plan_t* plan, int32_t* row_ptr_host, int32_t* col_idx_host);
+
+/* Physical tiles of one head, for the coverage check (a plan must preserve E(M), Section 2.2):
+ *   tile_row_ptr_host int32 [nQt + 1]  offsets into the two arrays below (relative to this head),
+ *   tile_col_host     int32 [cap]      KV tile index, ascending and unique inside a row,
+ *   tile_member_host  uint64 [cap]     membership bits: bit (a * sK + b) set iff logical sub-block
+ *                                      (a, b) of the tile is active, sK = max(1, T_KV / B_KV),
+ *                                      a < max(1, T_Q / B_Q), b < sK.
+ * `cap` is the capacity of the two arrays in entries; *ntiles_out receives the number needed
+ * (call with cap = 0 and NULL arrays to size them). */
+BSA_API bsa_status_t bsa_plan_export_tiles(const bsa_plan_t* plan, int head, int32_t* tile_row_ptr_host,
+                                   int32_t* tile_col_host, uint64_t* tile_member_host, int64_t cap,
+                                   int64_t* ntiles_out);
+
+/* Work items in queue order: 8 int32 per item {head, q_tile, tile_begin, tile_end, part, nparts,
+ * ws_slot, ntiles}; tile_begin/end index the plan's global tile arrays.  Sizing as above. */
+BSA_API bsa_status_t bsa_plan_export_items(const bsa_plan_t* plan, int32_t* items_host, int64_t cap, int64_t* nitems_out);
+
+/* ---------------------------------------------------------------------------------------------
+ * Catalog C_A and plan table Pi_A (Section 4.4, Section 5).
+ */
+BSA_API int bsa_catalog_size(void);
+BSA_API bsa_status_t bsa_catalog_get(int index, bsa_plan_desc_t* out);
+/* Eligible(P, R) (Section 4.4): geometry, head dim, membership format and workspace. */
+BSA_API int bsa_plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_workspace_bytes);
+/* Base plan of a request key (eligible for every request with that key). */
+BSA_API int bsa_base_plan(int B_Q, int B_KV, int d);
+/* Hash of the catalog contents; a plan table built for another catalog is rejected. */
+BSA_API uint64_t bsa_catalog_hash(void);
+
+/* Load the versioned plan table (text file written by the offline profiler).  Replaces any table
+ * loaded before.  On error the previous table is dropped and base plans are used. */
+BSA_API bsa_status_t bsa_lut_load(const char* path);
+BSA_API void bsa_lut_clear(void);
+BSA_API int bsa_lut_num_regimes(void);
+/* Regime lookup + ranked fallback only (no GPU): returns the plan id Algorithm 2 selects for these
+ * request scalars, or -1 for no-eligible-plan.  *hit_out (optional) = 1 if the regime was found. */
+BSA_API int bsa_lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_coverage,
+                   double skew, int64_t max_workspace_bytes, int* hit_out);
+/* Bucket edges of the feature schema F_A, so the offline profiler partitions cases exactly as the
+ * runtime does: writes the bucket indices {N, density, skew, run coverage} for the given scalars. */
+BSA_API void bsa_lut_buckets(int64_t N, double density, double skew, double run_coverage, int32_t out[4]);
+
+/* Process-wide default used when options->force_plan_id is not given: >= 0 forces a plan,
+ * -1 restores Algorithm 2. */
+BSA_API void bsa_force_plan(int plan_id);
+
+BSA_API const char* bsa_status_string(bsa_status_t s);
+BSA_API const char* bsa_last_cuda_error(void);
+BSA_API const char* bsa_version(void);
+/* Number of this library's kernels launched since load (all plans, all streams). */
+BSA_API int64_t bsa_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BSA_H_ */

@@ -1,0 +1,250 @@
+"""Thin ctypes binding of libbsa.so: argument marshalling only.
+
+Every step of the request path (mask state, plan selection, launch preparation,
+attention, Split-K merge) runs inside the C-ABI library; torch is used here only
+to own device memory and streams.  Loading fails loudly if the library has not
+been built -- there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbsa.so")
+
+BSA_OK = 0
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "NO_ELIGIBLE_PLAN", 4: "OOM", 5: "CUDA",
+                6: "DEVICE_TIMEOUT", 7: "LUT"}
+MAP_NAMES = {0: "direct", 1: "coarsened", 2: "refined"}
+
+
+class PlanDesc(ctypes.Structure):
+    _fields_ = [("plan_id", ctypes.c_int32), ("T_Q", ctypes.c_int32), ("T_KV", ctypes.c_int32),
+                ("stages", ctypes.c_int32), ("split_tau", ctypes.c_int32), ("split_pmax", ctypes.c_int32),
+                ("order", ctypes.c_int32), ("kernel", ctypes.c_int32), ("name", ctypes.c_char * 48)]
+
+
+class Options(ctypes.Structure):
+    _fields_ = [("force_plan_id", ctypes.c_int32), ("reserved0", ctypes.c_int32),
+                ("max_workspace_bytes", ctypes.c_int64)]
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [("plan", PlanDesc), ("map_q", ctypes.c_int32), ("map_kv", ctypes.c_int32),
+                ("heads", ctypes.c_int32), ("d", ctypes.c_int32), ("B_Q", ctypes.c_int32), ("B_KV", ctypes.c_int32),
+                ("N", ctypes.c_int64),
+                ("nQb", ctypes.c_int32), ("nKb", ctypes.c_int32), ("nQt", ctypes.c_int32), ("nKt", ctypes.c_int32),
+                ("member_bits", ctypes.c_int32), ("lut_hit", ctypes.c_int32), ("regime_bucket", ctypes.c_int32 * 4),
+                ("nnz_blocks", ctypes.c_int64), ("blocks_in_runs", ctypes.c_int64),
+                ("max_row_nnz", ctypes.c_int32), ("reserved0", ctypes.c_int32),
+                ("density", ctypes.c_double), ("run_coverage", ctypes.c_double), ("skew", ctypes.c_double),
+                ("ntiles", ctypes.c_int64), ("nitems", ctypes.c_int64), ("nsplit_rows", ctypes.c_int64),
+                ("workspace_bytes", ctypes.c_int64), ("covered_pairs", ctypes.c_int64),
+                ("us_mask_state", ctypes.c_float), ("us_stats_sync", ctypes.c_float), ("us_lookup", ctypes.c_float),
+                ("us_launch_prep", ctypes.c_float), ("us_total", ctypes.c_float), ("device_status", ctypes.c_int32)]
+
+    def as_dict(self) -> Dict:
+        out = {}
+        for name, _ in self._fields_:
+            v = getattr(self, name)
+            if name == "plan":
+                v = {f: (getattr(v, f).decode() if f == "name" else getattr(v, f)) for f, _ in PlanDesc._fields_}
+            elif name == "regime_bucket":
+                v = list(v)
+            out[name] = v
+        return out
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libbsa.so (raises if it was not built: there is no other code path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_25869_b200.build` "
+                           "(nvcc, sm_100a). There is no CPU or PyTorch fallback.")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_double
+    L.bsa_plan_create.argtypes = [vp, i32, i32, i64, i32, i32, ctypes.POINTER(vp)]
+    L.bsa_plan_create_ex.argtypes = [vp, i32, i32, i64, i32, i32, ctypes.POINTER(Options), vp, ctypes.POINTER(vp)]
+    L.bsa_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.bsa_plan_destroy.argtypes = [vp]
+    L.bsa_request_host.argtypes = [vp, i32, i32, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.POINTER(Options),
+                                   ctypes.POINTER(PlanInfo)]
+    L.bsa_plan_get_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
+    L.bsa_plan_export_csr.argtypes = [vp, vp, vp]
+    L.bsa_plan_export_tiles.argtypes = [vp, i32, vp, vp, vp, i64, ctypes.POINTER(i64)]
+    L.bsa_plan_export_items.argtypes = [vp, vp, i64, ctypes.POINTER(i64)]
+    L.bsa_catalog_size.restype = i32
+    L.bsa_catalog_get.argtypes = [i32, ctypes.POINTER(PlanDesc)]
+    L.bsa_plan_eligible.argtypes = [i32, i32, i32, i64, i32, i32, i64]
+    L.bsa_base_plan.argtypes = [i32, i32, i32]
+    L.bsa_catalog_hash.restype = ctypes.c_uint64
+    L.bsa_lut_load.argtypes = [ctypes.c_char_p]
+    L.bsa_lut_clear.restype = None
+    L.bsa_lut_select.argtypes = [i32, i32, i64, i32, i32, f64, f64, f64, i64, ctypes.POINTER(i32)]
+    L.bsa_lut_buckets.argtypes = [i64, f64, f64, f64, ctypes.POINTER(ctypes.c_int32)]
+    L.bsa_lut_buckets.restype = None
+    L.bsa_force_plan.argtypes = [i32]
+    L.bsa_force_plan.restype = None
+    L.bsa_status_string.argtypes = [i32]
+    L.bsa_status_string.restype = ctypes.c_char_p
+    L.bsa_last_cuda_error.restype = ctypes.c_char_p
+    L.bsa_version.restype = ctypes.c_char_p
+    L.bsa_kernel_launch_count.restype = i64
+    _lib = L
+    return L
+
+
+class BsaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        detail = lib().bsa_last_cuda_error().decode() if status == 5 else ""
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} "
+                         f"({lib().bsa_status_string(status).decode()}) {detail}")
+
+
+def _check(status: int, where: str):
+    if status != BSA_OK:
+        raise BsaError(status, where)
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream or None
+    return getattr(stream, "cuda_stream", stream) or None
+
+
+class Plan:
+    """Handle of a prepared plan (``bsa_plan_create`` ... ``bsa_plan_destroy``)."""
+
+    def __init__(self, handle: int):
+        self._h = ctypes.c_void_p(handle)
+
+    def forward(self, Q, K, V, O=None, LSE=None, stream=None):
+        """``bsa_forward``: Q, K, V are bf16 CUDA tensors ``[heads, N, d]``; returns ``(O, LSE)``."""
+        import torch
+        assert Q.is_cuda and Q.dtype == torch.bfloat16 and Q.is_contiguous()
+        assert K.is_contiguous() and V.is_contiguous() and K.dtype == V.dtype == torch.bfloat16
+        if O is None:
+            O = torch.empty_like(Q)
+        if LSE is None:
+            LSE = torch.empty(Q.shape[:2], dtype=torch.float32, device=Q.device)
+        _check(lib().bsa_forward(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
+                                 _stream_ptr(stream)), "bsa_forward")
+        return O, LSE
+
+    def info(self) -> Dict:
+        inf = PlanInfo()
+        _check(lib().bsa_plan_get_info(self._h, ctypes.byref(inf)), "bsa_plan_get_info")
+        return inf.as_dict()
+
+    def export_csr(self) -> Tuple[np.ndarray, np.ndarray]:
+        inf = self.info()
+        rp = np.zeros(inf["heads"] * inf["nQb"] + 1, dtype=np.int32)
+        ci = np.zeros(max(1, inf["nnz_blocks"]), dtype=np.int32)
+        _check(lib().bsa_plan_export_csr(self._h, rp.ctypes.data, ci.ctypes.data), "bsa_plan_export_csr")
+        return rp, ci[: inf["nnz_blocks"]]
+
+    def export_tiles(self, head: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        n = ctypes.c_int64(0)
+        _check(lib().bsa_plan_export_tiles(self._h, head, None, None, None, 0, ctypes.byref(n)), "export_tiles(size)")
+        nQt = self.info()["nQt"]
+        rp = np.zeros(nQt + 1, dtype=np.int32)
+        tc = np.zeros(max(1, n.value), dtype=np.int32)
+        tm = np.zeros(max(1, n.value), dtype=np.uint64)
+        _check(lib().bsa_plan_export_tiles(self._h, head, rp.ctypes.data, tc.ctypes.data, tm.ctypes.data,
+                                           max(1, n.value), ctypes.byref(n)), "export_tiles")
+        return rp, tc[: n.value], tm[: n.value]
+
+    def export_items(self) -> np.ndarray:
+        n = ctypes.c_int64(0)
+        _check(lib().bsa_plan_export_items(self._h, None, 0, ctypes.byref(n)), "export_items(size)")
+        it = np.zeros((max(1, n.value), 8), dtype=np.int32)
+        _check(lib().bsa_plan_export_items(self._h, it.ctypes.data, max(1, n.value), ctypes.byref(n)), "export_items")
+        return it[: n.value]
+
+    def destroy(self):
+        if self._h:
+            _check(lib().bsa_plan_destroy(self._h), "bsa_plan_destroy")
+            self._h = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.destroy()
+
+
+def plan_create(mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1,
+                max_workspace_bytes: int = 0, stream=None) -> Plan:
+    """``bsa_plan_create_ex``: ``mask`` is a uint8/bool CUDA tensor ``[heads, nQb, nKb]``."""
+    import torch
+    assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool)
+    h = ctypes.c_void_p()
+    opt = Options(plan_id, 0, max_workspace_bytes)
+    _check(lib().bsa_plan_create_ex(mask.data_ptr(), B_Q, B_KV, N, heads, d, ctypes.byref(opt), _stream_ptr(stream),
+                                    ctypes.byref(h)), "bsa_plan_create")
+    return Plan(h.value)
+
+
+def request_host(mask: np.ndarray, B_Q: int, B_KV: int, N: int, heads: int, d: int, Q, K, V, O, LSE,
+                 plan_id: int = -1) -> Dict:
+    """``bsa_request_host``: all arguments are HOST buffers (torch CPU tensors or numpy arrays)."""
+    def ptr(x):
+        return x.data_ptr() if hasattr(x, "data_ptr") else x.ctypes.data
+    inf = PlanInfo()
+    opt = Options(plan_id, 0, 0)
+    _check(lib().bsa_request_host(ptr(mask), B_Q, B_KV, N, heads, d, ptr(Q), ptr(K), ptr(V), ptr(O), ptr(LSE),
+                                  ctypes.byref(opt), ctypes.byref(inf)), "bsa_request_host")
+    return inf.as_dict()
+
+
+def catalog() -> List[Dict]:
+    out = []
+    for i in range(lib().bsa_catalog_size()):
+        d = PlanDesc()
+        _check(lib().bsa_catalog_get(i, ctypes.byref(d)), "bsa_catalog_get")
+        out.append({f: (getattr(d, f).decode() if f == "name" else getattr(d, f)) for f, _ in PlanDesc._fields_})
+    return out
+
+
+def plan_eligible(plan_id, B_Q, B_KV, N, heads, d, max_workspace_bytes=0) -> bool:
+    return bool(lib().bsa_plan_eligible(plan_id, B_Q, B_KV, N, heads, d, max_workspace_bytes))
+
+
+def lut_load(path: str):
+    _check(lib().bsa_lut_load(path.encode()), "bsa_lut_load")
+
+
+def lut_clear():
+    lib().bsa_lut_clear()
+
+
+def lut_select(B_Q, B_KV, N, heads, d, density, run_coverage, skew, max_workspace_bytes=0) -> Tuple[int, bool]:
+    hit = ctypes.c_int(0)
+    pid = lib().bsa_lut_select(B_Q, B_KV, N, heads, d, density, run_coverage, skew, max_workspace_bytes,
+                               ctypes.byref(hit))
+    return pid, bool(hit.value)
+
+
+def lut_buckets(N, density, skew, run_coverage) -> List[int]:
+    out = (ctypes.c_int32 * 4)()
+    lib().bsa_lut_buckets(N, density, skew, run_coverage, out)
+    return list(out)
+
+
+def force_plan(plan_id: int):
+    lib().bsa_force_plan(plan_id)
+
+
+def kernel_launch_count() -> int:
+    return int(lib().bsa_kernel_launch_count())

@@ -1,0 +1,492 @@
+// C ABI: online request path (paper Section 3 "Online request path", Section 5.2, Algorithm 2).
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+#include <time.h>
+
+#include <atomic>
+#include <new>
+
+#include "bsa_common.h"
+
+namespace bsa {
+// bsa_lut.cpp
+const bsa_plan_desc_t* catalog_entry(int plan_id);
+bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int heads, MapGeom* g);
+int64_t plan_workspace_bytes(const bsa_plan_desc_t& P, int64_t N, int heads, int d);
+bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws);
+int base_plan(int B_Q, int B_KV, int d);
+uint64_t catalog_hash();
+void lut_buckets(int64_t N, double density, double skew, double run_cov, int32_t out[4]);
+void lut_clear();
+int lut_num_regimes();
+bsa_status_t lut_load(const char* path);
+void set_force_plan(int id);
+int get_force_plan();
+int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_cov, double skew,
+               int64_t max_ws, int* hit_out, int32_t buckets_out[4]);
+int catalog_size();
+
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static thread_local char g_cuda_err[256] = "";
+static void set_cuda_err(cudaError_t e, const char* where) {
+    snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", where, cudaGetErrorString(e));
+}
+
+static double now_us() {
+    timespec ts;
+    clock_gettime(CLOCK_MONOTONIC, &ts);
+    return ts.tv_sec * 1e6 + ts.tv_nsec * 1e-3;
+}
+
+static size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+}  // namespace bsa
+
+using namespace bsa;
+
+struct bsa_plan {
+    bsa_plan_desc_t desc;
+    MapGeom g;
+    int d;
+    int stages;
+    cudaStream_t stream;
+    int device;
+    int num_sms;
+    // arena 1 (allocated before the statistics copy)
+    uint8_t* arena1;
+    int32_t* row_nnz;
+    int32_t* row_ptr;
+    MaskStatsDev* stats;
+    PlanCountersDev* counters;
+    int32_t* head_counts;
+    // arena 2 (sized from the statistics)
+    uint8_t* arena2;
+    int32_t* col_idx;
+    int32_t* tile_begin;
+    int32_t* tile_cnt;
+    int32_t* row_parts;
+    int32_t* tile_col;
+    uint64_t* tile_member;
+    WorkItem* items_tmp;
+    WorkItem* items;
+    SplitRow* split_rows;
+    int64_t tile_cap;
+    int64_t max_items;
+    // Split-K workspace
+    float* ws_O;
+    float* ws_LSE;
+    int64_t ws_bytes;
+    // host-side record
+    MaskStatsDev hstats;
+    int lut_hit;
+    int32_t buckets[4];
+    float us_mask_state, us_stats_sync, us_lookup, us_launch_prep, us_total;
+};
+
+static bsa_status_t validate(const void* mask, int B_Q, int B_KV, int64_t N, int heads, int d, void* out) {
+    if (!mask || !out || N <= 0 || heads <= 0) return BSA_ERR_INVALID_ARG;
+    auto p2 = [](int v) { return v >= 16 && v <= 256 && (v & (v - 1)) == 0; };
+    if (!(d == 64 || d == 128) || !p2(B_Q) || !p2(B_KV)) return BSA_ERR_UNSUPPORTED;
+    if (N > (1ll << 30)) return BSA_ERR_UNSUPPORTED;
+    return BSA_OK;
+}
+
+static void free_plan(bsa_plan* p) {
+    if (!p) return;
+    if (p->arena1) cudaFreeAsync(p->arena1, p->stream);
+    if (p->arena2) cudaFreeAsync(p->arena2, p->stream);
+    if (p->ws_O) cudaFreeAsync(p->ws_O, p->stream);
+    delete p;
+}
+
+#define BSA_CUDA(call, where)            \
+    do {                                 \
+        cudaError_t e__ = (call);        \
+        if (e__ != cudaSuccess) {        \
+            set_cuda_err(e__, where);    \
+            free_plan(p);                \
+            return e__ == cudaErrorMemoryAllocation ? BSA_ERR_OOM : BSA_ERR_CUDA; \
+        }                                \
+    } while (0)
+
+extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int B_KV, int64_t N, int heads, int d,
+                                           const bsa_options_t* options, void* stream_v, bsa_plan_t** out_plan) {
+    bsa_status_t vs = validate(mask_dev, B_Q, B_KV, N, heads, d, out_plan);
+    if (vs != BSA_OK) return vs;
+    *out_plan = nullptr;
+    const double t0 = now_us();
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
+    bsa_plan* p = new (std::nothrow) bsa_plan();
+    if (!p) return BSA_ERR_OOM;
+    memset(p, 0, sizeof *p);
+    p->stream = stream;
+    p->d = d;
+    BSA_CUDA(cudaGetDevice(&p->device), "cudaGetDevice");
+    BSA_CUDA(cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, p->device), "device attribute");
+
+    const int nQb = (int)((N + B_Q - 1) / B_Q), nKb = (int)((N + B_KV - 1) / B_KV);
+    const int64_t nrows64 = (int64_t)heads * nQb;
+    if (nrows64 >= (1ll << 31) - 8) { delete p; return BSA_ERR_UNSUPPORTED; }
+    const int nrows = (int)nrows64;
+
+    // ---- Algorithm 2, line 1: shared mask state mu(M), part 1 (row counts + scalar statistics) ----
+    size_t o_nnz = 0, o_ptr = align_up(o_nnz + sizeof(int32_t) * (size_t)nrows);
+    size_t o_zero = align_up(o_ptr + sizeof(int32_t) * ((size_t)nrows + 1));
+    size_t o_stats = o_zero, o_cnt = o_stats + 256, o_hc = o_cnt + 256;
+    size_t a1_bytes = align_up(o_hc + sizeof(int32_t) * 3 * (size_t)heads);
+    BSA_CUDA(cudaMallocAsync(&p->arena1, a1_bytes, stream), "arena1");
+    p->row_nnz = reinterpret_cast<int32_t*>(p->arena1 + o_nnz);
+    p->row_ptr = reinterpret_cast<int32_t*>(p->arena1 + o_ptr);
+    p->stats = reinterpret_cast<MaskStatsDev*>(p->arena1 + o_stats);
+    p->counters = reinterpret_cast<PlanCountersDev*>(p->arena1 + o_cnt);
+    p->head_counts = reinterpret_cast<int32_t*>(p->arena1 + o_hc);
+    BSA_CUDA(cudaMemsetAsync(p->arena1 + o_zero, 0, a1_bytes - o_zero, stream), "memset");
+    BSA_CUDA(launch_mask_row_stats(mask_dev, nrows, nKb, p->row_nnz, p->stats, stream), "mask_row_stats");
+    const double t1 = now_us();
+
+    // ---- lines 3-5: only the scalars cross to the host ----
+    static thread_local MaskStatsDev* pinned = nullptr;
+    if (!pinned) BSA_CUDA(cudaMallocHost(&pinned, sizeof(MaskStatsDev)), "pinned stats");
+    BSA_CUDA(cudaMemcpyAsync(pinned, p->stats, sizeof(MaskStatsDev), cudaMemcpyDeviceToHost, stream), "stats copy");
+    BSA_CUDA(cudaStreamSynchronize(stream), "stats sync");
+    p->hstats = *pinned;
+    const double t2 = now_us();
+
+    // ---- lines 6-19: regime lookup, ranked fallback, eligibility ----
+    const double total_blocks = (double)nrows * nKb;
+    const double nnz = (double)p->hstats.nnz;
+    const double density = total_blocks > 0 ? nnz / total_blocks : 0.0;
+    const double run_cov = nnz > 0 ? (double)p->hstats.in_runs / nnz : 0.0;
+    const double skew = nnz > 0 ? (double)p->hstats.max_row_nnz / (nnz / (double)nrows) : 0.0;
+    const int64_t max_ws = options ? options->max_workspace_bytes : 0;
+    int forced = (options && options->force_plan_id >= 0) ? options->force_plan_id : get_force_plan();
+    int plan_id;
+    if (forced >= 0) {
+        plan_id = plan_eligible(forced, B_Q, B_KV, N, heads, d, max_ws) ? forced : -1;
+        lut_buckets(N, density, skew, run_cov, p->buckets);
+        p->lut_hit = 0;
+    } else {
+        plan_id = lut_select(B_Q, B_KV, N, heads, d, density, run_cov, skew, max_ws, &p->lut_hit, p->buckets);
+    }
+    if (plan_id < 0) { free_plan(p); return BSA_ERR_NO_ELIGIBLE_PLAN; }
+    p->desc = *catalog_entry(plan_id);
+    make_geom(p->desc, B_Q, B_KV, N, heads, &p->g);
+    p->stages = p->desc.stages > 0 ? p->desc.stages : attention_max_stages(d, p->desc.T_KV);
+    const double t3 = now_us();
+
+    // ---- launch preparation: derive only the selected plan's metadata from the block-CSR ----
+    const MapGeom& g = p->g;
+    const int64_t nnz_i = (int64_t)p->hstats.nnz;
+    p->tile_cap = nnz_i * g.rq * g.rk;
+    if (p->tile_cap >= (1ll << 31) - 8) { free_plan(p); return BSA_ERR_UNSUPPORTED; }
+    const int pmax = p->desc.split_pmax < 1 ? 1 : p->desc.split_pmax;
+    const int64_t trows = (int64_t)heads * g.nQt;
+    p->max_items = trows * pmax;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
+    const size_t o_col = take(sizeof(int32_t) * (size_t)(nnz_i + 1));
+    const size_t o_tb = take(sizeof(int32_t) * (size_t)trows);
+    const size_t o_tc = take(sizeof(int32_t) * (size_t)trows);
+    const size_t o_rp = take(sizeof(int32_t) * (size_t)trows);
+    const size_t o_tcol = take(sizeof(int32_t) * (size_t)(p->tile_cap + 1));
+    const size_t o_tmem = take(sizeof(uint64_t) * (size_t)(p->tile_cap + 1));
+    const size_t o_it0 = take(sizeof(WorkItem) * (size_t)p->max_items);
+    const size_t o_it1 = take(sizeof(WorkItem) * (size_t)p->max_items);
+    const size_t o_sr = take(sizeof(SplitRow) * (size_t)(pmax > 1 ? trows : 1));
+    BSA_CUDA(cudaMallocAsync(&p->arena2, o, stream), "arena2");
+    p->col_idx = reinterpret_cast<int32_t*>(p->arena2 + o_col);
+    p->tile_begin = reinterpret_cast<int32_t*>(p->arena2 + o_tb);
+    p->tile_cnt = reinterpret_cast<int32_t*>(p->arena2 + o_tc);
+    p->row_parts = reinterpret_cast<int32_t*>(p->arena2 + o_rp);
+    p->tile_col = reinterpret_cast<int32_t*>(p->arena2 + o_tcol);
+    p->tile_member = reinterpret_cast<uint64_t*>(p->arena2 + o_tmem);
+    p->items_tmp = reinterpret_cast<WorkItem*>(p->arena2 + o_it0);
+    p->items = reinterpret_cast<WorkItem*>(p->arena2 + o_it1);
+    p->split_rows = reinterpret_cast<SplitRow*>(p->arena2 + o_sr);
+    p->ws_bytes = plan_workspace_bytes(p->desc, N, heads, d);
+    if (p->ws_bytes > 0) {
+        BSA_CUDA(cudaMallocAsync(&p->ws_O, (size_t)p->ws_bytes, stream), "workspace");
+        p->ws_LSE = p->ws_O + (size_t)p->max_items * kTQ * d;
+    }
+    BSA_CUDA(launch_row_scan(p->row_nnz, nrows, p->row_ptr, stream), "row_scan");
+    BSA_CUDA(launch_csr_fill(mask_dev, nrows, nKb, p->row_ptr, p->col_idx, stream), "csr_fill");
+    BSA_CUDA(launch_tile_map(g, p->row_ptr, p->col_idx, p->desc.split_tau, pmax, p->tile_begin, p->tile_cnt,
+                             p->row_parts, p->tile_col, p->tile_member, p->head_counts, p->counters, stream),
+             "tile_map");
+    BSA_CUDA(launch_organize(g, p->desc.order, pmax, p->tile_begin, p->tile_cnt, p->row_parts, p->head_counts,
+                             p->items_tmp, p->items, p->split_rows, p->counters, stream),
+             "organize");
+    const double t4 = now_us();
+    p->us_mask_state = (float)(t1 - t0);
+    p->us_stats_sync = (float)(t2 - t1);
+    p->us_lookup = (float)(t3 - t2);
+    p->us_launch_prep = (float)(t4 - t3);
+    p->us_total = (float)(t4 - t0);
+    *out_plan = p;
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_plan_create(const uint8_t* mask_dev, int B_Q, int B_KV, int64_t N, int heads, int d,
+                                        bsa_plan_t** out_plan) {
+    return bsa_plan_create_ex(mask_dev, B_Q, B_KV, N, heads, d, nullptr, nullptr, out_plan);
+}
+
+extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const void* K, const void* V, void* O,
+                                    float* LSE, void* stream_v) {
+    if (!p || !Q || !K || !V || !O || !LSE) return BSA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V) |
+         reinterpret_cast<uintptr_t>(O)) & 15)
+        return BSA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(LSE) & 3) return BSA_ERR_INVALID_ARG;
+    ForwardArgs a;
+    memset(&a, 0, sizeof a);
+    a.Q = Q; a.K = K; a.V = V; a.O = O; a.LSE = LSE;
+    a.items = p->items;
+    a.split_rows = p->split_rows;
+    a.tile_col = p->tile_col;
+    a.tile_member = p->tile_member;
+    a.counters = p->counters;
+    a.ws_O = p->ws_O;
+    a.ws_LSE = p->ws_LSE;
+    a.g = p->g;
+    a.d = p->d;
+    a.stages = p->stages;
+    a.kernel = p->desc.kernel;
+    a.has_split = p->desc.split_pmax > 1;
+    a.max_items = (int32_t)(p->max_items < (1 << 30) ? p->max_items : (1 << 30));
+    a.max_split_rows = p->g.H * p->g.nQt;
+    a.num_sms = p->num_sms;
+    const char* detail = "launch";
+    cudaError_t e = launch_forward(a, reinterpret_cast<cudaStream_t>(stream_v), &detail);
+    if (e != cudaSuccess) {
+        set_cuda_err(e, detail);
+        return BSA_ERR_CUDA;
+    }
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_plan_destroy(bsa_plan_t* p) {
+    if (!p) return BSA_ERR_INVALID_ARG;
+    cudaStream_t s = p->stream;
+    free_plan(p);
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        set_cuda_err(e, "destroy sync");
+        return BSA_ERR_CUDA;
+    }
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_plan_get_info(const bsa_plan_t* p, bsa_plan_info_t* info) {
+    if (!p || !info) return BSA_ERR_INVALID_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    PlanCountersDev c;
+    if (e == cudaSuccess) e = cudaMemcpy(&c, p->counters, sizeof c, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) {
+        set_cuda_err(e, "get_info");
+        return BSA_ERR_CUDA;
+    }
+    memset(info, 0, sizeof *info);
+    info->plan = p->desc;
+    const MapGeom& g = p->g;
+    info->map_q = g.sQ > 1 ? BSA_MAP_COARSENED : (g.rq > 1 ? BSA_MAP_REFINED : BSA_MAP_DIRECT);
+    info->map_kv = g.sK > 1 ? BSA_MAP_COARSENED : (g.rk > 1 ? BSA_MAP_REFINED : BSA_MAP_DIRECT);
+    info->heads = g.H; info->d = p->d; info->B_Q = g.B_Q; info->B_KV = g.B_KV; info->N = g.N;
+    info->nQb = g.nQb; info->nKb = g.nKb; info->nQt = g.nQt; info->nKt = g.nKt;
+    info->member_bits = g.sQ * g.sK;
+    info->lut_hit = p->lut_hit;
+    memcpy(info->regime_bucket, p->buckets, sizeof p->buckets);
+    info->nnz_blocks = (int64_t)p->hstats.nnz;
+    info->blocks_in_runs = (int64_t)p->hstats.in_runs;
+    info->max_row_nnz = (int32_t)p->hstats.max_row_nnz;
+    const double nrows = (double)g.H * g.nQb;
+    const double nnz = (double)p->hstats.nnz;
+    info->density = nrows > 0 ? nnz / (nrows * g.nKb) : 0.0;
+    info->run_coverage = nnz > 0 ? (double)p->hstats.in_runs / nnz : 0.0;
+    info->skew = nnz > 0 ? (double)p->hstats.max_row_nnz / (nnz / nrows) : 0.0;
+    info->ntiles = (int64_t)c.ntiles;
+    info->nitems = c.nitems;
+    info->nsplit_rows = c.nsplit_rows;
+    info->workspace_bytes = p->ws_bytes;
+    info->covered_pairs = (int64_t)c.ntiles * kTQ * g.T_KV;
+    info->us_mask_state = p->us_mask_state;
+    info->us_stats_sync = p->us_stats_sync;
+    info->us_lookup = p->us_lookup;
+    info->us_launch_prep = p->us_launch_prep;
+    info->us_total = p->us_total;
+    info->device_status = c.status;
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_plan_export_csr(const bsa_plan_t* p, int32_t* row_ptr_host, int32_t* col_idx_host) {
+    if (!p) return BSA_ERR_INVALID_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    const size_t nrows = (size_t)p->g.H * p->g.nQb;
+    if (e == cudaSuccess && row_ptr_host)
+        e = cudaMemcpy(row_ptr_host, p->row_ptr, sizeof(int32_t) * (nrows + 1), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && col_idx_host && p->hstats.nnz)
+        e = cudaMemcpy(col_idx_host, p->col_idx, sizeof(int32_t) * (size_t)p->hstats.nnz, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) {
+        set_cuda_err(e, "export_csr");
+        return BSA_ERR_CUDA;
+    }
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_plan_export_tiles(const bsa_plan_t* p, int head, int32_t* tile_row_ptr_host,
+                                              int32_t* tile_col_host, uint64_t* tile_member_host, int64_t cap,
+                                              int64_t* ntiles_out) {
+    if (!p || head < 0 || head >= p->g.H || !ntiles_out) return BSA_ERR_INVALID_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    const int nQt = p->g.nQt;
+    int32_t* tb = new (std::nothrow) int32_t[2 * (size_t)nQt];
+    if (!tb) return BSA_ERR_OOM;
+    int32_t* tc = tb + nQt;
+    if (e == cudaSuccess)
+        e = cudaMemcpy(tb, p->tile_begin + (size_t)head * nQt, sizeof(int32_t) * nQt, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(tc, p->tile_cnt + (size_t)head * nQt, sizeof(int32_t) * nQt, cudaMemcpyDeviceToHost);
+    int64_t total = 0;
+    for (int t = 0; t < nQt && e == cudaSuccess; ++t) total += tc[t];
+    *ntiles_out = total;
+    bsa_status_t st = BSA_OK;
+    if (e == cudaSuccess && tile_row_ptr_host && tile_col_host && tile_member_host) {
+        if (cap < total) {
+            st = BSA_ERR_INVALID_ARG;
+        } else {
+            int64_t off = 0;
+            for (int t = 0; t < nQt && e == cudaSuccess; ++t) {
+                tile_row_ptr_host[t] = (int32_t)off;
+                if (tc[t]) {
+                    e = cudaMemcpy(tile_col_host + off, p->tile_col + tb[t], sizeof(int32_t) * tc[t],
+                                   cudaMemcpyDeviceToHost);
+                    if (e == cudaSuccess)
+                        e = cudaMemcpy(tile_member_host + off, p->tile_member + tb[t], sizeof(uint64_t) * tc[t],
+                                       cudaMemcpyDeviceToHost);
+                }
+                off += tc[t];
+            }
+            tile_row_ptr_host[nQt] = (int32_t)off;
+        }
+    }
+    delete[] tb;
+    if (e != cudaSuccess) {
+        set_cuda_err(e, "export_tiles");
+        return BSA_ERR_CUDA;
+    }
+    return st;
+}
+
+extern "C" bsa_status_t bsa_plan_export_items(const bsa_plan_t* p, int32_t* items_host, int64_t cap,
+                                              int64_t* nitems_out) {
+    if (!p || !nitems_out) return BSA_ERR_INVALID_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    PlanCountersDev c;
+    if (e == cudaSuccess) e = cudaMemcpy(&c, p->counters, sizeof c, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) {
+        set_cuda_err(e, "export_items");
+        return BSA_ERR_CUDA;
+    }
+    *nitems_out = c.nitems;
+    if (items_host) {
+        if (cap < c.nitems) return BSA_ERR_INVALID_ARG;
+        e = cudaMemcpy(items_host, p->items, sizeof(WorkItem) * (size_t)c.nitems, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) {
+            set_cuda_err(e, "export_items copy");
+            return BSA_ERR_CUDA;
+        }
+    }
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int B_KV, int64_t N, int heads, int d,
+                                         const void* Q_host, const void* K_host, const void* V_host, void* O_host,
+                                         float* LSE_host, const bsa_options_t* options, bsa_plan_info_t* info_out) {
+    if (!Q_host || !K_host || !V_host || !O_host || !LSE_host) return BSA_ERR_INVALID_ARG;
+    bsa_plan_t* dummy = nullptr;
+    bsa_status_t vs = validate(mask_host, B_Q, B_KV, N, heads, d, &dummy);
+    if (vs != BSA_OK) return vs;
+    const size_t nQb = (size_t)((N + B_Q - 1) / B_Q), nKb = (size_t)((N + B_KV - 1) / B_KV);
+    const size_t mbytes = (size_t)heads * nQb * nKb;
+    const size_t tbytes = (size_t)heads * (size_t)N * d * 2;
+    const size_t lbytes = (size_t)heads * (size_t)N * 4;
+    const size_t o_m = 0, o_q = align_up(mbytes), o_k = o_q + align_up(tbytes), o_v = o_k + align_up(tbytes),
+                 o_o = o_v + align_up(tbytes), o_l = o_o + align_up(tbytes), total = o_l + align_up(lbytes);
+    cudaStream_t s = nullptr;
+    uint8_t* buf = nullptr;
+    cudaError_t e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
+    if (e != cudaSuccess) { set_cuda_err(e, "stream"); return BSA_ERR_CUDA; }
+    bsa_status_t st = BSA_OK;
+    bsa_plan_t* plan = nullptr;
+    e = cudaMallocAsync(&buf, total, s);
+    if (e != cudaSuccess) { set_cuda_err(e, "request buffers"); cudaStreamDestroy(s); return BSA_ERR_OOM; }
+    e = cudaMemcpyAsync(buf + o_m, mask_host, mbytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_q, Q_host, tbytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_k, K_host, tbytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_v, V_host, tbytes, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) {
+        st = bsa_plan_create_ex(buf + o_m, B_Q, B_KV, N, heads, d, options, s, &plan);
+        if (st == BSA_OK)
+            st = bsa_forward(plan, buf + o_q, buf + o_k, buf + o_v, buf + o_o, reinterpret_cast<float*>(buf + o_l), s);
+        if (st == BSA_OK) {
+            e = cudaMemcpyAsync(O_host, buf + o_o, tbytes, cudaMemcpyDeviceToHost, s);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(LSE_host, buf + o_l, lbytes, cudaMemcpyDeviceToHost, s);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        }
+    }
+    if (st == BSA_OK && e == cudaSuccess && plan) {
+        bsa_plan_info_t info;
+        st = bsa_plan_get_info(plan, &info);
+        if (st == BSA_OK && info.device_status != 0) st = BSA_ERR_DEVICE_TIMEOUT;
+        if (info_out) *info_out = info;
+    }
+    if (plan) bsa_plan_destroy(plan);
+    cudaFreeAsync(buf, s);
+    cudaStreamSynchronize(s);
+    cudaStreamDestroy(s);
+    if (e != cudaSuccess) { set_cuda_err(e, "request"); return BSA_ERR_CUDA; }
+    return st;
+}
+
+extern "C" int bsa_catalog_size(void) { return catalog_size(); }
+extern "C" bsa_status_t bsa_catalog_get(int index, bsa_plan_desc_t* out) {
+    const bsa_plan_desc_t* e = catalog_entry(index);
+    if (!e || !out) return BSA_ERR_INVALID_ARG;
+    *out = *e;
+    return BSA_OK;
+}
+extern "C" int bsa_plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws) {
+    return plan_eligible(plan_id, B_Q, B_KV, N, heads, d, max_ws) ? 1 : 0;
+}
+extern "C" int bsa_base_plan(int B_Q, int B_KV, int d) { return base_plan(B_Q, B_KV, d); }
+extern "C" uint64_t bsa_catalog_hash(void) { return catalog_hash(); }
+extern "C" bsa_status_t bsa_lut_load(const char* path) { return lut_load(path); }
+extern "C" void bsa_lut_clear(void) { lut_clear(); }
+extern "C" int bsa_lut_num_regimes(void) { return lut_num_regimes(); }
+extern "C" int bsa_lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_coverage,
+                              double skew, int64_t max_ws, int* hit_out) {
+    return lut_select(B_Q, B_KV, N, heads, d, density, run_coverage, skew, max_ws, hit_out, nullptr);
+}
+extern "C" void bsa_lut_buckets(int64_t N, double density, double skew, double run_coverage, int32_t out[4]) {
+    lut_buckets(N, density, skew, run_coverage, out);
+}
+extern "C" void bsa_force_plan(int plan_id) { set_force_plan(plan_id); }
+
+extern "C" const char* bsa_status_string(bsa_status_t s) {
+    switch (s) {
+        case BSA_OK: return "ok";
+        case BSA_ERR_INVALID_ARG: return "invalid argument";
+        case BSA_ERR_UNSUPPORTED: return "unsupported geometry or head dimension";
+        case BSA_ERR_NO_ELIGIBLE_PLAN: return "no eligible plan";
+        case BSA_ERR_OOM: return "out of memory";
+        case BSA_ERR_CUDA: return "CUDA error";
+        case BSA_ERR_DEVICE_TIMEOUT: return "bounded device wait expired";
+        case BSA_ERR_LUT: return "plan table rejected";
+    }
+    return "unknown status";
+}
+extern "C" const char* bsa_last_cuda_error(void) { return g_cuda_err; }
+extern "C" const char* bsa_version(void) { return "bsa-b200 0.1 (sm_100a)"; }
+extern "C" int64_t bsa_kernel_launch_count(void) { return g_launches.load(); }

@@ -1,0 +1,549 @@
+// Main attention kernel and Split-K reduction kernel for sm_100a (paper Section 4: "Native CUDA
+// catalog"; Section 2.3 data-compute pipeline; Section 4.3 Split-K).
+//
+// One persistent CTA per SM walks the ordered work-item list.  Inside a CTA the roles are
+// warp-specialised:
+//   warps 0-3  softmax / correction / epilogue: one thread per query row (TMEM lane), reads the
+//              score tile S from tensor memory, applies the intra-tile membership mask, keeps the
+//              online-softmax state (m, l) in registers, writes bf16 P back into tensor memory;
+//   warp 4     TMA producer: gathers K and V tiles by tile index into shared-memory rings
+//              (128-byte swizzle), and the Q tile once per work item;
+//   warp 5     MMA issuer: tcgen05.mma S = Q K^T (both operands in shared memory) and
+//              O += P V (P from tensor memory, V from shared memory, MN-major), fp32 accumulators
+//              in tensor memory; tcgen05.commit signals the mbarriers.
+// S is double-buffered so Q K^T of tile j+1 overlaps the softmax of tile j.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "bsa_common.h"
+#include "sm100_ptx.cuh"
+
+namespace bsa {
+
+using namespace ptx;
+
+namespace {
+
+constexpr int kMaxStages = 6;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units: P stays below 2^8 between rescales
+
+struct AttnParams {
+    const WorkItem* items;
+    const int32_t* tile_col;
+    const uint64_t* tile_member;
+    PlanCountersDev* counters;
+    __nv_bfloat16* O;
+    float* LSE;
+    float* ws_O;
+    float* ws_LSE;
+    unsigned long long full_member;
+    int32_t N;
+    int32_t lgBQ;   // log2(B_Q) when B_Q < 128, else 31 (row >> 31 == 0)
+    int32_t lgBKV;  // log2(B_KV) when B_KV < T_KV, else 31
+    int32_t sK;     // logical KV sub-blocks per tile
+    int32_t stages;
+    float scale_log2;  // log2(e) / sqrt(d)
+};
+
+struct __align__(8) Barriers {
+    uint64_t q_full, q_empty, o_free;
+    uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
+    uint64_t s_full[2], p_ready[2], pv_done[2];
+};
+
+template <int D, int TK>
+__global__ void __launch_bounds__(kThreads, 1)
+bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                     const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+    constexpr int NSUB = D / 64;              // 64-column (128-byte) sub-tiles per row
+    constexpr int Q_SUB = kTQ * 128;          // bytes of one [128][64] bf16 sub-tile
+    constexpr int KV_SUB = TK * 128;          // bytes of one [TK][64] bf16 sub-tile
+    constexpr int KV_TILE = NSUB * KV_SUB;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sQ = smem;
+    uint8_t* sK = sQ + NSUB * Q_SUB;
+    uint8_t* sV = sK + p.stages * KV_TILE;
+    __shared__ Barriers bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ uint32_t abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int NS = p.stages;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bars.q_full), 1);
+        mbar_init(smem_u32(&bars.q_empty), 1);
+        mbar_init(smem_u32(&bars.o_free), 128);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&bars.k_full[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_full[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&bars.s_full[s]), 1);
+            mbar_init(smem_u32(&bars.p_ready[s]), 128);
+            mbar_init(smem_u32(&bars.pv_done[s]), 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(&tmem_base_s), kTmemCols);
+        tmem_relinquish();
+    }
+    if (warp == 4 && lane == 0) {
+        prefetch_tensormap(&tmQ);
+        prefetch_tensormap(&tmK);
+        prefetch_tensormap(&tmV);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    volatile uint32_t* abortp = &abort_flag;
+    const int n_items = p.counters->nitems;
+
+    if (warp == 4) {
+        // =========================== TMA producer ===========================
+        if (lane == 0) {
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const WorkItem it = p.items[idx];
+                if (it.ntiles == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1, abortp);
+                if (!ok) break;
+                mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
+                for (int s = 0; s < NSUB; ++s)
+                    tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, it.q_tile * kTQ, it.head);
+                for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
+                    const int stage = g % NS;
+                    const uint32_t ph = (g / NS) & 1;
+                    const int kv0 = p.tile_col[j] * TK;
+                    ok = mbar_wait(smem_u32(&bars.k_empty[stage]), ph ^ 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), KV_TILE);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sK + stage * KV_TILE + s * KV_SUB), &tmK, smem_u32(&bars.k_full[stage]),
+                                    s * 64, kv0, it.head);
+                    ok = mbar_wait(smem_u32(&bars.v_empty[stage]), ph ^ 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), KV_TILE);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sV + stage * KV_TILE + s * KV_SUB), &tmV, smem_u32(&bars.v_full[stage]),
+                                    s * 64, kv0, it.head);
+                }
+                ++itq;
+            }
+            if (!ok) {
+                // let copies in flight land before the CTA's shared memory goes away
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        }
+    } else if (warp == 5) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
+            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
+            const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
+            const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const int n = p.items[idx].ntiles;
+                if (n == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
+                if (!ok) break;
+                for (int j = 0; j <= n && ok; ++j) {
+                    if (j < n) {
+                        const uint32_t gs = g + j;
+                        const int stage = gs % NS;
+                        const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
+                        ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
+                        if (!ok) break;
+                        tc_fence_after();
+                        // S[sb] = Q K^T.  The previous user of S[sb] (P of tile gs-2, read by its PV MMA)
+                        // precedes this MMA in issue order on the same pipe.
+                        const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint64_t a = descQ + (uint64_t)(((k / 4) * Q_SUB + (k % 4) * 32) >> 4);
+                            const uint64_t b = descK + (uint64_t)((stage * KV_TILE + (k / 4) * KV_SUB + (k % 4) * 32) >> 4);
+                            mma_ss(d_s, a, b, idesc_qk, k > 0);
+                        }
+                        mma_commit(smem_u32(&bars.k_empty[stage]));
+                        mma_commit(smem_u32(&bars.s_full[sb]));
+                        if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
+                    }
+                    if (j >= 1) {
+                        const uint32_t gp = g + j - 1;
+                        const int stage = gp % NS;
+                        const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
+                        ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
+                        if (!ok) break;
+                        ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
+                        if (!ok) break;
+                        if (j == 1) {
+                            ok = mbar_wait(smem_u32(&bars.o_free), (itq & 1) ^ 1, abortp);
+                            if (!ok) break;
+                        }
+                        tc_fence_after();
+                        const uint32_t a_p = tmem + (sb ? kColS1 : kColS0);
+#pragma unroll
+                        for (int k = 0; k < TK / 16; ++k) {
+                            const uint64_t b = descV + (uint64_t)((stage * KV_TILE + k * 2048) >> 4);
+                            mma_ts(tmem + kColO, a_p + k * 8, b, idesc_pv, (j > 1 || k > 0) ? 1u : 0u);
+                        }
+                        mma_commit(smem_u32(&bars.v_empty[stage]));
+                        mma_commit(smem_u32(&bars.pv_done[sb]));
+                    }
+                }
+                g += n;
+                ++itq;
+            }
+        }
+    } else {
+        // =========================== softmax / correction / epilogue ===========================
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        uint32_t itq = 0, g = 0;
+        bool ok = true;
+        const float c2 = p.scale_log2;
+        const unsigned long long sub_mask = (p.sK >= 64) ? ~0ull : ((1ull << p.sK) - 1ull);
+        for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            const WorkItem it = p.items[idx];
+            const int row = it.q_tile * kTQ + tid;
+            const bool row_ok = row < p.N;
+            if (it.ntiles == 0) {
+                // no physical tile touches this Q tile row: O = 0, LSE = -inf
+                if (row_ok) {
+                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D);
+#pragma unroll
+                    for (int c = 0; c < D / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
+                    p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
+                }
+                continue;
+            }
+            float m_ref = -INFINITY, l = 0.f;
+            for (int j = 0; j < it.ntiles; ++j) {
+                const uint32_t gs = g + j, sb = gs & 1;
+                const int kv0 = p.tile_col[it.tile_begin + j] * TK;
+                const unsigned long long member = p.tile_member[it.tile_begin + j];
+                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
+                const uint32_t row_bits = (uint32_t)((member >> ((tid >> p.lgBQ) * p.sK)) & sub_mask);
+                const int n_valid = p.N - kv0;  // columns >= n_valid do not exist
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[sb]), (gs >> 1) & 1, abortp));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_s = tmem + lane_base + (sb ? kColS1 : kColS0);
+                // ---- pass 1: row maximum over the tile ----
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < TK / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(t_s + c * 32, r);
+                    tc_wait_ld();
+                    if (need_mask) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int col = c * 32 + i;
+                            const bool act = ((row_bits >> (col >> p.lgBKV)) & 1u) && (col < n_valid);
+                            mx = fmaxf(mx, act ? __uint_as_float(r[i]) : -INFINITY);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+                    }
+                }
+                // ---- reference maximum: move it only when the tile maximum exceeds it by the threshold ----
+                const float mx2 = mx * c2;
+                float alpha = 1.f;
+                bool rescale = false;
+                if (mx2 > m_ref + kRescaleThreshold) {
+                    alpha = ex2_approx(m_ref - mx2);  // m_ref = -inf -> 0
+                    rescale = (j > 0) && (m_ref != -INFINITY);
+                    m_ref = mx2;
+                }
+                const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                // ---- pass 2: P = exp2(s * c2 - m), bf16, written over S in place ----
+                float rowsum = 0.f;
+#pragma unroll
+                for (int c = 0; c < TK / 32; ++c) {
+                    uint32_t r[32];
+                    uint32_t pk[16];
+                    tmem_ld32(t_s + c * 32, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float s0 = __uint_as_float(r[i]), s1 = __uint_as_float(r[i + 1]);
+                        if (need_mask) {
+                            const int col = c * 32 + i;
+                            const bool a0 = ((row_bits >> (col >> p.lgBKV)) & 1u) && (col < n_valid);
+                            const bool a1 = ((row_bits >> ((col + 1) >> p.lgBKV)) & 1u) && (col + 1 < n_valid);
+                            s0 = a0 ? s0 : -INFINITY;
+                            s1 = a1 ? s1 : -INFINITY;
+                        }
+                        const float p0 = ex2_approx(fmaf(s0, c2, -m_use));
+                        const float p1 = ex2_approx(fmaf(s1, c2, -m_use));
+                        rowsum += p0 + p1;
+                        pk[i >> 1] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st16(t_s + c * 16, pk);
+                }
+                l = l * alpha + rowsum;
+                // ---- correction: rescale the running output when the reference moved ----
+                if (j > 0 && __any_sync(0xffffffffu, rescale)) {
+                    const uint32_t gp = gs - 1;
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[gp & 1]), (gp >> 1) & 1, abortp));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t t_o = tmem + lane_base + kColO;
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(t_o + c * 32, r);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        tmem_st32(t_o + c * 32, r);
+                    }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.p_ready[sb]));
+            }
+            if (!ok) break;
+            // ---- epilogue ----
+            {
+                const uint32_t gl = g + it.ntiles - 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[gl & 1]), (gl >> 1) & 1, abortp));
+                if (!ok) break;
+                tc_fence_after();
+                const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+                const float lse = (l > 0.f) ? fmaf(m_ref, 0.6931471805599453f, logf(l)) : -INFINITY;
+                const uint32_t t_o = tmem + lane_base + kColO;
+                if (it.nparts == 1) {
+                    __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D;
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(t_o + c * 32, r);
+                        tc_wait_ld();
+                        if (row_ok) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                uint4 v;
+                                v.x = pack_bf16x2(__uint_as_float(r[q * 8 + 0]) * inv_l, __uint_as_float(r[q * 8 + 1]) * inv_l);
+                                v.y = pack_bf16x2(__uint_as_float(r[q * 8 + 2]) * inv_l, __uint_as_float(r[q * 8 + 3]) * inv_l);
+                                v.z = pack_bf16x2(__uint_as_float(r[q * 8 + 4]) * inv_l, __uint_as_float(r[q * 8 + 5]) * inv_l);
+                                v.w = pack_bf16x2(__uint_as_float(r[q * 8 + 6]) * inv_l, __uint_as_float(r[q * 8 + 7]) * inv_l);
+                                *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = v;
+                            }
+                        }
+                    }
+                    if (row_ok) p.LSE[(size_t)it.head * p.N + row] = lse;
+                } else {
+                    float* orow = p.ws_O + ((size_t)it.ws_slot * kTQ + tid) * D;
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(t_o + c * 32, r);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            float4 v = make_float4(__uint_as_float(r[q * 4 + 0]) * inv_l, __uint_as_float(r[q * 4 + 1]) * inv_l,
+                                                   __uint_as_float(r[q * 4 + 2]) * inv_l, __uint_as_float(r[q * 4 + 3]) * inv_l);
+                            *reinterpret_cast<float4*>(orow + c * 32 + q * 4) = v;
+                        }
+                    }
+                    p.ws_LSE[(size_t)it.ws_slot * kTQ + tid] = lse;
+                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.o_free));
+            }
+            g += it.ntiles;
+            ++itq;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && abort_flag) atomicExch(&p.counters->status, (int)BSA_ERR_DEVICE_TIMEOUT);
+    if (warp == 5) tmem_dealloc(tmem, kTmemCols);
+}
+
+// ------------------------------------------------------------------------------------------
+// Split-K reduction (Section 4.3): partial states were stored as (normalised O_p, LSE_p), so
+// rescaling to the common maximum, merging and normalising is
+//     LSE = log sum_p exp(LSE_p),  O = sum_p exp(LSE_p - LSE) O_p,
+// taken in fixed partition order (bitwise reproducible).  One CTA per split Q tile row.
+// ------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) bsa_merge_kernel(const SplitRow* __restrict__ split_rows,
+                                                         const PlanCountersDev* __restrict__ counters,
+                                                         const float* __restrict__ ws_O, const float* __restrict__ ws_LSE,
+                                                         __nv_bfloat16* __restrict__ O, float* __restrict__ LSE, int N) {
+    constexpr int GROUPS = D / 8;  // 8 output columns (16 bytes of bf16) per thread step
+    const int n_rows = counters->nsplit_rows;
+    for (int sr = blockIdx.x; sr < n_rows; sr += gridDim.x) {
+        const SplitRow s = split_rows[sr];
+        for (int u = threadIdx.x; u < kTQ * GROUPS; u += blockDim.x) {
+            const int r = u / GROUPS, gcol = (u % GROUPS) * 8;
+            const int row = s.q_tile * kTQ + r;
+            if (row >= N) continue;
+            float m = -INFINITY;
+            for (int q = 0; q < s.nparts; ++q) m = fmaxf(m, ws_LSE[(size_t)(s.ws_slot + q) * kTQ + r]);
+            const float m_use = (m == -INFINITY) ? 0.f : m;
+            float tot = 0.f;
+            float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            for (int q = 0; q < s.nparts; ++q) {
+                const float w = __expf(ws_LSE[(size_t)(s.ws_slot + q) * kTQ + r] - m_use);
+                tot += w;
+                const float4* src = reinterpret_cast<const float4*>(ws_O + ((size_t)(s.ws_slot + q) * kTQ + r) * D + gcol);
+                const float4 a = src[0], b = src[1];
+                acc[0] = fmaf(w, a.x, acc[0]); acc[1] = fmaf(w, a.y, acc[1]);
+                acc[2] = fmaf(w, a.z, acc[2]); acc[3] = fmaf(w, a.w, acc[3]);
+                acc[4] = fmaf(w, b.x, acc[4]); acc[5] = fmaf(w, b.y, acc[5]);
+                acc[6] = fmaf(w, b.z, acc[6]); acc[7] = fmaf(w, b.w, acc[7]);
+            }
+            const float inv = (tot > 0.f) ? 1.f / tot : 0.f;
+            uint4 v;
+            v.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+            v.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+            v.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
+            v.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+            *reinterpret_cast<uint4*>(O + ((size_t)s.head * N + row) * D + gcol) = v;
+            if (gcol == 0) LSE[(size_t)s.head * N + row] = (tot > 0.f) ? m_use + logf(tot) : -INFINITY;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 [heads][N][d] viewed as a 3-D tensor {d, N, heads}; box = {64, rows, 1}; rows beyond N read as zero.
+bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)heads};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * (cuuint64_t)d * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, int TK>
+cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t stream, const char** err) {
+    CUtensorMap tq, tk, tv;
+    if (!encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ) || !encode_map(&tk, a.K, a.g.N, a.g.H, D, TK) ||
+        !encode_map(&tv, a.V, a.g.N, a.g.H, D, TK)) {
+        *err = "cuTensorMapEncodeTiled failed";
+        return cudaErrorInvalidValue;
+    }
+    const int smem = attention_smem_bytes(D, TK, p.stages);
+    static int attr_bytes = 0;  // per instantiation; grows to the largest request seen
+    if (smem > attr_bytes) {
+        cudaError_t e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             smem);
+        if (e != cudaSuccess) {
+            *err = "cudaFuncSetAttribute(max dynamic shared memory)";
+            return e;
+        }
+        attr_bytes = smem;
+    }
+    int grid = a.num_sms < a.max_items ? a.num_sms : a.max_items;
+    if (grid < 1) grid = 1;
+    bsa_attention_kernel<D, TK><<<grid, kThreads, smem, stream>>>(tq, tk, tv, p);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int attention_smem_bytes(int d, int T_KV, int stages) {
+    const int q = kTQ * d * 2;
+    const int kv = T_KV * d * 2;
+    int need = q + 2 * stages * kv + 1024;
+    // more than half of the SM's shared memory, so exactly one CTA (and one 512-column TMEM allocation) per SM
+    if (need < 120 * 1024) need = 120 * 1024;
+    return need;
+}
+
+int attention_max_stages(int d, int T_KV) {
+    const int q = kTQ * d * 2;
+    const int kv = T_KV * d * 2;
+    // 227 KB per CTA minus the kernel's static shared memory (barriers) and alignment slack
+    int s = (232448 - 2048 - 1024 - q) / (2 * kv);
+    if (s > kMaxStages) s = kMaxStages;
+    return s;
+}
+
+cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char** err_detail) {
+    AttnParams p;
+    p.items = a.items;
+    p.tile_col = a.tile_col;
+    p.tile_member = a.tile_member;
+    p.counters = a.counters;
+    p.O = reinterpret_cast<__nv_bfloat16*>(a.O);
+    p.LSE = a.LSE;
+    p.ws_O = a.ws_O;
+    p.ws_LSE = a.ws_LSE;
+    const int bits = a.g.sQ * a.g.sK;
+    p.full_member = (bits >= 64) ? ~0ull : ((1ull << bits) - 1ull);
+    p.N = (int32_t)a.g.N;
+    p.lgBQ = (a.g.sQ > 1) ? a.g.lgBQ : 31;
+    p.lgBKV = (a.g.sK > 1) ? a.g.lgBKV : 31;
+    p.sK = a.g.sK;
+    p.stages = a.stages;
+    p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)a.d));
+    cudaError_t e;
+    if (a.d == 128 && a.g.T_KV == 128) e = launch_attn<128, 128>(a, p, stream, err_detail);
+    else if (a.d == 128 && a.g.T_KV == 64) e = launch_attn<128, 64>(a, p, stream, err_detail);
+    else if (a.d == 64 && a.g.T_KV == 128) e = launch_attn<64, 128>(a, p, stream, err_detail);
+    else if (a.d == 64 && a.g.T_KV == 64) e = launch_attn<64, 64>(a, p, stream, err_detail);
+    else {
+        *err_detail = "no kernel for this (d, T_KV)";
+        return cudaErrorInvalidValue;
+    }
+    if (e != cudaSuccess) return e;
+    if (a.has_split) {
+        int grid = a.max_split_rows < 4 * a.num_sms ? a.max_split_rows : 4 * a.num_sms;
+        if (grid < 1) grid = 1;
+        if (a.d == 128)
+            bsa_merge_kernel<128><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
+                                                            reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N);
+        else
+            bsa_merge_kernel<64><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
+                                                           reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N);
+        count_launch();
+        e = cudaGetLastError();
+    }
+    return e;
+}
+
+}  // namespace bsa

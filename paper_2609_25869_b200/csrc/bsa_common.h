@@ -1,0 +1,102 @@
+// Internal declarations shared by the planner, the attention kernels and the C ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/bsa.h"
+
+namespace bsa {
+
+constexpr int kTQ = 128;  // physical Q tile height of every catalog kernel (one MMA M=128 per CTA)
+
+// One unit of work for a persistent CTA: one Q tile row of one head, restricted to the KV tiles
+// [tile_begin, tile_end) of the plan's tile arrays (a Split-K partition when nparts > 1).
+struct WorkItem {
+    int32_t head;
+    int32_t q_tile;
+    int32_t tile_begin;
+    int32_t tile_end;
+    int32_t part;
+    int32_t nparts;
+    int32_t ws_slot;  // workspace slot of this partition (valid when nparts > 1)
+    int32_t ntiles;   // tile_end - tile_begin (sort key)
+};
+static_assert(sizeof(WorkItem) == 32, "WorkItem must be 32 bytes");
+
+struct SplitRow {
+    int32_t head;
+    int32_t q_tile;
+    int32_t ws_slot;  // first slot; partitions are consecutive
+    int32_t nparts;
+};
+
+// Scalars produced on the device during plan creation.
+struct MaskStatsDev {
+    unsigned long long nnz;
+    unsigned long long in_runs;
+    unsigned int max_row_nnz;
+    unsigned int pad;
+};
+struct PlanCountersDev {
+    unsigned long long ntiles;
+    int32_t nitems;
+    int32_t nsplit_rows;
+    int32_t nslots;
+    int32_t status;  // set by kernels when a bounded wait expires (0 = ok)
+};
+
+// Geometry of the logical -> physical mapping of one plan instance.
+struct MapGeom {
+    int32_t H, nQb, nKb, nQt, nKt;
+    int32_t B_Q, B_KV, T_KV;
+    int32_t sQ, rq;  // logical rows per tile row (coarsened) / tile rows per logical row (refined)
+    int32_t sK, rk;  // same for columns
+    int32_t lgBQ, lgBKV, lgSK;
+    int64_t N;
+};
+
+// ---- planner entry points (bsa_planner.cu); all launch on `stream`, none synchronises -------
+cudaError_t launch_mask_row_stats(const uint8_t* mask, int nrows, int nKb, int32_t* row_nnz, MaskStatsDev* stats,
+                                  cudaStream_t stream);
+cudaError_t launch_row_scan(const int32_t* row_nnz, int nrows, int32_t* row_ptr, cudaStream_t stream);
+cudaError_t launch_csr_fill(const uint8_t* mask, int nrows, int nKb, const int32_t* row_ptr, int32_t* col_idx,
+                            cudaStream_t stream);
+cudaError_t launch_tile_map(const MapGeom& g, const int32_t* row_ptr, const int32_t* col_idx, int split_tau,
+                            int split_pmax, int32_t* tile_begin, int32_t* tile_cnt, int32_t* row_parts,
+                            int32_t* tile_col, uint64_t* tile_member, int32_t* head_counts /* [3*H] */,
+                            PlanCountersDev* counters, cudaStream_t stream);
+cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const int32_t* tile_begin,
+                            const int32_t* tile_cnt, const int32_t* row_parts, const int32_t* head_counts, WorkItem* items_tmp,
+                            WorkItem* items, SplitRow* split_rows, PlanCountersDev* counters, cudaStream_t stream);
+size_t organize_smem_bytes(const MapGeom& g, int order, int split_pmax);
+
+// ---- attention + merge (bsa_attention.cu) ----------------------------------------------------
+struct ForwardArgs {
+    const void* Q;
+    const void* K;
+    const void* V;
+    void* O;
+    float* LSE;
+    const WorkItem* items;
+    const SplitRow* split_rows;
+    const int32_t* tile_col;
+    const uint64_t* tile_member;
+    PlanCountersDev* counters;
+    float* ws_O;    // [nslots][128][d] fp32, normalised partial outputs
+    float* ws_LSE;  // [nslots][128]    fp32, partial log-sum-exp
+    MapGeom g;
+    int32_t d;
+    int32_t stages;
+    int32_t kernel;
+    int32_t has_split;
+    int32_t max_items;       // host-side upper bound of the item count
+    int32_t max_split_rows;  // host-side upper bound
+    int32_t num_sms;
+};
+cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char** err_detail);
+int attention_max_stages(int d, int T_KV);
+int attention_smem_bytes(int d, int T_KV, int stages);
+
+void count_launch(int n = 1);
+
+}  // namespace bsa

@@ -1,0 +1,254 @@
+// Catalog C_A, eligibility, feature schema F_A and plan table Pi_A with the online selection of
+// Algorithm 2 (paper Section 4.4 and Section 5.2).  Host code only.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <map>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "bsa_common.h"
+
+namespace bsa {
+
+// ---------------------------------------------------------------------------------------------
+// catalog: every entry is a precompiled kernel + organisation; plan_id == index
+// ---------------------------------------------------------------------------------------------
+static const bsa_plan_desc_t kCatalog[] = {
+    //  id  T_Q  T_KV stages tau pmax order                       kernel name
+    {0, 128, 128, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 0, "q128k128"},
+    {1, 128, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 0, "q128k64"},
+    {2, 128, 128, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 0, "q128k128_split4x8"},
+    {3, 128, 64, 0, 8, 8, BSA_ORDER_HEAD_MAJOR_LPT, 0, "q128k64_split8x8"},
+    {4, 128, 128, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 0, "q128k128_global"},
+    {5, 128, 64, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 0, "q128k64_global"},
+    {6, 128, 128, 2, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 0, "q128k128_s2"},
+    {7, 128, 64, 3, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 0, "q128k64_s3"},
+    {8, 128, 128, 0, 16, 4, BSA_ORDER_GLOBAL_LPT, 0, "q128k128_split16x4_global"},
+    {9, 128, 64, 0, 2, 16, BSA_ORDER_HEAD_MAJOR_LPT, 0, "q128k64_split2x16"},
+};
+static const int kCatalogSize = (int)(sizeof(kCatalog) / sizeof(kCatalog[0]));
+static const int64_t kDefaultWorkspace = 2ll << 30;
+static const size_t kPlannerSmemLimit = 200 * 1024;
+
+static bool pow2_in(int v, int lo, int hi) { return v >= lo && v <= hi && (v & (v - 1)) == 0; }
+
+const bsa_plan_desc_t* catalog_entry(int plan_id) {
+    if (plan_id < 0 || plan_id >= kCatalogSize) return nullptr;
+    return &kCatalog[plan_id];
+}
+
+int ilog2(int v) {
+    int l = 0;
+    while ((1 << l) < v) ++l;
+    return l;
+}
+
+bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int heads, MapGeom* g) {
+    g->H = heads;
+    g->N = N;
+    g->B_Q = B_Q;
+    g->B_KV = B_KV;
+    g->T_KV = P.T_KV;
+    g->nQb = (int)((N + B_Q - 1) / B_Q);
+    g->nKb = (int)((N + B_KV - 1) / B_KV);
+    g->nQt = (int)((N + kTQ - 1) / kTQ);
+    g->nKt = (int)((N + P.T_KV - 1) / P.T_KV);
+    g->sQ = B_Q < kTQ ? kTQ / B_Q : 1;
+    g->rq = B_Q > kTQ ? B_Q / kTQ : 1;
+    g->sK = B_KV < P.T_KV ? P.T_KV / B_KV : 1;
+    g->rk = B_KV > P.T_KV ? B_KV / P.T_KV : 1;
+    g->lgBQ = ilog2(B_Q);
+    g->lgBKV = ilog2(B_KV);
+    g->lgSK = ilog2(g->sK);
+    return true;
+}
+
+int64_t plan_workspace_bytes(const bsa_plan_desc_t& P, int64_t N, int heads, int d) {
+    if (P.split_pmax <= 1) return 0;
+    const int64_t nQt = (N + kTQ - 1) / kTQ;
+    return (int64_t)heads * nQt * P.split_pmax * kTQ * (int64_t)(d + 1) * 4;
+}
+
+// Eligible(P, R), Section 4.4: logical geometry, tensor properties, metadata format, workspace.
+bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws) {
+    const bsa_plan_desc_t* P = catalog_entry(plan_id);
+    if (!P) return false;
+    if (!(d == 64 || d == 128)) return false;
+    if (!pow2_in(B_Q, 16, 256) || !pow2_in(B_KV, 16, 256)) return false;
+    if (N <= 0 || heads <= 0 || N > (1ll << 30)) return false;
+    MapGeom g;
+    make_geom(*P, B_Q, B_KV, N, heads, &g);
+    if (g.sQ * g.sK > 64) return false;  // membership word is 64 bits
+    const int max_st = attention_max_stages(d, P->T_KV);
+    if (max_st < 2) return false;
+    if (P->stages > max_st) return false;
+    if ((size_t)g.nKt * 8 > kPlannerSmemLimit) return false;
+    if (organize_smem_bytes(g, P->order, P->split_pmax) > kPlannerSmemLimit) return false;
+    if ((int64_t)heads * g.nQt * (P->split_pmax < 1 ? 1 : P->split_pmax) >= (1ll << 31)) return false;
+    if (max_ws <= 0) max_ws = kDefaultWorkspace;
+    if (plan_workspace_bytes(*P, N, heads, d) > max_ws) return false;
+    return true;
+}
+
+int base_plan(int B_Q, int B_KV, int d) {
+    (void)B_Q;
+    (void)B_KV;
+    (void)d;
+    return 0;  // q128k128: eligible for every supported geometry (membership <= 64 bits), no workspace
+}
+
+uint64_t catalog_hash() {
+    uint64_t h = 1469598103934665603ull;
+    const unsigned char* p = reinterpret_cast<const unsigned char*>(kCatalog);
+    for (size_t i = 0; i < sizeof(kCatalog); ++i) {
+        h ^= p[i];
+        h *= 1099511628211ull;
+    }
+    return h;
+}
+
+// ---------------------------------------------------------------------------------------------
+// feature schema F_A: fixed bucket edges (Section 5.1: "predefined intervals")
+// ---------------------------------------------------------------------------------------------
+static const double kDensityEdges[] = {0.02, 0.05, 0.08, 0.15, 0.25, 0.45};
+static const double kSkewEdges[] = {1.5, 3.0, 6.0};
+static const double kRunCovEdges[] = {0.5};
+
+static int bucket_of(double v, const double* edges, int n) {
+    int b = 0;
+    while (b < n && v >= edges[b]) ++b;
+    return b;
+}
+
+void lut_buckets(int64_t N, double density, double skew, double run_cov, int32_t out[4]) {
+    int nb = 0;
+    while ((1ll << (nb + 1)) <= N) ++nb;  // floor(log2 N)
+    out[0] = nb;
+    out[1] = bucket_of(density, kDensityEdges, 6);
+    out[2] = bucket_of(skew, kSkewEdges, 3);
+    out[3] = bucket_of(run_cov, kRunCovEdges, 1);
+}
+
+// ---------------------------------------------------------------------------------------------
+// plan table Pi_A
+// ---------------------------------------------------------------------------------------------
+struct RegimeKey {
+    int B_Q, B_KV, d;      // request key k_A(R) (architecture and dtype are fixed: sm_100a, bf16)
+    int nb, hb;            // bucketed request dimensions u_A(R): floor(log2 N), head bucket
+    int db, sb, rb;        // bucketed mask statistics s_A(M)
+    bool operator<(const RegimeKey& o) const {
+        return memcmp(this, &o, sizeof(RegimeKey)) < 0;
+    }
+};
+static std::map<RegimeKey, std::vector<int>> g_table;
+static std::mutex g_mu;
+static int g_force_plan = -1;
+
+static int head_bucket(int heads) { return heads <= 4 ? 0 : (heads <= 16 ? 1 : 2); }
+
+void lut_clear() {
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_table.clear();
+}
+
+int lut_num_regimes() {
+    std::lock_guard<std::mutex> lk(g_mu);
+    return (int)g_table.size();
+}
+
+// File format (text, one record per line):
+//   BSA_LUT 1
+//   catalog <hex hash>
+//   gpu <free text>
+//   regime B_Q B_KV d nb hb db sb rb : id id id ...
+bsa_status_t lut_load(const char* path) {
+    lut_clear();
+    if (!path) return BSA_ERR_INVALID_ARG;
+    FILE* f = fopen(path, "r");
+    if (!f) return BSA_ERR_LUT;
+    char line[1024];
+    bool header = false, hash_ok = false;
+    std::map<RegimeKey, std::vector<int>> table;
+    bsa_status_t st = BSA_OK;
+    while (fgets(line, sizeof line, f)) {
+        if (line[0] == '#' || line[0] == '\n') continue;
+        if (!strncmp(line, "BSA_LUT", 7)) {
+            int ver = 0;
+            if (sscanf(line + 7, "%d", &ver) != 1 || ver != 1) { st = BSA_ERR_LUT; break; }
+            header = true;
+        } else if (!strncmp(line, "catalog", 7)) {
+            unsigned long long hsh = 0;
+            if (sscanf(line + 7, "%llx", &hsh) != 1 || hsh != catalog_hash()) { st = BSA_ERR_LUT; break; }
+            hash_ok = true;
+        } else if (!strncmp(line, "gpu", 3)) {
+            continue;
+        } else if (!strncmp(line, "regime", 6)) {
+            RegimeKey k;
+            memset(&k, 0, sizeof k);
+            int used = 0;
+            if (sscanf(line + 6, "%d %d %d %d %d %d %d %d :%n", &k.B_Q, &k.B_KV, &k.d, &k.nb, &k.hb, &k.db, &k.sb, &k.rb,
+                       &used) != 8 || used == 0) { st = BSA_ERR_LUT; break; }
+            std::vector<int> ids;
+            const char* q = line + 6 + used;
+            char* end = nullptr;
+            while (true) {
+                long v = strtol(q, &end, 10);
+                if (end == q) break;
+                if (v < 0 || v >= kCatalogSize) { st = BSA_ERR_LUT; break; }
+                ids.push_back((int)v);
+                q = end;
+            }
+            if (st != BSA_OK || ids.empty()) { st = BSA_ERR_LUT; break; }
+            table[k] = ids;
+        } else {
+            st = BSA_ERR_LUT;
+            break;
+        }
+    }
+    fclose(f);
+    if (st == BSA_OK && !(header && hash_ok)) st = BSA_ERR_LUT;
+    if (st != BSA_OK) return st;
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_table.swap(table);
+    return BSA_OK;
+}
+
+void set_force_plan(int id) { g_force_plan = id; }
+int get_force_plan() { return g_force_plan; }
+
+// Algorithm 2, lines 6-19: z = <k, u, s>; r = rho(z); ranked list or base plan; first eligible.
+int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_cov, double skew,
+               int64_t max_ws, int* hit_out, int32_t buckets_out[4]) {
+    int32_t b[4];
+    lut_buckets(N, density, skew, run_cov, b);
+    if (buckets_out) memcpy(buckets_out, b, sizeof b);
+    RegimeKey k;
+    memset(&k, 0, sizeof k);
+    k.B_Q = B_Q; k.B_KV = B_KV; k.d = d;
+    k.nb = b[0]; k.hb = head_bucket(heads);
+    k.db = b[1]; k.sb = b[2]; k.rb = b[3];
+    std::vector<int> ranked;
+    bool hit = false;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_table.find(k);
+        if (it != g_table.end()) {
+            ranked = it->second;
+            hit = true;
+        }
+    }
+    if (!hit) ranked.push_back(base_plan(B_Q, B_KV, d));
+    if (hit_out) *hit_out = hit ? 1 : 0;
+    for (int id : ranked)
+        if (plan_eligible(id, B_Q, B_KV, N, heads, d, max_ws)) return id;
+    return -1;
+}
+
+int lut_head_bucket(int heads) { return head_bucket(heads); }
+int catalog_size() { return kCatalogSize; }
+
+}  // namespace bsa

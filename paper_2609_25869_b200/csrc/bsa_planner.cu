@@ -1,0 +1,442 @@
+// Plan construction on the GPU (paper Section 5.2 "Regime lookup" / "Launch preparation",
+// Section 4.2 physical mapping, Section 4.3 task organisation).
+//
+//   mask_row_stats : M -> active blocks per row + scalar statistics s_A(M) (density inputs,
+//                    active-block-run coverage, max row nnz)
+//   row_scan       : exclusive scan -> block-CSR offsets
+//   csr_fill       : sorted active KV column indices (block-CSR of the shared mask state mu(M))
+//   tile_map       : block-CSR -> physical tiles with membership bits (Direct / Coarsened / Refined)
+//                    + Split-K partition count of every Q tile row
+//   organize       : work items (Q tile row x KV partition), ordered longest-first
+//
+// All kernels are integer-only and bandwidth-bound; none needs the host between them.
+#include "bsa_common.h"
+
+namespace bsa {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+// ------------------------------------------------------------------------------------------
+// mask_row_stats: one warp per (head, query-block) row.
+// A block counts towards run coverage iff its left or right neighbour in the same row is active.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __restrict__ mask, int nrows, int nKb,
+                                                              int32_t* __restrict__ row_nnz, MaskStatsDev* stats) {
+    __shared__ unsigned s_nnz[8], s_runs[8], s_max[8];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + warp;
+    unsigned nnz = 0, runs = 0;
+    if (row < nrows) {
+        const uint8_t* m = mask + (size_t)row * nKb;
+        for (int j0 = 0; j0 < nKb; j0 += 32) {
+            const int j = j0 + lane;
+            const bool a = (j < nKb) && m[j] != 0;
+            const unsigned bits = __ballot_sync(kFull, a);
+            unsigned left = bits << 1, right = bits >> 1;
+            // neighbours across the 32-block chunk boundary (same row only)
+            if (j0 > 0 && m[j0 - 1] != 0) left |= 1u;
+            if (j0 + 32 < nKb && m[j0 + 32] != 0) right |= 0x80000000u;
+            nnz += __popc(bits);
+            runs += __popc(bits & (left | right));
+        }
+        if (lane == 0) row_nnz[row] = (int32_t)nnz;
+    }
+    if (lane == 0) {
+        s_nnz[warp] = nnz;
+        s_runs[warp] = runs;
+        s_max[warp] = nnz;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long tn = 0, tr = 0;
+        unsigned mx = 0;
+        for (int w = 0; w < 8; ++w) {
+            tn += s_nnz[w];
+            tr += s_runs[w];
+            mx = max(mx, s_max[w]);
+        }
+        if (tn) {
+            atomicAdd(&stats->nnz, tn);
+            atomicAdd(&stats->in_runs, tr);
+            atomicMax(&stats->max_row_nnz, mx);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// row_scan: exclusive scan of row_nnz by one CTA (rows are few: heads * query blocks).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) row_scan_kernel(const int32_t* __restrict__ row_nnz, int nrows,
+                                                        int32_t* __restrict__ row_ptr) {
+    __shared__ int32_t warp_sums[32];
+    __shared__ int32_t carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = (nrows + 1023) / 1024;
+    const int b = tid * per, e = min(nrows, b + per);
+    int32_t sum = 0;
+    for (int i = b; i < e; ++i) sum += row_nnz[i];
+    int32_t incl = sum;
+    for (int o = 1; o < 32; o <<= 1) {
+        int32_t v = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int32_t w = warp_sums[lane];
+        int32_t wi = w;
+        for (int o = 1; o < 32; o <<= 1) {
+            int32_t v = __shfl_up_sync(kFull, wi, o);
+            if (lane >= o) wi += v;
+        }
+        warp_sums[lane] = wi - w;
+        if (lane == 31) carry_s = wi;
+    }
+    __syncthreads();
+    int32_t run = warp_sums[warp] + incl - sum;
+    for (int i = b; i < e; ++i) {
+        row_ptr[i] = run;
+        run += row_nnz[i];
+    }
+    if (tid == 0) row_ptr[nrows] = carry_s;
+}
+
+// ------------------------------------------------------------------------------------------
+// csr_fill: one warp per row, ballot compaction keeps columns ascending.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) csr_fill_kernel(const uint8_t* __restrict__ mask, int nrows, int nKb,
+                                                        const int32_t* __restrict__ row_ptr,
+                                                        int32_t* __restrict__ col_idx) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + warp;
+    if (row >= nrows) return;
+    const uint8_t* m = mask + (size_t)row * nKb;
+    int32_t out = row_ptr[row];
+    for (int j0 = 0; j0 < nKb; j0 += 32) {
+        const int j = j0 + lane;
+        const bool a = (j < nKb) && m[j] != 0;
+        const unsigned bits = __ballot_sync(kFull, a);
+        if (a) col_idx[out + __popc(bits & ((1u << lane) - 1u))] = j;
+        out += __popc(bits);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// tile_map: one CTA per physical Q tile row.  A shared-memory array holds one membership word
+// per KV tile column; the active blocks of the tile row's logical rows OR their bit into it
+// (Coarsened), or name `rk` finer tile columns each (Refined, column c -> c*rk .. c*rk+rk-1).
+// Non-zero words are then compacted in column order.  Output position of tile row t is a
+// capacity offset computed from the block-CSR alone, so no second scan is needed.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t* __restrict__ row_ptr,
+                                                        const int32_t* __restrict__ col_idx, int split_tau,
+                                                        int split_pmax, int32_t* __restrict__ tile_begin,
+                                                        int32_t* __restrict__ tile_cnt, int32_t* __restrict__ row_parts,
+                                                        int32_t* __restrict__ tile_col,
+                                                        uint64_t* __restrict__ tile_member,
+                                                        int32_t* __restrict__ head_counts, PlanCountersDev* counters) {
+    extern __shared__ unsigned long long bm[];  // [nKt]
+    __shared__ int32_t warp_cnt[8];
+    __shared__ int32_t running;
+    const int trow = blockIdx.x;
+    const int h = trow / g.nQt, t = trow % g.nQt;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < g.nKt; i += blockDim.x) bm[i] = 0ull;
+    if (tid == 0) running = 0;
+    __syncthreads();
+
+    int32_t cap_begin;
+    if (g.rq == 1) {
+        const int r0 = t * g.sQ;
+        const int r1 = min(r0 + g.sQ, g.nQb);
+        const int32_t base = row_ptr[h * g.nQb + r0];
+        cap_begin = base * g.rk;
+        for (int r = r0; r < r1; ++r) {
+            const int a = r - r0;
+            const int32_t b = row_ptr[h * g.nQb + r], e = row_ptr[h * g.nQb + r + 1];
+            for (int32_t i = b + tid; i < e; i += blockDim.x) {
+                const int c = col_idx[i];
+                if (g.rk == 1) {
+                    const int tc = c >> g.lgSK;
+                    const int bit = a * g.sK + (c & (g.sK - 1));
+                    atomicOr(&bm[tc], 1ull << bit);
+                } else {
+                    for (int k = 0; k < g.rk; ++k) {
+                        const int tc = c * g.rk + k;
+                        if (tc < g.nKt) atomicOr(&bm[tc], 1ull << a);
+                    }
+                }
+            }
+        }
+    } else {
+        const int r = t / g.rq, sub = t % g.rq;
+        const int32_t b = row_ptr[h * g.nQb + r], e = row_ptr[h * g.nQb + r + 1];
+        cap_begin = (b * g.rq + sub * (e - b)) * g.rk;
+        for (int32_t i = b + tid; i < e; i += blockDim.x) {
+            const int c = col_idx[i];
+            if (g.rk == 1) {
+                const int tc = c >> g.lgSK;
+                atomicOr(&bm[tc], 1ull << (c & (g.sK - 1)));
+            } else {
+                for (int k = 0; k < g.rk; ++k) {
+                    const int tc = c * g.rk + k;
+                    if (tc < g.nKt) bm[tc] = 1ull;
+                }
+            }
+        }
+    }
+    __syncthreads();
+
+    for (int i0 = 0; i0 < g.nKt; i0 += blockDim.x) {
+        const int i = i0 + tid;
+        const unsigned long long w = (i < g.nKt) ? bm[i] : 0ull;
+        const unsigned bits = __ballot_sync(kFull, w != 0ull);
+        if (lane == 0) warp_cnt[warp] = __popc(bits);
+        __syncthreads();
+        int32_t before = running;
+        int32_t total = 0;
+        for (int k = 0; k < 8; ++k) {
+            if (k < warp) before += warp_cnt[k];
+            total += warp_cnt[k];
+        }
+        if (w != 0ull) {
+            const int32_t pos = cap_begin + before + __popc(bits & ((1u << lane) - 1u));
+            tile_col[pos] = i;
+            tile_member[pos] = w;
+        }
+        __syncthreads();
+        if (tid == 0) running += total;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        const int32_t cnt = running;
+        tile_begin[trow] = cap_begin;
+        tile_cnt[trow] = cnt;
+        int32_t P = 1;
+        if (split_pmax > 1 && cnt > split_tau) P = min(split_pmax, (cnt + split_tau - 1) / split_tau);
+        row_parts[trow] = P;
+        atomicAdd(&head_counts[3 * h + 0], P);
+        if (P > 1) {
+            atomicAdd(&head_counts[3 * h + 1], 1);
+            atomicAdd(&head_counts[3 * h + 2], P);
+        }
+        if (cnt) atomicAdd(&counters->ntiles, (unsigned long long)cnt);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// organize: one CTA per group of Q tile rows (a head, or all heads for the global order).
+//   A. scan the rows' partition counts -> unsorted items (row-major, partition-minor), Split-K
+//      row list and workspace slots;
+//   B. histogram of item lengths, suffix-summed so longer items come first;
+//   C. one warp walks the items in order and assigns each its rank inside its length bucket
+//      (stable: ties keep (head, q_tile, part) order), then all threads scatter.
+// Shared memory: bins [nKt + 2] then one int per item of the group.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int32_t block_excl_scan(int32_t v, int32_t* warp_buf, int32_t* total_out) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    int32_t incl = v;
+    for (int o = 1; o < 32; o <<= 1) {
+        int32_t x = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += x;
+    }
+    __syncthreads();
+    if (lane == 31) warp_buf[warp] = incl;
+    __syncthreads();
+    int32_t before = 0, total = 0;
+    for (int k = 0; k < nw; ++k) {
+        const int32_t s = warp_buf[k];
+        if (k < warp) before += s;
+        total += s;
+    }
+    *total_out = total;
+    return before + incl - v;
+}
+
+__global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, const int32_t* __restrict__ tile_begin,
+                                                         const int32_t* __restrict__ tile_cnt,
+                                                         const int32_t* __restrict__ row_parts,
+                                                         const int32_t* __restrict__ head_counts,
+                                                         WorkItem* __restrict__ items_tmp, WorkItem* __restrict__ items,
+                                                         SplitRow* __restrict__ split_rows, PlanCountersDev* counters) {
+    extern __shared__ int32_t sm[];
+    __shared__ int32_t warp_buf[32];
+    const int nbins = g.nKt + 2;
+    int32_t* bins = sm;            // [nbins]
+    int32_t* key = sm + nbins;     // [items of the group]: length, then rank
+    const int tid = threadIdx.x;
+    const int grp = blockIdx.x;
+    int row0, row1, item_base = 0, split_base = 0, slot_base = 0;
+    if (order == BSA_ORDER_GLOBAL_LPT) {
+        row0 = 0;
+        row1 = g.H * g.nQt;
+    } else {
+        row0 = grp * g.nQt;
+        row1 = row0 + g.nQt;
+        for (int hh = 0; hh < grp; ++hh) {
+            item_base += head_counts[3 * hh + 0];
+            split_base += head_counts[3 * hh + 1];
+            slot_base += head_counts[3 * hh + 2];
+        }
+    }
+    for (int i = tid; i < nbins; i += blockDim.x) bins[i] = 0;
+    __syncthreads();
+
+    // ---- A: unsorted items ----
+    int32_t run_items = 0, run_split = 0, run_slots = 0;
+    for (int r0 = row0; r0 < row1; r0 += blockDim.x) {
+        const int r = r0 + tid;
+        const int32_t P = (r < row1) ? row_parts[r] : 0;
+        int32_t tot_i, tot_s, tot_w;
+        const int32_t off_i = block_excl_scan(P, warp_buf, &tot_i);
+        const int32_t off_s = block_excl_scan(P > 1 ? 1 : 0, warp_buf, &tot_s);
+        const int32_t off_w = block_excl_scan(P > 1 ? P : 0, warp_buf, &tot_w);
+        if (r < row1) {
+            const int32_t tb = tile_begin[r], cnt = tile_cnt[r];
+            const int32_t slot = slot_base + run_slots + off_w;
+            for (int p = 0; p < P; ++p) {
+                WorkItem it;
+                it.head = r / g.nQt;
+                it.q_tile = r % g.nQt;
+                it.tile_begin = tb + (int32_t)(((int64_t)cnt * p) / P);
+                it.tile_end = tb + (int32_t)(((int64_t)cnt * (p + 1)) / P);
+                it.part = p;
+                it.nparts = P;
+                it.ws_slot = (P > 1) ? slot + p : -1;
+                it.ntiles = it.tile_end - it.tile_begin;
+                const int32_t li = run_items + off_i + p;
+                items_tmp[item_base + li] = it;
+                key[li] = it.ntiles;
+                atomicAdd(&bins[it.ntiles], 1);
+            }
+            if (P > 1) {
+                SplitRow s;
+                s.head = r / g.nQt;
+                s.q_tile = r % g.nQt;
+                s.ws_slot = slot;
+                s.nparts = P;
+                split_rows[split_base + run_split + off_s] = s;
+            }
+        }
+        run_items += tot_i;
+        run_split += tot_s;
+        run_slots += tot_w;
+    }
+    __syncthreads();
+    const int32_t n_items = run_items;
+
+    // ---- B: bucket starts, longest first ----
+    if (tid < 32) {
+        int32_t carry = 0;
+        for (int hi = nbins - 1; hi >= 0; hi -= 32) {
+            const int b = hi - tid;
+            const int32_t c = (b >= 0) ? bins[b] : 0;
+            int32_t incl = c;
+            for (int o = 1; o < 32; o <<= 1) {
+                int32_t x = __shfl_up_sync(kFull, incl, o);
+                if (tid >= o) incl += x;
+            }
+            if (b >= 0) bins[b] = carry + incl - c;
+            carry += __shfl_sync(kFull, incl, 31);
+        }
+    }
+    __syncthreads();
+
+    // ---- C1: stable rank, one warp, items in order ----
+    if (tid < 32) {
+        for (int i0 = 0; i0 < n_items; i0 += 32) {
+            const int i = i0 + tid;
+            const bool valid = i < n_items;
+            const int32_t k = valid ? key[i] : -1 - tid;  // invalid lanes get unique keys
+            const unsigned peers = __match_any_sync(kFull, k);
+            int32_t rank = 0;
+            if (valid) {
+                rank = bins[k] + __popc(peers & ((1u << tid) - 1u));
+            }
+            __syncwarp();
+            if (valid && (peers >> tid) <= 1u) bins[k] += __popc(peers);  // highest lane of the peer set
+            __syncwarp();
+            if (valid) key[i] = rank;
+        }
+    }
+    __syncthreads();
+
+    // ---- C2: scatter ----
+    for (int i = tid; i < n_items; i += blockDim.x) items[item_base + key[i]] = items_tmp[item_base + i];
+
+    if (tid == 0) {
+        if (order == BSA_ORDER_GLOBAL_LPT) {
+            counters->nitems = n_items;
+            counters->nsplit_rows = run_split;
+            counters->nslots = run_slots;
+        } else if (grp == gridDim.x - 1) {
+            counters->nitems = item_base + n_items;
+            counters->nsplit_rows = split_base + run_split;
+            counters->nslots = slot_base + run_slots;
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_mask_row_stats(const uint8_t* mask, int nrows, int nKb, int32_t* row_nnz, MaskStatsDev* stats,
+                                  cudaStream_t stream) {
+    mask_row_stats_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, nrows, nKb, row_nnz, stats);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_row_scan(const int32_t* row_nnz, int nrows, int32_t* row_ptr, cudaStream_t stream) {
+    row_scan_kernel<<<1, 1024, 0, stream>>>(row_nnz, nrows, row_ptr);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_csr_fill(const uint8_t* mask, int nrows, int nKb, const int32_t* row_ptr, int32_t* col_idx,
+                            cudaStream_t stream) {
+    csr_fill_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, nrows, nKb, row_ptr, col_idx);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tile_map(const MapGeom& g, const int32_t* row_ptr, const int32_t* col_idx, int split_tau,
+                            int split_pmax, int32_t* tile_begin, int32_t* tile_cnt, int32_t* row_parts,
+                            int32_t* tile_col, uint64_t* tile_member, int32_t* head_counts, PlanCountersDev* counters,
+                            cudaStream_t stream) {
+    const size_t smem = (size_t)g.nKt * sizeof(unsigned long long);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(tile_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    tile_map_kernel<<<g.H * g.nQt, 256, smem, stream>>>(g, row_ptr, col_idx, split_tau, split_pmax, tile_begin,
+                                                        tile_cnt, row_parts, tile_col, tile_member, head_counts,
+                                                        counters);
+    count_launch();
+    return cudaGetLastError();
+}
+
+size_t organize_smem_bytes(const MapGeom& g, int order, int split_pmax) {
+    const size_t rows = (order == BSA_ORDER_GLOBAL_LPT) ? (size_t)g.H * g.nQt : (size_t)g.nQt;
+    return ((size_t)g.nKt + 2 + rows * (size_t)(split_pmax < 1 ? 1 : split_pmax)) * sizeof(int32_t);
+}
+
+cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const int32_t* tile_begin,
+                            const int32_t* tile_cnt, const int32_t* row_parts, const int32_t* head_counts,
+                            WorkItem* items_tmp, WorkItem* items, SplitRow* split_rows, PlanCountersDev* counters,
+                            cudaStream_t stream) {
+    // the caller checked organize_smem_bytes() against the device limit when it chose `order`
+    const size_t smem = organize_smem_bytes(g, order, split_pmax);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(organize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    const int grid = (order == BSA_ORDER_GLOBAL_LPT) ? 1 : g.H;
+    organize_kernel<<<grid, 1024, smem, stream>>>(g, order, tile_begin, tile_cnt, row_parts, head_counts, items_tmp,
+                                                   items, split_rows, counters);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace bsa
