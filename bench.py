@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Benchmark of the dynamic block-sparse attention request path on B200.
+
+A *step* is one complete request through the C ABI: ``bsa_plan_create`` (mask
+state, statistics copy, regime lookup, launch preparation) followed by
+``bsa_forward`` (attention kernel + Split-K merge) on synthetic vDiT-shaped
+inputs already resident in HBM.  ``value`` is the effective TFLOP/s over the
+active token pairs (4*d flops per pair) of that whole step; the forward-only
+("kernel") figure, the request breakdown and the roofline of the attention
+kernel ride along in the same JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mid|hunyuan|...]
+    python bench.py --impl reference   # the fp64 CPU oracle on a bounded sample
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch on the bench workload,
+# from the ncu capture summarised under profiles/ (None until a capture exists for the workload)
+NCU_TRAFFIC_BYTES = {"mid": None}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def make_request(workload: str, rank: int):
+    from paper_2609_25869_b200 import inputs as I
+    if workload.startswith("sweep"):
+        req = I.config_sweep(int(workload[5:] or 0) + 50 * rank)
+    else:
+        req = I.CONFIGS[workload]()
+    if rank:
+        req.qkv_seed += 7919 * rank
+    return req
+
+
+def count_active_pairs(req) -> int:
+    """In-range token pairs of E(M): the work the metric counts (4*d flops each)."""
+    import numpy as np
+    rq = np.minimum(req.B_Q, req.N - np.arange(req.nQb) * req.B_Q).astype(np.int64)
+    ck = np.minimum(req.B_KV, req.N - np.arange(req.nKb) * req.B_KV).astype(np.int64)
+    return int(np.einsum("hij,i,j->", (req.mask != 0).astype(np.int64), rq, ck))
+
+
+def oracle_sample(req, qkv, nblocks: int, seed: int = 123):
+    """Time the CPU oracle as it stands on a bounded sample of query blocks."""
+    from oracle import oracle
+    from paper_2609_25869_b200 import inputs as I
+    import numpy as np
+    Qb, Kb, Vb = (I.bf16_bits(t) for t in qkv)
+    per_head = max(1, nblocks // req.H)
+    smp = I.sample_query_blocks(seed, req.H, req.nQb, per_head)
+    sel = [(h, int(b)) for h in range(req.H) for b in smp[h]]
+    t0 = time.perf_counter()
+    _, _, pairs = oracle.attention_blocks(req.mask, req.B_Q, req.B_KV, req.N, req.d, Qb, Kb, Vb, sel)
+    dt = time.perf_counter() - t0
+    return pairs, dt, len(sel), oracle.num_threads()
+
+
+def run_reference(args):
+    """--impl reference: the oracle, unmodified, on host cores; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import oracle
+    req = make_request(args.workload, 0)
+    qkv = req.qkv()
+    nblocks = args.ref_blocks
+    oracle_sample(req, qkv, min(nblocks, 8))  # builds/loads the library
+    for _ in range(args.warmup):
+        oracle_sample(req, qkv, nblocks)
+    times, pairs = [], 0
+    for _ in range(args.steps):
+        pairs, dt, nsel, thr = oracle_sample(req, qkv, nblocks)
+        times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    val = 4.0 * req.d * pairs / (ms * 1e-3) / 1e12
+    line = {
+        "impl": "reference", "metric": "effective TFLOP/s on active blocks (4*d flops per active token pair)",
+        "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(req, args.workload),
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": thr, "kind": "oracle",
+                         "sample": f"{nsel} of {req.H * req.nQb} query blocks per step ({pairs} active pairs)"},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(req, name):
+    return {"workload": f"{name}: heads={req.H} N={req.N} d={req.d} B=({req.B_Q},{req.B_KV}) {req.note}",
+            "l2": "256 MiB buffer written between timed iterations (L2 flush)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", default="mid")
+    ap.add_argument("--plan", type=int, default=-1, help="force a catalog plan id (-1: Algorithm 2)")
+    ap.add_argument("--lut", default=os.path.join(ROOT, "paper_2609_25869_b200", "plan_table_b200.lut"))
+    ap.add_argument("--ref-blocks", type=int, default=256, help="query blocks per reference step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--extra", default="", help="comma list of extra workloads reported under 'others'")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2609_25869_b200 import bsa
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    bsa.lib()  # fail loudly if the CUDA library is missing
+    if os.path.exists(args.lut):
+        bsa.lut_load(args.lut)
+    peaks = load_peaks()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def bench_workload(name, steps, warmup, with_e2e):
+        req = make_request(name, rank)
+        q, k, v = req.qkv()
+        mask_d = torch.from_numpy(req.mask).cuda()
+        qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+        O = torch.empty_like(qd)
+        LSE = torch.empty((req.H, req.N), dtype=torch.float32, device="cuda")
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        stream = torch.cuda.current_stream()
+        pairs = count_active_pairs(req)
+        flops = 4.0 * req.d * pairs
+
+        def step():
+            plan = bsa.plan_create(mask_d, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=args.plan)
+            plan.forward(qd, kd, vd, O, LSE)
+            return plan
+
+        for _ in range(warmup):
+            step().destroy()
+        barrier()
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        launches0 = bsa.kernel_launch_count()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        host_us = []
+        plans = []
+        for i in range(steps):
+            flush.fill_(i & 0xFF)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            ev[i][0].record(stream)
+            plans.append(step())
+            ev[i][1].record(stream)
+            ev[i][1].synchronize()
+            host_us.append((time.perf_counter() - t0) * 1e6)
+        barrier()
+        launches = bsa.kernel_launch_count() - launches0
+        step_ms = [a.elapsed_time(b) for a, b in ev]
+        info = plans[-1].info()
+        for p in plans[:-1]:
+            p.destroy()
+        plan = plans[-1]
+        # forward only (warm plan): the attention kernel (+ merge) timed alone, L2 flushed in between
+        kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for _ in range(3):
+            plan.forward(qd, kd, vd, O, LSE)
+        for i in range(steps):
+            flush.fill_(i & 0xFF)
+            kev[i][0].record(stream)
+            plan.forward(qd, kd, vd, O, LSE)
+            kev[i][1].record(stream)
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        k_ms = [a.elapsed_time(b) for a, b in kev]
+        info2 = plan.info()
+        assert info2["device_status"] == 0, "a bounded device wait expired during the bench"
+        plan.destroy()
+        res = {"req": req, "pairs": pairs, "flops": flops, "step_ms": sum(step_ms) / len(step_ms),
+               "step_ms_median": statistics.median(step_ms), "host_us": statistics.median(host_us),
+               "kernel_ms": sum(k_ms) / len(k_ms), "kernel_ms_median": statistics.median(k_ms), "info": info,
+               "launches": launches, "clocks": clocks, "qkv": (q, k, v)}
+        if with_e2e:
+            qp, kp, vp = q.pin_memory(), k.pin_memory(), v.pin_memory()
+            Oh = torch.empty_like(q).pin_memory()
+            Lh = torch.empty((req.H, req.N), dtype=torch.float32).pin_memory()
+            mh = torch.from_numpy(req.mask).pin_memory()
+            for _ in range(2):
+                bsa.request_host(mh, req.B_Q, req.B_KV, req.N, req.H, req.d, qp, kp, vp, Oh, Lh, plan_id=args.plan)
+            ts = []
+            for _ in range(max(3, steps // 2)):
+                barrier()
+                t0 = time.perf_counter()
+                bsa.request_host(mh, req.B_Q, req.B_KV, req.N, req.H, req.d, qp, kp, vp, Oh, Lh, plan_id=args.plan)
+                ts.append(time.perf_counter() - t0)
+            res["e2e_s"] = sum(ts) / len(ts)
+            res["h2d"] = req.mask.nbytes + 3 * q.numel() * 2
+            res["d2h"] = q.numel() * 2 + req.H * req.N * 4
+        return res
+
+    r = bench_workload(args.workload, args.steps, args.warmup, True)
+    req = r["req"]
+
+    def maxr(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    step_ms = maxr(r["step_ms"])
+    kernel_ms = maxr(r["kernel_ms"])
+    e2e_s = maxr(r["e2e_s"])
+    value = world * r["flops"] / (step_ms * 1e-3) / 1e12
+    kernel_tflops = r["flops"] / (kernel_ms * 1e-3) / 1e12
+    inf = r["info"]
+    line = {
+        "metric": "effective TFLOP/s on active blocks (4*d flops per active token pair), whole request: "
+                  "plan create + forward",
+        "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic", "config": workload_config(req, args.workload),
+        "clocks": r["clocks"],
+        "e2e": {"value": world * r["flops"] / e2e_s / 1e12, "unit": "TFLOP/s",
+                "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"], "ms_per_request": e2e_s * 1e3},
+        "gpu_launches": r["launches"],
+        "roofline": {"bound": "tensor", "kernel": "bsa_attention_kernel", "achieved": kernel_tflops,
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": kernel_tflops / peaks["bf16_tflops"],
+                     "frac_of_sustained": kernel_tflops / peaks["bf16_tflops_sustained"],
+                     "peak_source": peaks["_source"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                     "launch_ms": kernel_ms, "flops_per_launch": r["flops"]},
+        "request": {"us_per_request_gpu": step_ms * 1e3, "us_per_request_host_median": r["host_us"],
+                    "us_forward": kernel_ms * 1e3, "us_plan_create_host": inf["us_total"],
+                    "us_mask_state": inf["us_mask_state"], "us_stats_sync": inf["us_stats_sync"],
+                    "us_lookup": inf["us_lookup"], "us_launch_prep": inf["us_launch_prep"],
+                    "planning_fraction": max(0.0, 1.0 - kernel_ms / step_ms),
+                    "plan": inf["plan"]["name"], "lut_hit": inf["lut_hit"], "ntiles": inf["ntiles"],
+                    "nitems": inf["nitems"], "active_pairs": r["pairs"], "covered_pairs": inf["covered_pairs"],
+                    "density": inf["density"]},
+    }
+    others = {}
+    for name in [x for x in args.extra.split(",") if x]:
+        o = bench_workload(name, max(3, args.steps // 4), 3, False)
+        others[name] = {"kernel_tflops": o["flops"] / (o["kernel_ms"] * 1e-3) / 1e12, "kernel_ms": o["kernel_ms"],
+                        "request_ms": o["step_ms"], "frac_of_peak": o["flops"] / (o["kernel_ms"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                        "plan": o["info"]["plan"]["name"], "us_plan_create_host": o["info"]["us_total"]}
+    if others:
+        line["others"] = others
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        pairs, dt, nsel, thr = oracle_sample(req, r["qkv"], req.H * req.nQb if args.workload in ("tiny", "mid") else 512)
+        line["cpu_baseline"] = {"value": 4.0 * req.d * pairs / dt / 1e12, "unit": "TFLOP/s", "cores": thr,
+                                "kind": "oracle", "seconds": dt,
+                                "sample": f"{nsel} of {req.H * req.nQb} query blocks ({pairs} active pairs)"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

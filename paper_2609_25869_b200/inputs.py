@@ -170,7 +170,7 @@ def config_hunyuan(seed: int = 2, H: int = 24) -> Request:
 def _runs_row(nKb: int, target: int, seed: int, h: int, i: int) -> np.ndarray:
     """One row of the clustered mask: R ~ U{4..12} runs, lengths ~ Geom(0.3)
     rescaled to sum to ``target``, placed with at least one gap between runs."""
-    R = 4 + int(hash_u32(seed, 10, h, i)) % 9
+    R = min(4 + int(hash_u32(seed, 10, h, i)) % 9, max(1, target), max(1, (nKb - target + 1)))
     u = uniform01(seed, 11, np.full(R, h), np.full(R, i), np.arange(R))
     lens = np.floor(np.log(u) / np.log(0.7)).astype(np.int64) + 1  # geometric(p=0.3), support >= 1
     # rescale to the density target, keeping every run >= 1

@@ -1,0 +1,173 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element, on the
+same seeded inputs; the tile plan's coverage against E(M), bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_25869_b200 import bsa
+from paper_2609_25869_b200 import inputs as I
+from tests import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+
+def _sample(req, per_head, seed=77, heads=None):
+    smp = I.sample_query_blocks(seed, req.H, req.nQb, per_head)
+    hs = range(req.H) if heads is None else heads
+    return [(h, int(b)) for h in hs for b in smp[h]]
+
+
+# ---------------------------------------------------------------- the five configurations
+@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9])
+def test_tiny_full_oracle_every_plan(plan_id):
+    res = Hh.run_request(I.config_tiny(), plan_id=plan_id)
+    assert res["pairs"] == res["info"]["nnz_blocks"] * 64 * 64
+
+
+@pytest.mark.parametrize("plan_id", [0, 1, 2])
+def test_mid_full_oracle(plan_id):
+    Hh.run_request(I.config_mid(), plan_id=plan_id)
+
+
+def test_hunyuan_shaped_sampled_oracle():
+    req = I.config_hunyuan()
+    # 64 seeded query blocks per head; structure (coverage, CSR, items) on three heads to bound host time
+    Hh.run_request(req, plan_id=-1, sel=_sample(req, 64), heads=[0, 11, 23])
+
+
+@pytest.mark.parametrize("plan_id", [0, 1])
+def test_stress_a_coarsened(plan_id):
+    req = I.config_stress_a()
+    res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64), heads=[0, 15])
+    assert res["info"]["map_q"] == 1  # Coarsened along Q: 8 logical rows of 16 per 128-row tile
+
+
+@pytest.mark.parametrize("plan_id", [0, 1])
+def test_stress_b_refined(plan_id):
+    req = I.config_stress_b()
+    res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64))
+    assert res["info"]["map_q"] == 2 and res["info"]["map_kv"] == 2  # Refined in both dimensions
+
+
+@pytest.mark.parametrize("r,B,rho", [(0, (32, 32), 0.03), (1, (64, 128), 0.10), (2, (128, 64), 0.30),
+                                     (3, (256, 256), 0.60), (4, (128, 128), 0.03)])
+def test_sweep_requests_ragged_n(r, B, rho):
+    # N = 75600 is not a multiple of any block size; 6 heads keep the host-side mask generation short
+    req = I.config_sweep(r, H=6, B=B, rho=rho)
+    Hh.run_request(req, plan_id=-1, sel=_sample(req, 8), row_step=4, heads=[0, 5])
+
+
+# ---------------------------------------------------------------- small geometries spanning tiles + ragged tails
+@pytest.mark.parametrize("B_Q,B_KV,N,d,plan_id", [
+    (16, 16, 1000, 64, 0), (16, 16, 1000, 64, 1), (32, 64, 777, 128, 0), (64, 32, 1300, 128, 1),
+    (128, 256, 2100, 64, 0), (256, 128, 2100, 128, 1), (256, 16, 900, 64, 3), (16, 256, 900, 128, 2),
+    (64, 64, 130, 64, 0), (128, 128, 127, 128, 0), (128, 128, 1, 64, 1),
+])
+def test_geometries_with_ragged_tail(B_Q, B_KV, N, d, plan_id):
+    H = 3
+    M = I.random_mask(B_Q * 131 + B_KV + N, H, I.cdiv(N, B_Q), I.cdiv(N, B_KV), 0.35, diag=True, empty_rows=0.15)
+    req = I.Request("geom", H, N, d, B_Q, B_KV, M, qkv_seed=N + d)
+    Hh.run_request(req, plan_id=plan_id)
+
+
+# ---------------------------------------------------------------- degenerate masks
+@pytest.mark.parametrize("kind", ["empty", "full", "one_block", "empty_head"])
+def test_degenerate_masks(kind):
+    H, N, d, B = 2, 512, 64, 64
+    nb = N // B
+    M = np.zeros((H, nb, nb), np.uint8)
+    if kind == "full":
+        M[:] = 1
+    elif kind == "one_block":
+        M[1, 3, 5] = 1
+    elif kind == "empty_head":
+        M[0] = I.random_mask(1, 1, nb, nb, 0.5)[0]
+    req = I.Request(kind, H, N, d, B, B, M, qkv_seed=3)
+    for plan_id in (0, 3):
+        Hh.run_request(req, plan_id=plan_id)
+
+
+# ---------------------------------------------------------------- closed forms on the GPU path
+@pytest.mark.parametrize("B_Q,B_KV,N,d,plan_id", [(16, 64, 1000, 64, 0), (32, 32, 700, 128, 1), (256, 256, 1100, 128, 9)])
+def test_zero_keys_give_log_count_and_mean_value(B_Q, B_KV, N, d, plan_id):
+    """K = 0: every score is 0, so LSE = ln(#reachable keys) exactly and O = mean of reachable V.
+    Catches any off-by-one in ragged-edge or membership masking (one key off moves LSE by ~1/count)."""
+    H = 2
+    M = I.random_mask(5, H, I.cdiv(N, B_Q), I.cdiv(N, B_KV), 0.3, diag=True, empty_rows=0.1)
+    q, k, v = I.make_qkv(1, H, N, d)
+    mask = torch.from_numpy(M).cuda()
+    with bsa.plan_create(mask, B_Q, B_KV, N, H, d, plan_id=plan_id) as plan:
+        O, LSE = plan.forward(q.cuda(), torch.zeros_like(k).cuda(), v.cuda())
+        torch.cuda.synchronize()
+    ck = np.minimum(B_KV, N - np.arange(M.shape[2]) * B_KV)
+    cnt = np.repeat((M * ck[None, None, :]).sum(axis=2), B_Q, axis=1)[:, :N]
+    LSE = LSE.cpu().numpy()
+    nz = cnt > 0
+    assert np.array_equal(np.isneginf(LSE), ~nz)
+    np.testing.assert_allclose(LSE[nz], np.log(cnt[nz]), atol=2e-6, rtol=0)
+    # O = mean of the reachable values (bf16 output rounding only)
+    E = np.repeat(np.repeat(M[0] != 0, B_Q, axis=0), B_KV, axis=1)[:N, :N]
+    v64 = v[0].double().numpy()
+    mean = (E @ v64) / np.maximum(cnt[0], 1)[:, None]
+    np.testing.assert_allclose(O[0].float().cpu().numpy()[nz[0]], mean[nz[0]], atol=4e-3, rtol=0)
+
+
+def test_constant_values_come_back():
+    H, N, d = 2, 900, 128
+    M = I.random_mask(8, H, I.cdiv(N, 64), I.cdiv(N, 32), 0.4, diag=True)
+    q, k, v = I.make_qkv(2, H, N, d)
+    vc = torch.full_like(v, 0.75)
+    with bsa.plan_create(torch.from_numpy(M).cuda(), 64, 32, N, H, d, plan_id=0) as plan:
+        O, _ = plan.forward(q.cuda(), k.cuda(), vc.cuda())
+        torch.cuda.synchronize()
+    assert torch.allclose(O.float(), torch.full_like(O.float(), 0.75), atol=4e-3)
+
+
+def test_sharp_scores_stay_within_tolerance():
+    # 4x larger scores: a much peakier softmax, more rescaling of the running output
+    req = I.config_tiny(seed=21)
+    q, k, v = req.qkv()
+    res = Hh.run_request(req, plan_id=1, qkv=((q * 2).to(torch.bfloat16), (k * 2).to(torch.bfloat16), v), guards=False)
+    assert res["lse_max"] < 2e-4
+
+
+# ---------------------------------------------------------------- boundary behaviour
+def test_invalid_arguments_never_touch_the_gpu():
+    import ctypes
+    L = bsa.lib()
+    h = ctypes.c_void_p()
+    m = torch.zeros((1, 2, 2), dtype=torch.uint8, device="cuda")
+    assert L.bsa_plan_create(None, 64, 64, 128, 1, 64, ctypes.byref(h)) == 1
+    assert L.bsa_plan_create(m.data_ptr(), 64, 64, 0, 1, 64, ctypes.byref(h)) == 1
+    assert L.bsa_plan_create(m.data_ptr(), 48, 64, 128, 1, 64, ctypes.byref(h)) == 2
+    assert L.bsa_plan_create(m.data_ptr(), 64, 64, 128, 1, 96, ctypes.byref(h)) == 2
+    assert L.bsa_plan_create(m.data_ptr(), 64, 512, 128, 1, 64, ctypes.byref(h)) == 2
+    with pytest.raises(bsa.BsaError) as e:
+        bsa.plan_create(m, 64, 64, 128, 1, 64, plan_id=2, max_workspace_bytes=1024)  # workspace too small
+    assert e.value.status == 3
+    with bsa.plan_create(m, 64, 64, 128, 1, 64) as plan:
+        q = torch.zeros((1, 128, 64), dtype=torch.bfloat16, device="cuda")
+        assert L.bsa_forward(plan._h, q.data_ptr() + 2, q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None) == 1
+        assert L.bsa_forward(plan._h, None, q.data_ptr(), q.data_ptr(), q.data_ptr(), q.data_ptr(), None) == 1
+
+
+def test_request_from_host_buffers_matches_device_path():
+    req = I.config_tiny(seed=4, N=1536)
+    q, k, v = req.qkv()
+    O = torch.empty_like(q)
+    LSE = torch.empty((req.H, req.N), dtype=torch.float32)
+    inf = bsa.request_host(req.mask, req.B_Q, req.B_KV, req.N, req.H, req.d, q, k, v, O, LSE)
+    assert inf["device_status"] == 0
+    Hh.compare_with_oracle(req, O, LSE, (q, k, v))
+
+
+def test_launch_counter_counts_our_kernels():
+    req = I.config_tiny()
+    mask, q, k, v, _ = Hh.to_dev(req)
+    n0 = bsa.kernel_launch_count()
+    with bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=2) as plan:
+        n1 = bsa.kernel_launch_count()
+        plan.forward(q, k, v)
+        n2 = bsa.kernel_launch_count()
+    assert n1 - n0 == 5   # row stats, row scan, CSR fill, tile map, organise
+    assert n2 - n1 == 2   # attention + Split-K merge

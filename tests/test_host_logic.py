@@ -1,0 +1,133 @@
+"""CPU-only tests: the C-ABI library loads and exports what include/bsa.h declares, the catalog and
+eligibility rules, and the plan-table lookup (Algorithm 2) against the oracle's restatement of it."""
+import os
+import re
+import subprocess
+
+import pytest
+
+from oracle import oracle
+from paper_2609_25869_b200 import bsa
+from paper_2609_25869_b200 import build as bsa_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    bsa_build.build()
+    bsa.lut_clear()
+    yield
+    bsa.lut_clear()
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "bsa.h")).read()
+    declared = set(re.findall(r"BSA_API\s+[\w\s\*]+?\b(bsa_\w+)\s*\(", hdr))
+    assert {"bsa_plan_create", "bsa_forward", "bsa_plan_destroy"} <= declared and len(declared) >= 20
+    out = subprocess.check_output(["nm", "-D", "--defined-only", bsa.LIB_PATH], text=True)
+    exported = set(l.split()[-1] for l in out.splitlines() if " T " in l)
+    assert declared <= exported, declared - exported
+    assert all(s.startswith("bsa_") for s in exported), "only the C ABI is exported"
+    L = bsa.lib()
+    for name in declared:
+        assert hasattr(L, name)
+
+
+def test_catalog_and_eligibility():
+    cat = bsa.catalog()
+    assert len(cat) >= 6 and [c["plan_id"] for c in cat] == list(range(len(cat)))
+    assert len(set(c["name"] for c in cat)) == len(cat)
+    assert {c["T_KV"] for c in cat} == {64, 128} and all(c["T_Q"] == 128 for c in cat)
+    base = bsa.lib().bsa_base_plan(128, 128, 128)
+    # the base plan is eligible for every supported request key
+    for B_Q in (16, 32, 64, 128, 256):
+        for B_KV in (16, 32, 64, 128, 256):
+            for d in (64, 128):
+                assert bsa.plan_eligible(base, B_Q, B_KV, 75600, 24, d)
+    assert not bsa.plan_eligible(base, 8, 64, 1024, 1, 64)       # block size below 16
+    assert not bsa.plan_eligible(base, 64, 64, 1024, 1, 96)      # head dim outside the catalog
+    assert not bsa.plan_eligible(len(cat), 64, 64, 1024, 1, 64)  # unknown plan
+    split = next(c for c in cat if c["split_pmax"] > 1)
+    assert bsa.plan_eligible(split["plan_id"], 64, 64, 2048, 2, 64)
+    assert not bsa.plan_eligible(split["plan_id"], 64, 64, 2048, 2, 64, max_workspace_bytes=4096)  # workspace
+    assert not bsa.plan_eligible(split["plan_id"], 128, 128, 115200, 24, 128)  # default workspace limit
+
+
+def test_feature_schema_buckets():
+    assert bsa.lut_buckets(16384, 0.15, 1.5, 0.8) == [14, 4, 1, 1]
+    assert bsa.lut_buckets(16383, 0.0199, 1.49, 0.49) == [13, 0, 0, 0]
+    assert bsa.lut_buckets(115200, 0.9, 100.0, 1.0) == [16, 6, 3, 1]
+
+
+def _write_lut(path, regimes, catalog_hash=None, version=1):
+    h = bsa.lib().bsa_catalog_hash() if catalog_hash is None else catalog_hash
+    with open(path, "w") as f:
+        f.write(f"BSA_LUT {version}\ncatalog {h:x}\ngpu test\n")
+        for key, ids in regimes.items():
+            f.write("regime " + " ".join(str(x) for x in key) + " : " + " ".join(str(i) for i in ids) + "\n")
+
+
+def test_plan_table_lookup_matches_algorithm_2(tmp_path):
+    # regime key: B_Q B_KV d floor(log2 N) head-bucket density-bucket skew-bucket runcov-bucket
+    regimes = {
+        (64, 64, 64, 11, 0, 5, 1, 0): [3, 1, 0],
+        (128, 128, 128, 16, 2, 2, 0, 1): [2, 1, 0],   # plan 2 needs a workspace this request cannot bind
+    }
+    p = str(tmp_path / "t.lut")
+    _write_lut(p, regimes)
+    bsa.lut_load(p)
+    assert bsa.lib().bsa_lut_num_regimes() == 2
+    base = {("k64",): 0}
+    # hit: first eligible plan of the ranking
+    pid, hit = bsa.lut_select(64, 64, 2048, 2, 64, 0.27, 0.4, 1.6)
+    assert (pid, hit) == (3, True)
+    assert pid == oracle.select_plan({(("k64",), "b"): [3, 1, 0]}, base, ("k64",), "b", lambda q: True)
+    # ranked fallback: plan 2 is not eligible (workspace over the default limit) -> next in rank order
+    pid, hit = bsa.lut_select(128, 128, 115200, 24, 128, 0.066, 0.9, 1.2)
+    assert (pid, hit) == (1, True)
+    assert pid == oracle.select_plan({(("k",), "b"): [2, 1, 0]}, {("k",): 0}, ("k",), "b", lambda q: q != 2)
+    # miss: the base plan alone
+    pid, hit = bsa.lut_select(64, 64, 2048, 2, 64, 0.01, 0.4, 1.6)
+    assert (pid, hit) == (0, False)
+    assert pid == oracle.select_plan({}, base, ("k64",), "other", lambda q: True)
+    # nothing eligible -> no-eligible-plan
+    pid, hit = bsa.lut_select(64, 64, 2048, 2, 96, 0.27, 0.4, 1.6)
+    assert pid == -1
+    assert oracle.select_plan({}, base, ("k64",), "other", lambda q: False) is None
+    bsa.lut_clear()
+    assert bsa.lut_select(64, 64, 2048, 2, 64, 0.27, 0.4, 1.6) == (0, False)
+
+
+def test_plan_table_rejects_foreign_or_malformed_files(tmp_path):
+    good = {(64, 64, 64, 11, 0, 5, 1, 0): [1, 0]}
+    p = str(tmp_path / "bad.lut")
+    _write_lut(p, good, catalog_hash=0x1234)          # built for another catalog
+    with pytest.raises(bsa.BsaError) as e:
+        bsa.lut_load(p)
+    assert e.value.status == 7 and bsa.lib().bsa_lut_num_regimes() == 0
+    _write_lut(p, good, version=2)                    # unknown version
+    with pytest.raises(bsa.BsaError):
+        bsa.lut_load(p)
+    _write_lut(p, {(64, 64, 64, 11, 0, 5, 1, 0): [999]})  # unknown plan id
+    with pytest.raises(bsa.BsaError):
+        bsa.lut_load(p)
+    with pytest.raises(bsa.BsaError):
+        bsa.lut_load(str(tmp_path / "missing.lut"))
+    _write_lut(p, good)
+    bsa.lut_load(p)
+    assert bsa.lib().bsa_lut_num_regimes() == 1
+    bsa.lut_clear()
+
+
+def test_status_strings_and_version():
+    L = bsa.lib()
+    assert L.bsa_status_string(0) == b"ok" and L.bsa_status_string(3) == b"no eligible plan"
+    assert b"sm_100a" in L.bsa_version()
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(bsa, "_lib", None)
+    monkeypatch.setattr(bsa, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        bsa.lib()
