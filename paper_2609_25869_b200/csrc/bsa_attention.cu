@@ -55,6 +55,61 @@ struct __align__(8) Barriers {
     uint64_t s_full[2], p_ready[2], pv_done[2];
 };
 
+// One score tile of one query row (thread = row = TMEM lane): mask, running reference maximum,
+// P = exp2(s * c2 - m_ref) rounded to bf16 and written over S in place, running sum.
+// The reference maximum moves only when the tile maximum exceeds it by kRescaleThreshold (log2
+// units), so P stays below 2^8 and the running output needs rescaling (by `alpha`) only then.
+template <int TK>
+__device__ __forceinline__ void softmax_tile(uint32_t t_s, bool need_mask, uint32_t row_bits, int lgBKV, int n_valid,
+                                             float c2, bool not_first, float& m_ref, float& l, float& alpha,
+                                             bool& rescale) {
+    uint32_t r[TK];
+#pragma unroll
+    for (int c = 0; c < TK / 32; ++c) tmem_ld32(t_s + c * 32, &r[c * 32]);
+    tc_wait_ld();
+    if (need_mask) {
+#pragma unroll
+        for (int i = 0; i < TK; ++i) {
+            const bool act = ((row_bits >> (i >> lgBKV)) & 1u) && (i < n_valid);
+            r[i] = act ? r[i] : 0xff800000u;  // -inf
+        }
+    }
+    float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < TK; i += 4) {
+        m0 = fmaxf(m0, __uint_as_float(r[i]));
+        m1 = fmaxf(m1, __uint_as_float(r[i + 1]));
+        m2 = fmaxf(m2, __uint_as_float(r[i + 2]));
+        m3 = fmaxf(m3, __uint_as_float(r[i + 3]));
+    }
+    const float mx2 = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c2;
+    alpha = 1.f;
+    rescale = false;
+    if (mx2 > m_ref + kRescaleThreshold) {
+        alpha = ex2_approx(m_ref - mx2);  // m_ref = -inf -> 0
+        rescale = not_first && (m_ref != -INFINITY);
+        m_ref = mx2;
+    }
+    const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+    for (int i = 0; i < TK; i += 4) {
+        const float p0 = ex2_approx(fmaf(__uint_as_float(r[i]), c2, neg_m));
+        const float p1 = ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, neg_m));
+        const float p2 = ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, neg_m));
+        const float p3 = ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, neg_m));
+        s0 += p0;
+        s1 += p1;
+        s2 += p2;
+        s3 += p3;
+        r[i / 2] = pack_bf16x2(p0, p1);
+        r[i / 2 + 1] = pack_bf16x2(p2, p3);
+    }
+#pragma unroll
+    for (int c = 0; c < TK / 32; ++c) tmem_st16(t_s + c * 16, &r[c * 16]);
+    l = l * alpha + ((s0 + s1) + (s2 + s3));
+}
+
 template <int D, int TK>
 __global__ void __launch_bounds__(kThreads, 1)
 bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -243,61 +298,9 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t t_s = tmem + lane_base + (sb ? kColS1 : kColS0);
-                // ---- pass 1: row maximum over the tile ----
-                float mx = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < TK / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(t_s + c * 32, r);
-                    tc_wait_ld();
-                    if (need_mask) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int col = c * 32 + i;
-                            const bool act = ((row_bits >> (col >> p.lgBKV)) & 1u) && (col < n_valid);
-                            mx = fmaxf(mx, act ? __uint_as_float(r[i]) : -INFINITY);
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
-                    }
-                }
-                // ---- reference maximum: move it only when the tile maximum exceeds it by the threshold ----
-                const float mx2 = mx * c2;
-                float alpha = 1.f;
-                bool rescale = false;
-                if (mx2 > m_ref + kRescaleThreshold) {
-                    alpha = ex2_approx(m_ref - mx2);  // m_ref = -inf -> 0
-                    rescale = (j > 0) && (m_ref != -INFINITY);
-                    m_ref = mx2;
-                }
-                const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-                // ---- pass 2: P = exp2(s * c2 - m), bf16, written over S in place ----
-                float rowsum = 0.f;
-#pragma unroll
-                for (int c = 0; c < TK / 32; ++c) {
-                    uint32_t r[32];
-                    uint32_t pk[16];
-                    tmem_ld32(t_s + c * 32, r);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float s0 = __uint_as_float(r[i]), s1 = __uint_as_float(r[i + 1]);
-                        if (need_mask) {
-                            const int col = c * 32 + i;
-                            const bool a0 = ((row_bits >> (col >> p.lgBKV)) & 1u) && (col < n_valid);
-                            const bool a1 = ((row_bits >> ((col + 1) >> p.lgBKV)) & 1u) && (col + 1 < n_valid);
-                            s0 = a0 ? s0 : -INFINITY;
-                            s1 = a1 ? s1 : -INFINITY;
-                        }
-                        const float p0 = ex2_approx(fmaf(s0, c2, -m_use));
-                        const float p1 = ex2_approx(fmaf(s1, c2, -m_use));
-                        rowsum += p0 + p1;
-                        pk[i >> 1] = pack_bf16x2(p0, p1);
-                    }
-                    tmem_st16(t_s + c * 16, pk);
-                }
-                l = l * alpha + rowsum;
+                float alpha;
+                bool rescale;
+                softmax_tile<TK>(t_s, need_mask, row_bits, p.lgBKV, n_valid, c2, j > 0, m_ref, l, alpha, rescale);
                 // ---- correction: rescale the running output when the reference moved ----
                 if (j > 0 && __any_sync(0xffffffffu, rescale)) {
                     const uint32_t gp = gs - 1;
