@@ -73,17 +73,17 @@ typedef struct bsa_plan_info {
     int32_t heads, d, B_Q, B_KV;
     int64_t N;
     int32_t nQb, nKb, nQt, nKt;   /* logical block grid and physical tile grid per head              */
-    int32_t member_bits;          /* membership bits per tile (1 = no intra-tile mask needed)        */
+    int32_t member_bits;          /* membership bits per 128-row slot (1 = no intra-tile mask needed) */
     int32_t lut_hit;              /* 1: regime found in the plan table; 0: base plan used            */
     int32_t regime_bucket[4];     /* N, density, skew, run-coverage bucket indices used for lookup   */
     int64_t nnz_blocks;           /* active logical blocks                                           */
     int64_t blocks_in_runs;       /* active blocks in runs of length >= 2                            */
     int32_t max_row_nnz;
-    int32_t reserved0;
+    int32_t member_words;         /* 64-bit membership words per tile: one per 128-row slot (T_Q / 128) */
     double density, run_coverage, skew;
     int64_t ntiles;               /* physical tiles                                                  */
     int64_t nitems;               /* work items (Q tile rows x KV partitions)                        */
-    int64_t nsplit_rows;          /* Q tile rows with more than one partition                        */
+    int64_t nsplit_rows;          /* 128-row tile rows merged by the Split-K reduction kernel        */
     int64_t workspace_bytes;      /* Split-K workspace owned by the plan                             */
     int64_t covered_pairs;        /* token pairs the tiles compute, incl. masked-out ones            */
     /* host wall time of bsa_plan_create, microseconds */
@@ -169,9 +169,10 @@ BSA_API bsa_status_t bsa_plan_export_csr(const bsa_plan_t* plan, int32_t* row_pt
 /* Physical tiles of one head, for the coverage check (a plan must preserve E(M), Section 2.2):
  *   tile_row_ptr_host int32 [nQt + 1]  offsets into the two arrays below (relative to this head),
  *   tile_col_host     int32 [cap]      KV tile index, ascending and unique inside a row,
- *   tile_member_host  uint64 [cap]     membership bits: bit (a * sK + b) set iff logical sub-block
- *                                      (a, b) of the tile is active, sK = max(1, T_KV / B_KV),
- *                                      a < max(1, T_Q / B_Q), b < sK.
+ *   tile_member_host  uint64 [cap * W] membership words, W = T_Q / 128 per tile (info.member_words), one
+ *                                      per 128-row slot of the tile: bit (a * sK + b) of word s set iff
+ *                                      logical sub-block (a, b) of slot s is active, sK = max(1, T_KV / B_KV),
+ *                                      a < max(1, 128 / B_Q), b < sK.  A zero word: the slot skips the tile.
  * `cap` is the capacity of the two arrays in entries; *ntiles_out receives the number needed
  * (call with cap = 0 and NULL arrays to size them). */
 BSA_API bsa_status_t bsa_plan_export_tiles(const bsa_plan_t* plan, int head, int32_t* tile_row_ptr_host,

@@ -40,7 +40,7 @@ class PlanInfo(ctypes.Structure):
                 ("nQb", ctypes.c_int32), ("nKb", ctypes.c_int32), ("nQt", ctypes.c_int32), ("nKt", ctypes.c_int32),
                 ("member_bits", ctypes.c_int32), ("lut_hit", ctypes.c_int32), ("regime_bucket", ctypes.c_int32 * 4),
                 ("nnz_blocks", ctypes.c_int64), ("blocks_in_runs", ctypes.c_int64),
-                ("max_row_nnz", ctypes.c_int32), ("reserved0", ctypes.c_int32),
+                ("max_row_nnz", ctypes.c_int32), ("member_words", ctypes.c_int32),
                 ("density", ctypes.c_double), ("run_coverage", ctypes.c_double), ("skew", ctypes.c_double),
                 ("ntiles", ctypes.c_int64), ("nitems", ctypes.c_int64), ("nsplit_rows", ctypes.c_int64),
                 ("workspace_bytes", ctypes.c_int64), ("covered_pairs", ctypes.c_int64),
@@ -154,13 +154,16 @@ class Plan:
         _check(lib().bsa_plan_export_csr(self._h, rp.ctypes.data, ci.ctypes.data), "bsa_plan_export_csr")
         return rp, ci[: inf["nnz_blocks"]]
 
-    def export_tiles(self, head: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    def export_tiles(self, head: int):
+        """Tiles of one head: ``(tile_row_ptr [nQt+1], tile_col [n], tile_member [n, W] uint64)`` with
+        ``W = T_Q / 128`` membership words per tile (one per 128-row slot)."""
         n = ctypes.c_int64(0)
         _check(lib().bsa_plan_export_tiles(self._h, head, None, None, None, 0, ctypes.byref(n)), "export_tiles(size)")
-        nQt = self.info()["nQt"]
+        inf = self.info()
+        nQt, W = inf["nQt"], inf["member_words"]
         rp = np.zeros(nQt + 1, dtype=np.int32)
         tc = np.zeros(max(1, n.value), dtype=np.int32)
-        tm = np.zeros(max(1, n.value), dtype=np.uint64)
+        tm = np.zeros((max(1, n.value), W), dtype=np.uint64)
         _check(lib().bsa_plan_export_tiles(self._h, head, rp.ctypes.data, tc.ctypes.data, tm.ctypes.data,
                                            max(1, n.value), ctypes.byref(n)), "export_tiles")
         return rp, tc[: n.value], tm[: n.value]

@@ -173,7 +173,7 @@ extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int
     if (plan_id < 0) { free_plan(p); return BSA_ERR_NO_ELIGIBLE_PLAN; }
     p->desc = *catalog_entry(plan_id);
     make_geom(p->desc, B_Q, B_KV, N, heads, &p->g);
-    p->stages = p->desc.stages > 0 ? p->desc.stages : attention_max_stages(d, p->desc.T_KV);
+    p->stages = p->desc.stages > 0 ? p->desc.stages : attention_max_stages(d, p->desc.T_KV, p->desc.kernel);
     const double t3 = now_us();
 
     // ---- launch preparation: derive only the selected plan's metadata from the block-CSR ----
@@ -191,10 +191,10 @@ extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int
     const size_t o_tc = take(sizeof(int32_t) * (size_t)trows);
     const size_t o_rp = take(sizeof(int32_t) * (size_t)trows);
     const size_t o_tcol = take(sizeof(int32_t) * (size_t)(p->tile_cap + 1));
-    const size_t o_tmem = take(sizeof(uint64_t) * (size_t)(p->tile_cap + 1));
+    const size_t o_tmem = take(sizeof(uint64_t) * (size_t)(p->tile_cap + 1) * g.slots);
     const size_t o_it0 = take(sizeof(WorkItem) * (size_t)p->max_items);
     const size_t o_it1 = take(sizeof(WorkItem) * (size_t)p->max_items);
-    const size_t o_sr = take(sizeof(SplitRow) * (size_t)(pmax > 1 ? trows : 1));
+    const size_t o_sr = take(sizeof(SplitRow) * (size_t)(pmax > 1 ? trows * g.slots : 1));
     BSA_CUDA(cudaMallocAsync(&p->arena2, o, stream), "arena2");
     p->col_idx = reinterpret_cast<int32_t*>(p->arena2 + o_col);
     p->tile_begin = reinterpret_cast<int32_t*>(p->arena2 + o_tb);
@@ -208,7 +208,7 @@ extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int
     p->ws_bytes = plan_workspace_bytes(p->desc, N, heads, d);
     if (p->ws_bytes > 0) {
         BSA_CUDA(cudaMallocAsync(&p->ws_O, (size_t)p->ws_bytes, stream), "workspace");
-        p->ws_LSE = p->ws_O + (size_t)p->max_items * kTQ * d;
+        p->ws_LSE = p->ws_O + (size_t)p->max_items * g.T_Q * d;
     }
     BSA_CUDA(launch_row_scan(p->row_nnz, nrows, p->row_ptr, stream), "row_scan");
     BSA_CUDA(launch_csr_fill(mask_dev, nrows, nKb, p->row_ptr, p->col_idx, stream), "csr_fill");
@@ -256,7 +256,7 @@ extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const vo
     a.kernel = p->desc.kernel;
     a.has_split = p->desc.split_pmax > 1;
     a.max_items = (int32_t)(p->max_items < (1 << 30) ? p->max_items : (1 << 30));
-    a.max_split_rows = p->g.H * p->g.nQt;
+    a.max_split_rows = p->g.H * p->g.nQt * p->g.slots;
     a.num_sms = p->num_sms;
     const char* detail = "launch";
     cudaError_t e = launch_forward(a, reinterpret_cast<cudaStream_t>(stream_v), &detail);
@@ -295,7 +295,8 @@ extern "C" bsa_status_t bsa_plan_get_info(const bsa_plan_t* p, bsa_plan_info_t* 
     info->map_kv = g.sK > 1 ? BSA_MAP_COARSENED : (g.rk > 1 ? BSA_MAP_REFINED : BSA_MAP_DIRECT);
     info->heads = g.H; info->d = p->d; info->B_Q = g.B_Q; info->B_KV = g.B_KV; info->N = g.N;
     info->nQb = g.nQb; info->nKb = g.nKb; info->nQt = g.nQt; info->nKt = g.nKt;
-    info->member_bits = g.sQ * g.sK;
+    info->member_bits = g.sQ128 * g.sK;
+    info->member_words = g.slots;
     info->lut_hit = p->lut_hit;
     memcpy(info->regime_bucket, p->buckets, sizeof p->buckets);
     info->nnz_blocks = (int64_t)p->hstats.nnz;
@@ -308,9 +309,9 @@ extern "C" bsa_status_t bsa_plan_get_info(const bsa_plan_t* p, bsa_plan_info_t* 
     info->skew = nnz > 0 ? (double)p->hstats.max_row_nnz / (nnz / nrows) : 0.0;
     info->ntiles = (int64_t)c.ntiles;
     info->nitems = c.nitems;
-    info->nsplit_rows = c.nsplit_rows;
+    info->nsplit_rows = c.nsplit_rows;  // physical tile rows with more than one partition
     info->workspace_bytes = p->ws_bytes;
-    info->covered_pairs = (int64_t)c.ntiles * kTQ * g.T_KV;
+    info->covered_pairs = (int64_t)c.nslot_tiles * kTQ * g.T_KV;
     info->us_mask_state = p->us_mask_state;
     info->us_stats_sync = p->us_stats_sync;
     info->us_lookup = p->us_lookup;
@@ -363,8 +364,8 @@ extern "C" bsa_status_t bsa_plan_export_tiles(const bsa_plan_t* p, int head, int
                     e = cudaMemcpy(tile_col_host + off, p->tile_col + tb[t], sizeof(int32_t) * tc[t],
                                    cudaMemcpyDeviceToHost);
                     if (e == cudaSuccess)
-                        e = cudaMemcpy(tile_member_host + off, p->tile_member + tb[t], sizeof(uint64_t) * tc[t],
-                                       cudaMemcpyDeviceToHost);
+                        e = cudaMemcpy(tile_member_host + off * p->g.slots, p->tile_member + (size_t)tb[t] * p->g.slots,
+                                       sizeof(uint64_t) * tc[t] * p->g.slots, cudaMemcpyDeviceToHost);
                 }
                 off += tc[t];
             }

@@ -45,7 +45,8 @@ struct AttnParams {
     int32_t lgBQ;   // log2(B_Q) when B_Q < 128, else 31 (row >> 31 == 0)
     int32_t lgBKV;  // log2(B_KV) when B_KV < T_KV, else 31
     int32_t sK;     // logical KV sub-blocks per tile
-    int32_t stages;
+    int32_t stages;    // K ring depth (and V ring depth for the single-tile kernel)
+    int32_t stages_v;  // V ring depth of the paired kernel
     float scale_log2;  // log2(e) / sqrt(d)
 };
 
@@ -382,6 +383,336 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     if (warp == 5) tmem_dealloc(tmem, kTmemCols);
 }
 
+// ==========================================================================================
+// Paired kernel: one CTA owns a 256-row physical Q tile as two 128-row MMA slots.  Both slots
+// walk the same (merged) KV tile list, so every K/V tile is fetched into shared memory once and
+// feeds up to two Q tiles; a slot whose membership word for a tile is zero skips it.  Each slot
+// has its own softmax warpgroup, S/P columns and O accumulator in tensor memory; the single MMA
+// warp alternates between the slots (PV of the previous tile, then Q K^T of the next), so one
+// slot's softmax runs under the other slot's MMAs.
+//   warps 0-3 / 4-7 : softmax + correction + epilogue of slot 0 / slot 1 (more registers)
+//   warp 8          : TMA producer          warp 9 : MMA issuer (both give registers back)
+// Register budget: 384 threads launch with 168 registers each (504 per lane across the three
+// warpgroups); setmaxnreg moves them to 216 + 216 + 72 = 504.  The sum must not exceed the launch
+// allocation, otherwise the second setmaxnreg.inc never gets its registers and the CTA stalls.
+// ==========================================================================================
+constexpr int kPairThreads = 384;
+
+struct __align__(8) PairBarriers {
+    uint64_t q_full, q_empty;
+    uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
+    uint64_t s_full[2], p_ready[2], pv_done[2], o_free[2];
+};
+
+template <int R>
+__device__ __forceinline__ void reg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(R));
+}
+template <int R>
+__device__ __forceinline__ void reg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(R));
+}
+
+template <int D, int TK>
+__global__ void __launch_bounds__(kPairThreads, 1)
+bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                          const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+    constexpr int NSUB = D / 64;
+    constexpr int Q_SUB = kTQ * 128;
+    constexpr int Q_TILE = NSUB * Q_SUB;
+    constexpr int KV_SUB = TK * 128;
+    constexpr int KV_TILE = NSUB * KV_SUB;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sQ = smem;                       // [2 slots][NSUB][128][64]
+    uint8_t* sK = sQ + 2 * Q_TILE;            // [stages][NSUB][TK][64]
+    uint8_t* sV = sK + p.stages * KV_TILE;    // [stages_v][NSUB][TK][64]
+    __shared__ PairBarriers bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ uint32_t abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int NSK = p.stages, NSV = p.stages_v;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bars.q_full), 1);
+        mbar_init(smem_u32(&bars.q_empty), 1);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&bars.k_full[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_full[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&bars.s_full[s]), 1);
+            mbar_init(smem_u32(&bars.p_ready[s]), 128);
+            mbar_init(smem_u32(&bars.pv_done[s]), 1);
+            mbar_init(smem_u32(&bars.o_free[s]), 128);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 9) {
+        tmem_alloc(smem_u32(&tmem_base_s), kTmemCols);
+        tmem_relinquish();
+    }
+    if (warp == 8 && lane == 0) {
+        prefetch_tensormap(&tmQ);
+        prefetch_tensormap(&tmK);
+        prefetch_tensormap(&tmV);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    volatile uint32_t* abortp = &abort_flag;
+    const int n_items = p.counters->nitems;
+
+    if (warp >= 8) {
+        reg_dec<72>();
+        if (warp == 8 && lane == 0) {
+            // =========================== TMA producer ===========================
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const WorkItem it = p.items[idx];
+                if (it.ntiles == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1, abortp);
+                if (!ok) break;
+                mbar_arrive_expect_tx(smem_u32(&bars.q_full), 2 * Q_TILE);
+                for (int x = 0; x < 2; ++x)
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sQ + x * Q_TILE + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64,
+                                    it.q_tile * (2 * kTQ) + x * kTQ, it.head);
+                for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
+                    const int sk = g % NSK, sv = g % NSV;
+                    const uint32_t phk = (g / NSK) & 1, phv = (g / NSV) & 1;
+                    const int kv0 = p.tile_col[j] * TK;
+                    ok = mbar_wait(smem_u32(&bars.k_empty[sk]), phk ^ 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(smem_u32(&bars.k_full[sk]), KV_TILE);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sK + sk * KV_TILE + s * KV_SUB), &tmK, smem_u32(&bars.k_full[sk]), s * 64,
+                                    kv0, it.head);
+                    ok = mbar_wait(smem_u32(&bars.v_empty[sv]), phv ^ 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(smem_u32(&bars.v_full[sv]), KV_TILE);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sV + sv * KV_TILE + s * KV_SUB), &tmV, smem_u32(&bars.v_full[sv]), s * 64,
+                                    kv0, it.head);
+                }
+                ++itq;
+            }
+            if (!ok) {
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        } else if (warp == 9 && lane == 0) {
+            // =========================== MMA issuer ===========================
+            constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
+            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
+            const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
+            const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
+            uint32_t itq = 0, g = 0;
+            uint32_t npv[2] = {0, 0};  // PV MMAs issued per slot: phase of p_ready / pv_done
+            uint32_t oit[2] = {0, 0};  // items in which the slot had tiles: phase of o_free
+            int pend[2] = {-1, -1};    // global tile index whose PV is still to be issued, or -1
+            bool started[2] = {false, false};
+            bool ok = true;
+            // PV of slot x for its pending tile: O_x (+)= P_x V
+            auto issue_pv = [&](int x) -> bool {
+                const uint32_t gp = (uint32_t)pend[x];
+                const int sv = gp % NSV;
+                if (!mbar_wait(smem_u32(&bars.p_ready[x]), npv[x] & 1, abortp)) return false;
+                if (!mbar_wait(smem_u32(&bars.v_full[sv]), (gp / NSV) & 1, abortp)) return false;
+                if (!started[x] && !mbar_wait(smem_u32(&bars.o_free[x]), (oit[x] & 1) ^ 1, abortp)) return false;
+                tc_fence_after();
+                const uint32_t d_o = tmem + kColO + x * 128, a_p = tmem + x * 128;
+#pragma unroll
+                for (int k = 0; k < TK / 16; ++k) {
+                    const uint64_t b = descV + (uint64_t)((sv * KV_TILE + k * 2048) >> 4);
+                    mma_ts(d_o, a_p + k * 8, b, idesc_pv, (started[x] || k > 0) ? 1u : 0u);
+                }
+                // the V stage is free once the last slot that uses this tile has issued its PV
+                if (!(x == 0 && pend[1] == pend[0])) mma_commit(smem_u32(&bars.v_empty[sv]));
+                mma_commit(smem_u32(&bars.pv_done[x]));
+                ++npv[x];
+                started[x] = true;
+                pend[x] = -1;
+                return true;
+            };
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const WorkItem it = p.items[idx];
+                const int n = it.ntiles;
+                if (n == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
+                if (!ok) break;
+                pend[0] = pend[1] = -1;
+                started[0] = started[1] = false;
+                for (int j = 0; j < n && ok; ++j) {
+                    const uint32_t gj = g + j;
+                    const int sk = gj % NSK;
+                    const ulonglong2 mem = *reinterpret_cast<const ulonglong2*>(p.tile_member + (size_t)(it.tile_begin + j) * 2);
+                    bool k_waited = false;
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        if (pend[x] >= 0) {
+                            ok = issue_pv(x);
+                            if (!ok) break;
+                        }
+                        if ((x == 0 ? mem.x : mem.y) != 0ull) {
+                            if (!k_waited) {
+                                ok = mbar_wait(smem_u32(&bars.k_full[sk]), (gj / NSK) & 1, abortp);
+                                if (!ok) break;
+                                k_waited = true;
+                            }
+                            tc_fence_after();
+                            const uint32_t d_s = tmem + x * 128;
+#pragma unroll
+                            for (int k = 0; k < D / 16; ++k) {
+                                const uint64_t a = descQ + (uint64_t)((x * Q_TILE + (k / 4) * Q_SUB + (k % 4) * 32) >> 4);
+                                const uint64_t b = descK + (uint64_t)((sk * KV_TILE + (k / 4) * KV_SUB + (k % 4) * 32) >> 4);
+                                mma_ss(d_s, a, b, idesc_qk, k > 0);
+                            }
+                            mma_commit(smem_u32(&bars.s_full[x]));
+                            pend[x] = (int)gj;
+                        }
+                    }
+                    if (!ok) break;
+                    mma_commit(smem_u32(&bars.k_empty[sk]));
+                }
+                if (!ok) break;
+                mma_commit(smem_u32(&bars.q_empty));
+                for (int x = 0; x < 2 && ok; ++x)
+                    if (pend[x] >= 0) ok = issue_pv(x);
+                for (int x = 0; x < 2; ++x)
+                    if (started[x]) ++oit[x];
+                g += n;
+                ++itq;
+            }
+        }
+    } else {
+        // =========================== softmax / correction / epilogue of slot x ===========================
+        reg_inc<216>();
+        const int x = warp >> 2;
+        const int tw = tid & 127;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t t_s = tmem + lane_base + x * 128;
+        const uint32_t t_o = tmem + lane_base + kColO + x * 128;
+        uint32_t cnt = 0;  // tiles this slot has processed: phase of s_full / p_ready / pv_done
+        bool ok = true;
+        const float c2 = p.scale_log2;
+        const unsigned long long sub_mask = (p.sK >= 64) ? ~0ull : ((1ull << p.sK) - 1ull);
+        for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            const WorkItem it = p.items[idx];
+            const int row = it.q_tile * (2 * kTQ) + x * kTQ + tw;
+            const bool row_ok = row < p.N;
+            float m_ref = -INFINITY, l = 0.f;
+            int nmine = 0;
+            for (int j = 0; j < it.ntiles; ++j) {
+                const unsigned long long member = p.tile_member[(size_t)(it.tile_begin + j) * 2 + x];
+                if (member == 0ull) continue;
+                const int kv0 = p.tile_col[it.tile_begin + j] * TK;
+                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
+                const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
+                const int n_valid = p.N - kv0;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), cnt & 1, abortp));
+                if (!ok) break;
+                tc_fence_after();
+                float alpha;
+                bool rescale;
+                softmax_tile<TK>(t_s, need_mask, row_bits, p.lgBKV, n_valid, c2, nmine > 0, m_ref, l, alpha, rescale);
+                if (nmine > 0 && __any_sync(0xffffffffu, rescale)) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x]), (cnt - 1) & 1, abortp));
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(t_o + c * 32, r);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        tmem_st32(t_o + c * 32, r);
+                    }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.p_ready[x]));
+                ++cnt;
+                ++nmine;
+            }
+            if (!ok) break;
+            if (nmine == 0) {
+                // no tile of this item reaches this slot's rows: O = 0, LSE = -inf (or an empty partial state)
+                if (it.nparts == 1) {
+                    if (row_ok) {
+                        uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D);
+#pragma unroll
+                        for (int c = 0; c < D / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
+                        p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
+                    }
+                } else {
+                    float4* o = reinterpret_cast<float4*>(p.ws_O + ((size_t)(it.ws_slot + x) * kTQ + tw) * D);
+#pragma unroll
+                    for (int c = 0; c < D / 4; ++c) o[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    p.ws_LSE[(size_t)(it.ws_slot + x) * kTQ + tw] = -INFINITY;
+                }
+                continue;
+            }
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x]), (cnt - 1) & 1, abortp));
+            if (!ok) break;
+            tc_fence_after();
+            const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
+            const float lse = (l > 0.f) ? fmaf(m_ref, 0.6931471805599453f, logf(l)) : -INFINITY;
+            if (it.nparts == 1) {
+                __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(t_o + c * 32, r);
+                    tc_wait_ld();
+                    if (row_ok) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            uint4 v;
+                            v.x = pack_bf16x2(__uint_as_float(r[q * 8 + 0]) * inv_l, __uint_as_float(r[q * 8 + 1]) * inv_l);
+                            v.y = pack_bf16x2(__uint_as_float(r[q * 8 + 2]) * inv_l, __uint_as_float(r[q * 8 + 3]) * inv_l);
+                            v.z = pack_bf16x2(__uint_as_float(r[q * 8 + 4]) * inv_l, __uint_as_float(r[q * 8 + 5]) * inv_l);
+                            v.w = pack_bf16x2(__uint_as_float(r[q * 8 + 6]) * inv_l, __uint_as_float(r[q * 8 + 7]) * inv_l);
+                            *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = v;
+                        }
+                    }
+                }
+                if (row_ok) p.LSE[(size_t)it.head * p.N + row] = lse;
+            } else {
+                float* orow = p.ws_O + ((size_t)(it.ws_slot + x) * kTQ + tw) * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(t_o + c * 32, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        float4 v = make_float4(__uint_as_float(r[q * 4 + 0]) * inv_l, __uint_as_float(r[q * 4 + 1]) * inv_l,
+                                               __uint_as_float(r[q * 4 + 2]) * inv_l, __uint_as_float(r[q * 4 + 3]) * inv_l);
+                        *reinterpret_cast<float4*>(orow + c * 32 + q * 4) = v;
+                    }
+                }
+                p.ws_LSE[(size_t)(it.ws_slot + x) * kTQ + tw] = lse;
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars.o_free[x]));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && abort_flag) atomicExch(&p.counters->status, (int)BSA_ERR_DEVICE_TIMEOUT);
+    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+}
+
 // ------------------------------------------------------------------------------------------
 // Split-K reduction (Section 4.3): partial states were stored as (normalised O_p, LSE_p), so
 // rescaling to the common maximum, merging and normalising is
@@ -397,19 +728,21 @@ __global__ void __launch_bounds__(256) bsa_merge_kernel(const SplitRow* __restri
     const int n_rows = counters->nsplit_rows;
     for (int sr = blockIdx.x; sr < n_rows; sr += gridDim.x) {
         const SplitRow s = split_rows[sr];
+        const int nparts = s.nparts & 0xffff, stride = s.nparts >> 16;
         for (int u = threadIdx.x; u < kTQ * GROUPS; u += blockDim.x) {
             const int r = u / GROUPS, gcol = (u % GROUPS) * 8;
             const int row = s.q_tile * kTQ + r;
             if (row >= N) continue;
             float m = -INFINITY;
-            for (int q = 0; q < s.nparts; ++q) m = fmaxf(m, ws_LSE[(size_t)(s.ws_slot + q) * kTQ + r]);
+            for (int q = 0; q < nparts; ++q) m = fmaxf(m, ws_LSE[(size_t)(s.ws_slot + q * stride) * kTQ + r]);
             const float m_use = (m == -INFINITY) ? 0.f : m;
             float tot = 0.f;
             float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            for (int q = 0; q < s.nparts; ++q) {
-                const float w = __expf(ws_LSE[(size_t)(s.ws_slot + q) * kTQ + r] - m_use);
+            for (int q = 0; q < nparts; ++q) {
+                const size_t slot = (size_t)(s.ws_slot + q * stride);
+                const float w = __expf(ws_LSE[slot * kTQ + r] - m_use);
                 tot += w;
-                const float4* src = reinterpret_cast<const float4*>(ws_O + ((size_t)(s.ws_slot + q) * kTQ + r) * D + gcol);
+                const float4* src = reinterpret_cast<const float4*>(ws_O + (slot * kTQ + r) * D + gcol);
                 const float4 a = src[0], b = src[1];
                 acc[0] = fmaf(w, a.x, acc[0]); acc[1] = fmaf(w, a.y, acc[1]);
                 acc[2] = fmaf(w, a.z, acc[2]); acc[3] = fmaf(w, a.w, acc[3]);
@@ -460,7 +793,7 @@ bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, i
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, int TK>
+template <int D, int TK, int KERNEL>
 cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t stream, const char** err) {
     CUtensorMap tq, tk, tv;
     if (!encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ) || !encode_map(&tk, a.K, a.g.N, a.g.H, D, TK) ||
@@ -468,11 +801,14 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
         *err = "cuTensorMapEncodeTiled failed";
         return cudaErrorInvalidValue;
     }
-    const int smem = attention_smem_bytes(D, TK, p.stages);
+    const int smem = attention_smem_bytes(D, TK, a.stages, KERNEL);
     static int attr_bytes = 0;  // per instantiation; grows to the largest request seen
     if (smem > attr_bytes) {
-        cudaError_t e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             smem);
+        cudaError_t e;
+        if (KERNEL == 0)
+            e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        else
+            e = cudaFuncSetAttribute(bsa_attention_pair_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) {
             *err = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
@@ -481,29 +817,44 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
     }
     int grid = a.num_sms < a.max_items ? a.num_sms : a.max_items;
     if (grid < 1) grid = 1;
-    bsa_attention_kernel<D, TK><<<grid, kThreads, smem, stream>>>(tq, tk, tv, p);
+    if (KERNEL == 0)
+        bsa_attention_kernel<D, TK><<<grid, kThreads, smem, stream>>>(tq, tk, tv, p);
+    else
+        bsa_attention_pair_kernel<D, TK><<<grid, kPairThreads, smem, stream>>>(tq, tk, tv, p);
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace
 
-int attention_smem_bytes(int d, int T_KV, int stages) {
-    const int q = kTQ * d * 2;
+// Shared-memory budget: 227 KB per CTA minus the kernels' static shared memory (barriers) and alignment slack.
+static int kv_buffers_that_fit(int d, int T_KV, int kernel) {
+    const int q = (kernel == 1 ? 2 : 1) * kTQ * d * 2;
     const int kv = T_KV * d * 2;
-    int need = q + 2 * stages * kv + 1024;
+    return (232448 - 2048 - 1024 - q) / kv;
+}
+
+static void split_stages(int total, int* nk, int* nv) {
+    *nk = total / 2;
+    *nv = total - *nk;  // V is held one step longer than K, it gets the odd buffer
+    if (*nk > kMaxStages) *nk = kMaxStages;
+    if (*nv > kMaxStages) *nv = kMaxStages;
+}
+
+int attention_max_stages(int d, int T_KV, int kernel) {
+    const int nb = kv_buffers_that_fit(d, T_KV, kernel);
+    if (kernel == 1) return nb > 2 * kMaxStages ? 2 * kMaxStages : nb;
+    const int s = nb / 2;
+    return s > kMaxStages ? kMaxStages : s;
+}
+
+int attention_smem_bytes(int d, int T_KV, int stages, int kernel) {
+    const int q = (kernel == 1 ? 2 : 1) * kTQ * d * 2;
+    const int kv = T_KV * d * 2;
+    int need = q + (kernel == 1 ? stages : 2 * stages) * kv + 1024;
     // more than half of the SM's shared memory, so exactly one CTA (and one 512-column TMEM allocation) per SM
     if (need < 120 * 1024) need = 120 * 1024;
     return need;
-}
-
-int attention_max_stages(int d, int T_KV) {
-    const int q = kTQ * d * 2;
-    const int kv = T_KV * d * 2;
-    // 227 KB per CTA minus the kernel's static shared memory (barriers) and alignment slack
-    int s = (232448 - 2048 - 1024 - q) / (2 * kv);
-    if (s > kMaxStages) s = kMaxStages;
-    return s;
 }
 
 cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char** err_detail) {
@@ -516,19 +867,26 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     p.LSE = a.LSE;
     p.ws_O = a.ws_O;
     p.ws_LSE = a.ws_LSE;
-    const int bits = a.g.sQ * a.g.sK;
+    const int bits = a.g.sQ128 * a.g.sK;
     p.full_member = (bits >= 64) ? ~0ull : ((1ull << bits) - 1ull);
     p.N = (int32_t)a.g.N;
-    p.lgBQ = (a.g.sQ > 1) ? a.g.lgBQ : 31;
+    p.lgBQ = (a.g.sQ128 > 1) ? a.g.lgBQ : 31;
     p.lgBKV = (a.g.sK > 1) ? a.g.lgBKV : 31;
     p.sK = a.g.sK;
     p.stages = a.stages;
+    p.stages_v = a.stages;
+    if (a.kernel == 1) split_stages(a.stages, &p.stages, &p.stages_v);
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)a.d));
     cudaError_t e;
-    if (a.d == 128 && a.g.T_KV == 128) e = launch_attn<128, 128>(a, p, stream, err_detail);
-    else if (a.d == 128 && a.g.T_KV == 64) e = launch_attn<128, 64>(a, p, stream, err_detail);
-    else if (a.d == 64 && a.g.T_KV == 128) e = launch_attn<64, 128>(a, p, stream, err_detail);
-    else if (a.d == 64 && a.g.T_KV == 64) e = launch_attn<64, 64>(a, p, stream, err_detail);
+    const int key = a.kernel * 1000 + a.d + a.g.T_KV / 64;  // kernel, d, T_KV
+    if (key == 128 + 2) e = launch_attn<128, 128, 0>(a, p, stream, err_detail);
+    else if (key == 128 + 1) e = launch_attn<128, 64, 0>(a, p, stream, err_detail);
+    else if (key == 64 + 2) e = launch_attn<64, 128, 0>(a, p, stream, err_detail);
+    else if (key == 64 + 1) e = launch_attn<64, 64, 0>(a, p, stream, err_detail);
+    else if (key == 1000 + 128 + 2) e = launch_attn<128, 128, 1>(a, p, stream, err_detail);
+    else if (key == 1000 + 128 + 1) e = launch_attn<128, 64, 1>(a, p, stream, err_detail);
+    else if (key == 1000 + 64 + 2) e = launch_attn<64, 128, 1>(a, p, stream, err_detail);
+    else if (key == 1000 + 64 + 1) e = launch_attn<64, 64, 1>(a, p, stream, err_detail);
     else {
         *err_detail = "no kernel for this (d, T_KV)";
         return cudaErrorInvalidValue;

@@ -25,9 +25,9 @@ static_assert(sizeof(WorkItem) == 32, "WorkItem must be 32 bytes");
 
 struct SplitRow {
     int32_t head;
-    int32_t q_tile;
-    int32_t ws_slot;  // first slot; partitions are consecutive
-    int32_t nparts;
+    int32_t q_tile;   // 128-row tile index
+    int32_t ws_slot;  // workspace slot (128 rows each) of partition 0
+    int32_t nparts;   // low 16 bits: partitions; high 16 bits: slot stride between partitions
 };
 
 // Scalars produced on the device during plan creation.
@@ -38,7 +38,8 @@ struct MaskStatsDev {
     unsigned int pad;
 };
 struct PlanCountersDev {
-    unsigned long long ntiles;
+    unsigned long long ntiles;       // physical tiles (a 256-row tile counts once)
+    unsigned long long nslot_tiles;  // 128-row MMA tiles actually computed
     int32_t nitems;
     int32_t nsplit_rows;
     int32_t nslots;
@@ -48,7 +49,9 @@ struct PlanCountersDev {
 // Geometry of the logical -> physical mapping of one plan instance.
 struct MapGeom {
     int32_t H, nQb, nKb, nQt, nKt;
-    int32_t B_Q, B_KV, T_KV;
+    int32_t B_Q, B_KV, T_Q, T_KV;
+    int32_t slots;   // 128-row MMA slots per physical tile row (T_Q / 128)
+    int32_t sQ128;   // logical rows per 128-row slot (1 when B_Q >= 128)
     int32_t sQ, rq;  // logical rows per tile row (coarsened) / tile rows per logical row (refined)
     int32_t sK, rk;  // same for columns
     int32_t lgBQ, lgBKV, lgSK;
@@ -94,8 +97,9 @@ struct ForwardArgs {
     int32_t num_sms;
 };
 cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char** err_detail);
-int attention_max_stages(int d, int T_KV);
-int attention_smem_bytes(int d, int T_KV, int stages);
+// `stages` counts K buffers plus V buffers for the paired kernel (kernel 1), K = V ring depth for kernel 0
+int attention_max_stages(int d, int T_KV, int kernel);
+int attention_smem_bytes(int d, int T_KV, int stages, int kernel);
 
 void count_launch(int n = 1);
 

@@ -29,6 +29,11 @@ static const bsa_plan_desc_t kCatalog[] = {
     {7, 128, 64, 3, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 0, "q128k64_s3"},
     {8, 128, 128, 0, 16, 4, BSA_ORDER_GLOBAL_LPT, 0, "q128k128_split16x4_global"},
     {9, 128, 64, 0, 2, 16, BSA_ORDER_HEAD_MAJOR_LPT, 0, "q128k64_split2x16"},
+    // two 128-row Q tiles per CTA sharing one K/V ring, two softmax warpgroups
+    {10, 256, 128, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 1, "q256k128"},
+    {11, 256, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 1, "q256k64"},
+    {12, 256, 128, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 1, "q256k128_split4x8"},
+    {13, 256, 128, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 1, "q256k128_global"},
 };
 static const int kCatalogSize = (int)(sizeof(kCatalog) / sizeof(kCatalog[0]));
 static const int64_t kDefaultWorkspace = 2ll << 30;
@@ -52,13 +57,16 @@ bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int heads
     g->N = N;
     g->B_Q = B_Q;
     g->B_KV = B_KV;
+    g->T_Q = P.T_Q;
     g->T_KV = P.T_KV;
+    g->slots = P.T_Q / kTQ;
+    g->sQ128 = B_Q < kTQ ? kTQ / B_Q : 1;
     g->nQb = (int)((N + B_Q - 1) / B_Q);
     g->nKb = (int)((N + B_KV - 1) / B_KV);
-    g->nQt = (int)((N + kTQ - 1) / kTQ);
+    g->nQt = (int)((N + P.T_Q - 1) / P.T_Q);
     g->nKt = (int)((N + P.T_KV - 1) / P.T_KV);
-    g->sQ = B_Q < kTQ ? kTQ / B_Q : 1;
-    g->rq = B_Q > kTQ ? B_Q / kTQ : 1;
+    g->sQ = B_Q < P.T_Q ? P.T_Q / B_Q : 1;
+    g->rq = B_Q > P.T_Q ? B_Q / P.T_Q : 1;
     g->sK = B_KV < P.T_KV ? P.T_KV / B_KV : 1;
     g->rk = B_KV > P.T_KV ? B_KV / P.T_KV : 1;
     g->lgBQ = ilog2(B_Q);
@@ -69,8 +77,8 @@ bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int heads
 
 int64_t plan_workspace_bytes(const bsa_plan_desc_t& P, int64_t N, int heads, int d) {
     if (P.split_pmax <= 1) return 0;
-    const int64_t nQt = (N + kTQ - 1) / kTQ;
-    return (int64_t)heads * nQt * P.split_pmax * kTQ * (int64_t)(d + 1) * 4;
+    const int64_t nQt = (N + P.T_Q - 1) / P.T_Q;
+    return (int64_t)heads * nQt * P.split_pmax * P.T_Q * (int64_t)(d + 1) * 4;
 }
 
 // Eligible(P, R), Section 4.4: logical geometry, tensor properties, metadata format, workspace.
@@ -82,11 +90,11 @@ bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, 
     if (N <= 0 || heads <= 0 || N > (1ll << 30)) return false;
     MapGeom g;
     make_geom(*P, B_Q, B_KV, N, heads, &g);
-    if (g.sQ * g.sK > 64) return false;  // membership word is 64 bits
-    const int max_st = attention_max_stages(d, P->T_KV);
+    if (g.sQ128 * g.sK > 64) return false;  // one 64-bit membership word per 128-row slot
+    const int max_st = attention_max_stages(d, P->T_KV, P->kernel);
     if (max_st < 2) return false;
     if (P->stages > max_st) return false;
-    if ((size_t)g.nKt * 8 > kPlannerSmemLimit) return false;
+    if ((size_t)g.nKt * 8 * g.slots > kPlannerSmemLimit) return false;
     if (organize_smem_bytes(g, P->order, P->split_pmax) > kPlannerSmemLimit) return false;
     if ((int64_t)heads * g.nQt * (P->split_pmax < 1 ? 1 : P->split_pmax) >= (1ll << 31)) return false;
     if (max_ws <= 0) max_ws = kDefaultWorkspace;

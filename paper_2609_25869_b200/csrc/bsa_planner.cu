@@ -137,14 +137,19 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
                                                         int32_t* __restrict__ tile_col,
                                                         uint64_t* __restrict__ tile_member,
                                                         int32_t* __restrict__ head_counts, PlanCountersDev* counters) {
-    extern __shared__ unsigned long long bm[];  // [nKt]
+    extern __shared__ unsigned long long bm[];  // [slots][nKt]: one membership word per 128-row slot
     __shared__ int32_t warp_cnt[8];
+    __shared__ int32_t warp_slot_cnt[8];
     __shared__ int32_t running;
+    __shared__ int32_t running_slots;
     const int trow = blockIdx.x;
     const int h = trow / g.nQt, t = trow % g.nQt;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int i = tid; i < g.nKt; i += blockDim.x) bm[i] = 0ull;
-    if (tid == 0) running = 0;
+    for (int i = tid; i < g.nKt * g.slots; i += blockDim.x) bm[i] = 0ull;
+    if (tid == 0) {
+        running = 0;
+        running_slots = 0;
+    }
     __syncthreads();
 
     int32_t cap_begin;
@@ -155,30 +160,35 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
         cap_begin = base * g.rk;
         for (int r = r0; r < r1; ++r) {
             const int a = r - r0;
+            // which 128-row slot(s) the logical row feeds, and its sub-row inside the slot
+            const int slot_lo = (g.B_Q >= g.T_Q) ? 0 : a / g.sQ128;
+            const int slot_hi = (g.B_Q >= g.T_Q) ? g.slots - 1 : slot_lo;
+            const int arow = a % g.sQ128;
             const int32_t b = row_ptr[h * g.nQb + r], e = row_ptr[h * g.nQb + r + 1];
             for (int32_t i = b + tid; i < e; i += blockDim.x) {
                 const int c = col_idx[i];
-                if (g.rk == 1) {
-                    const int tc = c >> g.lgSK;
-                    const int bit = a * g.sK + (c & (g.sK - 1));
-                    atomicOr(&bm[tc], 1ull << bit);
-                } else {
-                    for (int k = 0; k < g.rk; ++k) {
-                        const int tc = c * g.rk + k;
-                        if (tc < g.nKt) atomicOr(&bm[tc], 1ull << a);
+                for (int sl = slot_lo; sl <= slot_hi; ++sl) {
+                    unsigned long long* w = bm + (size_t)sl * g.nKt;
+                    if (g.rk == 1) {
+                        atomicOr(&w[c >> g.lgSK], 1ull << (arow * g.sK + (c & (g.sK - 1))));
+                    } else {
+                        for (int k = 0; k < g.rk; ++k) {
+                            const int tc = c * g.rk + k;
+                            if (tc < g.nKt) atomicOr(&w[tc], 1ull << arow);
+                        }
                     }
                 }
             }
         }
     } else {
+        // Refined along Q (B_Q > T_Q): tile row t is the `sub`-th part of logical row r; one slot
         const int r = t / g.rq, sub = t % g.rq;
         const int32_t b = row_ptr[h * g.nQb + r], e = row_ptr[h * g.nQb + r + 1];
         cap_begin = (b * g.rq + sub * (e - b)) * g.rk;
         for (int32_t i = b + tid; i < e; i += blockDim.x) {
             const int c = col_idx[i];
             if (g.rk == 1) {
-                const int tc = c >> g.lgSK;
-                atomicOr(&bm[tc], 1ull << (c & (g.sK - 1)));
+                atomicOr(&bm[c >> g.lgSK], 1ull << (c & (g.sK - 1)));
             } else {
                 for (int k = 0; k < g.rk; ++k) {
                     const int tc = c * g.rk + k;
@@ -191,23 +201,34 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
 
     for (int i0 = 0; i0 < g.nKt; i0 += blockDim.x) {
         const int i = i0 + tid;
-        const unsigned long long w = (i < g.nKt) ? bm[i] : 0ull;
-        const unsigned bits = __ballot_sync(kFull, w != 0ull);
-        if (lane == 0) warp_cnt[warp] = __popc(bits);
+        const unsigned long long w0 = (i < g.nKt) ? bm[i] : 0ull;
+        const unsigned long long w1 = (i < g.nKt && g.slots == 2) ? bm[g.nKt + i] : 0ull;
+        const bool any = (w0 | w1) != 0ull;
+        const unsigned bits = __ballot_sync(kFull, any);
+        const unsigned sbits0 = __ballot_sync(kFull, w0 != 0ull), sbits1 = __ballot_sync(kFull, w1 != 0ull);
+        if (lane == 0) {
+            warp_cnt[warp] = __popc(bits);
+            warp_slot_cnt[warp] = __popc(sbits0) + __popc(sbits1);
+        }
         __syncthreads();
         int32_t before = running;
-        int32_t total = 0;
+        int32_t total = 0, total_slots = 0;
         for (int k = 0; k < 8; ++k) {
             if (k < warp) before += warp_cnt[k];
             total += warp_cnt[k];
+            total_slots += warp_slot_cnt[k];
         }
-        if (w != 0ull) {
+        if (any) {
             const int32_t pos = cap_begin + before + __popc(bits & ((1u << lane) - 1u));
             tile_col[pos] = i;
-            tile_member[pos] = w;
+            tile_member[(size_t)pos * g.slots] = w0;
+            if (g.slots == 2) tile_member[(size_t)pos * 2 + 1] = w1;
         }
         __syncthreads();
-        if (tid == 0) running += total;
+        if (tid == 0) {
+            running += total;
+            running_slots += total_slots;
+        }
         __syncthreads();
     }
     if (tid == 0) {
@@ -222,7 +243,10 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
             atomicAdd(&head_counts[3 * h + 1], 1);
             atomicAdd(&head_counts[3 * h + 2], P);
         }
-        if (cnt) atomicAdd(&counters->ntiles, (unsigned long long)cnt);
+        if (cnt) {
+            atomicAdd(&counters->ntiles, (unsigned long long)cnt);
+            atomicAdd(&counters->nslot_tiles, (unsigned long long)running_slots);
+        }
     }
 }
 
@@ -304,7 +328,7 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, co
                 it.tile_end = tb + (int32_t)(((int64_t)cnt * (p + 1)) / P);
                 it.part = p;
                 it.nparts = P;
-                it.ws_slot = (P > 1) ? slot + p : -1;
+                it.ws_slot = (P > 1) ? (slot + p) * g.slots : -1;  // 128-row workspace slots
                 it.ntiles = it.tile_end - it.tile_begin;
                 const int32_t li = run_items + off_i + p;
                 items_tmp[item_base + li] = it;
@@ -312,12 +336,14 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, co
                 atomicAdd(&bins[it.ntiles], 1);
             }
             if (P > 1) {
-                SplitRow s;
-                s.head = r / g.nQt;
-                s.q_tile = r % g.nQt;
-                s.ws_slot = slot;
-                s.nparts = P;
-                split_rows[split_base + run_split + off_s] = s;
+                for (int sl = 0; sl < g.slots; ++sl) {
+                    SplitRow s;
+                    s.head = r / g.nQt;
+                    s.q_tile = (r % g.nQt) * g.slots + sl;
+                    s.ws_slot = slot * g.slots + sl;
+                    s.nparts = P | (g.slots << 16);
+                    split_rows[(size_t)(split_base + run_split + off_s) * g.slots + sl] = s;
+                }
             }
         }
         run_items += tot_i;
@@ -369,11 +395,11 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, co
     if (tid == 0) {
         if (order == BSA_ORDER_GLOBAL_LPT) {
             counters->nitems = n_items;
-            counters->nsplit_rows = run_split;
+            counters->nsplit_rows = run_split * g.slots;
             counters->nslots = run_slots;
         } else if (grp == gridDim.x - 1) {
             counters->nitems = item_base + n_items;
-            counters->nsplit_rows = split_base + run_split;
+            counters->nsplit_rows = (split_base + run_split) * g.slots;
             counters->nslots = slot_base + run_slots;
         }
     }
@@ -405,7 +431,7 @@ cudaError_t launch_tile_map(const MapGeom& g, const int32_t* row_ptr, const int3
                             int split_pmax, int32_t* tile_begin, int32_t* tile_cnt, int32_t* row_parts,
                             int32_t* tile_col, uint64_t* tile_member, int32_t* head_counts, PlanCountersDev* counters,
                             cudaStream_t stream) {
-    const size_t smem = (size_t)g.nKt * sizeof(unsigned long long);
+    const size_t smem = (size_t)g.nKt * g.slots * sizeof(unsigned long long);
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(tile_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;

@@ -36,6 +36,7 @@ def check_plan_structure(req, plan, heads=None):
     orp, oci = oracle.block_csr(req.mask)
     assert np.array_equal(rp, orp) and np.array_equal(ci, oci)
     T_Q, T_KV = inf["plan"]["T_Q"], inf["plan"]["T_KV"]
+    W, bits = inf["member_words"], inf["member_bits"]
     hs = range(req.H) if heads is None else heads
     tiles = {}
     ntiles = 0
@@ -44,7 +45,16 @@ def check_plan_structure(req, plan, heads=None):
         for t in range(len(trp) - 1):
             cols = tc[trp[t]:trp[t + 1]]
             assert (np.diff(cols) > 0).all(), "tile columns must be ascending and unique"
-        tiles[h] = (trp, tc, tm)
+        assert (tm.astype(object).sum(axis=1) != 0).all() if len(tm) else True, "a listed tile must have an active slot"
+        # one Python integer per tile: slot s of a 256-row tile holds sub-rows [s*sQ128, (s+1)*sQ128)
+        if W == 1:
+            mem = [int(v) for v in tm[:, 0]]
+        elif req.B_Q >= T_Q:  # one logical row block spans both slots: their words must agree
+            assert np.array_equal(tm[:, 0], tm[:, 1])
+            mem = [int(v) for v in tm[:, 0]]
+        else:
+            mem = [int(a) | (int(b) << bits) for a, b in tm]
+        tiles[h] = (trp, tc, mem)
         ntiles += len(tc)
     cover = oracle.coverage_counts(req.H, req.N, req.B_Q, req.B_KV, T_Q, T_KV, tiles)
     expect = oracle.expected_cell_cover(req.mask, req.N, req.B_Q, req.B_KV, T_Q, T_KV)
@@ -66,9 +76,9 @@ def check_plan_structure(req, plan, heads=None):
         parts.sort()
         assert [p[0] for p in parts] == list(range(parts[0][3]))
         for a, b in zip(parts[:-1], parts[1:]):
-            assert a[2] == b[1] and b[4] == a[4] + 1
+            assert a[2] == b[1] and b[4] == a[4] + W
         nsplit += len(parts) > 1
-    assert nsplit == inf["nsplit_rows"]
+    assert nsplit * W == inf["nsplit_rows"]
     return inf
 
 

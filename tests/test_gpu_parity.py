@@ -18,13 +18,13 @@ def _sample(req, per_head, seed=77, heads=None):
 
 
 # ---------------------------------------------------------------- the five configurations
-@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9])
+@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9, 10, 11, 12, 13])
 def test_tiny_full_oracle_every_plan(plan_id):
     res = Hh.run_request(I.config_tiny(), plan_id=plan_id)
     assert res["pairs"] == res["info"]["nnz_blocks"] * 64 * 64
 
 
-@pytest.mark.parametrize("plan_id", [0, 1, 2])
+@pytest.mark.parametrize("plan_id", [0, 1, 2, 10, 12])
 def test_mid_full_oracle(plan_id):
     Hh.run_request(I.config_mid(), plan_id=plan_id)
 
@@ -35,18 +35,19 @@ def test_hunyuan_shaped_sampled_oracle():
     Hh.run_request(req, plan_id=-1, sel=_sample(req, 64), heads=[0, 11, 23])
 
 
-@pytest.mark.parametrize("plan_id", [0, 1])
+@pytest.mark.parametrize("plan_id", [0, 1, 10])
 def test_stress_a_coarsened(plan_id):
     req = I.config_stress_a()
     res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64), heads=[0, 15])
     assert res["info"]["map_q"] == 1  # Coarsened along Q: 8 logical rows of 16 per 128-row tile
 
 
-@pytest.mark.parametrize("plan_id", [0, 1])
+@pytest.mark.parametrize("plan_id", [0, 1, 10, 11])
 def test_stress_b_refined(plan_id):
     req = I.config_stress_b()
     res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64))
-    assert res["info"]["map_q"] == 2 and res["info"]["map_kv"] == 2  # Refined in both dimensions
+    # B = (256,256): Refined along KV always; along Q Refined for 128-row tiles, Direct for 256-row tiles
+    assert res["info"]["map_kv"] == 2 and res["info"]["map_q"] == (2 if res["info"]["plan"]["T_Q"] == 128 else 0)
 
 
 @pytest.mark.parametrize("r,B,rho", [(0, (32, 32), 0.03), (1, (64, 128), 0.10), (2, (128, 64), 0.30),
@@ -62,6 +63,9 @@ def test_sweep_requests_ragged_n(r, B, rho):
     (16, 16, 1000, 64, 0), (16, 16, 1000, 64, 1), (32, 64, 777, 128, 0), (64, 32, 1300, 128, 1),
     (128, 256, 2100, 64, 0), (256, 128, 2100, 128, 1), (256, 16, 900, 64, 3), (16, 256, 900, 128, 2),
     (64, 64, 130, 64, 0), (128, 128, 127, 128, 0), (128, 128, 1, 64, 1),
+    (16, 16, 1000, 64, 10), (32, 64, 777, 128, 11), (64, 32, 1300, 128, 10), (128, 256, 2100, 64, 11),
+    (256, 128, 2100, 128, 10), (256, 16, 900, 64, 12), (16, 256, 900, 128, 12), (128, 128, 127, 128, 10),
+    (128, 128, 129, 64, 10), (64, 64, 300, 128, 13),
 ])
 def test_geometries_with_ragged_tail(B_Q, B_KV, N, d, plan_id):
     H = 3
@@ -83,12 +87,13 @@ def test_degenerate_masks(kind):
     elif kind == "empty_head":
         M[0] = I.random_mask(1, 1, nb, nb, 0.5)[0]
     req = I.Request(kind, H, N, d, B, B, M, qkv_seed=3)
-    for plan_id in (0, 3):
+    for plan_id in (0, 3, 10, 12):
         Hh.run_request(req, plan_id=plan_id)
 
 
 # ---------------------------------------------------------------- closed forms on the GPU path
-@pytest.mark.parametrize("B_Q,B_KV,N,d,plan_id", [(16, 64, 1000, 64, 0), (32, 32, 700, 128, 1), (256, 256, 1100, 128, 9)])
+@pytest.mark.parametrize("B_Q,B_KV,N,d,plan_id", [(16, 64, 1000, 64, 0), (32, 32, 700, 128, 1), (256, 256, 1100, 128, 9),
+                                                  (16, 64, 1000, 64, 10), (64, 32, 700, 128, 11), (256, 256, 1100, 128, 12)])
 def test_zero_keys_give_log_count_and_mean_value(B_Q, B_KV, N, d, plan_id):
     """K = 0: every score is 0, so LSE = ln(#reachable keys) exactly and O = mean of reachable V.
     Catches any off-by-one in ragged-edge or membership masking (one key off moves LSE by ~1/count)."""
