@@ -119,8 +119,8 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     constexpr int Q_SUB = kTQ * 128;          // bytes of one [128][64] bf16 sub-tile
     constexpr int KV_SUB = TK * 128;          // bytes of one [TK][64] bf16 sub-tile
     constexpr int KV_TILE = NSUB * KV_SUB;
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // dynamic shared memory starts on a 1024-byte boundary (the swizzled tiles need it); checked below
+    extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* sQ = smem;
     uint8_t* sK = sQ + NSUB * Q_SUB;
     uint8_t* sV = sK + p.stages * KV_TILE;
@@ -129,6 +129,10 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     __shared__ uint32_t abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (smem_u32(smem) & 1023u) {  // never expected; fail with a status instead of corrupting tiles
+        if (tid == 0) atomicExch(&p.counters->status, (int)BSA_ERR_CUDA);
+        return;
+    }
     const int NS = p.stages;
 
     if (tid == 0) {
@@ -422,8 +426,8 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     constexpr int Q_TILE = NSUB * Q_SUB;
     constexpr int KV_SUB = TK * 128;
     constexpr int KV_TILE = NSUB * KV_SUB;
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // dynamic shared memory starts on a 1024-byte boundary (the swizzled tiles need it); checked below
+    extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* sQ = smem;                       // [2 slots][NSUB][128][64]
     uint8_t* sK = sQ + 2 * Q_TILE;            // [stages][NSUB][TK][64]
     uint8_t* sV = sK + p.stages * KV_TILE;    // [stages_v][NSUB][TK][64]
@@ -432,6 +436,10 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     __shared__ uint32_t abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (smem_u32(smem) & 1023u) {  // never expected; fail with a status instead of corrupting tiles
+        if (tid == 0) atomicExch(&p.counters->status, (int)BSA_ERR_CUDA);
+        return;
+    }
     const int NSK = p.stages, NSV = p.stages_v;
 
     if (tid == 0) {
@@ -713,6 +721,367 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
     if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
+// ==========================================================================================
+// Column-split kernel: same work decomposition as bsa_attention_kernel (one 128-row Q tile per
+// CTA, S double-buffered), but TWO threads per query row: softmax warps 0-3 take the left half of
+// the score tile's columns, warps 4-7 the right half (both may read the same TMEM lanes).  The two
+// threads of a row exchange their half-row maxima through shared memory so they take identical
+// reference-maximum decisions; each keeps a partial sum, added up once in the epilogue.  P goes to
+// its own TMEM columns (the halves of S being read by the partner must not be overwritten).
+//   warps 0-7 : softmax / correction / epilogue    warp 8 : TMA producer    warp 9 : MMA issuer
+// ==========================================================================================
+constexpr int kCsThreads = 320;
+constexpr uint32_t kColP0 = 384, kColP1 = 448;
+
+struct __align__(8) CsBarriers {
+    uint64_t q_full, q_empty, o_free, xchg;
+    uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
+    uint64_t s_full[2], p_ready[2], pv_done[2];
+};
+
+template <int D, int TK>
+__global__ void __launch_bounds__(kCsThreads, 1)
+bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                        const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+    constexpr int NSUB = D / 64;
+    constexpr int Q_SUB = kTQ * 128;
+    constexpr int KV_SUB = TK * 128;
+    constexpr int KV_TILE = NSUB * KV_SUB;
+    constexpr int NC = TK / 2;  // score columns per softmax thread
+    constexpr int DC = D / 2;   // output columns per softmax thread
+    // dynamic shared memory starts on a 1024-byte boundary (the swizzled tiles need it); checked below
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint8_t* sQ = smem;
+    uint8_t* sK = sQ + NSUB * Q_SUB;
+    uint8_t* sV = sK + p.stages * KV_TILE;
+    __shared__ CsBarriers bars;
+    __shared__ float xbuf[2][2][kTQ];  // [use parity][column half][row]: half-row maxima / partial sums
+    __shared__ uint32_t tmem_base_s;
+    __shared__ uint32_t abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (smem_u32(smem) & 1023u) {  // never expected; fail with a status instead of corrupting tiles
+        if (tid == 0) atomicExch(&p.counters->status, (int)BSA_ERR_CUDA);
+        return;
+    }
+    const int NS = p.stages;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bars.q_full), 1);
+        mbar_init(smem_u32(&bars.q_empty), 1);
+        mbar_init(smem_u32(&bars.o_free), 256);
+        mbar_init(smem_u32(&bars.xchg), 256);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&bars.k_full[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_full[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&bars.s_full[s]), 1);
+            mbar_init(smem_u32(&bars.p_ready[s]), 256);
+            mbar_init(smem_u32(&bars.pv_done[s]), 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 9) {
+        tmem_alloc(smem_u32(&tmem_base_s), kTmemCols);
+        tmem_relinquish();
+    }
+    if (warp == 8 && lane == 0) {
+        prefetch_tensormap(&tmQ);
+        prefetch_tensormap(&tmK);
+        prefetch_tensormap(&tmV);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    volatile uint32_t* abortp = &abort_flag;
+    const int n_items = p.counters->nitems;
+
+    if (warp == 8) {
+        // =========================== TMA producer ===========================
+        if (lane == 0) {
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const WorkItem it = p.items[idx];
+                if (it.ntiles == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1, abortp);
+                if (!ok) break;
+                mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
+                for (int s = 0; s < NSUB; ++s)
+                    tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, it.q_tile * kTQ, it.head);
+                for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
+                    const int stage = g % NS;
+                    const uint32_t ph = (g / NS) & 1;
+                    const int kv0 = p.tile_col[j] * TK;
+                    ok = mbar_wait(smem_u32(&bars.k_empty[stage]), ph ^ 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), KV_TILE);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sK + stage * KV_TILE + s * KV_SUB), &tmK, smem_u32(&bars.k_full[stage]),
+                                    s * 64, kv0, it.head);
+                    ok = mbar_wait(smem_u32(&bars.v_empty[stage]), ph ^ 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), KV_TILE);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sV + stage * KV_TILE + s * KV_SUB), &tmV, smem_u32(&bars.v_full[stage]),
+                                    s * 64, kv0, it.head);
+                }
+                ++itq;
+            }
+            if (!ok) {
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        }
+    } else if (warp == 9) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
+            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
+            const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
+            const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const int n = p.items[idx].ntiles;
+                if (n == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
+                if (!ok) break;
+                for (int j = 0; j <= n && ok; ++j) {
+                    if (j < n) {
+                        const uint32_t gs = g + j;
+                        const int stage = gs % NS;
+                        const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
+                        ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
+                        if (!ok) break;
+                        if (gs >= 2) {
+                            // S[sb] was last read by the softmax of tile gs-2, which arrived on p_ready before
+                            // the PV of that tile was issued: already ordered before this point
+                        }
+                        tc_fence_after();
+                        const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint64_t a = descQ + (uint64_t)(((k / 4) * Q_SUB + (k % 4) * 32) >> 4);
+                            const uint64_t b = descK + (uint64_t)((stage * KV_TILE + (k / 4) * KV_SUB + (k % 4) * 32) >> 4);
+                            mma_ss(d_s, a, b, idesc_qk, k > 0);
+                        }
+                        mma_commit(smem_u32(&bars.k_empty[stage]));
+                        mma_commit(smem_u32(&bars.s_full[sb]));
+                        if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
+                    }
+                    if (j >= 1) {
+                        const uint32_t gp = g + j - 1;
+                        const int stage = gp % NS;
+                        const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
+                        ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
+                        if (!ok) break;
+                        ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
+                        if (!ok) break;
+                        if (j == 1) {
+                            ok = mbar_wait(smem_u32(&bars.o_free), (itq & 1) ^ 1, abortp);
+                            if (!ok) break;
+                        }
+                        tc_fence_after();
+                        const uint32_t a_p = tmem + (sb ? kColP1 : kColP0);
+#pragma unroll
+                        for (int k = 0; k < TK / 16; ++k) {
+                            const uint64_t b = descV + (uint64_t)((stage * KV_TILE + k * 2048) >> 4);
+                            mma_ts(tmem + kColO, a_p + k * 8, b, idesc_pv, (j > 1 || k > 0) ? 1u : 0u);
+                        }
+                        mma_commit(smem_u32(&bars.v_empty[stage]));
+                        mma_commit(smem_u32(&bars.pv_done[sb]));
+                    }
+                }
+                g += n;
+                ++itq;
+            }
+        }
+    } else {
+        // =========================== softmax / correction / epilogue ===========================
+        const int half = warp >> 2;   // which half of the columns this thread owns
+        const int tw = tid & 127;     // query row inside the tile = TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        uint32_t itq = 0, g = 0, xuse = 0;
+        bool ok = true;
+        const float c2 = p.scale_log2;
+        const unsigned long long sub_mask = (p.sK >= 64) ? ~0ull : ((1ull << p.sK) - 1ull);
+        // exchange one float with the partner thread of this row (bounded wait, no hardware barrier)
+        auto exchange = [&](float mine, float& other) -> bool {
+            const uint32_t par = xuse & 1;
+            xbuf[par][half][tw] = mine;
+            mbar_arrive(smem_u32(&bars.xchg));
+            const bool got = mbar_wait(smem_u32(&bars.xchg), par, abortp);
+            other = xbuf[par][half ^ 1][tw];
+            ++xuse;
+            return got;
+        };
+        for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            const WorkItem it = p.items[idx];
+            const int row = it.q_tile * kTQ + tw;
+            const bool row_ok = row < p.N;
+            if (it.ntiles == 0) {
+                if (row_ok) {
+                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D + half * DC);
+#pragma unroll
+                    for (int c = 0; c < DC / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
+                    if (half == 0) p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
+                }
+                continue;
+            }
+            float m_ref = -INFINITY, l = 0.f;
+            for (int j = 0; j < it.ntiles; ++j) {
+                const uint32_t gs = g + j, sb = gs & 1;
+                const int kv0 = p.tile_col[it.tile_begin + j] * TK;
+                const unsigned long long member = p.tile_member[it.tile_begin + j];
+                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
+                const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
+                const int n_valid = p.N - kv0;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[sb]), (gs >> 1) & 1, abortp));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_s = tmem + lane_base + (sb ? kColS1 : kColS0) + half * NC;
+                const uint32_t t_p = tmem + lane_base + (sb ? kColP1 : kColP0) + half * (NC / 2);
+                uint32_t r[NC];
+#pragma unroll
+                for (int c = 0; c < NC / 32; ++c) tmem_ld32(t_s + c * 32, &r[c * 32]);
+                tc_wait_ld();
+                if (need_mask) {
+#pragma unroll
+                    for (int i = 0; i < NC; ++i) {
+                        const int col = half * NC + i;
+                        const bool act = ((row_bits >> (col >> p.lgBKV)) & 1u) && (col < n_valid);
+                        r[i] = act ? r[i] : 0xff800000u;
+                    }
+                }
+                float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < NC; i += 4) {
+                    m0 = fmaxf(m0, __uint_as_float(r[i]));
+                    m1 = fmaxf(m1, __uint_as_float(r[i + 1]));
+                    m2 = fmaxf(m2, __uint_as_float(r[i + 2]));
+                    m3 = fmaxf(m3, __uint_as_float(r[i + 3]));
+                }
+                float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)), mx_other;
+                ok = __all_sync(0xffffffffu, exchange(mx, mx_other));
+                if (!ok) break;
+                const float mx2 = fmaxf(mx, mx_other) * c2;
+                float alpha = 1.f;
+                bool rescale = false;
+                if (mx2 > m_ref + kRescaleThreshold) {
+                    alpha = ex2_approx(m_ref - mx2);
+                    rescale = (j > 0) && (m_ref != -INFINITY);
+                    m_ref = mx2;
+                }
+                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int i = 0; i < NC; i += 8) {
+                    float t[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) t[k] = fmaf(__uint_as_float(r[i + k]), c2, neg_m);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) t[k] = ex2_approx(t[k]);
+                    s0 += t[0] + t[4];
+                    s1 += t[1] + t[5];
+                    s2 += t[2] + t[6];
+                    s3 += t[3] + t[7];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) r[i / 2 + k] = pack_bf16x2(t[2 * k], t[2 * k + 1]);
+                }
+#pragma unroll
+                for (int c = 0; c < NC / 32; ++c) tmem_st16(t_p + c * 16, &r[c * 16]);
+                l = l * alpha + ((s0 + s1) + (s2 + s3));
+                if (j > 0 && __any_sync(0xffffffffu, rescale)) {
+                    const uint32_t gp = gs - 1;
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[gp & 1]), (gp >> 1) & 1, abortp));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t t_o = tmem + lane_base + kColO + half * DC;
+#pragma unroll
+                    for (int c = 0; c < DC / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(t_o + c * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(t_o + c * 32, o);
+                    }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.p_ready[sb]));
+            }
+            if (!ok) break;
+            // ---- epilogue: add the two partial sums, normalise, store this thread's half of the row ----
+            {
+                float l_other;
+                ok = __all_sync(0xffffffffu, exchange(l, l_other));
+                if (!ok) break;
+                const float l_tot = (half == 0) ? (l + l_other) : (l_other + l);
+                const uint32_t gl = g + it.ntiles - 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[gl & 1]), (gl >> 1) & 1, abortp));
+                if (!ok) break;
+                tc_fence_after();
+                const float inv_l = (l_tot > 0.f) ? 1.f / l_tot : 0.f;
+                const float lse = (l_tot > 0.f) ? fmaf(m_ref, 0.6931471805599453f, logf(l_tot)) : -INFINITY;
+                const uint32_t t_o = tmem + lane_base + kColO + half * DC;
+                if (it.nparts == 1) {
+                    __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D + half * DC;
+#pragma unroll
+                    for (int c = 0; c < DC / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(t_o + c * 32, o);
+                        tc_wait_ld();
+                        if (row_ok) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                uint4 v;
+                                v.x = pack_bf16x2(__uint_as_float(o[q * 8 + 0]) * inv_l, __uint_as_float(o[q * 8 + 1]) * inv_l);
+                                v.y = pack_bf16x2(__uint_as_float(o[q * 8 + 2]) * inv_l, __uint_as_float(o[q * 8 + 3]) * inv_l);
+                                v.z = pack_bf16x2(__uint_as_float(o[q * 8 + 4]) * inv_l, __uint_as_float(o[q * 8 + 5]) * inv_l);
+                                v.w = pack_bf16x2(__uint_as_float(o[q * 8 + 6]) * inv_l, __uint_as_float(o[q * 8 + 7]) * inv_l);
+                                *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = v;
+                            }
+                        }
+                    }
+                    if (row_ok && half == 0) p.LSE[(size_t)it.head * p.N + row] = lse;
+                } else {
+                    float* orow = p.ws_O + ((size_t)it.ws_slot * kTQ + tw) * D + half * DC;
+#pragma unroll
+                    for (int c = 0; c < DC / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(t_o + c * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            float4 v = make_float4(__uint_as_float(o[q * 4 + 0]) * inv_l, __uint_as_float(o[q * 4 + 1]) * inv_l,
+                                                   __uint_as_float(o[q * 4 + 2]) * inv_l, __uint_as_float(o[q * 4 + 3]) * inv_l);
+                            *reinterpret_cast<float4*>(orow + c * 32 + q * 4) = v;
+                        }
+                    }
+                    if (half == 0) p.ws_LSE[(size_t)it.ws_slot * kTQ + tw] = lse;
+                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.o_free));
+            }
+            g += it.ntiles;
+            ++itq;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && abort_flag) atomicExch(&p.counters->status, (int)BSA_ERR_DEVICE_TIMEOUT);
+    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+}
+
 // ------------------------------------------------------------------------------------------
 // Split-K reduction (Section 4.3): partial states were stored as (normalised O_p, LSE_p), so
 // rescaling to the common maximum, merging and normalising is
@@ -807,8 +1176,10 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
         cudaError_t e;
         if (KERNEL == 0)
             e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        else
+        else if (KERNEL == 1)
             e = cudaFuncSetAttribute(bsa_attention_pair_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        else
+            e = cudaFuncSetAttribute(bsa_attention_cs_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) {
             *err = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
@@ -819,19 +1190,24 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
     if (grid < 1) grid = 1;
     if (KERNEL == 0)
         bsa_attention_kernel<D, TK><<<grid, kThreads, smem, stream>>>(tq, tk, tv, p);
-    else
+    else if (KERNEL == 1)
         bsa_attention_pair_kernel<D, TK><<<grid, kPairThreads, smem, stream>>>(tq, tk, tv, p);
+    else
+        bsa_attention_cs_kernel<D, TK><<<grid, kCsThreads, smem, stream>>>(tq, tk, tv, p);
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace
 
-// Shared-memory budget: 227 KB per CTA minus the kernels' static shared memory (barriers) and alignment slack.
+// Shared-memory budget: 227 KB per CTA minus each kernel's static shared memory (barriers, exchange
+// buffer), which the compiler rounds up to the 1024-byte alignment of the dynamic part.
+static int static_smem_bytes(int kernel) { return kernel == 2 ? 3072 : 1024; }
+
 static int kv_buffers_that_fit(int d, int T_KV, int kernel) {
     const int q = (kernel == 1 ? 2 : 1) * kTQ * d * 2;
     const int kv = T_KV * d * 2;
-    return (232448 - 2048 - 1024 - q) / kv;
+    return (232448 - static_smem_bytes(kernel) - q) / kv;
 }
 
 static void split_stages(int total, int* nk, int* nv) {
@@ -851,7 +1227,7 @@ int attention_max_stages(int d, int T_KV, int kernel) {
 int attention_smem_bytes(int d, int T_KV, int stages, int kernel) {
     const int q = (kernel == 1 ? 2 : 1) * kTQ * d * 2;
     const int kv = T_KV * d * 2;
-    int need = q + (kernel == 1 ? stages : 2 * stages) * kv + 1024;
+    int need = q + (kernel == 1 ? stages : 2 * stages) * kv;
     // more than half of the SM's shared memory, so exactly one CTA (and one 512-column TMEM allocation) per SM
     if (need < 120 * 1024) need = 120 * 1024;
     return need;
@@ -887,6 +1263,10 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     else if (key == 1000 + 128 + 1) e = launch_attn<128, 64, 1>(a, p, stream, err_detail);
     else if (key == 1000 + 64 + 2) e = launch_attn<64, 128, 1>(a, p, stream, err_detail);
     else if (key == 1000 + 64 + 1) e = launch_attn<64, 64, 1>(a, p, stream, err_detail);
+    else if (key == 2000 + 128 + 2) e = launch_attn<128, 128, 2>(a, p, stream, err_detail);
+    else if (key == 2000 + 128 + 1) e = launch_attn<128, 64, 2>(a, p, stream, err_detail);
+    else if (key == 2000 + 64 + 2) e = launch_attn<64, 128, 2>(a, p, stream, err_detail);
+    else if (key == 2000 + 64 + 1) e = launch_attn<64, 64, 2>(a, p, stream, err_detail);
     else {
         *err_detail = "no kernel for this (d, T_KV)";
         return cudaErrorInvalidValue;

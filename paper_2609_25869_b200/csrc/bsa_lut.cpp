@@ -34,6 +34,11 @@ static const bsa_plan_desc_t kCatalog[] = {
     {11, 256, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 1, "q256k64"},
     {12, 256, 128, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 1, "q256k128_split4x8"},
     {13, 256, 128, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 1, "q256k128_global"},
+    // one 128-row Q tile per CTA, two softmax threads per query row (column halves)
+    {14, 128, 128, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 2, "q128k128_cs"},
+    {15, 128, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 2, "q128k64_cs"},
+    {16, 128, 128, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 2, "q128k128_cs_split4x8"},
+    {17, 128, 128, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 2, "q128k128_cs_global"},
 };
 static const int kCatalogSize = (int)(sizeof(kCatalog) / sizeof(kCatalog[0]));
 static const int64_t kDefaultWorkspace = 2ll << 30;
