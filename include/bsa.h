@@ -158,6 +158,36 @@ BSA_API bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int B_K
                               bsa_plan_info_t* info_out);
 
 /* ---------------------------------------------------------------------------------------------
+ * bsa_mask_stats_noalloc -- the scalar mask statistics s_A(M) for callers that cannot allocate.
+ * (The paper has no counterpart: its runtime always builds the statistics as part of plan selection.)
+ *
+ * Meant for hosts where a call into the CUDA allocator is off limits: a serving process that gave
+ * all device memory to its own pool at start-up, a plug-in that lives under another component's
+ * allocation policy, a loop that cannot afford the device-wide synchronisation or the late failure
+ * of a cudaMalloc.  This call performs no cudaMalloc / cudaMallocAsync / cudaFree and uses no
+ * allocating library routine.  Its scratch memory (one int32 counter per mask row plus three
+ * accumulators) is a fixed array inside the library's device image: 256 + 4 * BSA_NOALLOC_MAX_ROWS
+ * bytes (about 4 MiB), resident on every GPU that loads the library until the process exits.
+ *
+ *   mask_dev      : uint8 [heads, nQb, nKb], nonzero = active block (device, borrowed).
+ *   stats_out_dev : int64 [4] in DEVICE memory, written on `stream`:
+ *                   {active blocks, active blocks in runs of length >= 2, largest row count,
+ *                    rows with no active block}.
+ *   heads * nQb must not exceed BSA_NOALLOC_MAX_ROWS; larger masks are rejected with
+ *   BSA_ERR_UNSUPPORTED before anything is launched.
+ *
+ * The first call on a device resolves the array's device address (cudaGetSymbolAddress) with that
+ * device current; make that first call before starting any stream capture.  All calls on a device
+ * share the one array, which still holds the previous call's data: the accumulators are cleared
+ * on `stream` at the start of every call.  Two calls whose GPU work overlaps (different streams, or
+ * different host threads) race on the array and give wrong results: keep them stream-ordered.
+ * Errors: INVALID_ARG (null pointers, non-positive sizes), UNSUPPORTED (too many rows), CUDA.
+ */
+#define BSA_NOALLOC_MAX_ROWS (1 << 20)
+BSA_API bsa_status_t bsa_mask_stats_noalloc(const uint8_t* mask_dev, int heads, int nQb, int nKb,
+                                    int64_t* stats_out_dev, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Introspection (tests, benches, the offline profiler).  These synchronise with the plan's stream.
  */
 BSA_API bsa_status_t bsa_plan_get_info(const bsa_plan_t* plan, bsa_plan_info_t* info_out);

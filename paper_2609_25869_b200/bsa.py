@@ -78,6 +78,7 @@ def lib() -> ctypes.CDLL:
     L.bsa_plan_destroy.argtypes = [vp]
     L.bsa_request_host.argtypes = [vp, i32, i32, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.POINTER(Options),
                                    ctypes.POINTER(PlanInfo)]
+    L.bsa_mask_stats_noalloc.argtypes = [vp, i32, i32, i32, vp, vp]
     L.bsa_plan_get_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
     L.bsa_plan_export_csr.argtypes = [vp, vp, vp]
     L.bsa_plan_export_tiles.argtypes = [vp, i32, vp, vp, vp, i64, ctypes.POINTER(i64)]
@@ -209,6 +210,24 @@ def request_host(mask: np.ndarray, B_Q: int, B_KV: int, N: int, heads: int, d: i
     _check(lib().bsa_request_host(ptr(mask), B_Q, B_KV, N, heads, d, ptr(Q), ptr(K), ptr(V), ptr(O), ptr(LSE),
                                   ctypes.byref(opt), ctypes.byref(inf)), "bsa_request_host")
     return inf.as_dict()
+
+
+NOALLOC_MAX_ROWS = 1 << 20
+
+
+def mask_stats_noalloc(mask, out=None, stream=None):
+    """``bsa_mask_stats_noalloc``: statistics of a uint8/bool CUDA mask ``[heads, nQb, nKb]`` into an int64
+    CUDA tensor of 4 entries, using the library's built-in scratch (no allocation inside the call when
+    ``out`` is given).  Returns ``out``; raises ``BsaError`` (UNSUPPORTED) beyond ``NOALLOC_MAX_ROWS`` rows."""
+    import torch
+    assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool) and mask.dim() == 3
+    if out is None:
+        out = torch.empty(4, dtype=torch.int64, device=mask.device)
+    assert out.is_cuda and out.dtype == torch.int64 and out.numel() >= 4 and out.is_contiguous()
+    h, nq, nk = mask.shape
+    _check(lib().bsa_mask_stats_noalloc(mask.data_ptr(), h, nq, nk, out.data_ptr(), _stream_ptr(stream)),
+           "bsa_mask_stats_noalloc")
+    return out
 
 
 def catalog() -> List[Dict]:
