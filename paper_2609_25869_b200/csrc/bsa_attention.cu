@@ -23,12 +23,28 @@ namespace bsa {
 
 using namespace ptx;
 
+// Optional timeline tracing (compile with -DBSA_TRACE): CTA 0 records clock64() at barrier events of the
+// single-tile kernel, per role, into a device buffer that bsa_debug_trace_copy() reads back.
+#ifdef BSA_TRACE
+__device__ long long g_trace[6][4096];  // producer, MMA issuer, softmax warps 0-3
+__device__ long long g_trace_aux[12][4];  // last tile's stamps inside softmax_tile, per warp
+#define BSA_TRACE_DECL(n) int n = 0
+#define BSA_TRACE_POINT(role, n, tag)                                              \
+    do {                                                                           \
+        if (blockIdx.x == 0 && (n) < 4096) g_trace[role][(n)++] = (clock64() << 8) | (tag); \
+    } while (0)
+#else
+#define BSA_TRACE_DECL(n)
+#define BSA_TRACE_POINT(role, n, tag)
+#endif
+
 namespace {
 
 constexpr int kMaxStages = 6;
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256;
+constexpr uint32_t kColP0 = 384, kColP1 = 448;  // separate bf16 P buffers of the column-split kernel
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: P stays below 2^8 between rescales
 
 struct AttnParams {
@@ -57,17 +73,20 @@ struct __align__(8) Barriers {
 };
 
 // One score tile of one query row (thread = row = TMEM lane): mask, running reference maximum,
-// P = exp2(s * c2 - m_ref) rounded to bf16 and written over S in place, running sum.
+// P = exp2(s * c2 - m_ref) rounded to bf16 and written to t_p (over S in place when t_p == t_s), running sum.
 // The reference maximum moves only when the tile maximum exceeds it by kRescaleThreshold (log2
 // units), so P stays below 2^8 and the running output needs rescaling (by `alpha`) only then.
 template <int TK>
-__device__ __forceinline__ void softmax_tile(uint32_t t_s, bool need_mask, uint32_t row_bits, int lgBKV, int n_valid,
+__device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, bool need_mask, uint32_t row_bits, int lgBKV, int n_valid,
                                              float c2, bool not_first, float& m_ref, float& l, float& alpha,
                                              bool& rescale) {
     uint32_t r[TK];
 #pragma unroll
     for (int c = 0; c < TK / 32; ++c) tmem_ld32(t_s + c * 32, &r[c * 32]);
     tc_wait_ld();
+#ifdef BSA_TRACE
+    if ((threadIdx.x & 31) == 0 && blockIdx.x == 0) g_trace_aux[threadIdx.x >> 5][0] = clock64();
+#endif
     if (need_mask) {
 #pragma unroll
         for (int i = 0; i < TK; ++i) {
@@ -92,27 +111,49 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, bool need_mask, uint3
         m_ref = mx2;
     }
     const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+#ifdef BSA_TRACE
+    if ((threadIdx.x & 31) == 0 && blockIdx.x == 0) g_trace_aux[threadIdx.x >> 5][1] = clock64();
+#endif
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
     for (int i = 0; i < TK; i += 4) {
-        const float p0 = ex2_approx(fmaf(__uint_as_float(r[i]), c2, neg_m));
-        const float p1 = ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, neg_m));
-        const float p2 = ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, neg_m));
-        const float p3 = ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, neg_m));
+#ifdef BSA_EXP_NOMUFU
+#define BSA_EX2(x) (x)
+#else
+#define BSA_EX2(x) ex2_approx(x)
+#endif
+        const float p0 = BSA_EX2(fmaf(__uint_as_float(r[i]), c2, neg_m));
+        const float p1 = BSA_EX2(fmaf(__uint_as_float(r[i + 1]), c2, neg_m));
+        const float p2 = BSA_EX2(fmaf(__uint_as_float(r[i + 2]), c2, neg_m));
+        const float p3 = BSA_EX2(fmaf(__uint_as_float(r[i + 3]), c2, neg_m));
         s0 += p0;
         s1 += p1;
         s2 += p2;
         s3 += p3;
+#ifdef BSA_EXP_NOPACK
+        r[i / 2] = __float_as_uint(p0) ^ __float_as_uint(p1);
+        r[i / 2 + 1] = __float_as_uint(p2) ^ __float_as_uint(p3);
+#else
         r[i / 2] = pack_bf16x2(p0, p1);
         r[i / 2 + 1] = pack_bf16x2(p2, p3);
+#endif
     }
+#ifdef BSA_TRACE
+    if ((threadIdx.x & 31) == 0 && blockIdx.x == 0) g_trace_aux[threadIdx.x >> 5][2] = clock64();
+#endif
+#ifdef BSA_EXP_NOST
+    if (c2 == 12345.f)
+#endif
 #pragma unroll
-    for (int c = 0; c < TK / 32; ++c) tmem_st16(t_s + c * 16, &r[c * 16]);
+    for (int c = 0; c < TK / 32; ++c) tmem_st16(t_p + c * 16, &r[c * 16]);
     l = l * alpha + ((s0 + s1) + (s2 + s3));
 }
 
-template <int D, int TK>
-__global__ void __launch_bounds__(kThreads, 1)
+// DUAL = true adds a seventh warp so that Q K^T and P V are issued by two different threads: the
+// Q K^T issuer runs up to two tiles ahead (S is double-buffered) instead of stalling behind the wait
+// for the softmax of the previous tile; ordering between the two issuers is carried by mbarriers only.
+template <int D, int TK, bool DUAL>
+__global__ void __launch_bounds__(DUAL ? kThreads + 32 : kThreads, 1)
 bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
     constexpr int NSUB = D / 64;              // 64-column (128-byte) sub-tiles per row
@@ -174,6 +215,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         if (lane == 0) {
             uint32_t itq = 0, g = 0;
             bool ok = true;
+            BSA_TRACE_DECL(tn);
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
                 const WorkItem it = p.items[idx];
                 if (it.ntiles == 0) continue;
@@ -182,18 +224,23 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
                 for (int s = 0; s < NSUB; ++s)
                     tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, it.q_tile * kTQ, it.head);
+                int col_next = p.tile_col[it.tile_begin];  // tile metadata is fetched one tile ahead of its use
                 for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
+                    const int col_cur = col_next;
+                    if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
                     const int stage = g % NS;
                     const uint32_t ph = (g / NS) & 1;
-                    const int kv0 = p.tile_col[j] * TK;
+                    const int kv0 = col_cur * TK;
                     ok = mbar_wait(smem_u32(&bars.k_empty[stage]), ph ^ 1, abortp);
                     if (!ok) break;
+                    BSA_TRACE_POINT(0, tn, 20);
                     mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), KV_TILE);
                     for (int s = 0; s < NSUB; ++s)
                         tma_load_3d(smem_u32(sK + stage * KV_TILE + s * KV_SUB), &tmK, smem_u32(&bars.k_full[stage]),
                                     s * 64, kv0, it.head);
                     ok = mbar_wait(smem_u32(&bars.v_empty[stage]), ph ^ 1, abortp);
                     if (!ok) break;
+                    BSA_TRACE_POINT(0, tn, 22);
                     mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), KV_TILE);
                     for (int s = 0; s < NSUB; ++s)
                         tma_load_3d(smem_u32(sV + stage * KV_TILE + s * KV_SUB), &tmV, smem_u32(&bars.v_full[stage]),
@@ -207,7 +254,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 5 && !DUAL) {
         // =========================== MMA issuer ===========================
         if (lane == 0) {
             constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
@@ -217,6 +264,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
             uint32_t itq = 0, g = 0;
             bool ok = true;
+            BSA_TRACE_DECL(tn);
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
                 const int n = p.items[idx].ntiles;
                 if (n == 0) continue;
@@ -229,6 +277,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
                         ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
                         if (!ok) break;
+                        BSA_TRACE_POINT(1, tn, 1);
                         tc_fence_after();
                         // S[sb] = Q K^T.  The previous user of S[sb] (P of tile gs-2, read by its PV MMA)
                         // precedes this MMA in issue order on the same pipe.
@@ -241,6 +290,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         }
                         mma_commit(smem_u32(&bars.k_empty[stage]));
                         mma_commit(smem_u32(&bars.s_full[sb]));
+                        BSA_TRACE_POINT(1, tn, 2);
                         if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
                     }
                     if (j >= 1) {
@@ -249,8 +299,10 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
                         ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
                         if (!ok) break;
+                        BSA_TRACE_POINT(1, tn, 3);
                         ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
                         if (!ok) break;
+                        BSA_TRACE_POINT(1, tn, 4);
                         if (j == 1) {
                             ok = mbar_wait(smem_u32(&bars.o_free), (itq & 1) ^ 1, abortp);
                             if (!ok) break;
@@ -264,7 +316,86 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         }
                         mma_commit(smem_u32(&bars.v_empty[stage]));
                         mma_commit(smem_u32(&bars.pv_done[sb]));
+                        BSA_TRACE_POINT(1, tn, 5);
                     }
+                }
+                g += n;
+                ++itq;
+            }
+        }
+    } else if (warp == 5) {
+        // =========================== Q K^T issuer (DUAL) ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
+            const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
+            const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const int n = p.items[idx].ntiles;
+                if (n == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
+                if (!ok) break;
+                for (int j = 0; j < n; ++j) {
+                    const uint32_t gs = g + j;
+                    const int stage = gs % NS;
+                    const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
+                    ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
+                    if (!ok) break;
+                    // S[sb] still holds P of tile gs-2 (written in place) until that tile's P V has completed.
+                    // (Measured: giving P its own columns so that Q K^T may start right after the softmax of
+                    // tile gs-2 was slower -- the early Q K^T delays the P V the softmax chain is waiting for.)
+                    if (gs >= 2) {
+                        ok = mbar_wait(smem_u32(&bars.pv_done[sb]), ((gs >> 1) - 1) & 1, abortp);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint64_t a = descQ + (uint64_t)(((k / 4) * Q_SUB + (k % 4) * 32) >> 4);
+                        const uint64_t b = descK + (uint64_t)((stage * KV_TILE + (k / 4) * KV_SUB + (k % 4) * 32) >> 4);
+                        mma_ss(d_s, a, b, idesc_qk, k > 0);
+                    }
+                    mma_commit(smem_u32(&bars.k_empty[stage]));
+                    mma_commit(smem_u32(&bars.s_full[sb]));
+                    if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
+                }
+                g += n;
+                ++itq;
+            }
+        }
+    } else if (warp == 6) {
+        // =========================== P V issuer (DUAL) ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const int n = p.items[idx].ntiles;
+                if (n == 0) continue;
+                for (int j = 0; j < n; ++j) {
+                    const uint32_t gp = g + j;
+                    const int stage = gp % NS;
+                    const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
+                    ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
+                    if (!ok) break;
+                    ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
+                    if (!ok) break;
+                    if (j == 0) {
+                        ok = mbar_wait(smem_u32(&bars.o_free), (itq & 1) ^ 1, abortp);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    const uint32_t a_p = tmem + (sb ? kColS1 : kColS0);
+#pragma unroll
+                    for (int k = 0; k < TK / 16; ++k) {
+                        const uint64_t b = descV + (uint64_t)((stage * KV_TILE + k * 2048) >> 4);
+                        mma_ts(tmem + kColO, a_p + k * 8, b, idesc_pv, (j > 0 || k > 0) ? 1u : 0u);
+                    }
+                    mma_commit(smem_u32(&bars.v_empty[stage]));
+                    mma_commit(smem_u32(&bars.pv_done[sb]));
                 }
                 g += n;
                 ++itq;
@@ -275,6 +406,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         uint32_t itq = 0, g = 0;
         bool ok = true;
+        BSA_TRACE_DECL(tn);
         const float c2 = p.scale_log2;
         const unsigned long long sub_mask = (p.sK >= 64) ? ~0ull : ((1ull << p.sK) - 1ull);
         for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
@@ -292,20 +424,35 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 continue;
             }
             float m_ref = -INFINITY, l = 0.f;
+            int col_next = p.tile_col[it.tile_begin];  // tile metadata is fetched one tile ahead of its use
+            unsigned long long member_next = p.tile_member[it.tile_begin];
             for (int j = 0; j < it.ntiles; ++j) {
                 const uint32_t gs = g + j, sb = gs & 1;
-                const int kv0 = p.tile_col[it.tile_begin + j] * TK;
-                const unsigned long long member = p.tile_member[it.tile_begin + j];
+                const int kv0 = col_next * TK;
+                const unsigned long long member = member_next;
+                if (j + 1 < it.ntiles) {
+                    col_next = p.tile_col[it.tile_begin + j + 1];
+                    member_next = p.tile_member[it.tile_begin + j + 1];
+                }
                 const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
                 const uint32_t row_bits = (uint32_t)((member >> ((tid >> p.lgBQ) * p.sK)) & sub_mask);
                 const int n_valid = p.N - kv0;  // columns >= n_valid do not exist
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[sb]), (gs >> 1) & 1, abortp));
                 if (!ok) break;
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 10);
                 tc_fence_after();
                 const uint32_t t_s = tmem + lane_base + (sb ? kColS1 : kColS0);
                 float alpha;
                 bool rescale;
-                softmax_tile<TK>(t_s, need_mask, row_bits, p.lgBKV, n_valid, c2, j > 0, m_ref, l, alpha, rescale);
+                softmax_tile<TK>(t_s, t_s, need_mask, row_bits, p.lgBKV, n_valid, c2, j > 0, m_ref, l, alpha, rescale);
+#ifdef BSA_TRACE
+                if (lane == 0 && blockIdx.x == 0 && tn + 3 < 4096) {
+                    g_trace[2 + warp][tn++] = (g_trace_aux[warp][0] << 8) | 11;
+                    g_trace[2 + warp][tn++] = (g_trace_aux[warp][1] << 8) | 12;
+                    g_trace[2 + warp][tn++] = (g_trace_aux[warp][2] << 8) | 14;
+                }
+#endif
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 13);
                 // ---- correction: rescale the running output when the reference moved ----
                 if (j > 0 && __any_sync(0xffffffffu, rescale)) {
                     const uint32_t gp = gs - 1;
@@ -326,6 +473,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.p_ready[sb]));
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 16);
             }
             if (!ok) break;
             // ---- epilogue ----
@@ -492,10 +640,13 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
                     for (int s = 0; s < NSUB; ++s)
                         tma_load_3d(smem_u32(sQ + x * Q_TILE + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64,
                                     it.q_tile * (2 * kTQ) + x * kTQ, it.head);
+                int col_next = p.tile_col[it.tile_begin];  // tile metadata is fetched one tile ahead of its use
                 for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
+                    const int col_cur = col_next;
+                    if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
                     const int sk = g % NSK, sv = g % NSV;
                     const uint32_t phk = (g / NSK) & 1, phv = (g / NSV) & 1;
-                    const int kv0 = p.tile_col[j] * TK;
+                    const int kv0 = col_cur * TK;
                     ok = mbar_wait(smem_u32(&bars.k_empty[sk]), phk ^ 1, abortp);
                     if (!ok) break;
                     mbar_arrive_expect_tx(smem_u32(&bars.k_full[sk]), KV_TILE);
@@ -558,10 +709,13 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
                 if (!ok) break;
                 pend[0] = pend[1] = -1;
                 started[0] = started[1] = false;
+                ulonglong2 mem_next = *reinterpret_cast<const ulonglong2*>(p.tile_member + (size_t)it.tile_begin * 2);
                 for (int j = 0; j < n && ok; ++j) {
                     const uint32_t gj = g + j;
                     const int sk = gj % NSK;
-                    const ulonglong2 mem = *reinterpret_cast<const ulonglong2*>(p.tile_member + (size_t)(it.tile_begin + j) * 2);
+                    const ulonglong2 mem = mem_next;
+                    if (j + 1 < n)
+                        mem_next = *reinterpret_cast<const ulonglong2*>(p.tile_member + (size_t)(it.tile_begin + j + 1) * 2);
                     bool k_waited = false;
 #pragma unroll
                     for (int x = 0; x < 2; ++x) {
@@ -618,10 +772,20 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
             const bool row_ok = row < p.N;
             float m_ref = -INFINITY, l = 0.f;
             int nmine = 0;
+            int col_next = 0;
+            unsigned long long member_next = 0ull;
+            if (it.ntiles > 0) {  // tile metadata is fetched one tile ahead of its use
+                col_next = p.tile_col[it.tile_begin];
+                member_next = p.tile_member[(size_t)it.tile_begin * 2 + x];
+            }
             for (int j = 0; j < it.ntiles; ++j) {
-                const unsigned long long member = p.tile_member[(size_t)(it.tile_begin + j) * 2 + x];
+                const unsigned long long member = member_next;
+                const int kv0 = col_next * TK;
+                if (j + 1 < it.ntiles) {
+                    col_next = p.tile_col[it.tile_begin + j + 1];
+                    member_next = p.tile_member[(size_t)(it.tile_begin + j + 1) * 2 + x];
+                }
                 if (member == 0ull) continue;
-                const int kv0 = p.tile_col[it.tile_begin + j] * TK;
                 const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
                 const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
                 const int n_valid = p.N - kv0;
@@ -630,7 +794,7 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
                 tc_fence_after();
                 float alpha;
                 bool rescale;
-                softmax_tile<TK>(t_s, need_mask, row_bits, p.lgBKV, n_valid, c2, nmine > 0, m_ref, l, alpha, rescale);
+                softmax_tile<TK>(t_s, t_s, need_mask, row_bits, p.lgBKV, n_valid, c2, nmine > 0, m_ref, l, alpha, rescale);
                 if (nmine > 0 && __any_sync(0xffffffffu, rescale)) {
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x]), (cnt - 1) & 1, abortp));
                     if (!ok) break;
@@ -728,10 +892,10 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
 // threads of a row exchange their half-row maxima through shared memory so they take identical
 // reference-maximum decisions; each keeps a partial sum, added up once in the epilogue.  P goes to
 // its own TMEM columns (the halves of S being read by the partner must not be overwritten).
-//   warps 0-7 : softmax / correction / epilogue    warp 8 : TMA producer    warp 9 : MMA issuer
+//   warps 0-7 : softmax / correction / epilogue    warp 8 : TMA producer
+//   warp 9 : Q K^T issuer    warp 10 : P V issuer (separate threads, ordered through mbarriers only)
 // ==========================================================================================
-constexpr int kCsThreads = 320;
-constexpr uint32_t kColP0 = 384, kColP1 = 448;
+constexpr int kCsThreads = 352;
 
 struct __align__(8) CsBarriers {
     uint64_t q_full, q_empty, o_free, xchg;
@@ -814,10 +978,13 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
                 for (int s = 0; s < NSUB; ++s)
                     tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, it.q_tile * kTQ, it.head);
+                int col_next = p.tile_col[it.tile_begin];  // tile metadata is fetched one tile ahead of its use
                 for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
+                    const int col_cur = col_next;
+                    if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
                     const int stage = g % NS;
                     const uint32_t ph = (g / NS) & 1;
-                    const int kv0 = p.tile_col[j] * TK;
+                    const int kv0 = col_cur * TK;
                     ok = mbar_wait(smem_u32(&bars.k_empty[stage]), ph ^ 1, abortp);
                     if (!ok) break;
                     mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), KV_TILE);
@@ -839,13 +1006,11 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             }
         }
     } else if (warp == 9) {
-        // =========================== MMA issuer ===========================
+        // =========================== Q K^T issuer ===========================
         if (lane == 0) {
             constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
-            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
             const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
             const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
-            const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
             uint32_t itq = 0, g = 0;
             bool ok = true;
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
@@ -853,51 +1018,65 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (n == 0) continue;
                 ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
                 if (!ok) break;
-                for (int j = 0; j <= n && ok; ++j) {
-                    if (j < n) {
-                        const uint32_t gs = g + j;
-                        const int stage = gs % NS;
-                        const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
-                        ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
+                for (int j = 0; j < n; ++j) {
+                    const uint32_t gs = g + j;
+                    const int stage = gs % NS;
+                    const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
+                    ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
+                    if (!ok) break;
+                    // S[sb] was last read by the softmax of tile gs-2; P lives in its own columns, so the
+                    // buffer is free as soon as that softmax has arrived on p_ready
+                    if (gs >= 2) {
+                        ok = mbar_wait(smem_u32(&bars.p_ready[sb]), ((gs >> 1) - 1) & 1, abortp);
                         if (!ok) break;
-                        if (gs >= 2) {
-                            // S[sb] was last read by the softmax of tile gs-2, which arrived on p_ready before
-                            // the PV of that tile was issued: already ordered before this point
-                        }
-                        tc_fence_after();
-                        const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
-#pragma unroll
-                        for (int k = 0; k < D / 16; ++k) {
-                            const uint64_t a = descQ + (uint64_t)(((k / 4) * Q_SUB + (k % 4) * 32) >> 4);
-                            const uint64_t b = descK + (uint64_t)((stage * KV_TILE + (k / 4) * KV_SUB + (k % 4) * 32) >> 4);
-                            mma_ss(d_s, a, b, idesc_qk, k > 0);
-                        }
-                        mma_commit(smem_u32(&bars.k_empty[stage]));
-                        mma_commit(smem_u32(&bars.s_full[sb]));
-                        if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
                     }
-                    if (j >= 1) {
-                        const uint32_t gp = g + j - 1;
-                        const int stage = gp % NS;
-                        const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
-                        ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
-                        if (!ok) break;
-                        ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
-                        if (!ok) break;
-                        if (j == 1) {
-                            ok = mbar_wait(smem_u32(&bars.o_free), (itq & 1) ^ 1, abortp);
-                            if (!ok) break;
-                        }
-                        tc_fence_after();
-                        const uint32_t a_p = tmem + (sb ? kColP1 : kColP0);
+                    tc_fence_after();
+                    const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
 #pragma unroll
-                        for (int k = 0; k < TK / 16; ++k) {
-                            const uint64_t b = descV + (uint64_t)((stage * KV_TILE + k * 2048) >> 4);
-                            mma_ts(tmem + kColO, a_p + k * 8, b, idesc_pv, (j > 1 || k > 0) ? 1u : 0u);
-                        }
-                        mma_commit(smem_u32(&bars.v_empty[stage]));
-                        mma_commit(smem_u32(&bars.pv_done[sb]));
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint64_t a = descQ + (uint64_t)(((k / 4) * Q_SUB + (k % 4) * 32) >> 4);
+                        const uint64_t b = descK + (uint64_t)((stage * KV_TILE + (k / 4) * KV_SUB + (k % 4) * 32) >> 4);
+                        mma_ss(d_s, a, b, idesc_qk, k > 0);
                     }
+                    mma_commit(smem_u32(&bars.k_empty[stage]));
+                    mma_commit(smem_u32(&bars.s_full[sb]));
+                    if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
+                }
+                g += n;
+                ++itq;
+            }
+        }
+    } else if (warp == 10) {
+        // =========================== P V issuer ===========================
+        if (lane == 0) {
+            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const int n = p.items[idx].ntiles;
+                if (n == 0) continue;
+                for (int j = 0; j < n; ++j) {
+                    const uint32_t gp = g + j;
+                    const int stage = gp % NS;
+                    const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
+                    ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
+                    if (!ok) break;
+                    ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
+                    if (!ok) break;
+                    if (j == 0) {
+                        ok = mbar_wait(smem_u32(&bars.o_free), (itq & 1) ^ 1, abortp);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    const uint32_t a_p = tmem + (sb ? kColP1 : kColP0);
+#pragma unroll
+                    for (int k = 0; k < TK / 16; ++k) {
+                        const uint64_t b = descV + (uint64_t)((stage * KV_TILE + k * 2048) >> 4);
+                        mma_ts(tmem + kColO, a_p + k * 8, b, idesc_pv, (j > 0 || k > 0) ? 1u : 0u);
+                    }
+                    mma_commit(smem_u32(&bars.v_empty[stage]));
+                    mma_commit(smem_u32(&bars.pv_done[sb]));
                 }
                 g += n;
                 ++itq;
@@ -936,10 +1115,16 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 continue;
             }
             float m_ref = -INFINITY, l = 0.f;
+            int col_next = p.tile_col[it.tile_begin];  // tile metadata is fetched one tile ahead of its use
+            unsigned long long member_next = p.tile_member[it.tile_begin];
             for (int j = 0; j < it.ntiles; ++j) {
                 const uint32_t gs = g + j, sb = gs & 1;
-                const int kv0 = p.tile_col[it.tile_begin + j] * TK;
-                const unsigned long long member = p.tile_member[it.tile_begin + j];
+                const int kv0 = col_next * TK;
+                const unsigned long long member = member_next;
+                if (j + 1 < it.ntiles) {
+                    col_next = p.tile_col[it.tile_begin + j + 1];
+                    member_next = p.tile_member[it.tile_begin + j + 1];
+                }
                 const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
                 const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
                 const int n_valid = p.N - kv0;
@@ -994,6 +1179,11 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     s3 += t[3] + t[7];
 #pragma unroll
                     for (int k = 0; k < 4; ++k) r[i / 2 + k] = pack_bf16x2(t[2 * k], t[2 * k + 1]);
+                }
+                // P[sb] was last read by the P V of tile gs-2, issued by another thread than Q K^T: make sure it is done
+                if (gs >= 2) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[sb]), ((gs >> 1) - 1) & 1, abortp));
+                    if (!ok) break;
                 }
 #pragma unroll
                 for (int c = 0; c < NC / 32; ++c) tmem_st16(t_p + c * 16, &r[c * 16]);
@@ -1175,7 +1365,9 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
     if (smem > attr_bytes) {
         cudaError_t e;
         if (KERNEL == 0)
-            e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        else if (KERNEL == 3)
+            e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         else if (KERNEL == 1)
             e = cudaFuncSetAttribute(bsa_attention_pair_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         else
@@ -1189,7 +1381,9 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
     int grid = a.num_sms < a.max_items ? a.num_sms : a.max_items;
     if (grid < 1) grid = 1;
     if (KERNEL == 0)
-        bsa_attention_kernel<D, TK><<<grid, kThreads, smem, stream>>>(tq, tk, tv, p);
+        bsa_attention_kernel<D, TK, false><<<grid, kThreads, smem, stream>>>(tq, tk, tv, p);
+    else if (KERNEL == 3)
+        bsa_attention_kernel<D, TK, true><<<grid, kThreads + 32, smem, stream>>>(tq, tk, tv, p);
     else if (KERNEL == 1)
         bsa_attention_pair_kernel<D, TK><<<grid, kPairThreads, smem, stream>>>(tq, tk, tv, p);
     else
@@ -1233,6 +1427,12 @@ int attention_smem_bytes(int d, int T_KV, int stages, int kernel) {
     return need;
 }
 
+#ifdef BSA_TRACE
+extern "C" __attribute__((visibility("default"))) int bsa_debug_trace_copy(long long* host, int role) {
+    return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * 4096, sizeof(long long) * 4096 * role);
+}
+#endif
+
 cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char** err_detail) {
     AttnParams p;
     p.items = a.items;
@@ -1267,6 +1467,10 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     else if (key == 2000 + 128 + 1) e = launch_attn<128, 64, 2>(a, p, stream, err_detail);
     else if (key == 2000 + 64 + 2) e = launch_attn<64, 128, 2>(a, p, stream, err_detail);
     else if (key == 2000 + 64 + 1) e = launch_attn<64, 64, 2>(a, p, stream, err_detail);
+    else if (key == 3000 + 128 + 2) e = launch_attn<128, 128, 3>(a, p, stream, err_detail);
+    else if (key == 3000 + 128 + 1) e = launch_attn<128, 64, 3>(a, p, stream, err_detail);
+    else if (key == 3000 + 64 + 2) e = launch_attn<64, 128, 3>(a, p, stream, err_detail);
+    else if (key == 3000 + 64 + 1) e = launch_attn<64, 64, 3>(a, p, stream, err_detail);
     else {
         *err_detail = "no kernel for this (d, T_KV)";
         return cudaErrorInvalidValue;

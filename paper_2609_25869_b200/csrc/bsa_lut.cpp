@@ -39,6 +39,11 @@ static const bsa_plan_desc_t kCatalog[] = {
     {15, 128, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 2, "q128k64_cs"},
     {16, 128, 128, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 2, "q128k128_cs_split4x8"},
     {17, 128, 128, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 2, "q128k128_cs_global"},
+    // one 128-row Q tile per CTA, separate issuing threads for Q K^T and P V
+    {18, 128, 128, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 3, "q128k128_di"},
+    {19, 128, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 3, "q128k64_di"},
+    {20, 128, 128, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 3, "q128k128_di_split4x8"},
+    {21, 128, 128, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 3, "q128k128_di_global"},
 };
 static const int kCatalogSize = (int)(sizeof(kCatalog) / sizeof(kCatalog[0]));
 static const int64_t kDefaultWorkspace = 2ll << 30;
@@ -111,7 +116,7 @@ int base_plan(int B_Q, int B_KV, int d) {
     (void)B_Q;
     (void)B_KV;
     (void)d;
-    return 0;  // q128k128: eligible for every supported geometry (membership <= 64 bits), no workspace
+    return 18;  // q128k128_di: eligible for every supported geometry (membership <= 64 bits), no workspace
 }
 
 uint64_t catalog_hash() {

@@ -18,13 +18,13 @@ def _sample(req, per_head, seed=77, heads=None):
 
 
 # ---------------------------------------------------------------- the five configurations
-@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9, 10, 11, 12, 13, 14, 15, 16, 17])
+@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21])
 def test_tiny_full_oracle_every_plan(plan_id):
     res = Hh.run_request(I.config_tiny(), plan_id=plan_id)
     assert res["pairs"] == res["info"]["nnz_blocks"] * 64 * 64
 
 
-@pytest.mark.parametrize("plan_id", [0, 1, 2, 10, 12, 14, 16])
+@pytest.mark.parametrize("plan_id", [0, 1, 2, 10, 12, 14, 16, 18, 20])
 def test_mid_full_oracle(plan_id):
     Hh.run_request(I.config_mid(), plan_id=plan_id)
 
@@ -35,14 +35,14 @@ def test_hunyuan_shaped_sampled_oracle():
     Hh.run_request(req, plan_id=-1, sel=_sample(req, 64), heads=[0, 11, 23])
 
 
-@pytest.mark.parametrize("plan_id", [0, 1, 10, 14])
+@pytest.mark.parametrize("plan_id", [0, 1, 10, 14, 18])
 def test_stress_a_coarsened(plan_id):
     req = I.config_stress_a()
     res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64), heads=[0, 15])
     assert res["info"]["map_q"] == 1  # Coarsened along Q: 8 logical rows of 16 per 128-row tile
 
 
-@pytest.mark.parametrize("plan_id", [0, 1, 10, 11, 14, 15])
+@pytest.mark.parametrize("plan_id", [0, 1, 10, 11, 14, 15, 18, 19])
 def test_stress_b_refined(plan_id):
     req = I.config_stress_b()
     res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64))
@@ -68,6 +68,8 @@ def test_sweep_requests_ragged_n(r, B, rho):
     (128, 128, 129, 64, 10), (64, 64, 300, 128, 13),
     (16, 16, 1000, 64, 14), (32, 64, 777, 128, 15), (64, 32, 1300, 128, 14), (128, 256, 2100, 64, 15),
     (256, 128, 2100, 128, 14), (256, 16, 900, 64, 16), (16, 256, 900, 128, 16), (128, 128, 127, 128, 17),
+    (16, 16, 1000, 64, 18), (32, 64, 777, 128, 19), (64, 32, 1300, 128, 18), (128, 256, 2100, 64, 19),
+    (256, 128, 2100, 128, 18), (256, 16, 900, 64, 20), (16, 256, 900, 128, 20), (128, 128, 127, 128, 21),
 ])
 def test_geometries_with_ragged_tail(B_Q, B_KV, N, d, plan_id):
     H = 3
@@ -89,14 +91,15 @@ def test_degenerate_masks(kind):
     elif kind == "empty_head":
         M[0] = I.random_mask(1, 1, nb, nb, 0.5)[0]
     req = I.Request(kind, H, N, d, B, B, M, qkv_seed=3)
-    for plan_id in (0, 3, 10, 12, 14, 16):
+    for plan_id in (0, 3, 10, 12, 14, 16, 18, 20):
         Hh.run_request(req, plan_id=plan_id)
 
 
 # ---------------------------------------------------------------- closed forms on the GPU path
 @pytest.mark.parametrize("B_Q,B_KV,N,d,plan_id", [(16, 64, 1000, 64, 0), (32, 32, 700, 128, 1), (256, 256, 1100, 128, 9),
                                                   (16, 64, 1000, 64, 10), (64, 32, 700, 128, 11), (256, 256, 1100, 128, 12),
-                                                  (16, 64, 1000, 64, 14), (64, 32, 700, 128, 15), (256, 256, 1100, 128, 16)])
+                                                  (16, 64, 1000, 64, 14), (64, 32, 700, 128, 15), (256, 256, 1100, 128, 16),
+                                                  (16, 64, 1000, 64, 18), (64, 32, 700, 128, 19), (256, 256, 1100, 128, 20)])
 def test_zero_keys_give_log_count_and_mean_value(B_Q, B_KV, N, d, plan_id):
     """K = 0: every score is 0, so LSE = ln(#reachable keys) exactly and O = mean of reachable V.
     Catches any off-by-one in ragged-edge or membership masking (one key off moves LSE by ~1/count)."""

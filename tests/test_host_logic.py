@@ -39,7 +39,7 @@ def test_catalog_and_eligibility():
     assert len(cat) >= 6 and [c["plan_id"] for c in cat] == list(range(len(cat)))
     assert len(set(c["name"] for c in cat)) == len(cat)
     assert {c["T_KV"] for c in cat} == {64, 128} and {c["T_Q"] for c in cat} == {128, 256}
-    assert {c["kernel"] for c in cat} == {0, 1, 2}
+    assert {c["kernel"] for c in cat} == {0, 1, 2, 3}
     base = bsa.lib().bsa_base_plan(128, 128, 128)
     # the base plan is eligible for every supported request key
     for B_Q in (16, 32, 64, 128, 256):
@@ -79,7 +79,8 @@ def test_plan_table_lookup_matches_algorithm_2(tmp_path):
     _write_lut(p, regimes)
     bsa.lut_load(p)
     assert bsa.lib().bsa_lut_num_regimes() == 2
-    base = {("k64",): 0}
+    BASE = bsa.lib().bsa_base_plan(64, 64, 64)
+    base = {("k64",): BASE}
     # hit: first eligible plan of the ranking
     pid, hit = bsa.lut_select(64, 64, 2048, 2, 64, 0.27, 0.4, 1.6)
     assert (pid, hit) == (3, True)
@@ -87,17 +88,17 @@ def test_plan_table_lookup_matches_algorithm_2(tmp_path):
     # ranked fallback: plan 2 is not eligible (workspace over the default limit) -> next in rank order
     pid, hit = bsa.lut_select(128, 128, 115200, 24, 128, 0.066, 0.9, 1.2)
     assert (pid, hit) == (1, True)
-    assert pid == oracle.select_plan({(("k",), "b"): [2, 1, 0]}, {("k",): 0}, ("k",), "b", lambda q: q != 2)
+    assert pid == oracle.select_plan({(("k",), "b"): [2, 1, 0]}, {("k",): BASE}, ("k",), "b", lambda q: q != 2)
     # miss: the base plan alone
     pid, hit = bsa.lut_select(64, 64, 2048, 2, 64, 0.01, 0.4, 1.6)
-    assert (pid, hit) == (0, False)
+    assert (pid, hit) == (BASE, False)
     assert pid == oracle.select_plan({}, base, ("k64",), "other", lambda q: True)
     # nothing eligible -> no-eligible-plan
     pid, hit = bsa.lut_select(64, 64, 2048, 2, 96, 0.27, 0.4, 1.6)
     assert pid == -1
     assert oracle.select_plan({}, base, ("k64",), "other", lambda q: False) is None
     bsa.lut_clear()
-    assert bsa.lut_select(64, 64, 2048, 2, 64, 0.27, 0.4, 1.6) == (0, False)
+    assert bsa.lut_select(64, 64, 2048, 2, 64, 0.27, 0.4, 1.6) == (BASE, False)
 
 
 def test_plan_table_rejects_foreign_or_malformed_files(tmp_path):
