@@ -153,6 +153,64 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Dynamic-request sweep: every request is cold (new mask): latency = plan build + lookup + forward.
+    Reports per-request host latency and its planning share; one JSON line."""
+    import numpy as np
+    import torch
+    from paper_2609_25869_b200 import bsa, inputs as I
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    bsa.lib()
+    peaks = load_peaks()
+    rows = []
+    qkv = None
+    for r in range(args.sweep_requests):
+        req = I.config_sweep(r, H=args.sweep_heads)
+        if qkv is None:
+            qkv = tuple(t.cuda() for t in req.qkv())  # tensors are reused; only the mask changes per request
+        q, k, v = qkv
+        mask = torch.from_numpy(req.mask).cuda()
+        O = torch.empty_like(q)
+        L = torch.empty((req.H, req.N), dtype=torch.float32, device="cuda")
+        pairs = count_active_pairs(req)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        plan = bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d)
+        t1 = time.perf_counter()
+        plan.forward(q, k, v, O, L)
+        torch.cuda.synchronize()
+        t2 = time.perf_counter()
+        ts = []
+        for _ in range(3):  # warm exact repeats (prepared plan reused)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            plan.forward(q, k, v, O, L)
+            b.record()
+            b.synchronize()
+            ts.append(a.elapsed_time(b))
+        inf = plan.info()
+        assert inf["device_status"] == 0
+        plan.destroy()
+        kern_ms = statistics.median(ts)
+        rows.append({"r": r, "B": [req.B_Q, req.B_KV], "density": round(inf["density"], 4), "skew": round(inf["skew"], 2),
+                     "plan": inf["plan"]["name"], "lut_hit": inf["lut_hit"], "cold_request_us": (t2 - t0) * 1e6,
+                     "plan_create_us": (t1 - t0) * 1e6, "lookup_us": inf["us_lookup"], "warm_forward_us": kern_ms * 1e3,
+                     "tflops_warm": 4.0 * req.d * pairs / (kern_ms * 1e-3) / 1e12})
+    cold = [x["cold_request_us"] for x in rows]
+    plan_frac = [x["plan_create_us"] / x["cold_request_us"] for x in rows]
+    line = {"metric": "per-request us incl. planning (cold unique requests), dynamic-request sweep", "unit": "us",
+            "value": statistics.mean(cold), "p50": statistics.median(cold), "p95": sorted(cold)[int(0.95 * (len(cold) - 1))],
+            "higher_is_better": False, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"sweep: {len(rows)} requests, heads={args.sweep_heads} N=75600 d=128, B and density drawn per request"},
+            "plan_create_us_mean": statistics.mean(x["plan_create_us"] for x in rows),
+            "lookup_us_mean": statistics.mean(x["lookup_us"] for x in rows),
+            "planning_fraction_mean": statistics.mean(plan_frac), "planning_fraction_max": max(plan_frac),
+            "tflops_warm_mean": statistics.mean(x["tflops_warm"] for x in rows),
+            "frac_of_peak_warm_mean": statistics.mean(x["tflops_warm"] for x in rows) / peaks["bf16_tflops"],
+            "lut_hits": sum(x["lut_hit"] for x in rows), "requests": rows}
+    print(json.dumps(line), flush=True)
+
+
 def workload_config(req, name):
     return {"workload": f"{name}: heads={req.H} N={req.N} d={req.d} B=({req.B_Q},{req.B_KV}) {req.note}",
             "l2": "256 MiB buffer written between timed iterations (L2 flush)"}
@@ -166,15 +224,20 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="mid")
     ap.add_argument("--plan", type=int, default=-1, help="force a catalog plan id (-1: Algorithm 2)")
-    ap.add_argument("--lut", default=os.path.join(ROOT, "paper_2609_25869_b200", "plan_table_b200.lut"))
+    ap.add_argument("--lut", default="", help="plan table to load instead of the packaged one")
     ap.add_argument("--ref-blocks", type=int, default=256, help="query blocks per reference step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extra", default="", help="comma list of extra workloads reported under 'others'")
+    ap.add_argument("--sweep-requests", type=int, default=50)
+    ap.add_argument("--sweep-heads", type=int, default=24)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.workload == "sweep":
+        run_sweep(args)
         return
 
     import torch
@@ -187,9 +250,10 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    bsa.lib()  # fail loudly if the CUDA library is missing
-    if os.path.exists(args.lut):
+    bsa.lib()  # fail loudly if the CUDA library is missing; loads the packaged plan table if it matches the catalog
+    if args.lut:
         bsa.lut_load(args.lut)
+    lut_regimes = int(bsa.lib().bsa_lut_num_regimes())
     peaks = load_peaks()
 
     def barrier():
@@ -312,7 +376,8 @@ def main():
                     "us_mask_state": inf["us_mask_state"], "us_stats_sync": inf["us_stats_sync"],
                     "us_lookup": inf["us_lookup"], "us_launch_prep": inf["us_launch_prep"],
                     "planning_fraction": max(0.0, 1.0 - kernel_ms / step_ms),
-                    "plan": inf["plan"]["name"], "lut_hit": inf["lut_hit"], "ntiles": inf["ntiles"],
+                    "plan": inf["plan"]["name"], "lut_hit": inf["lut_hit"], "lut_regimes": lut_regimes,
+                    "ntiles": inf["ntiles"],
                     "nitems": inf["nitems"], "active_pairs": r["pairs"], "covered_pairs": inf["covered_pairs"],
                     "density": inf["density"]},
     }

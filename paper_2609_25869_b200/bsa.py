@@ -101,7 +101,19 @@ def lib() -> ctypes.CDLL:
     L.bsa_version.restype = ctypes.c_char_p
     L.bsa_kernel_launch_count.restype = i64
     _lib = L
+    load_default_table()
     return L
+
+
+DEFAULT_TABLE = os.path.join(_HERE, "plan_table_b200.lut")
+
+
+def load_default_table() -> bool:
+    """Load the plan table shipped with the package (written by ``lut_build.py`` on a B200).  A table built
+    for another catalog is rejected by the library; base plans are used then.  Returns True if loaded."""
+    if _lib is None or not os.path.exists(DEFAULT_TABLE):
+        return False
+    return _lib.bsa_lut_load(DEFAULT_TABLE.encode()) == BSA_OK
 
 
 class BsaError(RuntimeError):

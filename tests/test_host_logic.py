@@ -133,3 +133,33 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(bsa, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         bsa.lib()
+
+
+def test_offline_table_compilation_matches_algorithm_1(tmp_path):
+    """lut_build.compile_table (product) against the oracle's restatement of Algorithm 1, and the
+    written file loads back into the runtime with the same rankings."""
+    from paper_2609_25869_b200 import lut_build
+    import random
+    rnd = random.Random(3)
+    keys = [(128, 128, 128), (64, 64, 64)]
+    cases, lat, bucket = [], {}, {}
+    for n in range(24):
+        key = keys[n % 2]
+        cid = f"case{n}"
+        cases.append((cid, key))
+        bucket[cid] = (14, 1, n % 3, 0, 1)
+        for pid in range(6):
+            if rnd.random() < 0.15:
+                continue  # failed validation / not eligible on this case
+            lat[(cid, pid)] = rnd.choice([1.0, 2.0, 4.0]) * (1 + (pid == 3))
+    base = {keys[0]: 0, keys[1]: 1}
+    got = lut_build.compile_table(cases, lat, base, bucket.get)
+    want = oracle.compile_table(cases, lat, base, bucket.get)
+    assert got == want and len(got) >= 4
+    for ranked in got.values():
+        assert ranked[-1] in (0, 1) and len(set(ranked[:-1])) == len(ranked) - 1
+    path = str(tmp_path / "t.lut")
+    lut_build.write_table(path, got, int(bsa.lib().bsa_catalog_hash()), "test-gpu")
+    bsa.lut_load(path)
+    assert bsa.lib().bsa_lut_num_regimes() == len(got)
+    bsa.lut_clear()
