@@ -125,6 +125,21 @@ extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int
     p->d = d;
     BSA_CUDA(cudaGetDevice(&p->device), "cudaGetDevice");
     BSA_CUDA(cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, p->device), "device attribute");
+    {
+        // Plans are created and destroyed per request: keep freed arena memory in this process's default
+        // stream-ordered pool instead of handing it back to the driver at every synchronisation (the
+        // default threshold of 0 makes each larger request pay a fresh driver allocation, 10-80 ms).
+        static std::atomic<unsigned long long> pool_ready_mask{0};
+        const unsigned long long bit = 1ull << (p->device & 63);
+        if (!(pool_ready_mask.load(std::memory_order_relaxed) & bit)) {
+            cudaMemPool_t pool;
+            if (cudaDeviceGetDefaultMemPool(&pool, p->device) == cudaSuccess) {
+                unsigned long long keep = ~0ull;
+                cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+            }
+            pool_ready_mask.fetch_or(bit, std::memory_order_relaxed);
+        }
+    }
 
     const int nQb = (int)((N + B_Q - 1) / B_Q), nKb = (int)((N + B_KV - 1) / B_KV);
     const int64_t nrows64 = (int64_t)heads * nQb;

@@ -19,6 +19,31 @@ namespace {
 constexpr unsigned kFull = 0xffffffffu;
 
 // ------------------------------------------------------------------------------------------
+// Both mask passes read a row as aligned 16-byte words, one word per lane and step (512 bytes per
+// warp step); bytes of a word that fall outside the row are masked off.  `row_word_bits` returns,
+// for the word at index `w` (in 16-byte units of the flat mask array), a 16-bit mask of the bytes
+// that belong to [row_begin, row_end) and are non-zero.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned row_word_bits(const uint4* __restrict__ words, long long w, long long row_begin,
+                                                  long long row_end) {
+    const long long byte0 = w * 16;
+    if (byte0 >= row_end || byte0 + 16 <= row_begin) return 0u;
+    const uint4 v = __ldg(words + w);
+    unsigned bits = 0;
+    const unsigned parts[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const unsigned ne = __vcmpne4(parts[q], 0u);  // 0xff per non-zero byte
+        bits |= ((ne & 1u) | ((ne >> 7) & 2u) | ((ne >> 14) & 4u) | ((ne >> 21) & 8u)) << (4 * q);
+    }
+    // keep only the bytes inside the row
+    const int lo = row_begin > byte0 ? (int)(row_begin - byte0) : 0;
+    const int hi = row_end < byte0 + 16 ? (int)(row_end - byte0) : 16;
+    const unsigned keep = (hi >= 16 ? 0xffffu : ((1u << hi) - 1u)) & ~((1u << lo) - 1u);
+    return bits & keep;
+}
+
+// ------------------------------------------------------------------------------------------
 // mask_row_stats: one warp per (head, query-block) row.
 // A block counts towards run coverage iff its left or right neighbour in the same row is active.
 // ------------------------------------------------------------------------------------------
@@ -29,17 +54,27 @@ __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __re
     const int row = blockIdx.x * 8 + warp;
     unsigned nnz = 0, runs = 0;
     if (row < nrows) {
-        const uint8_t* m = mask + (size_t)row * nKb;
-        for (int j0 = 0; j0 < nKb; j0 += 32) {
-            const int j = j0 + lane;
-            const bool a = (j < nKb) && m[j] != 0;
-            const unsigned bits = __ballot_sync(kFull, a);
-            unsigned left = bits << 1, right = bits >> 1;
-            // neighbours across the 32-block chunk boundary (same row only)
-            if (j0 > 0 && m[j0 - 1] != 0) left |= 1u;
-            if (j0 + 32 < nKb && m[j0 + 32] != 0) right |= 0x80000000u;
-            nnz += __popc(bits);
-            runs += __popc(bits & (left | right));
+        // the mask base may be unaligned: address words relative to the enclosing 16-byte grid
+        const unsigned long long base = reinterpret_cast<unsigned long long>(mask);
+        const uint4* words = reinterpret_cast<const uint4*>(base & ~15ull);
+        const long long rb = (long long)(base & 15ull) + (long long)row * nKb, re = rb + nKb;
+        const long long w0 = rb >> 4, w1 = (re + 15) >> 4;
+        unsigned carry = 0;  // last byte of the previous step (bit 0)
+        for (long long w = w0; w < w1; w += 32) {
+            const unsigned m = row_word_bits(words, w + lane, rb, re);
+            // neighbours across lanes: previous lane's bit 15, next lane's bit 0
+            unsigned prev15 = __shfl_up_sync(kFull, m >> 15, 1);
+            unsigned next0 = __shfl_down_sync(kFull, m & 1u, 1);
+            if (lane == 0) prev15 = carry;
+            if (lane == 31) next0 = (w + 32 < w1) ? (row_word_bits(words, w + 32, rb, re) & 1u) : 0u;
+            const unsigned left = ((m << 1) | prev15) & 0xffffu, right = (m >> 1) | (next0 << 15);
+            nnz += __popc(m);
+            runs += __popc(m & (left | right));
+            carry = __shfl_sync(kFull, m >> 15, 31);
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            nnz += __shfl_down_sync(kFull, nnz, o);
+            runs += __shfl_down_sync(kFull, runs, o);
         }
         if (lane == 0) row_nnz[row] = (int32_t)nnz;
     }
@@ -104,7 +139,7 @@ __global__ void __launch_bounds__(1024) row_scan_kernel(const int32_t* __restric
 }
 
 // ------------------------------------------------------------------------------------------
-// csr_fill: one warp per row, ballot compaction keeps columns ascending.
+// csr_fill: one warp per row; a warp scan over the lanes' popcounts keeps columns ascending.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) csr_fill_kernel(const uint8_t* __restrict__ mask, int nrows, int nKb,
                                                         const int32_t* __restrict__ row_ptr,
@@ -112,14 +147,27 @@ __global__ void __launch_bounds__(256) csr_fill_kernel(const uint8_t* __restrict
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row = blockIdx.x * 8 + warp;
     if (row >= nrows) return;
-    const uint8_t* m = mask + (size_t)row * nKb;
+    const unsigned long long base = reinterpret_cast<unsigned long long>(mask);
+    const uint4* words = reinterpret_cast<const uint4*>(base & ~15ull);
+    const long long rb = (long long)(base & 15ull) + (long long)row * nKb, re = rb + nKb;
+    const long long w0 = rb >> 4, w1 = (re + 15) >> 4;
     int32_t out = row_ptr[row];
-    for (int j0 = 0; j0 < nKb; j0 += 32) {
-        const int j = j0 + lane;
-        const bool a = (j < nKb) && m[j] != 0;
-        const unsigned bits = __ballot_sync(kFull, a);
-        if (a) col_idx[out + __popc(bits & ((1u << lane) - 1u))] = j;
-        out += __popc(bits);
+    for (long long w = w0; w < w1; w += 32) {
+        unsigned m = row_word_bits(words, w + lane, rb, re);
+        const int cnt = __popc(m);
+        int incl = cnt;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int x = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl += x;
+        }
+        int pos = out + incl - cnt;
+        const int col0 = (int)((w + lane) * 16 - rb);  // column of this word's byte 0
+        while (m) {
+            const int b = __ffs(m) - 1;
+            col_idx[pos++] = col0 + b;
+            m &= m - 1;
+        }
+        out += __shfl_sync(kFull, incl, 31);
     }
 }
 
