@@ -106,36 +106,29 @@ __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __re
 __global__ void __launch_bounds__(1024) row_scan_kernel(const int32_t* __restrict__ row_nnz, int nrows,
                                                         int32_t* __restrict__ row_ptr) {
     __shared__ int32_t warp_sums[32];
-    __shared__ int32_t carry_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int per = (nrows + 1023) / 1024;
-    const int b = tid * per, e = min(nrows, b + per);
-    int32_t sum = 0;
-    for (int i = b; i < e; ++i) sum += row_nnz[i];
-    int32_t incl = sum;
-    for (int o = 1; o < 32; o <<= 1) {
-        int32_t v = __shfl_up_sync(kFull, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) warp_sums[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        int32_t w = warp_sums[lane];
-        int32_t wi = w;
+    int32_t carry = 0;  // sum of all rows before this step (same value in every thread)
+    for (int i0 = 0; i0 < nrows; i0 += 1024) {
+        const int i = i0 + tid;  // consecutive threads read consecutive rows
+        const int32_t v = (i < nrows) ? row_nnz[i] : 0;
+        int32_t incl = v;
         for (int o = 1; o < 32; o <<= 1) {
-            int32_t v = __shfl_up_sync(kFull, wi, o);
-            if (lane >= o) wi += v;
+            const int32_t x = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl += x;
         }
-        warp_sums[lane] = wi - w;
-        if (lane == 31) carry_s = wi;
+        __syncthreads();  // warp_sums of the previous step have been consumed
+        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();
+        int32_t before = 0, total = 0;
+        for (int k = 0; k < 32; ++k) {
+            const int32_t ws = warp_sums[k];
+            if (k < warp) before += ws;
+            total += ws;
+        }
+        if (i < nrows) row_ptr[i] = carry + before + incl - v;
+        carry += total;
     }
-    __syncthreads();
-    int32_t run = warp_sums[warp] + incl - sum;
-    for (int i = b; i < e; ++i) {
-        row_ptr[i] = run;
-        run += row_nnz[i];
-    }
-    if (tid == 0) row_ptr[nrows] = carry_s;
+    if (tid == 0) row_ptr[nrows] = carry;
 }
 
 // ------------------------------------------------------------------------------------------
