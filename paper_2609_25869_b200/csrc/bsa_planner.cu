@@ -105,28 +105,50 @@ __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __re
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) row_scan_kernel(const int32_t* __restrict__ row_nnz, int nrows,
                                                         int32_t* __restrict__ row_ptr) {
-    __shared__ int32_t warp_sums[32];
+    __shared__ int32_t warp_excl[32];
+    __shared__ int32_t step_total;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t carry = 0;  // sum of all rows before this step (same value in every thread)
-    for (int i0 = 0; i0 < nrows; i0 += 1024) {
-        const int i = i0 + tid;  // consecutive threads read consecutive rows
-        const int32_t v = (i < nrows) ? row_nnz[i] : 0;
-        int32_t incl = v;
+    for (int i0 = 0; i0 < nrows; i0 += 4096) {
+        const int i = i0 + tid * 4;  // four consecutive rows per thread, 16-byte accesses
+        int4 v = make_int4(0, 0, 0, 0);
+        if (i + 3 < nrows) {
+            v = *reinterpret_cast<const int4*>(row_nnz + i);
+        } else {
+            if (i < nrows) v.x = row_nnz[i];
+            if (i + 1 < nrows) v.y = row_nnz[i + 1];
+            if (i + 2 < nrows) v.z = row_nnz[i + 2];
+        }
+        const int32_t t = v.x + v.y + v.z + v.w;
+        int32_t incl = t;
         for (int o = 1; o < 32; o <<= 1) {
             const int32_t x = __shfl_up_sync(kFull, incl, o);
             if (lane >= o) incl += x;
         }
-        __syncthreads();  // warp_sums of the previous step have been consumed
-        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();  // the previous step's warp_excl / step_total have been consumed
+        if (lane == 31) warp_excl[warp] = incl;
         __syncthreads();
-        int32_t before = 0, total = 0;
-        for (int k = 0; k < 32; ++k) {
-            const int32_t ws = warp_sums[k];
-            if (k < warp) before += ws;
-            total += ws;
+        if (warp == 0) {
+            const int32_t w = warp_excl[lane];
+            int32_t wi = w;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t x = __shfl_up_sync(kFull, wi, o);
+                if (lane >= o) wi += x;
+            }
+            warp_excl[lane] = wi - w;
+            if (lane == 31) step_total = wi;
         }
-        if (i < nrows) row_ptr[i] = carry + before + incl - v;
-        carry += total;
+        __syncthreads();
+        const int32_t base = carry + warp_excl[warp] + incl - t;
+        const int4 o4 = make_int4(base, base + v.x, base + v.x + v.y, base + v.x + v.y + v.z);
+        if (i + 3 < nrows) {
+            *reinterpret_cast<int4*>(row_ptr + i) = o4;
+        } else {
+            if (i < nrows) row_ptr[i] = o4.x;
+            if (i + 1 < nrows) row_ptr[i + 1] = o4.y;
+            if (i + 2 < nrows) row_ptr[i + 2] = o4.z;
+        }
+        carry += step_total;
     }
     if (tid == 0) row_ptr[nrows] = carry;
 }
