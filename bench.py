@@ -211,6 +211,24 @@ def run_sweep(args):
     print(json.dumps(line), flush=True)
 
 
+def aggregate_over_ranks(step_ms: float, flops_per_rank: float, dist=None, device="cuda"):
+    """Weak scaling by replication: every rank runs its own request, no data-path collective.
+    The job's time is the MAX over ranks; the job's work is the SUM.  Returns (max_ms, total TFLOP/s)."""
+    world = 1
+    if dist is not None and dist.is_initialized():
+        import torch
+        world = dist.get_world_size()
+        t = torch.tensor([step_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        step_ms = float(t.item())
+        f = torch.tensor([flops_per_rank], dtype=torch.float64, device=device)
+        dist.all_reduce(f, op=dist.ReduceOp.SUM)
+        total = float(f.item())
+    else:
+        total = flops_per_rank
+    return step_ms, total / (step_ms * 1e-3) / 1e12, world
+
+
 def workload_config(req, name):
     return {"workload": f"{name}: heads={req.H} N={req.N} d={req.d} B=({req.B_Q},{req.B_KV}) {req.note}",
             "l2": "256 MiB buffer written between timed iterations (L2 flush)"}
@@ -350,10 +368,9 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    step_ms = maxr(r["step_ms"])
+    step_ms, value, _ = aggregate_over_ranks(r["step_ms"], r["flops"], dist)
     kernel_ms = maxr(r["kernel_ms"])
     e2e_s = maxr(r["e2e_s"])
-    value = world * r["flops"] / (step_ms * 1e-3) / 1e12
     kernel_tflops = r["flops"] / (kernel_ms * 1e-3) / 1e12
     inf = r["info"]
     line = {
