@@ -26,7 +26,7 @@ using namespace ptx;
 // Optional timeline tracing (compile with -DBSA_TRACE): CTA 0 records clock64() at barrier events of the
 // single-tile kernel, per role, into a device buffer that bsa_debug_trace_copy() reads back.
 #ifdef BSA_TRACE
-__device__ long long g_trace[6][4096];  // producer, MMA issuer, softmax warps 0-3
+__device__ long long g_trace[7][4096];  // producer, MMA (or Q K^T) issuer, softmax warps 0-3, P V issuer
 __device__ long long g_trace_aux[12][4];  // last tile's stamps inside softmax_tile, per warp
 #define BSA_TRACE_DECL(n) int n = 0
 #define BSA_TRACE_POINT(role, n, tag)                                              \
@@ -331,6 +331,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
             uint32_t itq = 0, g = 0;
             bool ok = true;
+            BSA_TRACE_DECL(tn);
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
                 const int n = p.items[idx].ntiles;
                 if (n == 0) continue;
@@ -342,6 +343,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
                     ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
                     if (!ok) break;
+                    BSA_TRACE_POINT(1, tn, 1);
                     // S[sb] still holds P of tile gs-2 (written in place) until that tile's P V has completed.
                     // (Measured: giving P its own columns so that Q K^T may start right after the softmax of
                     // tile gs-2 was slower -- the early Q K^T delays the P V the softmax chain is waiting for.)
@@ -349,6 +351,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         ok = mbar_wait(smem_u32(&bars.pv_done[sb]), ((gs >> 1) - 1) & 1, abortp);
                         if (!ok) break;
                     }
+                    BSA_TRACE_POINT(1, tn, 6);
                     tc_fence_after();
                     const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
 #pragma unroll
@@ -359,6 +362,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     }
                     mma_commit(smem_u32(&bars.k_empty[stage]));
                     mma_commit(smem_u32(&bars.s_full[sb]));
+                    BSA_TRACE_POINT(1, tn, 2);
                     if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
                 }
                 g += n;
@@ -372,6 +376,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
             uint32_t itq = 0, g = 0;
             bool ok = true;
+            BSA_TRACE_DECL(tn);
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
                 const int n = p.items[idx].ntiles;
                 if (n == 0) continue;
@@ -381,6 +386,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
                     ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
                     if (!ok) break;
+                    BSA_TRACE_POINT(6, tn, 3);
                     ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
                     if (!ok) break;
                     if (j == 0) {
@@ -396,6 +402,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     }
                     mma_commit(smem_u32(&bars.v_empty[stage]));
                     mma_commit(smem_u32(&bars.pv_done[sb]));
+                    BSA_TRACE_POINT(6, tn, 5);
                 }
                 g += n;
                 ++itq;
@@ -543,7 +550,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 // warp alternates between the slots (PV of the previous tile, then Q K^T of the next), so one
 // slot's softmax runs under the other slot's MMAs.
 //   warps 0-3 / 4-7 : softmax + correction + epilogue of slot 0 / slot 1 (more registers)
-//   warp 8          : TMA producer          warp 9 : MMA issuer (both give registers back)
+//   warp 8          : TMA producer    warp 9 : Q K^T issuer    warp 10 : P V issuer (this warpgroup gives registers back)
 // Register budget: 384 threads launch with 168 registers each (504 per lane across the three
 // warpgroups); setmaxnreg moves them to 216 + 216 + 72 = 504.  The sum must not exceed the launch
 // allocation, otherwise the second setmaxnreg.inc never gets its registers and the CTA stalls.
@@ -667,48 +674,19 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
                 while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
             }
         } else if (warp == 9 && lane == 0) {
-            // =========================== MMA issuer ===========================
+            // =========================== Q K^T issuer (both slots) ===========================
             constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
-            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
             const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
             const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
-            const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
             uint32_t itq = 0, g = 0;
-            uint32_t npv[2] = {0, 0};  // PV MMAs issued per slot: phase of p_ready / pv_done
-            uint32_t oit[2] = {0, 0};  // items in which the slot had tiles: phase of o_free
-            int pend[2] = {-1, -1};    // global tile index whose PV is still to be issued, or -1
-            bool started[2] = {false, false};
+            uint32_t nqk[2] = {0, 0};  // Q K^T tiles issued per slot
             bool ok = true;
-            // PV of slot x for its pending tile: O_x (+)= P_x V
-            auto issue_pv = [&](int x) -> bool {
-                const uint32_t gp = (uint32_t)pend[x];
-                const int sv = gp % NSV;
-                if (!mbar_wait(smem_u32(&bars.p_ready[x]), npv[x] & 1, abortp)) return false;
-                if (!mbar_wait(smem_u32(&bars.v_full[sv]), (gp / NSV) & 1, abortp)) return false;
-                if (!started[x] && !mbar_wait(smem_u32(&bars.o_free[x]), (oit[x] & 1) ^ 1, abortp)) return false;
-                tc_fence_after();
-                const uint32_t d_o = tmem + kColO + x * 128, a_p = tmem + x * 128;
-#pragma unroll
-                for (int k = 0; k < TK / 16; ++k) {
-                    const uint64_t b = descV + (uint64_t)((sv * KV_TILE + k * 2048) >> 4);
-                    mma_ts(d_o, a_p + k * 8, b, idesc_pv, (started[x] || k > 0) ? 1u : 0u);
-                }
-                // the V stage is free once the last slot that uses this tile has issued its PV
-                if (!(x == 0 && pend[1] == pend[0])) mma_commit(smem_u32(&bars.v_empty[sv]));
-                mma_commit(smem_u32(&bars.pv_done[x]));
-                ++npv[x];
-                started[x] = true;
-                pend[x] = -1;
-                return true;
-            };
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
                 const WorkItem it = p.items[idx];
                 const int n = it.ntiles;
                 if (n == 0) continue;
                 ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
                 if (!ok) break;
-                pend[0] = pend[1] = -1;
-                started[0] = started[1] = false;
                 ulonglong2 mem_next = *reinterpret_cast<const ulonglong2*>(p.tile_member + (size_t)it.tile_begin * 2);
                 for (int j = 0; j < n && ok; ++j) {
                     const uint32_t gj = g + j;
@@ -716,42 +694,84 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
                     const ulonglong2 mem = mem_next;
                     if (j + 1 < n)
                         mem_next = *reinterpret_cast<const ulonglong2*>(p.tile_member + (size_t)(it.tile_begin + j + 1) * 2);
-                    bool k_waited = false;
+                    ok = mbar_wait(smem_u32(&bars.k_full[sk]), (gj / NSK) & 1, abortp);
+                    if (!ok) break;
 #pragma unroll
                     for (int x = 0; x < 2; ++x) {
-                        if (pend[x] >= 0) {
-                            ok = issue_pv(x);
+                        if ((x == 0 ? mem.x : mem.y) == 0ull) continue;
+                        // S_x holds the bf16 P of the slot's previous tile until that tile's P V has completed
+                        if (nqk[x] >= 1) {
+                            ok = mbar_wait(smem_u32(&bars.pv_done[x]), (nqk[x] - 1) & 1, abortp);
                             if (!ok) break;
                         }
-                        if ((x == 0 ? mem.x : mem.y) != 0ull) {
-                            if (!k_waited) {
-                                ok = mbar_wait(smem_u32(&bars.k_full[sk]), (gj / NSK) & 1, abortp);
-                                if (!ok) break;
-                                k_waited = true;
-                            }
-                            tc_fence_after();
-                            const uint32_t d_s = tmem + x * 128;
+                        tc_fence_after();
+                        const uint32_t d_s = tmem + x * 128;
 #pragma unroll
-                            for (int k = 0; k < D / 16; ++k) {
-                                const uint64_t a = descQ + (uint64_t)((x * Q_TILE + (k / 4) * Q_SUB + (k % 4) * 32) >> 4);
-                                const uint64_t b = descK + (uint64_t)((sk * KV_TILE + (k / 4) * KV_SUB + (k % 4) * 32) >> 4);
-                                mma_ss(d_s, a, b, idesc_qk, k > 0);
-                            }
-                            mma_commit(smem_u32(&bars.s_full[x]));
-                            pend[x] = (int)gj;
+                        for (int k = 0; k < D / 16; ++k) {
+                            const uint64_t a = descQ + (uint64_t)((x * Q_TILE + (k / 4) * Q_SUB + (k % 4) * 32) >> 4);
+                            const uint64_t b = descK + (uint64_t)((sk * KV_TILE + (k / 4) * KV_SUB + (k % 4) * 32) >> 4);
+                            mma_ss(d_s, a, b, idesc_qk, k > 0);
                         }
+                        mma_commit(smem_u32(&bars.s_full[x]));
+                        ++nqk[x];
                     }
                     if (!ok) break;
                     mma_commit(smem_u32(&bars.k_empty[sk]));
                 }
                 if (!ok) break;
                 mma_commit(smem_u32(&bars.q_empty));
-                for (int x = 0; x < 2 && ok; ++x)
-                    if (pend[x] >= 0) ok = issue_pv(x);
+                g += n;
+                ++itq;
+            }
+        } else if (warp == 10 && lane == 0) {
+            // =========================== P V issuer (both slots) ===========================
+            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
+            uint32_t g = 0;
+            uint32_t npv[2] = {0, 0};  // P V tiles issued per slot: phase of p_ready / pv_done
+            uint32_t oit[2] = {0, 0};  // items in which the slot had tiles: phase of o_free
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const WorkItem it = p.items[idx];
+                const int n = it.ntiles;
+                if (n == 0) continue;
+                bool started[2] = {false, false};
+                ulonglong2 mem_next = *reinterpret_cast<const ulonglong2*>(p.tile_member + (size_t)it.tile_begin * 2);
+                for (int j = 0; j < n && ok; ++j) {
+                    const uint32_t gj = g + j;
+                    const int sv = gj % NSV;
+                    const ulonglong2 mem = mem_next;
+                    if (j + 1 < n)
+                        mem_next = *reinterpret_cast<const ulonglong2*>(p.tile_member + (size_t)(it.tile_begin + j + 1) * 2);
+                    ok = mbar_wait(smem_u32(&bars.v_full[sv]), (gj / NSV) & 1, abortp);
+                    if (!ok) break;
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        if ((x == 0 ? mem.x : mem.y) == 0ull) continue;
+                        ok = mbar_wait(smem_u32(&bars.p_ready[x]), npv[x] & 1, abortp);
+                        if (!ok) break;
+                        if (!started[x]) {
+                            ok = mbar_wait(smem_u32(&bars.o_free[x]), (oit[x] & 1) ^ 1, abortp);
+                            if (!ok) break;
+                        }
+                        tc_fence_after();
+                        const uint32_t d_o = tmem + kColO + x * 128, a_p = tmem + x * 128;
+#pragma unroll
+                        for (int k = 0; k < TK / 16; ++k) {
+                            const uint64_t b = descV + (uint64_t)((sv * KV_TILE + k * 2048) >> 4);
+                            mma_ts(d_o, a_p + k * 8, b, idesc_pv, (started[x] || k > 0) ? 1u : 0u);
+                        }
+                        mma_commit(smem_u32(&bars.pv_done[x]));
+                        ++npv[x];
+                        started[x] = true;
+                    }
+                    if (!ok) break;
+                    mma_commit(smem_u32(&bars.v_empty[sv]));
+                }
+                if (!ok) break;
                 for (int x = 0; x < 2; ++x)
                     if (started[x]) ++oit[x];
                 g += n;
-                ++itq;
             }
         }
     } else {
@@ -1024,10 +1044,12 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
                     ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
                     if (!ok) break;
-                    // S[sb] was last read by the softmax of tile gs-2; P lives in its own columns, so the
-                    // buffer is free as soon as that softmax has arrived on p_ready
+                    // S[sb] was last read by the softmax of tile gs-2.  P lives in its own columns, so Q K^T could
+                    // start as soon as that softmax has arrived on p_ready, but issuing it ahead of the P V of
+                    // tile gs-2 delays the P V the softmax chain waits for (measured slower): keep the order
+                    // P V (gs-2) -> Q K^T (gs)
                     if (gs >= 2) {
-                        ok = mbar_wait(smem_u32(&bars.p_ready[sb]), ((gs >> 1) - 1) & 1, abortp);
+                        ok = mbar_wait(smem_u32(&bars.pv_done[sb]), ((gs >> 1) - 1) & 1, abortp);
                         if (!ok) break;
                     }
                     tc_fence_after();
