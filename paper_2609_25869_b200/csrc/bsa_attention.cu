@@ -1294,6 +1294,427 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
+// ==========================================================================================
+// Ping-pong kernel: one 128-row Q tile per CTA, TWO softmax warpgroups that take alternate KV
+// tiles (warpgroup x owns the tiles whose running index has parity x, and with them S buffer x
+// and P buffer x).  While one warpgroup is in its exponential phase the other loads its scores,
+// finds its row maxima and waits for nothing but the previous tile's reference maximum, so the
+// XU pipe and the tensor pipe both stay fed.  One O accumulator is shared: both warpgroups
+// follow the SAME reference maximum per row, handed from tile to tile through shared memory
+// (`mref`, one float per row, published right after a tile's max phase).  Each warpgroup keeps a
+// partial row sum, converted whenever the reference it last saw has moved; the sums are added in
+// the epilogue.  P has its own TMEM columns, so S[x] is free again as soon as warpgroup x has
+// read it into registers (`s_free`).
+//   warps 0-3 / 4-7 : softmax warpgroups 0 / 1      warp 8 : TMA producer
+//   warp 9 : Q K^T issuer      warp 10 : P V issuer  (warps 8-11 give registers back)
+// TMEM columns: S0 0, S1 128, O 256, P0 384, P1 448.
+// ==========================================================================================
+constexpr int kPpThreads = 384;
+
+struct __align__(8) PpBarriers {
+    uint64_t q_full, q_empty, o_free, l_bar;
+    uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
+    uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2], mx_bar[2];
+};
+
+template <int D, int TK>
+__global__ void __launch_bounds__(kPpThreads, 1)
+bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                        const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+    constexpr int NSUB = D / 64;
+    constexpr int Q_SUB = kTQ * 128;
+    constexpr int KV_SUB = TK * 128;
+    constexpr int KV_TILE = NSUB * KV_SUB;
+    constexpr int DC = D / 2;  // output columns each warpgroup stores in the epilogue
+    // dynamic shared memory starts on a 1024-byte boundary (the swizzled tiles need it); checked below
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint8_t* sQ = smem;
+    uint8_t* sK = sQ + NSUB * Q_SUB;
+    uint8_t* sV = sK + p.stages * KV_TILE;
+    __shared__ PpBarriers bars;
+    __shared__ float mref[2][kTQ];   // [publishing warpgroup][row]: reference maximum after that warpgroup's latest tile
+    __shared__ float lsum[2][kTQ];   // [warpgroup][row]: partial row sums, exchanged in the epilogue
+    __shared__ uint32_t tmem_base_s;
+    __shared__ uint32_t abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (smem_u32(smem) & 1023u) {  // never expected; fail with a status instead of corrupting tiles
+        if (tid == 0) atomicExch(&p.counters->status, (int)BSA_ERR_CUDA);
+        return;
+    }
+    const int NS = p.stages;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bars.q_full), 1);
+        mbar_init(smem_u32(&bars.q_empty), 1);
+        mbar_init(smem_u32(&bars.o_free), 256);
+        mbar_init(smem_u32(&bars.l_bar), 256);
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(smem_u32(&bars.k_full[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_full[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&bars.s_full[s]), 1);
+            mbar_init(smem_u32(&bars.s_free[s]), 128);
+            mbar_init(smem_u32(&bars.p_ready[s]), 128);
+            mbar_init(smem_u32(&bars.pv_done[s]), 1);
+            mbar_init(smem_u32(&bars.mx_bar[s]), 128);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 9) {
+        tmem_alloc(smem_u32(&tmem_base_s), kTmemCols);
+        tmem_relinquish();
+    }
+    if (warp == 8 && lane == 0) {
+        prefetch_tensormap(&tmQ);
+        prefetch_tensormap(&tmK);
+        prefetch_tensormap(&tmV);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+    volatile uint32_t* abortp = &abort_flag;
+    const int n_items = p.counters->nitems;
+
+    if (warp >= 8) {
+        reg_dec<72>();
+        if (warp == 8 && lane == 0) {
+            // =========================== TMA producer ===========================
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const WorkItem it = p.items[idx];
+                if (it.ntiles == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1, abortp);
+                if (!ok) break;
+                mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
+                for (int s = 0; s < NSUB; ++s)
+                    tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, it.q_tile * kTQ, it.head);
+                int col_next = p.tile_col[it.tile_begin];
+                for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
+                    const int col_cur = col_next;
+                    if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
+                    const int stage = g % NS;
+                    const uint32_t ph = (g / NS) & 1;
+                    const int kv0 = col_cur * TK;
+                    ok = mbar_wait(smem_u32(&bars.k_empty[stage]), ph ^ 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), KV_TILE);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sK + stage * KV_TILE + s * KV_SUB), &tmK, smem_u32(&bars.k_full[stage]),
+                                    s * 64, kv0, it.head);
+                    ok = mbar_wait(smem_u32(&bars.v_empty[stage]), ph ^ 1, abortp);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), KV_TILE);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sV + stage * KV_TILE + s * KV_SUB), &tmV, smem_u32(&bars.v_full[stage]),
+                                    s * 64, kv0, it.head);
+                }
+                ++itq;
+            }
+            if (!ok) {
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        } else if (warp == 9 && lane == 0) {
+            // =========================== Q K^T issuer ===========================
+            constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
+            const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
+            const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const int n = p.items[idx].ntiles;
+                if (n == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
+                if (!ok) break;
+                for (int j = 0; j < n; ++j) {
+                    const uint32_t gs = g + j;
+                    const int stage = gs % NS;
+                    const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
+                    ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
+                    if (!ok) break;
+                    if (gs >= 2) {  // S[sb] has been read into registers by the softmax of tile gs-2
+                        ok = mbar_wait(smem_u32(&bars.s_free[sb]), ((gs >> 1) - 1) & 1, abortp);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint64_t a = descQ + (uint64_t)(((k / 4) * Q_SUB + (k % 4) * 32) >> 4);
+                        const uint64_t b = descK + (uint64_t)((stage * KV_TILE + (k / 4) * KV_SUB + (k % 4) * 32) >> 4);
+                        mma_ss(d_s, a, b, idesc_qk, k > 0);
+                    }
+                    mma_commit(smem_u32(&bars.k_empty[stage]));
+                    mma_commit(smem_u32(&bars.s_full[sb]));
+                    if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
+                }
+                g += n;
+                ++itq;
+            }
+        } else if (warp == 10 && lane == 0) {
+            // =========================== P V issuer ===========================
+            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
+            uint32_t itq = 0, g = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const int n = p.items[idx].ntiles;
+                if (n == 0) continue;
+                for (int j = 0; j < n; ++j) {
+                    const uint32_t gp = g + j;
+                    const int stage = gp % NS;
+                    const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
+                    ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
+                    if (!ok) break;
+                    ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
+                    if (!ok) break;
+                    if (j == 0) {
+                        ok = mbar_wait(smem_u32(&bars.o_free), (itq & 1) ^ 1, abortp);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    const uint32_t a_p = tmem + (sb ? kColP1 : kColP0);
+#pragma unroll
+                    for (int k = 0; k < TK / 16; ++k) {
+                        const uint64_t b = descV + (uint64_t)((stage * KV_TILE + k * 2048) >> 4);
+                        mma_ts(tmem + kColO, a_p + k * 8, b, idesc_pv, (j > 0 || k > 0) ? 1u : 0u);
+                    }
+                    mma_commit(smem_u32(&bars.v_empty[stage]));
+                    mma_commit(smem_u32(&bars.pv_done[sb]));
+                }
+                g += n;
+                ++itq;
+            }
+        }
+    } else {
+        // =========================== softmax warpgroup x ===========================
+        reg_inc<216>();
+        const int x = warp >> 2;
+        const int tw = tid & 127;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t t_s = tmem + lane_base + (x ? kColS1 : kColS0);
+        const uint32_t t_p = tmem + lane_base + (x ? kColP1 : kColP0);
+        const uint32_t t_o = tmem + lane_base + kColO;
+        uint32_t g = 0;          // running tile index at the start of the current item (all warpgroups agree)
+        uint32_t seen = 0;       // publishes of the OTHER warpgroup already waited for (they are consumed in order)
+        uint32_t luse = 0;       // uses of l_bar
+        bool ok = true;
+        const float c2 = p.scale_log2;
+        const unsigned long long sub_mask = (p.sK >= 64) ? ~0ull : ((1ull << p.sK) - 1ull);
+        // wait until the other warpgroup has published the reference after global tile t (t has the other parity)
+        auto wait_publish = [&](uint32_t t) -> bool {
+            const uint32_t k = t >> 1;  // publish index inside the other warpgroup
+            if (seen > k) return true;
+            const bool got = mbar_wait(smem_u32(&bars.mx_bar[x ^ 1]), k & 1, abortp);
+            seen = k + 1;
+            return got;
+        };
+        for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            const WorkItem it = p.items[idx];
+            const int n = it.ntiles;
+            const int row = it.q_tile * kTQ + tw;
+            const bool row_ok = row < p.N;
+            if (n == 0) {
+                if (row_ok) {
+                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D + x * DC);
+#pragma unroll
+                    for (int c = 0; c < DC / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
+                    if (x == 0) p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
+                }
+                continue;
+            }
+            float m_know = -INFINITY;  // reference maximum this thread's partial sum l is expressed in
+            float l = 0.f;
+            // first local tile index of this warpgroup inside the item
+            const int j0 = ((g & 1) == (uint32_t)x) ? 0 : 1;
+            int col_next = 0;
+            unsigned long long member_next = 0ull;
+            if (j0 < n) {
+                col_next = p.tile_col[it.tile_begin + j0];
+                member_next = p.tile_member[it.tile_begin + j0];
+            }
+            for (int j = j0; j < n; j += 2) {
+                const uint32_t gs = g + j;
+                const int kv0 = col_next * TK;
+                const unsigned long long member = member_next;
+                if (j + 2 < n) {
+                    col_next = p.tile_col[it.tile_begin + j + 2];
+                    member_next = p.tile_member[it.tile_begin + j + 2];
+                }
+                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
+                const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
+                const int n_valid = p.N - kv0;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), (gs >> 1) & 1, abortp));
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t r[TK];
+#pragma unroll
+                for (int c = 0; c < TK / 32; ++c) tmem_ld32(t_s + c * 32, &r[c * 32]);
+                tc_wait_ld();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.s_free[x]));  // S[x] is in registers: the next Q K^T into it may start
+                if (need_mask) {
+#pragma unroll
+                    for (int i = 0; i < TK; ++i) {
+                        const bool act = ((row_bits >> (i >> p.lgBKV)) & 1u) && (i < n_valid);
+                        r[i] = act ? r[i] : 0xff800000u;
+                    }
+                }
+                float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < TK; i += 4) {
+                    m0 = fmaxf(m0, __uint_as_float(r[i]));
+                    m1 = fmaxf(m1, __uint_as_float(r[i + 1]));
+                    m2 = fmaxf(m2, __uint_as_float(r[i + 2]));
+                    m3 = fmaxf(m3, __uint_as_float(r[i + 3]));
+                }
+                const float mx2 = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c2;
+                // ---- reference maximum handed over from the previous tile (other warpgroup) ----
+                float m_prev = -INFINITY;
+                if (gs > 0) {
+                    ok = __all_sync(0xffffffffu, wait_publish(gs - 1));
+                    if (!ok) break;
+                    if (j > 0) m_prev = mref[x ^ 1][tw];  // the previous tile belongs to this item
+                }
+                if (m_prev != m_know) {  // the other warpgroup moved the reference since this thread last looked
+                    l *= ex2_approx(m_know - m_prev);  // m_know = -inf only while l = 0
+                    m_know = m_prev;
+                }
+                float alpha = 1.f;
+                bool rescale = false;
+                if (mx2 > m_know + kRescaleThreshold) {
+                    alpha = ex2_approx(m_know - mx2);
+                    rescale = (j > 0) && (m_know != -INFINITY);
+                    l *= alpha;
+                    m_know = mx2;
+                }
+                mref[x][tw] = m_know;
+                mbar_arrive(smem_u32(&bars.mx_bar[x]));  // publish: the next tile's warpgroup may take its decision
+                const float neg_m = (m_know == -INFINITY) ? 0.f : -m_know;
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int i = 0; i < TK; i += 4) {
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(r[i]), c2, neg_m));
+                    const float p1 = ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, neg_m));
+                    const float p2 = ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, neg_m));
+                    const float p3 = ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, neg_m));
+                    s0 += p0;
+                    s1 += p1;
+                    s2 += p2;
+                    s3 += p3;
+                    r[i / 2] = pack_bf16x2(p0, p1);
+                    r[i / 2 + 1] = pack_bf16x2(p2, p3);
+                }
+                l += (s0 + s1) + (s2 + s3);
+                // P[x] was last read by the P V of tile gs-2
+                if (gs >= 2) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x]), ((gs >> 1) - 1) & 1, abortp));
+                    if (!ok) break;
+                }
+#pragma unroll
+                for (int c = 0; c < TK / 32; ++c) tmem_st16(t_p + c * 16, &r[c * 16]);
+                // ---- the reference moved at this tile: rescale the running output (after the P V of tile gs-1) ----
+                if (j > 0 && __any_sync(0xffffffffu, rescale)) {
+                    const uint32_t gp = gs - 1;
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x ^ 1]), (gp >> 1) & 1, abortp));
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(t_o + c * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(t_o + c * 32, o);
+                    }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.p_ready[x]));
+            }
+            if (!ok) break;
+            // ---- epilogue: bring both partial sums to the final reference, add them, store half of the row each ----
+            {
+                const uint32_t gl = g + n - 1;  // last tile of the item
+                float m_final = m_know;
+                if ((gl & 1) != (uint32_t)x) {  // the other warpgroup took the last tile: its publish holds the final reference
+                    ok = __all_sync(0xffffffffu, wait_publish(gl));
+                    if (!ok) break;
+                    m_final = mref[x ^ 1][tw];
+                }
+                if (m_final != m_know) l *= ex2_approx(m_know - m_final);
+                // Wait for the item's last P V before touching `lsum`: that MMA could only be issued after BOTH
+                // warpgroups finished the previous item's epilogue (o_free), i.e. after they read the previous sums.
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[gl & 1]), (gl >> 1) & 1, abortp));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t par = luse & 1;
+                lsum[x][tw] = l;
+                mbar_arrive(smem_u32(&bars.l_bar));
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.l_bar), par, abortp));
+                if (!ok) break;
+                ++luse;
+                const float l_tot = lsum[0][tw] + lsum[1][tw];
+                const float inv_l = (l_tot > 0.f) ? 1.f / l_tot : 0.f;
+                const float lse = (l_tot > 0.f) ? fmaf(m_final, 0.6931471805599453f, logf(l_tot)) : -INFINITY;
+                const uint32_t t_oh = t_o + x * DC;
+                if (it.nparts == 1) {
+                    __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D + x * DC;
+#pragma unroll
+                    for (int c = 0; c < DC / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(t_oh + c * 32, o);
+                        tc_wait_ld();
+                        if (row_ok) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                uint4 v;
+                                v.x = pack_bf16x2(__uint_as_float(o[q * 8 + 0]) * inv_l, __uint_as_float(o[q * 8 + 1]) * inv_l);
+                                v.y = pack_bf16x2(__uint_as_float(o[q * 8 + 2]) * inv_l, __uint_as_float(o[q * 8 + 3]) * inv_l);
+                                v.z = pack_bf16x2(__uint_as_float(o[q * 8 + 4]) * inv_l, __uint_as_float(o[q * 8 + 5]) * inv_l);
+                                v.w = pack_bf16x2(__uint_as_float(o[q * 8 + 6]) * inv_l, __uint_as_float(o[q * 8 + 7]) * inv_l);
+                                *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = v;
+                            }
+                        }
+                    }
+                    if (row_ok && x == 0) p.LSE[(size_t)it.head * p.N + row] = lse;
+                } else {
+                    float* orow = p.ws_O + ((size_t)it.ws_slot * kTQ + tw) * D + x * DC;
+#pragma unroll
+                    for (int c = 0; c < DC / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(t_oh + c * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            float4 v = make_float4(__uint_as_float(o[q * 4 + 0]) * inv_l, __uint_as_float(o[q * 4 + 1]) * inv_l,
+                                                   __uint_as_float(o[q * 4 + 2]) * inv_l, __uint_as_float(o[q * 4 + 3]) * inv_l);
+                            *reinterpret_cast<float4*>(orow + c * 32 + q * 4) = v;
+                        }
+                    }
+                    if (x == 0) p.ws_LSE[(size_t)it.ws_slot * kTQ + tw] = lse;
+                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.o_free));
+            }
+            g += n;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && abort_flag) atomicExch(&p.counters->status, (int)BSA_ERR_DEVICE_TIMEOUT);
+    if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+}
+
 // ------------------------------------------------------------------------------------------
 // Split-K reduction (Section 4.3): partial states were stored as (normalised O_p, LSE_p), so
 // rescaling to the common maximum, merging and normalising is
@@ -1392,8 +1813,10 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
             e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         else if (KERNEL == 1)
             e = cudaFuncSetAttribute(bsa_attention_pair_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        else
+        else if (KERNEL == 2)
             e = cudaFuncSetAttribute(bsa_attention_cs_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        else
+            e = cudaFuncSetAttribute(bsa_attention_pp_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) {
             *err = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
@@ -1408,8 +1831,10 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
         bsa_attention_kernel<D, TK, true><<<grid, kThreads + 32, smem, stream>>>(tq, tk, tv, p);
     else if (KERNEL == 1)
         bsa_attention_pair_kernel<D, TK><<<grid, kPairThreads, smem, stream>>>(tq, tk, tv, p);
-    else
+    else if (KERNEL == 2)
         bsa_attention_cs_kernel<D, TK><<<grid, kCsThreads, smem, stream>>>(tq, tk, tv, p);
+    else
+        bsa_attention_pp_kernel<D, TK><<<grid, kPpThreads, smem, stream>>>(tq, tk, tv, p);
     count_launch();
     return cudaGetLastError();
 }
@@ -1418,7 +1843,7 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
 
 // Shared-memory budget: 227 KB per CTA minus each kernel's static shared memory (barriers, exchange
 // buffer), which the compiler rounds up to the 1024-byte alignment of the dynamic part.
-static int static_smem_bytes(int kernel) { return kernel == 2 ? 3072 : 1024; }
+static int static_smem_bytes(int kernel) { return (kernel == 2 || kernel == 4) ? 3072 : 1024; }
 
 static int kv_buffers_that_fit(int d, int T_KV, int kernel) {
     const int q = (kernel == 1 ? 2 : 1) * kTQ * d * 2;
@@ -1493,6 +1918,10 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     else if (key == 3000 + 128 + 1) e = launch_attn<128, 64, 3>(a, p, stream, err_detail);
     else if (key == 3000 + 64 + 2) e = launch_attn<64, 128, 3>(a, p, stream, err_detail);
     else if (key == 3000 + 64 + 1) e = launch_attn<64, 64, 3>(a, p, stream, err_detail);
+    else if (key == 4000 + 128 + 2) e = launch_attn<128, 128, 4>(a, p, stream, err_detail);
+    else if (key == 4000 + 128 + 1) e = launch_attn<128, 64, 4>(a, p, stream, err_detail);
+    else if (key == 4000 + 64 + 2) e = launch_attn<64, 128, 4>(a, p, stream, err_detail);
+    else if (key == 4000 + 64 + 1) e = launch_attn<64, 64, 4>(a, p, stream, err_detail);
     else {
         *err_detail = "no kernel for this (d, T_KV)";
         return cudaErrorInvalidValue;

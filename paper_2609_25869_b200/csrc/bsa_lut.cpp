@@ -44,6 +44,11 @@ static const bsa_plan_desc_t kCatalog[] = {
     {19, 128, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 3, "q128k64_di"},
     {20, 128, 128, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 3, "q128k128_di_split4x8"},
     {21, 128, 128, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 3, "q128k128_di_global"},
+    // one 128-row Q tile per CTA, two softmax warpgroups on alternate KV tiles, shared reference maximum
+    {22, 128, 128, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k128_pp"},
+    {23, 128, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k64_pp"},
+    {24, 128, 128, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k128_pp_split4x8"},
+    {25, 128, 128, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 4, "q128k128_pp_global"},
 };
 static const int kCatalogSize = (int)(sizeof(kCatalog) / sizeof(kCatalog[0]));
 static const int64_t kDefaultWorkspace = 2ll << 30;
@@ -116,7 +121,7 @@ int base_plan(int B_Q, int B_KV, int d) {
     (void)B_Q;
     (void)B_KV;
     (void)d;
-    return 18;  // q128k128_di: eligible for every supported geometry (membership <= 64 bits), no workspace
+    return 22;  // q128k128_pp: eligible for every supported geometry (membership <= 64 bits), no workspace
 }
 
 uint64_t catalog_hash() {

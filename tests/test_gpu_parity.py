@@ -18,13 +18,13 @@ def _sample(req, per_head, seed=77, heads=None):
 
 
 # ---------------------------------------------------------------- the five configurations
-@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21])
+@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25])
 def test_tiny_full_oracle_every_plan(plan_id):
     res = Hh.run_request(I.config_tiny(), plan_id=plan_id)
     assert res["pairs"] == res["info"]["nnz_blocks"] * 64 * 64
 
 
-@pytest.mark.parametrize("plan_id", [0, 1, 2, 10, 12, 14, 16, 18, 20])
+@pytest.mark.parametrize("plan_id", [0, 1, 2, 10, 12, 14, 16, 18, 20, 22, 24])
 def test_mid_full_oracle(plan_id):
     Hh.run_request(I.config_mid(), plan_id=plan_id)
 
@@ -35,14 +35,14 @@ def test_hunyuan_shaped_sampled_oracle():
     Hh.run_request(req, plan_id=-1, sel=_sample(req, 64), heads=[0, 11, 23])
 
 
-@pytest.mark.parametrize("plan_id", [0, 1, 10, 14, 18])
+@pytest.mark.parametrize("plan_id", [0, 1, 10, 14, 18, 22, 23])
 def test_stress_a_coarsened(plan_id):
     req = I.config_stress_a()
     res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64), heads=[0, 15])
     assert res["info"]["map_q"] == 1  # Coarsened along Q: 8 logical rows of 16 per 128-row tile
 
 
-@pytest.mark.parametrize("plan_id", [0, 1, 10, 11, 14, 15, 18, 19])
+@pytest.mark.parametrize("plan_id", [0, 1, 10, 11, 14, 15, 18, 19, 22, 23])
 def test_stress_b_refined(plan_id):
     req = I.config_stress_b()
     res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64))
@@ -70,6 +70,9 @@ def test_sweep_requests_ragged_n(r, B, rho):
     (256, 128, 2100, 128, 14), (256, 16, 900, 64, 16), (16, 256, 900, 128, 16), (128, 128, 127, 128, 17),
     (16, 16, 1000, 64, 18), (32, 64, 777, 128, 19), (64, 32, 1300, 128, 18), (128, 256, 2100, 64, 19),
     (256, 128, 2100, 128, 18), (256, 16, 900, 64, 20), (16, 256, 900, 128, 20), (128, 128, 127, 128, 21),
+    (16, 16, 1000, 64, 22), (32, 64, 777, 128, 23), (64, 32, 1300, 128, 22), (128, 256, 2100, 64, 23),
+    (256, 128, 2100, 128, 22), (256, 16, 900, 64, 24), (16, 256, 900, 128, 24), (128, 128, 127, 128, 25),
+    (64, 64, 130, 64, 22), (128, 128, 1, 64, 23), (128, 128, 129, 128, 22), (32, 32, 3000, 64, 25),
 ])
 def test_geometries_with_ragged_tail(B_Q, B_KV, N, d, plan_id):
     H = 3
@@ -91,7 +94,7 @@ def test_degenerate_masks(kind):
     elif kind == "empty_head":
         M[0] = I.random_mask(1, 1, nb, nb, 0.5)[0]
     req = I.Request(kind, H, N, d, B, B, M, qkv_seed=3)
-    for plan_id in (0, 3, 10, 12, 14, 16, 18, 20):
+    for plan_id in (0, 3, 10, 12, 14, 16, 18, 20, 22, 24):
         Hh.run_request(req, plan_id=plan_id)
 
 
@@ -99,7 +102,8 @@ def test_degenerate_masks(kind):
 @pytest.mark.parametrize("B_Q,B_KV,N,d,plan_id", [(16, 64, 1000, 64, 0), (32, 32, 700, 128, 1), (256, 256, 1100, 128, 9),
                                                   (16, 64, 1000, 64, 10), (64, 32, 700, 128, 11), (256, 256, 1100, 128, 12),
                                                   (16, 64, 1000, 64, 14), (64, 32, 700, 128, 15), (256, 256, 1100, 128, 16),
-                                                  (16, 64, 1000, 64, 18), (64, 32, 700, 128, 19), (256, 256, 1100, 128, 20)])
+                                                  (16, 64, 1000, 64, 18), (64, 32, 700, 128, 19), (256, 256, 1100, 128, 20),
+                                                  (16, 64, 1000, 64, 22), (64, 32, 700, 128, 23), (256, 256, 1100, 128, 24)])
 def test_zero_keys_give_log_count_and_mean_value(B_Q, B_KV, N, d, plan_id):
     """K = 0: every score is 0, so LSE = ln(#reachable keys) exactly and O = mean of reachable V.
     Catches any off-by-one in ragged-edge or membership masking (one key off moves LSE by ~1/count)."""
@@ -134,12 +138,29 @@ def test_constant_values_come_back():
     assert torch.allclose(O.float(), torch.full_like(O.float(), 0.75), atol=4e-3)
 
 
-def test_sharp_scores_stay_within_tolerance():
-    # 4x larger scores: a much peakier softmax, more rescaling of the running output
+@pytest.mark.parametrize("plan_id", [1, 18, 22, 23, 24])
+def test_sharp_scores_stay_within_tolerance(plan_id):
+    # 4x larger scores: a much peakier softmax, the reference maximum keeps moving and the running output is
+    # rescaled often (in the ping-pong kernel the reference is handed from one warpgroup to the other every tile)
     req = I.config_tiny(seed=21)
     q, k, v = req.qkv()
-    res = Hh.run_request(req, plan_id=1, qkv=((q * 2).to(torch.bfloat16), (k * 2).to(torch.bfloat16), v), guards=False)
+    res = Hh.run_request(req, plan_id=plan_id, qkv=((q * 2).to(torch.bfloat16), (k * 2).to(torch.bfloat16), v),
+                         guards=False)
     assert res["lse_max"] < 2e-4
+
+
+@pytest.mark.parametrize("plan_id", [18, 22])
+def test_growing_scores_force_a_rescale_at_every_tile(plan_id):
+    """Keys sorted by increasing magnitude along the sequence: every later tile raises the row maximum by more
+    than the rescale threshold, so the reference moves (and O is rescaled) tile after tile."""
+    H, N, d, B = 1, 1024, 128, 128
+    q, k, v = I.make_qkv(77, H, N, d)
+    ramp = torch.linspace(0.2, 6.0, N).view(1, N, 1)
+    k = (k * ramp).to(torch.bfloat16)
+    M = np.ones((H, N // B, N // B), np.uint8)
+    req = I.Request("ramp", H, N, d, B, B, M, qkv_seed=0)
+    res = Hh.run_request(req, plan_id=plan_id, qkv=(q, k, v), guards=False)
+    assert res["lse_max"] < 5e-4
 
 
 # ---------------------------------------------------------------- boundary behaviour

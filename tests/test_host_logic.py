@@ -39,7 +39,7 @@ def test_catalog_and_eligibility():
     assert len(cat) >= 6 and [c["plan_id"] for c in cat] == list(range(len(cat)))
     assert len(set(c["name"] for c in cat)) == len(cat)
     assert {c["T_KV"] for c in cat} == {64, 128} and {c["T_Q"] for c in cat} == {128, 256}
-    assert {c["kernel"] for c in cat} == {0, 1, 2, 3}
+    assert {c["kernel"] for c in cat} == {0, 1, 2, 3, 4}
     base = bsa.lib().bsa_base_plan(128, 128, 128)
     # the base plan is eligible for every supported request key
     for B_Q in (16, 32, 64, 128, 256):
