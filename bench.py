@@ -28,7 +28,7 @@ sys.path.insert(0, ROOT)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch on the bench workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists for the workload)
-NCU_TRAFFIC_BYTES = {"mid": 120.2e6}  # 101.1 MB read + 19.1 MB written (profiles/attention_kernel_mid.md, capture B3)
+NCU_TRAFFIC_BYTES = {"mid": 118.8e6}  # 101.0 MB read + 17.8 MB written (profiles/attention_kernel_mid.md, capture B)
 
 
 def load_peaks():
@@ -383,7 +383,7 @@ def main():
         "e2e": {"value": world * r["flops"] / e2e_s / 1e12, "unit": "TFLOP/s",
                 "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"], "ms_per_request": e2e_s * 1e3},
         "gpu_launches": r["launches"],
-        "roofline": {"bound": "tensor", "kernel": "bsa_attention_kernel", "achieved": kernel_tflops,
+        "roofline": {"bound": "tensor", "kernel": "bsa_attention_pp_kernel", "achieved": kernel_tflops,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": kernel_tflops / peaks["bf16_tflops"],
                      "frac_of_sustained": kernel_tflops / peaks["bf16_tflops_sustained"],
                      "peak_source": peaks["_source"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload),

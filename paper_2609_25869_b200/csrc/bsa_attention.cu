@@ -26,7 +26,7 @@ using namespace ptx;
 // Optional timeline tracing (compile with -DBSA_TRACE): CTA 0 records clock64() at barrier events of the
 // single-tile kernel, per role, into a device buffer that bsa_debug_trace_copy() reads back.
 #ifdef BSA_TRACE
-__device__ long long g_trace[7][4096];  // producer, MMA (or Q K^T) issuer, softmax warps 0-3, P V issuer
+__device__ long long g_trace[11][4096];  // producer, Q K^T (or single) issuer, softmax warps 0-7, P V issuer (role 6 in the 7-warp kernel)
 __device__ long long g_trace_aux[12][4];  // last tile's stamps inside softmax_tile, per warp
 #define BSA_TRACE_DECL(n) int n = 0
 #define BSA_TRACE_POINT(role, n, tag)                                              \
@@ -1428,6 +1428,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
             uint32_t itq = 0, g = 0;
             bool ok = true;
+            BSA_TRACE_DECL(tn);
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
                 const int n = p.items[idx].ntiles;
                 if (n == 0) continue;
@@ -1439,10 +1440,12 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
                     ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
                     if (!ok) break;
+                    BSA_TRACE_POINT(1, tn, 1);
                     if (gs >= 2) {  // S[sb] has been read into registers by the softmax of tile gs-2
                         ok = mbar_wait(smem_u32(&bars.s_free[sb]), ((gs >> 1) - 1) & 1, abortp);
                         if (!ok) break;
                     }
+                    BSA_TRACE_POINT(1, tn, 6);
                     tc_fence_after();
                     const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
 #pragma unroll
@@ -1453,6 +1456,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     }
                     mma_commit(smem_u32(&bars.k_empty[stage]));
                     mma_commit(smem_u32(&bars.s_full[sb]));
+                    BSA_TRACE_POINT(1, tn, 2);
                     if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
                 }
                 g += n;
@@ -1464,6 +1468,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
             uint32_t itq = 0, g = 0;
             bool ok = true;
+            BSA_TRACE_DECL(tn);
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
                 const int n = p.items[idx].ntiles;
                 if (n == 0) continue;
@@ -1473,6 +1478,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
                     ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
                     if (!ok) break;
+                    BSA_TRACE_POINT(10, tn, 3);
                     ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
                     if (!ok) break;
                     if (j == 0) {
@@ -1488,6 +1494,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     }
                     mma_commit(smem_u32(&bars.v_empty[stage]));
                     mma_commit(smem_u32(&bars.pv_done[sb]));
+                    BSA_TRACE_POINT(10, tn, 5);
                 }
                 g += n;
                 ++itq;
@@ -1506,6 +1513,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         uint32_t seen = 0;       // publishes of the OTHER warpgroup already waited for (they are consumed in order)
         uint32_t luse = 0;       // uses of l_bar
         bool ok = true;
+        BSA_TRACE_DECL(tn);
         const float c2 = p.scale_log2;
         const unsigned long long sub_mask = (p.sK >= 64) ? ~0ull : ((1ull << p.sK) - 1ull);
         // wait until the other warpgroup has published the reference after global tile t (t has the other parity)
@@ -1553,6 +1561,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const int n_valid = p.N - kv0;
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), (gs >> 1) & 1, abortp));
                 if (!ok) break;
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 10);
                 tc_fence_after();
                 uint32_t r[TK];
 #pragma unroll
@@ -1560,6 +1569,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 tc_wait_ld();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.s_free[x]));  // S[x] is in registers: the next Q K^T into it may start
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 11);
                 if (need_mask) {
 #pragma unroll
                     for (int i = 0; i < TK; ++i) {
@@ -1583,6 +1593,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     if (!ok) break;
                     if (j > 0) m_prev = mref[x ^ 1][tw];  // the previous tile belongs to this item
                 }
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 12);
                 if (m_prev != m_know) {  // the other warpgroup moved the reference since this thread last looked
                     l *= ex2_approx(m_know - m_prev);  // m_know = -inf only while l = 0
                     m_know = m_prev;
@@ -1613,6 +1624,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     r[i / 2 + 1] = pack_bf16x2(p2, p3);
                 }
                 l += (s0 + s1) + (s2 + s3);
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 14);
                 // P[x] was last read by the P V of tile gs-2
                 if (gs >= 2) {
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x]), ((gs >> 1) - 1) & 1, abortp));
@@ -1639,6 +1651,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.p_ready[x]));
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 16);
             }
             if (!ok) break;
             // ---- epilogue: bring both partial sums to the final reference, add them, store half of the row each ----
