@@ -96,11 +96,11 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, bool ne
     }
     float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < TK; i += 4) {
-        m0 = fmaxf(m0, __uint_as_float(r[i]));
-        m1 = fmaxf(m1, __uint_as_float(r[i + 1]));
-        m2 = fmaxf(m2, __uint_as_float(r[i + 2]));
-        m3 = fmaxf(m3, __uint_as_float(r[i + 3]));
+    for (int i = 0; i < TK; i += 8) {
+        m0 = max3(m0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+        m1 = max3(m1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+        m2 = max3(m2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+        m3 = max3(m3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
     }
     const float mx2 = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c2;
     alpha = 1.f;
@@ -114,35 +114,25 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, bool ne
 #ifdef BSA_TRACE
     if ((threadIdx.x & 31) == 0 && blockIdx.x == 0) g_trace_aux[threadIdx.x >> 5][1] = clock64();
 #endif
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    // scale-and-shift and the row sums run as packed two-lane fp32 operations
+    const uint64_t c22 = pack_f32x2(c2, c2), nm2 = pack_f32x2(neg_m, neg_m);
+    uint64_t sum01 = pack_f32x2(0.f, 0.f), sum23 = sum01;
 #pragma unroll
     for (int i = 0; i < TK; i += 4) {
-#ifdef BSA_EXP_NOMUFU
-#define BSA_EX2(x) (x)
-#else
-#define BSA_EX2(x) ex2_approx(x)
-#endif
-        const float p0 = BSA_EX2(fmaf(__uint_as_float(r[i]), c2, neg_m));
-        const float p1 = BSA_EX2(fmaf(__uint_as_float(r[i + 1]), c2, neg_m));
-        const float p2 = BSA_EX2(fmaf(__uint_as_float(r[i + 2]), c2, neg_m));
-        const float p3 = BSA_EX2(fmaf(__uint_as_float(r[i + 3]), c2, neg_m));
-        s0 += p0;
-        s1 += p1;
-        s2 += p2;
-        s3 += p3;
-#ifdef BSA_EXP_NOPACK
-        r[i / 2] = __float_as_uint(p0) ^ __float_as_uint(p1);
-        r[i / 2 + 1] = __float_as_uint(p2) ^ __float_as_uint(p3);
-#else
+        float x0, x1, x2, x3;
+        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), c22, nm2), x0, x1);
+        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), c22, nm2), x2, x3);
+        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
+        sum01 = add_f32x2(sum01, pack_f32x2(p0, p1));
+        sum23 = add_f32x2(sum23, pack_f32x2(p2, p3));
         r[i / 2] = pack_bf16x2(p0, p1);
         r[i / 2 + 1] = pack_bf16x2(p2, p3);
-#endif
     }
+    float s0, s1, s2, s3;
+    unpack_f32x2(sum01, s0, s1);
+    unpack_f32x2(sum23, s2, s3);
 #ifdef BSA_TRACE
     if ((threadIdx.x & 31) == 0 && blockIdx.x == 0) g_trace_aux[threadIdx.x >> 5][2] = clock64();
-#endif
-#ifdef BSA_EXP_NOST
-    if (c2 == 12345.f)
 #endif
 #pragma unroll
     for (int c = 0; c < TK / 32; ++c) tmem_st16(t_p + c * 16, &r[c * 16]);
@@ -1579,11 +1569,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 }
                 float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < TK; i += 4) {
-                    m0 = fmaxf(m0, __uint_as_float(r[i]));
-                    m1 = fmaxf(m1, __uint_as_float(r[i + 1]));
-                    m2 = fmaxf(m2, __uint_as_float(r[i + 2]));
-                    m3 = fmaxf(m3, __uint_as_float(r[i + 3]));
+                for (int i = 0; i < TK; i += 8) {
+                    m0 = max3(m0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                    m1 = max3(m1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                    m2 = max3(m2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+                    m3 = max3(m3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
                 }
                 const float mx2 = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c2;
                 // ---- reference maximum handed over from the previous tile (other warpgroup) ----
@@ -1609,20 +1599,22 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 mref[x][tw] = m_know;
                 mbar_arrive(smem_u32(&bars.mx_bar[x]));  // publish: the next tile's warpgroup may take its decision
                 const float neg_m = (m_know == -INFINITY) ? 0.f : -m_know;
-                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                const uint64_t c22 = pack_f32x2(c2, c2), nm2 = pack_f32x2(neg_m, neg_m);
+                uint64_t sum01 = pack_f32x2(0.f, 0.f), sum23 = sum01;
 #pragma unroll
                 for (int i = 0; i < TK; i += 4) {
-                    const float p0 = ex2_approx(fmaf(__uint_as_float(r[i]), c2, neg_m));
-                    const float p1 = ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, neg_m));
-                    const float p2 = ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, neg_m));
-                    const float p3 = ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, neg_m));
-                    s0 += p0;
-                    s1 += p1;
-                    s2 += p2;
-                    s3 += p3;
+                    float x0, x1, x2, x3;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), c22, nm2), x0, x1);
+                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), c22, nm2), x2, x3);
+                    const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
+                    sum01 = add_f32x2(sum01, pack_f32x2(p0, p1));
+                    sum23 = add_f32x2(sum23, pack_f32x2(p2, p3));
                     r[i / 2] = pack_bf16x2(p0, p1);
                     r[i / 2 + 1] = pack_bf16x2(p2, p3);
                 }
+                float s0, s1, s2, s3;
+                unpack_f32x2(sum01, s0, s1);
+                unpack_f32x2(sum23, s2, s3);
                 l += (s0 + s1) + (s2 + s3);
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 14);
                 // P[x] was last read by the P V of tile gs-2
@@ -1739,40 +1731,46 @@ __global__ void __launch_bounds__(256) bsa_merge_kernel(const SplitRow* __restri
                                                          const PlanCountersDev* __restrict__ counters,
                                                          const float* __restrict__ ws_O, const float* __restrict__ ws_LSE,
                                                          __nv_bfloat16* __restrict__ O, float* __restrict__ LSE, int N) {
-    constexpr int GROUPS = D / 8;  // 8 output columns (16 bytes of bf16) per thread step
-    const int n_rows = counters->nsplit_rows;
-    for (int sr = blockIdx.x; sr < n_rows; sr += gridDim.x) {
-        const SplitRow s = split_rows[sr];
+    constexpr int GROUPS = D / 8;                   // 8 output columns (16 bytes of bf16) per thread
+    constexpr int CHUNKS = kTQ * GROUPS / 256;      // CTAs' worth of work per merged 128-row tile
+    const int n_units = counters->nsplit_rows * CHUNKS;
+    for (int cu = blockIdx.x; cu < n_units; cu += gridDim.x) {
+        const SplitRow s = split_rows[cu / CHUNKS];
         const int nparts = s.nparts & 0xffff, stride = s.nparts >> 16;
-        for (int u = threadIdx.x; u < kTQ * GROUPS; u += blockDim.x) {
-            const int r = u / GROUPS, gcol = (u % GROUPS) * 8;
-            const int row = s.q_tile * kTQ + r;
-            if (row >= N) continue;
-            float m = -INFINITY;
-            for (int q = 0; q < nparts; ++q) m = fmaxf(m, ws_LSE[(size_t)(s.ws_slot + q * stride) * kTQ + r]);
-            const float m_use = (m == -INFINITY) ? 0.f : m;
-            float tot = 0.f;
-            float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            for (int q = 0; q < nparts; ++q) {
-                const size_t slot = (size_t)(s.ws_slot + q * stride);
-                const float w = __expf(ws_LSE[slot * kTQ + r] - m_use);
-                tot += w;
-                const float4* src = reinterpret_cast<const float4*>(ws_O + (slot * kTQ + r) * D + gcol);
-                const float4 a = src[0], b = src[1];
-                acc[0] = fmaf(w, a.x, acc[0]); acc[1] = fmaf(w, a.y, acc[1]);
-                acc[2] = fmaf(w, a.z, acc[2]); acc[3] = fmaf(w, a.w, acc[3]);
-                acc[4] = fmaf(w, b.x, acc[4]); acc[5] = fmaf(w, b.y, acc[5]);
-                acc[6] = fmaf(w, b.z, acc[6]); acc[7] = fmaf(w, b.w, acc[7]);
-            }
-            const float inv = (tot > 0.f) ? 1.f / tot : 0.f;
-            uint4 v;
-            v.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-            v.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
-            v.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
-            v.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
-            *reinterpret_cast<uint4*>(O + ((size_t)s.head * N + row) * D + gcol) = v;
-            if (gcol == 0) LSE[(size_t)s.head * N + row] = (tot > 0.f) ? m_use + logf(tot) : -INFINITY;
+        const int u = (cu % CHUNKS) * 256 + threadIdx.x;
+        const int r = u / GROUPS, gcol = (u % GROUPS) * 8;
+        const int row = s.q_tile * kTQ + r;
+        if (row >= N) continue;
+        // all partial LSEs of the row first (independent loads), then the weights, then the weighted sum
+        float lse_p[32];
+        float m = -INFINITY;
+#pragma unroll 4
+        for (int q = 0; q < nparts; ++q) {
+            lse_p[q & 31] = ws_LSE[(size_t)(s.ws_slot + q * stride) * kTQ + r];
+            m = fmaxf(m, lse_p[q & 31]);
         }
+        const float m_use = (m == -INFINITY) ? 0.f : m;
+        float tot = 0.f;
+        float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        for (int q = 0; q < nparts; ++q) {
+            const size_t slot = (size_t)(s.ws_slot + q * stride);
+            const float w = __expf(lse_p[q & 31] - m_use);
+            tot += w;
+            const float4* src = reinterpret_cast<const float4*>(ws_O + (slot * kTQ + r) * D + gcol);
+            const float4 a = src[0], b = src[1];
+            acc[0] = fmaf(w, a.x, acc[0]); acc[1] = fmaf(w, a.y, acc[1]);
+            acc[2] = fmaf(w, a.z, acc[2]); acc[3] = fmaf(w, a.w, acc[3]);
+            acc[4] = fmaf(w, b.x, acc[4]); acc[5] = fmaf(w, b.y, acc[5]);
+            acc[6] = fmaf(w, b.z, acc[6]); acc[7] = fmaf(w, b.w, acc[7]);
+        }
+        const float inv = (tot > 0.f) ? 1.f / tot : 0.f;
+        uint4 v;
+        v.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+        v.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+        v.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
+        v.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+        *reinterpret_cast<uint4*>(O + ((size_t)s.head * N + row) * D + gcol) = v;
+        if (gcol == 0) LSE[(size_t)s.head * N + row] = (tot > 0.f) ? m_use + logf(tot) : -INFINITY;
     }
 }
 
@@ -1941,7 +1939,9 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     }
     if (e != cudaSuccess) return e;
     if (a.has_split) {
-        int grid = a.max_split_rows < 4 * a.num_sms ? a.max_split_rows : 4 * a.num_sms;
+        // one CTA per 256 (row, 8-column) units of a merged tile, grid-strided beyond 8 waves
+        const long long want = (long long)a.max_split_rows * (kTQ * (a.d / 8) / 256);
+        int grid = want < 8ll * a.num_sms ? (int)want : 8 * a.num_sms;
         if (grid < 1) grid = 1;
         if (a.d == 128)
             bsa_merge_kernel<128><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,

@@ -49,6 +49,9 @@ static const bsa_plan_desc_t kCatalog[] = {
     {23, 128, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k64_pp"},
     {24, 128, 128, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k128_pp_split4x8"},
     {25, 128, 128, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 4, "q128k128_pp_global"},
+    {26, 128, 64, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 4, "q128k64_pp_global"},
+    {27, 128, 64, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k64_pp_split4x8"},
+    {28, 128, 64, 0, 2, 16, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k64_pp_split2x16"},
 };
 static const int kCatalogSize = (int)(sizeof(kCatalog) / sizeof(kCatalog[0]));
 static const int64_t kDefaultWorkspace = 2ll << 30;
@@ -106,6 +109,7 @@ bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, 
     MapGeom g;
     make_geom(*P, B_Q, B_KV, N, heads, &g);
     if (g.sQ128 * g.sK > 64) return false;  // one 64-bit membership word per 128-row slot
+    if (P->split_pmax > 32) return false;   // the merge kernel keeps up to 32 partial LSEs in registers
     const int max_st = attention_max_stages(d, P->T_KV, P->kernel);
     if (max_st < 2) return false;
     if (P->stages > max_st) return false;
