@@ -1295,11 +1295,27 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 // partial row sum, converted whenever the reference it last saw has moved; the sums are added in
 // the epilogue.  P has its own TMEM columns, so S[x] is free again as soon as warpgroup x has
 // read it into registers (`s_free`).
-//   warps 0-3 / 4-7 : softmax warpgroups 0 / 1      warp 8 : TMA producer
+//   warps 0-3 / 4-7 : softmax warpgroups 0 / 1      warp 8 : K/V TMA producer    warp 11 : Q TMA producer
 //   warp 9 : Q K^T issuer      warp 10 : P V issuer  (warps 8-11 give registers back)
 // TMEM columns: S0 0, S1 128, O 256, P0 384, P1 448.
 // ==========================================================================================
 constexpr int kPpThreads = 384;
+
+// Work item `idx` through the read-only path (items are written by the planner before the launch), or an
+// empty item past the end of the list.
+__device__ __forceinline__ WorkItem load_item(const WorkItem* items, int idx, int n_items) {
+    WorkItem it;
+    if (idx < n_items) {
+        const int4* src = reinterpret_cast<const int4*>(items + idx);
+        const int4 a = __ldg(src), b = __ldg(src + 1);
+        it.head = a.x; it.q_tile = a.y; it.tile_begin = a.z; it.tile_end = a.w;
+        it.part = b.x; it.nparts = b.y; it.ws_slot = b.z; it.ntiles = b.w;
+    } else {
+        it.head = it.q_tile = it.tile_begin = it.tile_end = it.part = it.ws_slot = it.ntiles = 0;
+        it.nparts = 1;
+    }
+    return it;
+}
 
 struct __align__(8) PpBarriers {
     uint64_t q_full, q_empty, o_free, l_bar;
@@ -1375,16 +1391,15 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         reg_dec<72>();
         if (warp == 8 && lane == 0) {
             // =========================== TMA producer ===========================
-            uint32_t itq = 0, g = 0;
+            // K and V only: this thread never waits for the Q buffer, so it keeps the rings full across work
+            // item boundaries (the Q tile is loaded by the thread of warp 11)
+            uint32_t g = 0;
             bool ok = true;
+            WorkItem it_next = load_item(p.items, blockIdx.x, n_items);  // work items are fetched one item ahead
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
-                const WorkItem it = p.items[idx];
+                const WorkItem it = it_next;
+                it_next = load_item(p.items, idx + gridDim.x, n_items);
                 if (it.ntiles == 0) continue;
-                ok = mbar_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1, abortp);
-                if (!ok) break;
-                mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
-                for (int s = 0; s < NSUB; ++s)
-                    tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, it.q_tile * kTQ, it.head);
                 int col_next = p.tile_col[it.tile_begin];
                 for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
                     const int col_cur = col_next;
@@ -1405,6 +1420,25 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         tma_load_3d(smem_u32(sV + stage * KV_TILE + s * KV_SUB), &tmV, smem_u32(&bars.v_full[stage]),
                                     s * 64, kv0, it.head);
                 }
+            }
+            if (!ok) {
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        } else if (warp == 11 && lane == 0) {
+            // =========================== Q producer ===========================
+            uint32_t itq = 0;
+            bool ok = true;
+            WorkItem it_next = load_item(p.items, blockIdx.x, n_items);
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const WorkItem it = it_next;
+                it_next = load_item(p.items, idx + gridDim.x, n_items);
+                if (it.ntiles == 0) continue;
+                ok = mbar_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1, abortp);
+                if (!ok) break;
+                mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
+                for (int s = 0; s < NSUB; ++s)
+                    tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, it.q_tile * kTQ, it.head);
                 ++itq;
             }
             if (!ok) {
@@ -1419,8 +1453,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             uint32_t itq = 0, g = 0;
             bool ok = true;
             BSA_TRACE_DECL(tn);
+            int n_next = load_item(p.items, blockIdx.x, n_items).ntiles;
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
-                const int n = p.items[idx].ntiles;
+                const int n = n_next;
+                n_next = load_item(p.items, idx + gridDim.x, n_items).ntiles;
                 if (n == 0) continue;
                 ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
                 if (!ok) break;
@@ -1459,8 +1495,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             uint32_t itq = 0, g = 0;
             bool ok = true;
             BSA_TRACE_DECL(tn);
+            int n_next = load_item(p.items, blockIdx.x, n_items).ntiles;
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
-                const int n = p.items[idx].ntiles;
+                const int n = n_next;
+                n_next = load_item(p.items, idx + gridDim.x, n_items).ntiles;
                 if (n == 0) continue;
                 for (int j = 0; j < n; ++j) {
                     const uint32_t gp = g + j;
@@ -1514,9 +1552,33 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             seen = k + 1;
             return got;
         };
+        // work items are fetched two items ahead and the first tile's metadata one item ahead, so that neither the
+        // item nor the metadata that depends on it is waited for at an item boundary
+        WorkItem it_next = load_item(p.items, blockIdx.x, n_items);
+        WorkItem it_next2 = load_item(p.items, blockIdx.x + gridDim.x, n_items);
+        int first_col = 0;
+        unsigned long long first_member = 0ull;
+        {
+            const int j0n = ((g & 1) == (uint32_t)x) ? 0 : 1;
+            if (j0n < it_next.ntiles) {
+                first_col = __ldg(p.tile_col + it_next.tile_begin + j0n);
+                first_member = __ldg(p.tile_member + it_next.tile_begin + j0n);
+            }
+        }
         for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
-            const WorkItem it = p.items[idx];
+            const WorkItem it = it_next;
+            it_next = it_next2;
+            it_next2 = load_item(p.items, idx + 2 * gridDim.x, n_items);
             const int n = it.ntiles;
+            int col_next = first_col;
+            unsigned long long member_next = first_member;
+            {   // the next item's first tile of this warpgroup: its parity follows from g + n
+                const int j0n = (((g + n) & 1) == (uint32_t)x) ? 0 : 1;
+                if (j0n < it_next.ntiles) {
+                    first_col = __ldg(p.tile_col + it_next.tile_begin + j0n);
+                    first_member = __ldg(p.tile_member + it_next.tile_begin + j0n);
+                }
+            }
             const int row = it.q_tile * kTQ + tw;
             const bool row_ok = row < p.N;
             if (n == 0) {
@@ -1532,12 +1594,6 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             float l = 0.f;
             // first local tile index of this warpgroup inside the item
             const int j0 = ((g & 1) == (uint32_t)x) ? 0 : 1;
-            int col_next = 0;
-            unsigned long long member_next = 0ull;
-            if (j0 < n) {
-                col_next = p.tile_col[it.tile_begin + j0];
-                member_next = p.tile_member[it.tile_begin + j0];
-            }
             for (int j = j0; j < n; j += 2) {
                 const uint32_t gs = g + j;
                 const int kv0 = col_next * TK;
@@ -1549,6 +1605,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
                 const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
                 const int n_valid = p.N - kv0;
+                if (lane == 0 && j == j0) BSA_TRACE_POINT(2 + warp, tn, 35);
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), (gs >> 1) & 1, abortp));
                 if (!ok) break;
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 10);
@@ -1655,60 +1712,64 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     if (!ok) break;
                     m_final = mref[x ^ 1][tw];
                 }
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 30);
                 if (m_final != m_know) l *= ex2_approx(m_know - m_final);
                 // Wait for the item's last P V before touching `lsum`: that MMA could only be issued after BOTH
                 // warpgroups finished the previous item's epilogue (o_free), i.e. after they read the previous sums.
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[gl & 1]), (gl >> 1) & 1, abortp));
                 if (!ok) break;
                 tc_fence_after();
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 31);
                 const uint32_t par = luse & 1;
                 lsum[x][tw] = l;
                 mbar_arrive(smem_u32(&bars.l_bar));
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.l_bar), par, abortp));
                 if (!ok) break;
                 ++luse;
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 32);
                 const float l_tot = lsum[0][tw] + lsum[1][tw];
                 const float inv_l = (l_tot > 0.f) ? 1.f / l_tot : 0.f;
                 const float lse = (l_tot > 0.f) ? fmaf(m_final, 0.6931471805599453f, logf(l_tot)) : -INFINITY;
                 const uint32_t t_oh = t_o + x * DC;
+                // this warpgroup's half of the accumulator goes to registers; the accumulator is then free for the
+                // next item's first P V while the scaling and the global stores proceed
+                uint32_t o[DC];
+#pragma unroll
+                for (int c = 0; c < DC / 32; ++c) tmem_ld32(t_oh + c * 32, &o[c * 32]);
+                tc_wait_ld();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.o_free));
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 33);
+#ifdef BSA_ABL_NOSTORE
+                if (inv_l == 12345.f)
+#endif
                 if (it.nparts == 1) {
-                    __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D + x * DC;
+                    if (row_ok) {
+                        __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D + x * DC;
+                        // 32-byte stores: every thread fills whole 32-byte sectors of its own row
 #pragma unroll
-                    for (int c = 0; c < DC / 32; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(t_oh + c * 32, o);
-                        tc_wait_ld();
-                        if (row_ok) {
+                        for (int q = 0; q < DC / 16; ++q) {
+                            uint32_t v[8];
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                uint4 v;
-                                v.x = pack_bf16x2(__uint_as_float(o[q * 8 + 0]) * inv_l, __uint_as_float(o[q * 8 + 1]) * inv_l);
-                                v.y = pack_bf16x2(__uint_as_float(o[q * 8 + 2]) * inv_l, __uint_as_float(o[q * 8 + 3]) * inv_l);
-                                v.z = pack_bf16x2(__uint_as_float(o[q * 8 + 4]) * inv_l, __uint_as_float(o[q * 8 + 5]) * inv_l);
-                                v.w = pack_bf16x2(__uint_as_float(o[q * 8 + 6]) * inv_l, __uint_as_float(o[q * 8 + 7]) * inv_l);
-                                *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = v;
-                            }
+                            for (int e = 0; e < 8; ++e)
+                                v[e] = pack_bf16x2(__uint_as_float(o[q * 16 + 2 * e]) * inv_l,
+                                                   __uint_as_float(o[q * 16 + 2 * e + 1]) * inv_l);
+                            st_global_v8(orow + q * 16, v);
                         }
+                        if (x == 0) p.LSE[(size_t)it.head * p.N + row] = lse;
                     }
-                    if (row_ok && x == 0) p.LSE[(size_t)it.head * p.N + row] = lse;
                 } else {
                     float* orow = p.ws_O + ((size_t)it.ws_slot * kTQ + tw) * D + x * DC;
 #pragma unroll
-                    for (int c = 0; c < DC / 32; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(t_oh + c * 32, o);
-                        tc_wait_ld();
+                    for (int q = 0; q < DC / 8; ++q) {
+                        uint32_t v[8];
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            float4 v = make_float4(__uint_as_float(o[q * 4 + 0]) * inv_l, __uint_as_float(o[q * 4 + 1]) * inv_l,
-                                                   __uint_as_float(o[q * 4 + 2]) * inv_l, __uint_as_float(o[q * 4 + 3]) * inv_l);
-                            *reinterpret_cast<float4*>(orow + c * 32 + q * 4) = v;
-                        }
+                        for (int e = 0; e < 8; ++e) v[e] = __float_as_uint(__uint_as_float(o[q * 8 + e]) * inv_l);
+                        st_global_v8(orow + q * 8, v);
                     }
                     if (x == 0) p.ws_LSE[(size_t)it.ws_slot * kTQ + tw] = lse;
                 }
-                tc_fence_before();
-                mbar_arrive(smem_u32(&bars.o_free));
+                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 34);
             }
             g += n;
         }
