@@ -23,10 +23,11 @@ namespace bsa {
 
 using namespace ptx;
 
+
 // Optional timeline tracing (compile with -DBSA_TRACE): CTA 0 records clock64() at barrier events of the
 // single-tile kernel, per role, into a device buffer that bsa_debug_trace_copy() reads back.
 #ifdef BSA_TRACE
-__device__ long long g_trace[11][4096];  // producer, Q K^T (or single) issuer, softmax warps 0-7, P V issuer (role 6 in the 7-warp kernel)
+__device__ long long g_trace[12][4096];  // producer, Q K^T (or single) issuer, softmax warps 0-7, P V issuer (role 6 in the 7-warp kernel)
 __device__ long long g_trace_aux[12][4];  // last tile's stamps inside softmax_tile, per warp
 #define BSA_TRACE_DECL(n) int n = 0
 #define BSA_TRACE_POINT(role, n, tag)                                              \
@@ -1292,14 +1293,20 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 // XU pipe and the tensor pipe both stay fed.  One O accumulator is shared: both warpgroups
 // follow the SAME reference maximum per row, handed from tile to tile through shared memory
 // (`mref`, one float per row, published right after a tile's max phase).  Each warpgroup keeps a
-// partial row sum, converted whenever the reference it last saw has moved; the sums are added in
-// the epilogue.  P has its own TMEM columns, so S[x] is free again as soon as warpgroup x has
-// read it into registers (`s_free`).
-//   warps 0-3 / 4-7 : softmax warpgroups 0 / 1      warp 8 : K/V TMA producer    warp 11 : Q TMA producer
-//   warp 9 : Q K^T issuer      warp 10 : P V issuer  (warps 8-11 give registers back)
+// partial row sum, converted whenever the reference it last saw has moved.  P has its own TMEM
+// columns, so S[x] is free again as soon as warpgroup x has read it into registers (`s_free`).
+// A third warpgroup owns the epilogue: at the end of a work item the softmax warpgroups only hand
+// over their row sums (expressed in the item's final reference) and move straight on to the next
+// item's tiles; the epilogue warpgroup waits for the item's last P V, drains the accumulator,
+// normalises and stores, and releases the accumulator for the next item's first P V, which cannot
+// be issued before that item's first softmax tile is done anyway.
+//   warps 0-3 / 4-7 : softmax warpgroups 0 / 1      warp 8 : K and Q TMA producer   warp 11 : V TMA producer
+//   warp 9 : Q K^T issuer      warp 10 : P V issuer    warps 12-15 : epilogue warpgroup
+// Registers (setmaxnreg): softmax 192, epilogue 80, producers and issuers 48 per thread; the sum over the CTA,
+// 256*192 + 128*80 + 128*48 = 65536, is exactly the launch allocation of 512 threads x 128.
 // TMEM columns: S0 0, S1 128, O 256, P0 384, P1 448.
 // ==========================================================================================
-constexpr int kPpThreads = 384;
+constexpr int kPpThreads = 512;
 
 // Work item `idx` through the read-only path (items are written by the planner before the launch), or an
 // empty item past the end of the list.
@@ -1318,7 +1325,7 @@ __device__ __forceinline__ WorkItem load_item(const WorkItem* items, int idx, in
 }
 
 struct __align__(8) PpBarriers {
-    uint64_t q_full, q_empty, o_free, l_bar;
+    uint64_t q_full, q_empty, o_free, o_full, e_ready, e_taken;
     uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
     uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2], mx_bar[2];
 };
@@ -1331,7 +1338,6 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     constexpr int Q_SUB = kTQ * 128;
     constexpr int KV_SUB = TK * 128;
     constexpr int KV_TILE = NSUB * KV_SUB;
-    constexpr int DC = D / 2;  // output columns each warpgroup stores in the epilogue
     // dynamic shared memory starts on a 1024-byte boundary (the swizzled tiles need it); checked below
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* sQ = smem;
@@ -1339,7 +1345,8 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     uint8_t* sV = sK + p.stages * KV_TILE;
     __shared__ PpBarriers bars;
     __shared__ float mref[2][kTQ];   // [publishing warpgroup][row]: reference maximum after that warpgroup's latest tile
-    __shared__ float lsum[2][kTQ];   // [warpgroup][row]: partial row sums, exchanged in the epilogue
+    __shared__ float lfin[2][kTQ];   // [warpgroup][row]: an item's partial row sums in its final reference
+    __shared__ float mfin[kTQ];      // the item's final reference maximum (log2 domain) per row
     __shared__ uint32_t tmem_base_s;
     __shared__ uint32_t abort_flag;
 
@@ -1354,8 +1361,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         abort_flag = 0;
         mbar_init(smem_u32(&bars.q_full), 1);
         mbar_init(smem_u32(&bars.q_empty), 1);
-        mbar_init(smem_u32(&bars.o_free), 256);
-        mbar_init(smem_u32(&bars.l_bar), 256);
+        mbar_init(smem_u32(&bars.o_free), 128);   // epilogue threads: accumulator drained
+        mbar_init(smem_u32(&bars.o_full), 1);     // P V issuer: the item's last P V has completed
+        mbar_init(smem_u32(&bars.e_ready), 256);  // softmax threads: row sums of the item are in shared memory
+        mbar_init(smem_u32(&bars.e_taken), 128);  // epilogue threads: row sums read
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(&bars.k_full[s]), 1);
             mbar_init(smem_u32(&bars.k_empty[s]), 1);
@@ -1387,15 +1396,157 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     volatile uint32_t* abortp = &abort_flag;
     const int n_items = p.counters->nitems;
 
-    if (warp >= 8) {
-        reg_dec<72>();
+    if (warp >= 12) {
+        // =========================== epilogue warpgroup ===========================
+        reg_dec<80>();
+        const int tw = tid & 127;
+        const uint32_t t_o = tmem + ((uint32_t)((warp & 3) * 32) << 16) + kColO;
+        uint32_t itn = 0;  // non-empty items seen
+        bool ok = true;
+        BSA_TRACE_DECL(tn);
+        WorkItem it_next = load_item(p.items, blockIdx.x, n_items);
+        for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            const WorkItem it = it_next;
+            it_next = load_item(p.items, idx + gridDim.x, n_items);
+            const int row = it.q_tile * kTQ + tw;
+            const bool row_ok = row < p.N;
+            if (it.ntiles == 0) {  // no active column: zero output, LSE = -inf
+                if (row_ok) {
+                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D);
+#pragma unroll
+                    for (int c = 0; c < D / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
+                    p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
+                }
+                continue;
+            }
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.e_ready), itn & 1, abortp));
+            if (!ok) break;
+            const float l_tot = lfin[0][tw] + lfin[1][tw];
+            const float m_final = mfin[tw];
+            mbar_arrive(smem_u32(&bars.e_taken));
+            const float inv_l = (l_tot > 0.f) ? 1.f / l_tot : 0.f;
+            const float lse = (l_tot > 0.f) ? fmaf(m_final, 0.6931471805599453f, logf(l_tot)) : -INFINITY;
+            if (lane == 0) BSA_TRACE_POINT(11, tn, 32);
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_full), itn & 1, abortp));
+            if (!ok) break;
+            tc_fence_after();
+            if (lane == 0) BSA_TRACE_POINT(11, tn, 31);
+            ++itn;
+            __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D;
+            float* wrow = p.ws_O + ((size_t)it.ws_slot * kTQ + tw) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(t_o + c * 32, o);
+                tc_wait_ld();
+                if (c == D / 32 - 1) {  // the accumulator is in registers: the next item's first P V may overwrite it
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&bars.o_free));
+                    if (lane == 0) BSA_TRACE_POINT(11, tn, 33);
+                }
+#ifdef BSA_ABL_NOSTORE
+                if (inv_l == 12345.f)
+#endif
+                if (it.nparts == 1) {
+                    if (row_ok) {  // 32-byte stores: every thread fills whole 32-byte sectors of its own row
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            uint32_t v[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                v[e] = pack_bf16x2(__uint_as_float(o[q * 16 + 2 * e]) * inv_l,
+                                                   __uint_as_float(o[q * 16 + 2 * e + 1]) * inv_l);
+                            st_global_v8(orow + c * 32 + q * 16, v);
+                        }
+                    }
+                } else {  // Split-K partial: normalised fp32 rows in the workspace
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t v[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) v[e] = __float_as_uint(__uint_as_float(o[q * 8 + e]) * inv_l);
+                        st_global_v8(wrow + c * 32 + q * 8, v);
+                    }
+                }
+            }
+            if (it.nparts == 1) {
+                if (row_ok) p.LSE[(size_t)it.head * p.N + row] = lse;
+            } else {
+                p.ws_LSE[(size_t)it.ws_slot * kTQ + tw] = lse;
+            }
+            if (lane == 0) BSA_TRACE_POINT(11, tn, 34);
+        }
+    } else if (warp >= 8) {
+        reg_dec<48>();
         if (warp == 8 && lane == 0) {
-            // =========================== TMA producer ===========================
-            // K and V only: this thread never waits for the Q buffer, so it keeps the rings full across work
-            // item boundaries (the Q tile is loaded by the thread of warp 11)
+            // =========================== K and Q producer ===========================
+            // K tiles run up to NS tiles ahead of the Q K^T issuer and never wait for V slots (the V tiles have a
+            // thread of their own in warp 11).  The Q tile of a new item may only be loaded once the previous
+            // item's last Q K^T has completed; that is the same event that frees the K slot NS-1 tiles into the new
+            // item, so pending Q loads are kept in a short queue and issued right before that K load: this thread
+            // never blocks on the Q buffer while K slots are still free.
+            uint32_t g = 0, itq = 0;
+            bool ok = true;
+            BSA_TRACE_DECL(tn);
+            int pq_row0 = 0, pq_row1 = 0, pq_row2 = 0, pq_head0 = 0, pq_head1 = 0, pq_head2 = 0;
+            int pq_need0 = 0, pq_need1 = 0, pq_need2 = 0, npend = 0;
+            auto issue_q = [&]() -> bool {  // loads the oldest pending Q tile
+                if (!mbar_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1, abortp)) return false;
+                mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
+                for (int s = 0; s < NSUB; ++s)
+                    tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, pq_row0, pq_head0);
+                ++itq;
+                pq_row0 = pq_row1; pq_head0 = pq_head1; pq_need0 = pq_need1;
+                pq_row1 = pq_row2; pq_head1 = pq_head2; pq_need1 = pq_need2;
+                --npend;
+                return true;
+            };
+            WorkItem it_next = load_item(p.items, blockIdx.x, n_items);  // work items are fetched one item ahead
+            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+                const WorkItem it = it_next;
+                it_next = load_item(p.items, idx + gridDim.x, n_items);
+                if (it.ntiles == 0) continue;
+                {   // queue this item's Q tile: it needs the Q K^T of global tile g-1 (the previous item's last)
+                    const int qrow = it.q_tile * kTQ, need = (int)g - 1;
+                    if (npend == 0) { pq_row0 = qrow; pq_head0 = it.head; pq_need0 = need; }
+                    else if (npend == 1) { pq_row1 = qrow; pq_head1 = it.head; pq_need1 = need; }
+                    else { pq_row2 = qrow; pq_head2 = it.head; pq_need2 = need; }
+                    ++npend;
+                    if (g == 0) ok = issue_q();  // the first item: the buffer is free
+                }
+                int col_next = p.tile_col[it.tile_begin];
+                for (int j = it.tile_begin; j < it.tile_end && ok; ++j, ++g) {
+                    const int col_cur = col_next;
+                    if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
+                    const int stage = g % NS;
+                    const uint32_t ph = (g / NS) & 1;
+                    // Q tiles whose condition is implied by this K slot's (Q K^T of tile g-NS done)
+                    // (or that are found free already: a Q tile takes priority over K tiles far ahead)
+                    while (ok && npend > 0 &&
+                           (pq_need0 <= (int)g - NS || mbar_test_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1)))
+                        ok = issue_q();
+                    if (!ok) break;
+                    BSA_TRACE_POINT(0, tn, 19);
+                    ok = mbar_wait(smem_u32(&bars.k_empty[stage]), ph ^ 1, abortp);
+                    if (!ok) break;
+                    BSA_TRACE_POINT(0, tn, 20);
+                    mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), KV_TILE);
+                    for (int s = 0; s < NSUB; ++s)
+                        tma_load_3d(smem_u32(sK + stage * KV_TILE + s * KV_SUB), &tmK, smem_u32(&bars.k_full[stage]),
+                                    s * 64, col_cur * TK, it.head);
+                    BSA_TRACE_POINT(0, tn, 21);
+                }
+            }
+            while (ok && npend > 0) ok = issue_q();
+            if (!ok) {
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        } else if (warp == 11 && lane == 0) {
+            // =========================== V producer ===========================
             uint32_t g = 0;
             bool ok = true;
-            WorkItem it_next = load_item(p.items, blockIdx.x, n_items);  // work items are fetched one item ahead
+            WorkItem it_next = load_item(p.items, blockIdx.x, n_items);
             for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
                 const WorkItem it = it_next;
                 it_next = load_item(p.items, idx + gridDim.x, n_items);
@@ -1406,40 +1557,13 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
                     const int stage = g % NS;
                     const uint32_t ph = (g / NS) & 1;
-                    const int kv0 = col_cur * TK;
-                    ok = mbar_wait(smem_u32(&bars.k_empty[stage]), ph ^ 1, abortp);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), KV_TILE);
-                    for (int s = 0; s < NSUB; ++s)
-                        tma_load_3d(smem_u32(sK + stage * KV_TILE + s * KV_SUB), &tmK, smem_u32(&bars.k_full[stage]),
-                                    s * 64, kv0, it.head);
                     ok = mbar_wait(smem_u32(&bars.v_empty[stage]), ph ^ 1, abortp);
                     if (!ok) break;
                     mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), KV_TILE);
                     for (int s = 0; s < NSUB; ++s)
                         tma_load_3d(smem_u32(sV + stage * KV_TILE + s * KV_SUB), &tmV, smem_u32(&bars.v_full[stage]),
-                                    s * 64, kv0, it.head);
+                                    s * 64, col_cur * TK, it.head);
                 }
-            }
-            if (!ok) {
-                const uint64_t t0 = globaltimer_ns();
-                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
-            }
-        } else if (warp == 11 && lane == 0) {
-            // =========================== Q producer ===========================
-            uint32_t itq = 0;
-            bool ok = true;
-            WorkItem it_next = load_item(p.items, blockIdx.x, n_items);
-            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
-                const WorkItem it = it_next;
-                it_next = load_item(p.items, idx + gridDim.x, n_items);
-                if (it.ntiles == 0) continue;
-                ok = mbar_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1, abortp);
-                if (!ok) break;
-                mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
-                for (int s = 0; s < NSUB; ++s)
-                    tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, it.q_tile * kTQ, it.head);
-                ++itq;
             }
             if (!ok) {
                 const uint64_t t0 = globaltimer_ns();
@@ -1509,6 +1633,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     BSA_TRACE_POINT(10, tn, 3);
                     ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
                     if (!ok) break;
+                    BSA_TRACE_POINT(10, tn, 4);
                     if (j == 0) {
                         ok = mbar_wait(smem_u32(&bars.o_free), (itq & 1) ^ 1, abortp);
                         if (!ok) break;
@@ -1522,6 +1647,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     }
                     mma_commit(smem_u32(&bars.v_empty[stage]));
                     mma_commit(smem_u32(&bars.pv_done[sb]));
+                    if (j == n - 1) mma_commit(smem_u32(&bars.o_full));
                     BSA_TRACE_POINT(10, tn, 5);
                 }
                 g += n;
@@ -1530,7 +1656,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         }
     } else {
         // =========================== softmax warpgroup x ===========================
-        reg_inc<216>();
+        reg_inc<192>();
         const int x = warp >> 2;
         const int tw = tid & 127;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -1539,7 +1665,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         const uint32_t t_o = tmem + lane_base + kColO;
         uint32_t g = 0;          // running tile index at the start of the current item (all warpgroups agree)
         uint32_t seen = 0;       // publishes of the OTHER warpgroup already waited for (they are consumed in order)
-        uint32_t luse = 0;       // uses of l_bar
+        uint32_t itn = 0;        // non-empty items finished
         bool ok = true;
         BSA_TRACE_DECL(tn);
         const float c2 = p.scale_log2;
@@ -1579,17 +1705,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     first_member = __ldg(p.tile_member + it_next.tile_begin + j0n);
                 }
             }
-            const int row = it.q_tile * kTQ + tw;
-            const bool row_ok = row < p.N;
-            if (n == 0) {
-                if (row_ok) {
-                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D + x * DC);
-#pragma unroll
-                    for (int c = 0; c < DC / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
-                    if (x == 0) p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
-                }
-                continue;
-            }
+            if (n == 0) continue;  // the epilogue warpgroup writes the empty rows
             float m_know = -INFINITY;  // reference maximum this thread's partial sum l is expressed in
             float l = 0.f;
             // first local tile index of this warpgroup inside the item
@@ -1633,6 +1749,9 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     m3 = max3(m3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
                 }
                 const float mx2 = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c2;
+#ifdef BSA_TRACE
+                if (lane == 0 && mx2 != 12345.f) BSA_TRACE_POINT(2 + warp, tn, 17);
+#endif
                 // ---- reference maximum handed over from the previous tile (other warpgroup) ----
                 float m_prev = -INFINITY;
                 if (gs > 0) {
@@ -1640,6 +1759,9 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     if (!ok) break;
                     if (j > 0) m_prev = mref[x ^ 1][tw];  // the previous tile belongs to this item
                 }
+#ifdef BSA_TRACE
+                if (lane == 0 && m_prev != 12345.f) BSA_TRACE_POINT(2 + warp, tn, 18);
+#endif
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 12);
                 if (m_prev != m_know) {  // the other warpgroup moved the reference since this thread last looked
                     l *= ex2_approx(m_know - m_prev);  // m_know = -inf only while l = 0
@@ -1703,73 +1825,25 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 16);
             }
             if (!ok) break;
-            // ---- epilogue: bring both partial sums to the final reference, add them, store half of the row each ----
+            // ---- hand this warpgroup's row sums, expressed in the item's final reference, to the epilogue warpgroup ----
             {
                 const uint32_t gl = g + n - 1;  // last tile of the item
+                const bool owner = (gl & 1) == (uint32_t)x;
                 float m_final = m_know;
-                if ((gl & 1) != (uint32_t)x) {  // the other warpgroup took the last tile: its publish holds the final reference
+                if (!owner) {  // the other warpgroup took the last tile: its publish holds the final reference
                     ok = __all_sync(0xffffffffu, wait_publish(gl));
                     if (!ok) break;
                     m_final = mref[x ^ 1][tw];
                 }
+                if (m_final != m_know) l *= ex2_approx(m_know - m_final);  // l = 0 whenever m_know = -inf
+                // the previous item's sums must have been read
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.e_taken), (itn & 1) ^ 1, abortp));
+                if (!ok) break;
+                lfin[x][tw] = l;
+                if (owner) mfin[tw] = m_final;
+                mbar_arrive(smem_u32(&bars.e_ready));
+                ++itn;
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 30);
-                if (m_final != m_know) l *= ex2_approx(m_know - m_final);
-                // Wait for the item's last P V before touching `lsum`: that MMA could only be issued after BOTH
-                // warpgroups finished the previous item's epilogue (o_free), i.e. after they read the previous sums.
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[gl & 1]), (gl >> 1) & 1, abortp));
-                if (!ok) break;
-                tc_fence_after();
-                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 31);
-                const uint32_t par = luse & 1;
-                lsum[x][tw] = l;
-                mbar_arrive(smem_u32(&bars.l_bar));
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.l_bar), par, abortp));
-                if (!ok) break;
-                ++luse;
-                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 32);
-                const float l_tot = lsum[0][tw] + lsum[1][tw];
-                const float inv_l = (l_tot > 0.f) ? 1.f / l_tot : 0.f;
-                const float lse = (l_tot > 0.f) ? fmaf(m_final, 0.6931471805599453f, logf(l_tot)) : -INFINITY;
-                const uint32_t t_oh = t_o + x * DC;
-                // this warpgroup's half of the accumulator goes to registers; the accumulator is then free for the
-                // next item's first P V while the scaling and the global stores proceed
-                uint32_t o[DC];
-#pragma unroll
-                for (int c = 0; c < DC / 32; ++c) tmem_ld32(t_oh + c * 32, &o[c * 32]);
-                tc_wait_ld();
-                tc_fence_before();
-                mbar_arrive(smem_u32(&bars.o_free));
-                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 33);
-#ifdef BSA_ABL_NOSTORE
-                if (inv_l == 12345.f)
-#endif
-                if (it.nparts == 1) {
-                    if (row_ok) {
-                        __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D + x * DC;
-                        // 32-byte stores: every thread fills whole 32-byte sectors of its own row
-#pragma unroll
-                        for (int q = 0; q < DC / 16; ++q) {
-                            uint32_t v[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                v[e] = pack_bf16x2(__uint_as_float(o[q * 16 + 2 * e]) * inv_l,
-                                                   __uint_as_float(o[q * 16 + 2 * e + 1]) * inv_l);
-                            st_global_v8(orow + q * 16, v);
-                        }
-                        if (x == 0) p.LSE[(size_t)it.head * p.N + row] = lse;
-                    }
-                } else {
-                    float* orow = p.ws_O + ((size_t)it.ws_slot * kTQ + tw) * D + x * DC;
-#pragma unroll
-                    for (int q = 0; q < DC / 8; ++q) {
-                        uint32_t v[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) v[e] = __float_as_uint(__uint_as_float(o[q * 8 + e]) * inv_l);
-                        st_global_v8(orow + q * 8, v);
-                    }
-                    if (x == 0) p.ws_LSE[(size_t)it.ws_slot * kTQ + tw] = lse;
-                }
-                if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 34);
             }
             g += n;
         }
