@@ -1327,7 +1327,7 @@ __device__ __forceinline__ WorkItem load_item(const WorkItem* items, int idx, in
 struct __align__(8) PpBarriers {
     uint64_t q_full, q_empty, o_free, o_full, e_ready, e_taken;
     uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
-    uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2], mx_bar[2];
+    uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2];
 };
 
 template <int D, int TK>
@@ -1344,7 +1344,12 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     uint8_t* sK = sQ + NSUB * Q_SUB;
     uint8_t* sV = sK + p.stages * KV_TILE;
     __shared__ PpBarriers bars;
-    __shared__ float mref[2][kTQ];   // [publishing warpgroup][row]: reference maximum after that warpgroup's latest tile
+    // [publishing warpgroup][row]: the reference maximum after that warpgroup's latest tile.  One 32-bit word per
+    // row carries value and sequence together: reference values keep their two lowest mantissa bits clear, and
+    // the word's two low bits hold (publish index + 1) mod 4, so the reader of the next tile (always the same
+    // row's thread of the other warpgroup, which consumes every publish in order) needs one shared-memory
+    // read, with no barrier in front of it, to know whether the value it got is the one it waits for.
+    __shared__ uint32_t mref[2][kTQ];
     __shared__ float lfin[2][kTQ];   // [warpgroup][row]: an item's partial row sums in its final reference
     __shared__ float mfin[kTQ];      // the item's final reference maximum (log2 domain) per row
     __shared__ uint32_t tmem_base_s;
@@ -1376,10 +1381,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             mbar_init(smem_u32(&bars.s_free[s]), 128);
             mbar_init(smem_u32(&bars.p_ready[s]), 128);
             mbar_init(smem_u32(&bars.pv_done[s]), 1);
-            mbar_init(smem_u32(&bars.mx_bar[s]), 128);
         }
         fence_mbar_init();
     }
+    if (tid < 2 * kTQ) (&mref[0][0])[tid] = 0u;  // tag 0: matches no first publish
     if (warp == 9) {
         tmem_alloc(smem_u32(&tmem_base_s), kTmemCols);
         tmem_relinquish();
@@ -1535,6 +1540,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         tma_load_3d(smem_u32(sK + stage * KV_TILE + s * KV_SUB), &tmK, smem_u32(&bars.k_full[stage]),
                                     s * 64, col_cur * TK, it.head);
                     BSA_TRACE_POINT(0, tn, 21);
+#ifdef BSA_TRACE_KLAT
+                    mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
+                    BSA_TRACE_POINT(0, tn, 23);
+#endif
                 }
             }
             while (ok && npend > 0) ok = issue_q();
@@ -1588,13 +1597,12 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     const uint32_t gs = g + j;
                     const int stage = gs % NS;
                     const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
-                    ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
+                    // K tile present, and S[sb] read into registers by the softmax of tile gs-2
+                    if (gs >= 2)
+                        ok = mbar_wait2(smem_u32(&bars.s_free[sb]), ((gs >> 1) - 1) & 1, smem_u32(&bars.k_full[stage]), ph, abortp);
+                    else
+                        ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
                     if (!ok) break;
-                    BSA_TRACE_POINT(1, tn, 1);
-                    if (gs >= 2) {  // S[sb] has been read into registers by the softmax of tile gs-2
-                        ok = mbar_wait(smem_u32(&bars.s_free[sb]), ((gs >> 1) - 1) & 1, abortp);
-                        if (!ok) break;
-                    }
                     BSA_TRACE_POINT(1, tn, 6);
                     tc_fence_after();
                     const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
@@ -1628,16 +1636,16 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     const uint32_t gp = g + j;
                     const int stage = gp % NS;
                     const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
-                    ok = mbar_wait(smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
-                    if (!ok) break;
-                    BSA_TRACE_POINT(10, tn, 3);
-                    ok = mbar_wait(smem_u32(&bars.v_full[stage]), ph, abortp);
-                    if (!ok) break;
-                    BSA_TRACE_POINT(10, tn, 4);
+                    // V tile present (normally long before), accumulator drained by the epilogue (first tile of an
+                    // item), and last the P tile, which is the one this thread normally waits for
                     if (j == 0) {
                         ok = mbar_wait(smem_u32(&bars.o_free), (itq & 1) ^ 1, abortp);
                         if (!ok) break;
                     }
+                    ok = mbar_wait2(smem_u32(&bars.v_full[stage]), ph, smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
+                    if (!ok) break;
+                    BSA_TRACE_POINT(10, tn, 3);
+
                     tc_fence_after();
                     const uint32_t a_p = tmem + (sb ? kColP1 : kColP0);
 #pragma unroll
@@ -1664,19 +1672,35 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         const uint32_t t_p = tmem + lane_base + (x ? kColP1 : kColP0);
         const uint32_t t_o = tmem + lane_base + kColO;
         uint32_t g = 0;          // running tile index at the start of the current item (all warpgroups agree)
-        uint32_t seen = 0;       // publishes of the OTHER warpgroup already waited for (they are consumed in order)
         uint32_t itn = 0;        // non-empty items finished
         bool ok = true;
         BSA_TRACE_DECL(tn);
         const float c2 = p.scale_log2;
         const unsigned long long sub_mask = (p.sK >= 64) ? ~0ull : ((1ull << p.sK) - 1ull);
-        // wait until the other warpgroup has published the reference after global tile t (t has the other parity)
-        auto wait_publish = [&](uint32_t t) -> bool {
-            const uint32_t k = t >> 1;  // publish index inside the other warpgroup
-            if (seen > k) return true;
-            const bool got = mbar_wait(smem_u32(&bars.mx_bar[x ^ 1]), k & 1, abortp);
-            seen = k + 1;
-            return got;
+        // The reference after global tile t (taken by the other warpgroup), given a word read earlier from its slot:
+        // if that word already carries the publish's tag it is used, else the slot is polled (bounded).
+        auto take_reference = [&](uint32_t t, uint32_t word, float& m_out) -> bool {
+            const uint32_t tag = ((t >> 1) + 1) & 3u;
+            if ((word & 3u) != tag) {
+                volatile uint32_t* slot = &mref[x ^ 1][tw];
+                long long t0 = 0;
+                uint32_t spins = 0;
+                while (true) {
+                    word = *slot;
+                    if ((word & 3u) == tag) break;
+                    if ((++spins & 63u) == 0) {
+                        if (*abortp) return false;
+                        const long long now = clock64();
+                        if (t0 == 0) t0 = now;
+                        if (now - t0 > 4000000000ll) {
+                            *abortp = 1;
+                            return false;
+                        }
+                    }
+                }
+            }
+            m_out = __uint_as_float(word & ~3u);
+            return true;
         };
         // work items are fetched two items ahead and the first tile's metadata one item ahead, so that neither the
         // item nor the metadata that depends on it is waited for at an item boundary
@@ -1733,6 +1757,9 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.s_free[x]));  // S[x] is in registers: the next Q K^T into it may start
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 11);
+                // The previous tile's reference has normally been published by now: its slot is read here and the
+                // word checked after the max phase, so that the shared-memory round trip overlaps that phase.
+                const uint32_t ref_word = *reinterpret_cast<volatile uint32_t*>(&mref[x ^ 1][tw]);
                 if (need_mask) {
 #pragma unroll
                     for (int i = 0; i < TK; ++i) {
@@ -1754,10 +1781,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 #endif
                 // ---- reference maximum handed over from the previous tile (other warpgroup) ----
                 float m_prev = -INFINITY;
-                if (gs > 0) {
-                    ok = __all_sync(0xffffffffu, wait_publish(gs - 1));
+                if (gs > 0) {  // every publish is consumed, in order, also across item boundaries (the tags rely on it)
+                    float m_taken;
+                    ok = __all_sync(0xffffffffu, take_reference(gs - 1, ref_word, m_taken));
                     if (!ok) break;
-                    if (j > 0) m_prev = mref[x ^ 1][tw];  // the previous tile belongs to this item
+                    if (j > 0) m_prev = m_taken;  // the previous tile belongs to this item
                 }
 #ifdef BSA_TRACE
                 if (lane == 0 && m_prev != 12345.f) BSA_TRACE_POINT(2 + warp, tn, 18);
@@ -1770,13 +1798,14 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 float alpha = 1.f;
                 bool rescale = false;
                 if (mx2 > m_know + kRescaleThreshold) {
-                    alpha = ex2_approx(m_know - mx2);
+                    const float m_new = __uint_as_float(__float_as_uint(mx2) & ~3u);  // two low bits clear (see mref)
+                    alpha = ex2_approx(m_know - m_new);
                     rescale = (j > 0) && (m_know != -INFINITY);
                     l *= alpha;
-                    m_know = mx2;
+                    m_know = m_new;
                 }
-                mref[x][tw] = m_know;
-                mbar_arrive(smem_u32(&bars.mx_bar[x]));  // publish: the next tile's warpgroup may take its decision
+                // publish: the next tile's warpgroup may take its decision
+                *reinterpret_cast<volatile uint32_t*>(&mref[x][tw]) = __float_as_uint(m_know) | (((gs >> 1) + 1) & 3u);
                 const float neg_m = (m_know == -INFINITY) ? 0.f : -m_know;
                 const uint64_t c22 = pack_f32x2(c2, c2), nm2 = pack_f32x2(neg_m, neg_m);
                 uint64_t sum01 = pack_f32x2(0.f, 0.f), sum23 = sum01;
@@ -1831,9 +1860,9 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const bool owner = (gl & 1) == (uint32_t)x;
                 float m_final = m_know;
                 if (!owner) {  // the other warpgroup took the last tile: its publish holds the final reference
-                    ok = __all_sync(0xffffffffu, wait_publish(gl));
+                    ok = __all_sync(0xffffffffu,
+                                    take_reference(gl, *reinterpret_cast<volatile uint32_t*>(&mref[x ^ 1][tw]), m_final));
                     if (!ok) break;
-                    m_final = mref[x ^ 1][tw];
                 }
                 if (m_final != m_know) l *= ex2_approx(m_know - m_final);  // l = 0 whenever m_know = -inf
                 // the previous item's sums must have been read

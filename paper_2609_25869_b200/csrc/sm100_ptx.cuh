@@ -93,6 +93,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Bounded wait for two barriers.  Both are tested first, back to back, so that when both phases have completed the
+// thread pays one shared-memory round trip instead of two dependent ones.
+__device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b,
+                                           volatile uint32_t* abort_flag) {
+    const bool a = mbar_test_wait(bar_a, parity_a);
+    const bool b = mbar_test_wait(bar_b, parity_b);
+    if (!a && !mbar_wait(bar_a, parity_a, abort_flag)) return false;
+    if (!b && !mbar_wait(bar_b, parity_b, abort_flag)) return false;
+    return true;
+}
+
 // ---------------------------------------------------------------- TMA
 __device__ __forceinline__ void prefetch_tensormap(const void* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");

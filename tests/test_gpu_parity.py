@@ -163,6 +163,24 @@ def test_growing_scores_force_a_rescale_at_every_tile(plan_id):
     assert res["lse_max"] < 5e-4
 
 
+@pytest.mark.parametrize("name,plan_id", [("stress_b", 22), ("stress_b", 23), ("stress_b", 18), ("mid", 22), ("mid", 24),
+                                          ("stress_a", 23), ("tiny", 27)])
+def test_repeated_runs_are_bitwise_identical(name, plan_id):
+    """No atomics and a fixed accumulation order: six forwards of one plan give the same bits.  Long work items
+    (Stress-B has about a hundred tiles per item) give a timing-dependent hand-off the most chances to show."""
+    req = I.CONFIGS[name]()
+    mask, q, k, v, _ = Hh.to_dev(req, None)
+    with bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=plan_id) as plan:
+        O0, L0 = plan.forward(q, k, v)
+        torch.cuda.synchronize()
+        O0, L0 = O0.clone(), L0.clone()
+        for _ in range(5):
+            O, L = plan.forward(q, k, v)
+            torch.cuda.synchronize()
+            assert torch.equal(O, O0) and torch.equal(L, L0)
+        assert plan.info()["device_status"] == 0
+
+
 # ---------------------------------------------------------------- boundary behaviour
 def test_invalid_arguments_never_touch_the_gpu():
     import ctypes
