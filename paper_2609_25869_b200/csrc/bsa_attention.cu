@@ -1308,8 +1308,13 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
 // ==========================================================================================
 constexpr int kPpThreads = 512;
 
-// Work item `idx` through the read-only path (items are written by the planner before the launch), or an
-// empty item past the end of the list.
+// The k-th work item of CTA b out of G: rounds of G consecutive items, alternately dealt forwards and backwards.
+// Items arrive longest first, so dealing every round in the same direction would hand CTA 0 the longest item of
+// every round and the last CTA the shortest; reversing every other round evens the per-CTA sums out.
+__device__ __forceinline__ int cta_item_index(int k, int b, int G) { return k * G + ((k & 1) ? (G - 1 - b) : b); }
+
+// Work item `idx` through the read-only path (items are written by the planner before the launch); past the end
+// of the list the item has ntiles = -1 (an item with ntiles = 0 is a real row without active columns).
 __device__ __forceinline__ WorkItem load_item(const WorkItem* items, int idx, int n_items) {
     WorkItem it;
     if (idx < n_items) {
@@ -1318,8 +1323,9 @@ __device__ __forceinline__ WorkItem load_item(const WorkItem* items, int idx, in
         it.head = a.x; it.q_tile = a.y; it.tile_begin = a.z; it.tile_end = a.w;
         it.part = b.x; it.nparts = b.y; it.ws_slot = b.z; it.ntiles = b.w;
     } else {
-        it.head = it.q_tile = it.tile_begin = it.tile_end = it.part = it.ws_slot = it.ntiles = 0;
+        it.head = it.q_tile = it.tile_begin = it.tile_end = it.part = it.ws_slot = 0;
         it.nparts = 1;
+        it.ntiles = -1;
     }
     return it;
 }
@@ -1400,6 +1406,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     const uint32_t tmem = tmem_base_s;
     volatile uint32_t* abortp = &abort_flag;
     const int n_items = p.counters->nitems;
+    const int n_rounds = (n_items + (int)gridDim.x - 1) / (int)gridDim.x;
 
     if (warp >= 12) {
         // =========================== epilogue warpgroup ===========================
@@ -1409,12 +1416,13 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         uint32_t itn = 0;  // non-empty items seen
         bool ok = true;
         BSA_TRACE_DECL(tn);
-        WorkItem it_next = load_item(p.items, blockIdx.x, n_items);
-        for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+        WorkItem it_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);
+        for (int kr = 0; kr < n_rounds && ok; ++kr) {
             const WorkItem it = it_next;
-            it_next = load_item(p.items, idx + gridDim.x, n_items);
+            it_next = load_item(p.items, cta_item_index(kr + 1, blockIdx.x, gridDim.x), n_items);
             const int row = it.q_tile * kTQ + tw;
             const bool row_ok = row < p.N;
+            if (it.ntiles < 0) continue;  // past the end of the list
             if (it.ntiles == 0) {  // no active column: zero output, LSE = -inf
                 if (row_ok) {
                     uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D);
@@ -1506,11 +1514,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 --npend;
                 return true;
             };
-            WorkItem it_next = load_item(p.items, blockIdx.x, n_items);  // work items are fetched one item ahead
-            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            WorkItem it_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);  // work items are fetched one item ahead
+            for (int kr = 0; kr < n_rounds && ok; ++kr) {
                 const WorkItem it = it_next;
-                it_next = load_item(p.items, idx + gridDim.x, n_items);
-                if (it.ntiles == 0) continue;
+                it_next = load_item(p.items, cta_item_index(kr + 1, blockIdx.x, gridDim.x), n_items);
+                if (it.ntiles <= 0) continue;
                 {   // queue this item's Q tile: it needs the Q K^T of global tile g-1 (the previous item's last)
                     const int qrow = it.q_tile * kTQ, need = (int)g - 1;
                     if (npend == 0) { pq_row0 = qrow; pq_head0 = it.head; pq_need0 = need; }
@@ -1555,11 +1563,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             // =========================== V producer ===========================
             uint32_t g = 0;
             bool ok = true;
-            WorkItem it_next = load_item(p.items, blockIdx.x, n_items);
-            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            WorkItem it_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);
+            for (int kr = 0; kr < n_rounds && ok; ++kr) {
                 const WorkItem it = it_next;
-                it_next = load_item(p.items, idx + gridDim.x, n_items);
-                if (it.ntiles == 0) continue;
+                it_next = load_item(p.items, cta_item_index(kr + 1, blockIdx.x, gridDim.x), n_items);
+                if (it.ntiles <= 0) continue;
                 int col_next = p.tile_col[it.tile_begin];
                 for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
                     const int col_cur = col_next;
@@ -1586,11 +1594,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             uint32_t itq = 0, g = 0;
             bool ok = true;
             BSA_TRACE_DECL(tn);
-            int n_next = load_item(p.items, blockIdx.x, n_items).ntiles;
-            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            int n_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items).ntiles;
+            for (int kr = 0; kr < n_rounds && ok; ++kr) {
                 const int n = n_next;
-                n_next = load_item(p.items, idx + gridDim.x, n_items).ntiles;
-                if (n == 0) continue;
+                n_next = load_item(p.items, cta_item_index(kr + 1, blockIdx.x, gridDim.x), n_items).ntiles;
+                if (n <= 0) continue;
                 ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
                 if (!ok) break;
                 for (int j = 0; j < n; ++j) {
@@ -1627,11 +1635,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             uint32_t itq = 0, g = 0;
             bool ok = true;
             BSA_TRACE_DECL(tn);
-            int n_next = load_item(p.items, blockIdx.x, n_items).ntiles;
-            for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+            int n_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items).ntiles;
+            for (int kr = 0; kr < n_rounds && ok; ++kr) {
                 const int n = n_next;
-                n_next = load_item(p.items, idx + gridDim.x, n_items).ntiles;
-                if (n == 0) continue;
+                n_next = load_item(p.items, cta_item_index(kr + 1, blockIdx.x, gridDim.x), n_items).ntiles;
+                if (n <= 0) continue;
                 for (int j = 0; j < n; ++j) {
                     const uint32_t gp = g + j;
                     const int stage = gp % NS;
@@ -1704,8 +1712,8 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         };
         // work items are fetched two items ahead and the first tile's metadata one item ahead, so that neither the
         // item nor the metadata that depends on it is waited for at an item boundary
-        WorkItem it_next = load_item(p.items, blockIdx.x, n_items);
-        WorkItem it_next2 = load_item(p.items, blockIdx.x + gridDim.x, n_items);
+        WorkItem it_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);
+        WorkItem it_next2 = load_item(p.items, cta_item_index(1, blockIdx.x, gridDim.x), n_items);
         int first_col = 0;
         unsigned long long first_member = 0ull;
         {
@@ -1715,10 +1723,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 first_member = __ldg(p.tile_member + it_next.tile_begin + j0n);
             }
         }
-        for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+        for (int kr = 0; kr < n_rounds && ok; ++kr) {
             const WorkItem it = it_next;
             it_next = it_next2;
-            it_next2 = load_item(p.items, idx + 2 * gridDim.x, n_items);
+            it_next2 = load_item(p.items, cta_item_index(kr + 2, blockIdx.x, gridDim.x), n_items);
             const int n = it.ntiles;
             int col_next = first_col;
             unsigned long long member_next = first_member;
@@ -1729,7 +1737,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     first_member = __ldg(p.tile_member + it_next.tile_begin + j0n);
                 }
             }
-            if (n == 0) continue;  // the epilogue warpgroup writes the empty rows
+            if (n <= 0) continue;  // the epilogue warpgroup writes the empty rows
             float m_know = -INFINITY;  // reference maximum this thread's partial sum l is expressed in
             float l = 0.f;
             // first local tile index of this warpgroup inside the item
