@@ -164,8 +164,13 @@ extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int
     // ---- lines 3-5: only the scalars cross to the host ----
     static thread_local MaskStatsDev* pinned = nullptr;
     if (!pinned) BSA_CUDA(cudaMallocHost(&pinned, sizeof(MaskStatsDev)), "pinned stats");
+    static thread_local cudaEvent_t stats_copied = nullptr;
+    if (!stats_copied) BSA_CUDA(cudaEventCreateWithFlags(&stats_copied, cudaEventDisableTiming), "stats event");
     BSA_CUDA(cudaMemcpyAsync(pinned, p->stats, sizeof(MaskStatsDev), cudaMemcpyDeviceToHost, stream), "stats copy");
-    BSA_CUDA(cudaStreamSynchronize(stream), "stats sync");
+    BSA_CUDA(cudaEventRecord(stats_copied, stream), "stats event record");
+    // the row-pointer scan needs nothing from the host: it runs while the host waits for the scalars
+    BSA_CUDA(launch_row_scan(p->row_nnz, nrows, p->row_ptr, stream), "row_scan");
+    BSA_CUDA(cudaEventSynchronize(stats_copied), "stats sync");
     p->hstats = *pinned;
     const double t2 = now_us();
 
@@ -225,7 +230,6 @@ extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int
         BSA_CUDA(cudaMallocAsync(&p->ws_O, (size_t)p->ws_bytes, stream), "workspace");
         p->ws_LSE = p->ws_O + (size_t)p->max_items * g.T_Q * d;
     }
-    BSA_CUDA(launch_row_scan(p->row_nnz, nrows, p->row_ptr, stream), "row_scan");
     BSA_CUDA(launch_csr_fill(mask_dev, nrows, nKb, p->row_ptr, p->col_idx, stream), "csr_fill");
     BSA_CUDA(launch_tile_map(g, p->row_ptr, p->col_idx, p->desc.split_tau, pmax, p->tile_begin, p->tile_cnt,
                              p->row_parts, p->tile_col, p->tile_member, p->head_counts, p->counters, stream),

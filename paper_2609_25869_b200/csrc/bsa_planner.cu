@@ -342,7 +342,8 @@ __device__ __forceinline__ int32_t block_excl_scan(int32_t v, int32_t* warp_buf,
     return before + incl - v;
 }
 
-__global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, const int32_t* __restrict__ tile_begin,
+__global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, int rank_warps, int key_cap,
+                                                         const int32_t* __restrict__ tile_begin,
                                                          const int32_t* __restrict__ tile_cnt,
                                                          const int32_t* __restrict__ row_parts,
                                                          const int32_t* __restrict__ head_counts,
@@ -433,8 +434,45 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, co
     }
     __syncthreads();
 
-    // ---- C1: stable rank, one warp, items in order ----
-    if (tid < 32) {
+    // ---- C1: stable rank ----
+    if (rank_warps >= 2) {
+        // The group's items are cut into `rank_warps` contiguous chunks, one per warp: per-warp histograms, then for
+        // every length the warps' counts are turned into start offsets (bucket start + counts of the earlier chunks),
+        // then every warp ranks its own chunk in order.  Same ranks as the one-warp walk below.
+        int32_t* whist = key + key_cap;  // [rank_warps][nbins]
+        const int warp = tid >> 5, lane = tid & 31;
+        const int chunk = (((n_items + rank_warps - 1) / rank_warps) + 31) & ~31;
+        for (int i = tid; i < rank_warps * nbins; i += blockDim.x) whist[i] = 0;
+        __syncthreads();
+        const int c0 = warp * chunk, c1 = min(n_items, c0 + chunk);
+        if (warp < rank_warps)
+            for (int i = c0 + lane; i < c1; i += 32) atomicAdd(&whist[warp * nbins + key[i]], 1);
+        __syncthreads();
+        for (int b = tid; b < nbins; b += blockDim.x) {
+            int32_t run = bins[b];
+            for (int w = 0; w < rank_warps; ++w) {
+                const int32_t c = whist[w * nbins + b];
+                whist[w * nbins + b] = run;
+                run += c;
+            }
+        }
+        __syncthreads();
+        if (warp < rank_warps) {
+            int32_t* wb = whist + warp * nbins;
+            for (int i0 = c0; i0 < c1; i0 += 32) {
+                const int i = i0 + lane;
+                const bool valid = i < c1;
+                const int32_t k = valid ? key[i] : -1 - lane;  // invalid lanes get unique keys
+                const unsigned peers = __match_any_sync(kFull, k);
+                int32_t rank = 0;
+                if (valid) rank = wb[k] + __popc(peers & ((1u << lane) - 1u));
+                __syncwarp();
+                if (valid && (peers >> lane) <= 1u) wb[k] += __popc(peers);  // highest lane of the peer set
+                __syncwarp();
+                if (valid) key[i] = rank;
+            }
+        }
+    } else if (tid < 32) {
         for (int i0 = 0; i0 < n_items; i0 += 32) {
             const int i = i0 + tid;
             const bool valid = i < n_items;
@@ -506,24 +544,38 @@ cudaError_t launch_tile_map(const MapGeom& g, const int32_t* row_ptr, const int3
     return cudaGetLastError();
 }
 
-size_t organize_smem_bytes(const MapGeom& g, int order, int split_pmax) {
+static size_t organize_key_cap(const MapGeom& g, int order, int split_pmax) {
     const size_t rows = (order == BSA_ORDER_GLOBAL_LPT) ? (size_t)g.H * g.nQt : (size_t)g.nQt;
-    return ((size_t)g.nKt + 2 + rows * (size_t)(split_pmax < 1 ? 1 : split_pmax)) * sizeof(int32_t);
+    return rows * (size_t)(split_pmax < 1 ? 1 : split_pmax);
+}
+
+// Minimum (one ranking warp): length histogram + one key per item of a group.
+size_t organize_smem_bytes(const MapGeom& g, int order, int split_pmax) {
+    return ((size_t)g.nKt + 2 + organize_key_cap(g, order, split_pmax)) * sizeof(int32_t);
 }
 
 cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const int32_t* tile_begin,
                             const int32_t* tile_cnt, const int32_t* row_parts, const int32_t* head_counts,
                             WorkItem* items_tmp, WorkItem* items, SplitRow* split_rows, PlanCountersDev* counters,
                             cudaStream_t stream) {
-    // the caller checked organize_smem_bytes() against the device limit when it chose `order`
-    const size_t smem = organize_smem_bytes(g, order, split_pmax);
-    if (smem > 48 * 1024) {
+    // the caller checked organize_smem_bytes() against the device limit when it chose `order`; whatever shared
+    // memory is left up to 200 KB holds per-warp histograms for the parallel ranking (up to one per warp)
+    const size_t base = organize_smem_bytes(g, order, split_pmax);
+    const size_t per_warp = ((size_t)g.nKt + 2) * sizeof(int32_t);
+    const size_t budget = 200 * 1024;
+    int rank_warps = base < budget ? (int)((budget - base) / per_warp) : 0;
+    if (rank_warps > 32) rank_warps = 32;
+    if (rank_warps < 2) rank_warps = 0;
+    const size_t smem = base + (size_t)rank_warps * per_warp;
+    static size_t attr_bytes = 48 * 1024;
+    if (smem > attr_bytes) {
         cudaError_t e = cudaFuncSetAttribute(organize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
+        attr_bytes = smem;
     }
     const int grid = (order == BSA_ORDER_GLOBAL_LPT) ? 1 : g.H;
-    organize_kernel<<<grid, 1024, smem, stream>>>(g, order, tile_begin, tile_cnt, row_parts, head_counts, items_tmp,
-                                                   items, split_rows, counters);
+    organize_kernel<<<grid, 1024, smem, stream>>>(g, order, rank_warps, (int)organize_key_cap(g, order, split_pmax), tile_begin,
+                                                   tile_cnt, row_parts, head_counts, items_tmp, items, split_rows, counters);
     count_launch();
     return cudaGetLastError();
 }
