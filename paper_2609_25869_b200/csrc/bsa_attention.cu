@@ -1623,6 +1623,12 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     mma_commit(smem_u32(&bars.k_empty[stage]));
                     mma_commit(smem_u32(&bars.s_full[sb]));
                     BSA_TRACE_POINT(1, tn, 2);
+#ifdef BSA_TRACE_LDS
+                    if (*abortp == 77u) ok = false;  // a dependent shared-memory read, to time one round trip
+                    BSA_TRACE_POINT(1, tn, 7);
+                    ok = mbar_wait(smem_u32(&bars.k_full[(gs + 1) % NS]), ((gs + 1) / NS) & 1, abortp) || true;
+                    BSA_TRACE_POINT(1, tn, 8);
+#endif
                     if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
                 }
                 g += n;
@@ -1817,6 +1823,15 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const float neg_m = (m_know == -INFINITY) ? 0.f : -m_know;
                 const uint64_t c22 = pack_f32x2(c2, c2), nm2 = pack_f32x2(neg_m, neg_m);
                 uint64_t sum01 = pack_f32x2(0.f, 0.f), sum23 = sum01;
+                // P[x] was last read by the P V of tile gs-2 (normally long complete).  With d = 64 it is waited for
+                // here and the P tile stored 32 columns at a time while the next columns are still being exponentiated
+                // (+4 % on Stress-B); with d = 128 the stores follow the loop (the split loop was 1-2 % slower there).
+                constexpr bool kStoreInLoop = (D == 64);
+                if (kStoreInLoop && gs >= 2) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x]), ((gs >> 1) - 1) & 1, abortp));
+                    if (!ok) break;
+                    tc_fence_after();
+                }
 #pragma unroll
                 for (int i = 0; i < TK; i += 4) {
                     float x0, x1, x2, x3;
@@ -1827,19 +1842,21 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     sum23 = add_f32x2(sum23, pack_f32x2(p2, p3));
                     r[i / 2] = pack_bf16x2(p0, p1);
                     r[i / 2 + 1] = pack_bf16x2(p2, p3);
+                    if (kStoreInLoop && (i & 31) == 28) tmem_st16(t_p + (i >> 5) * 16, &r[(i >> 5) * 16]);
                 }
                 float s0, s1, s2, s3;
                 unpack_f32x2(sum01, s0, s1);
                 unpack_f32x2(sum23, s2, s3);
                 l += (s0 + s1) + (s2 + s3);
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 14);
-                // P[x] was last read by the P V of tile gs-2
-                if (gs >= 2) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x]), ((gs >> 1) - 1) & 1, abortp));
-                    if (!ok) break;
-                }
+                if (!kStoreInLoop) {
+                    if (gs >= 2) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x]), ((gs >> 1) - 1) & 1, abortp));
+                        if (!ok) break;
+                    }
 #pragma unroll
-                for (int c = 0; c < TK / 32; ++c) tmem_st16(t_p + c * 16, &r[c * 16]);
+                    for (int c = 0; c < TK / 32; ++c) tmem_st16(t_p + c * 16, &r[c * 16]);
+                }
                 // ---- the reference moved at this tile: rescale the running output (after the P V of tile gs-1) ----
                 if (j > 0 && __any_sync(0xffffffffu, rescale)) {
                     const uint32_t gp = gs - 1;
