@@ -1623,12 +1623,6 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     mma_commit(smem_u32(&bars.k_empty[stage]));
                     mma_commit(smem_u32(&bars.s_full[sb]));
                     BSA_TRACE_POINT(1, tn, 2);
-#ifdef BSA_TRACE_LDS
-                    if (*abortp == 77u) ok = false;  // a dependent shared-memory read, to time one round trip
-                    BSA_TRACE_POINT(1, tn, 7);
-                    ok = mbar_wait(smem_u32(&bars.k_full[(gs + 1) % NS]), ((gs + 1) / NS) & 1, abortp) || true;
-                    BSA_TRACE_POINT(1, tn, 8);
-#endif
                     if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
                 }
                 g += n;

@@ -76,9 +76,6 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // consulted only every 64 failed polls (each poll already suspends the thread for a while), and the
 // slow %globaltimer is never read on this path.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
-#ifdef BSA_TEST_FIRST
-    if (mbar_test_wait(bar, parity)) return true;
-#endif
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = 0;
     uint32_t spins = 0;
