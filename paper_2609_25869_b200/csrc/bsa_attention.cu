@@ -89,10 +89,12 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, bool ne
     if ((threadIdx.x & 31) == 0 && blockIdx.x == 0) g_trace_aux[threadIdx.x >> 5][0] = clock64();
 #endif
     if (need_mask) {
+        // B_KV >= 16: a group of 16 key columns lies inside one logical block, so one activity bit serves the group
 #pragma unroll
-        for (int i = 0; i < TK; ++i) {
-            const bool act = ((row_bits >> (i >> lgBKV)) & 1u) && (i < n_valid);
-            r[i] = act ? r[i] : 0xff800000u;  // -inf
+        for (int gq = 0; gq < TK / 16; ++gq) {
+            const bool grp = (row_bits >> ((gq * 16) >> lgBKV)) & 1u;
+#pragma unroll
+            for (int i = gq * 16; i < gq * 16 + 16; ++i) r[i] = (grp && i < n_valid) ? r[i] : 0xff800000u;  // -inf
         }
     }
     float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
@@ -1330,8 +1332,24 @@ __device__ __forceinline__ WorkItem load_item(const WorkItem* items, int idx, in
     return it;
 }
 
+// The two fields of a work item the softmax warpgroups need, prefetched into registers with loads that stay put.
+struct ItemSpan {
+    int tile_begin, ntiles;  // ntiles = -1 past the end of the list
+};
+__device__ __forceinline__ ItemSpan load_item_span(const WorkItem* items, int idx, int n_items) {
+    ItemSpan r;
+    r.tile_begin = 0;
+    r.ntiles = -1;
+    if (idx < n_items) {
+        const int* w = reinterpret_cast<const int*>(items + idx);
+        r.tile_begin = ldg_pinned_s32(w + 2);
+        r.ntiles = ldg_pinned_s32(w + 7);
+    }
+    return r;
+}
+
 struct __align__(8) PpBarriers {
-    uint64_t q_full, q_empty, o_free, o_full, e_ready, e_taken;
+    uint64_t q_full[2], q_empty[2], o_free, o_full, e_ready, e_taken;
     uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
     uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2];
 };
@@ -1346,9 +1364,9 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     constexpr int KV_TILE = NSUB * KV_SUB;
     // dynamic shared memory starts on a 1024-byte boundary (the swizzled tiles need it); checked below
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint8_t* sQ = smem;
-    uint8_t* sK = sQ + NSUB * Q_SUB;
-    uint8_t* sV = sK + p.stages * KV_TILE;
+    uint8_t* sQ = smem;                      // two Q tiles: the next item's is loaded while this one's is in use
+    uint8_t* sK = sQ + 2 * NSUB * Q_SUB;     // NSK K tiles (a K tile lives from its load to the end of its Q K^T)
+    uint8_t* sV = sK + p.stages * KV_TILE;   // NSV V tiles (a V tile lives about two tiles longer, until its P V)
     __shared__ PpBarriers bars;
     // [publishing warpgroup][row]: the reference maximum after that warpgroup's latest tile.  One 32-bit word per
     // row carries value and sequence together: reference values keep their two lowest mantissa bits clear, and
@@ -1366,12 +1384,14 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         if (tid == 0) atomicExch(&p.counters->status, (int)BSA_ERR_CUDA);
         return;
     }
-    const int NS = p.stages;
+    const int NSK = p.stages, NSV = p.stages_v;
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(smem_u32(&bars.q_full), 1);
-        mbar_init(smem_u32(&bars.q_empty), 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bars.q_full[b]), 1);
+            mbar_init(smem_u32(&bars.q_empty[b]), 1);
+        }
         mbar_init(smem_u32(&bars.o_free), 128);   // epilogue threads: accumulator drained
         mbar_init(smem_u32(&bars.o_full), 1);     // P V issuer: the item's last P V has completed
         mbar_init(smem_u32(&bars.e_ready), 256);  // softmax threads: row sums of the item are in shared memory
@@ -1447,7 +1467,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             ++itn;
             __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D;
             float* wrow = p.ws_O + ((size_t)it.ws_slot * kTQ + tw) * D;
-#pragma unroll
+#pragma unroll 1  // once per item: a rolled loop keeps the kernel's code small
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[32];
                 tmem_ld32(t_o + c * 32, o);
@@ -1493,50 +1513,65 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         reg_dec<48>();
         if (warp == 8 && lane == 0) {
             // =========================== K and Q producer ===========================
-            // K tiles run up to NS tiles ahead of the Q K^T issuer and never wait for V slots (the V tiles have a
-            // thread of their own in warp 11).  The Q tile of a new item may only be loaded once the previous
-            // item's last Q K^T has completed; that is the same event that frees the K slot NS-1 tiles into the new
-            // item, so pending Q loads are kept in a short queue and issued right before that K load: this thread
-            // never blocks on the Q buffer while K slots are still free.
-            uint32_t g = 0, itq = 0;
+            // K tiles run up to NSK tiles ahead of the Q K^T issuer and never wait for V slots (the V tiles have a
+            // thread of their own in warp 11).  Q tiles alternate between two buffers: an item's Q tile may be
+            // loaded once the last Q K^T of the item two before it has completed, so it is queued when this thread
+            // enters the item BEFORE it and issued as soon as that condition is implied by a K slot this thread has
+            // already waited for (Q K^T of tile g-NSK done) or is found true: this thread never blocks on a Q buffer
+            // while K slots are free, and a new item's first Q K^T does not wait for its Q tile.
+            uint32_t g = 0, itq = 0;  // itq: Q tiles issued (buffer itq & 1)
+            uint32_t seq = 0;          // non-empty items entered
             bool ok = true;
             BSA_TRACE_DECL(tn);
             int pq_row0 = 0, pq_row1 = 0, pq_row2 = 0, pq_head0 = 0, pq_head1 = 0, pq_head2 = 0;
             int pq_need0 = 0, pq_need1 = 0, pq_need2 = 0, npend = 0;
+            uint32_t queued = 0;             // Q tiles queued so far (= sequence number of the next item to queue)
+            int buf_last0 = -1000000, buf_last1 = -1000000;  // last global tile of the item that last used each buffer
             auto issue_q = [&]() -> bool {  // loads the oldest pending Q tile
-                if (!mbar_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1, abortp)) return false;
-                mbar_arrive_expect_tx(smem_u32(&bars.q_full), NSUB * Q_SUB);
+                const uint32_t b = itq & 1;
+                if (!mbar_wait(smem_u32(&bars.q_empty[b]), ((itq >> 1) & 1) ^ 1, abortp)) return false;
+                mbar_arrive_expect_tx(smem_u32(&bars.q_full[b]), NSUB * Q_SUB);
                 for (int s = 0; s < NSUB; ++s)
-                    tma_load_3d(smem_u32(sQ + s * Q_SUB), &tmQ, smem_u32(&bars.q_full), s * 64, pq_row0, pq_head0);
+                    tma_load_3d(smem_u32(sQ + b * NSUB * Q_SUB + s * Q_SUB), &tmQ, smem_u32(&bars.q_full[b]), s * 64, pq_row0,
+                                pq_head0);
                 ++itq;
                 pq_row0 = pq_row1; pq_head0 = pq_head1; pq_need0 = pq_need1;
                 pq_row1 = pq_row2; pq_head1 = pq_head2; pq_need1 = pq_need2;
                 --npend;
                 return true;
             };
-            WorkItem it_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);  // work items are fetched one item ahead
+            // queue the Q tile of an item whose tiles are [first, first + n): it needs its buffer's previous user done
+            auto queue_q = [&](const WorkItem& w, int first, int n) -> bool {
+                while (npend >= 3)  // queue full (many short items ahead of the Q K^T issuer): wait for a buffer
+                    if (!issue_q()) return false;
+                const uint32_t b = queued & 1;
+                const int qrow = w.q_tile * kTQ, need = b ? buf_last1 : buf_last0;
+                if (npend == 0) { pq_row0 = qrow; pq_head0 = w.head; pq_need0 = need; }
+                else if (npend == 1) { pq_row1 = qrow; pq_head1 = w.head; pq_need1 = need; }
+                else { pq_row2 = qrow; pq_head2 = w.head; pq_need2 = need; }
+                ++npend;
+                if (b) buf_last1 = first + n - 1; else buf_last0 = first + n - 1;
+                ++queued;
+                return true;
+            };
+            WorkItem it_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);
             for (int kr = 0; kr < n_rounds && ok; ++kr) {
                 const WorkItem it = it_next;
                 it_next = load_item(p.items, cta_item_index(kr + 1, blockIdx.x, gridDim.x), n_items);
                 if (it.ntiles <= 0) continue;
-                {   // queue this item's Q tile: it needs the Q K^T of global tile g-1 (the previous item's last)
-                    const int qrow = it.q_tile * kTQ, need = (int)g - 1;
-                    if (npend == 0) { pq_row0 = qrow; pq_head0 = it.head; pq_need0 = need; }
-                    else if (npend == 1) { pq_row1 = qrow; pq_head1 = it.head; pq_need1 = need; }
-                    else { pq_row2 = qrow; pq_head2 = it.head; pq_need2 = need; }
-                    ++npend;
-                    if (g == 0) ok = issue_q();  // the first item: the buffer is free
-                }
+                if (queued == seq) ok = queue_q(it, (int)g, it.ntiles);  // not queued ahead (first item, or after an empty one)
+                if (ok && it_next.ntiles > 0 && queued == seq + 1) ok = queue_q(it_next, (int)g + it.ntiles, it_next.ntiles);
+                if (!ok) break;
+                ++seq;
                 int col_next = p.tile_col[it.tile_begin];
                 for (int j = it.tile_begin; j < it.tile_end && ok; ++j, ++g) {
                     const int col_cur = col_next;
                     if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
-                    const int stage = g % NS;
-                    const uint32_t ph = (g / NS) & 1;
-                    // Q tiles whose condition is implied by this K slot's (Q K^T of tile g-NS done)
-                    // (or that are found free already: a Q tile takes priority over K tiles far ahead)
+                    const int stage = g % NSK;
+                    const uint32_t ph = (g / NSK) & 1;
                     while (ok && npend > 0 &&
-                           (pq_need0 <= (int)g - NS || mbar_test_wait(smem_u32(&bars.q_empty), (itq & 1) ^ 1)))
+                           (pq_need0 <= (int)g - NSK ||
+                            mbar_test_wait(smem_u32(&bars.q_empty[itq & 1]), ((itq >> 1) & 1) ^ 1)))
                         ok = issue_q();
                     if (!ok) break;
                     BSA_TRACE_POINT(0, tn, 19);
@@ -1572,8 +1607,8 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
                     const int col_cur = col_next;
                     if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
-                    const int stage = g % NS;
-                    const uint32_t ph = (g / NS) & 1;
+                    const int stage = g % NSV;
+                    const uint32_t ph = (g / NSV) & 1;
                     ok = mbar_wait(smem_u32(&bars.v_empty[stage]), ph ^ 1, abortp);
                     if (!ok) break;
                     mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), KV_TILE);
@@ -1589,7 +1624,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         } else if (warp == 9 && lane == 0) {
             // =========================== Q K^T issuer ===========================
             constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
-            const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
+            const uint64_t descQ0 = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
             const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
             uint32_t itq = 0, g = 0;
             bool ok = true;
@@ -1599,12 +1634,14 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const int n = n_next;
                 n_next = load_item(p.items, cta_item_index(kr + 1, blockIdx.x, gridDim.x), n_items).ntiles;
                 if (n <= 0) continue;
-                ok = mbar_wait(smem_u32(&bars.q_full), itq & 1, abortp);
+                const uint32_t qb = itq & 1;  // this item's Q buffer
+                ok = mbar_wait(smem_u32(&bars.q_full[qb]), (itq >> 1) & 1, abortp);
                 if (!ok) break;
+                const uint64_t descQ = descQ0 + (uint64_t)((qb * NSUB * Q_SUB) >> 4);
                 for (int j = 0; j < n; ++j) {
                     const uint32_t gs = g + j;
-                    const int stage = gs % NS;
-                    const uint32_t ph = (gs / NS) & 1, sb = gs & 1;
+                    const int stage = gs % NSK;
+                    const uint32_t ph = (gs / NSK) & 1, sb = gs & 1;
                     // K tile present, and S[sb] read into registers by the softmax of tile gs-2
                     if (gs >= 2)
                         ok = mbar_wait2(smem_u32(&bars.s_free[sb]), ((gs >> 1) - 1) & 1, smem_u32(&bars.k_full[stage]), ph, abortp);
@@ -1623,7 +1660,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     mma_commit(smem_u32(&bars.k_empty[stage]));
                     mma_commit(smem_u32(&bars.s_full[sb]));
                     BSA_TRACE_POINT(1, tn, 2);
-                    if (j == n - 1) mma_commit(smem_u32(&bars.q_empty));
+                    if (j == n - 1) mma_commit(smem_u32(&bars.q_empty[qb]));
                 }
                 g += n;
                 ++itq;
@@ -1642,8 +1679,8 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (n <= 0) continue;
                 for (int j = 0; j < n; ++j) {
                     const uint32_t gp = g + j;
-                    const int stage = gp % NS;
-                    const uint32_t ph = (gp / NS) & 1, sb = gp & 1;
+                    const int stage = gp % NSV;
+                    const uint32_t ph = (gp / NSV) & 1, sb = gp & 1;
                     // V tile present (normally long before), accumulator drained by the epilogue (first tile of an
                     // item), and last the P tile, which is the one this thread normally waits for
                     if (j == 0) {
@@ -1712,29 +1749,29 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         };
         // work items are fetched two items ahead and the first tile's metadata one item ahead, so that neither the
         // item nor the metadata that depends on it is waited for at an item boundary
-        WorkItem it_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);
-        WorkItem it_next2 = load_item(p.items, cta_item_index(1, blockIdx.x, gridDim.x), n_items);
+        ItemSpan it_next = load_item_span(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);
+        ItemSpan it_next2 = load_item_span(p.items, cta_item_index(1, blockIdx.x, gridDim.x), n_items);
         int first_col = 0;
         unsigned long long first_member = 0ull;
         {
             const int j0n = ((g & 1) == (uint32_t)x) ? 0 : 1;
             if (j0n < it_next.ntiles) {
-                first_col = __ldg(p.tile_col + it_next.tile_begin + j0n);
-                first_member = __ldg(p.tile_member + it_next.tile_begin + j0n);
+                first_col = ldg_pinned_s32(p.tile_col + it_next.tile_begin + j0n);
+                first_member = ldg_pinned_u64(p.tile_member + it_next.tile_begin + j0n);
             }
         }
         for (int kr = 0; kr < n_rounds && ok; ++kr) {
-            const WorkItem it = it_next;
+            const ItemSpan it = it_next;
             it_next = it_next2;
-            it_next2 = load_item(p.items, cta_item_index(kr + 2, blockIdx.x, gridDim.x), n_items);
+            it_next2 = load_item_span(p.items, cta_item_index(kr + 2, blockIdx.x, gridDim.x), n_items);
             const int n = it.ntiles;
             int col_next = first_col;
             unsigned long long member_next = first_member;
             {   // the next item's first tile of this warpgroup: its parity follows from g + n
                 const int j0n = (((g + n) & 1) == (uint32_t)x) ? 0 : 1;
                 if (j0n < it_next.ntiles) {
-                    first_col = __ldg(p.tile_col + it_next.tile_begin + j0n);
-                    first_member = __ldg(p.tile_member + it_next.tile_begin + j0n);
+                    first_col = ldg_pinned_s32(p.tile_col + it_next.tile_begin + j0n);
+                    first_member = ldg_pinned_u64(p.tile_member + it_next.tile_begin + j0n);
                 }
             }
             if (n <= 0) continue;  // the epilogue warpgroup writes the empty rows
@@ -1747,8 +1784,8 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const int kv0 = col_next * TK;
                 const unsigned long long member = member_next;
                 if (j + 2 < n) {
-                    col_next = p.tile_col[it.tile_begin + j + 2];
-                    member_next = p.tile_member[it.tile_begin + j + 2];
+                    col_next = ldg_pinned_s32(p.tile_col + it.tile_begin + j + 2);
+                    member_next = ldg_pinned_u64(p.tile_member + it.tile_begin + j + 2);
                 }
                 const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
                 const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
@@ -1769,10 +1806,15 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 // word checked after the max phase, so that the shared-memory round trip overlaps that phase.
                 const uint32_t ref_word = *reinterpret_cast<volatile uint32_t*>(&mref[x ^ 1][tw]);
                 if (need_mask) {
+                    // B_KV >= 16, so a group of 16 key columns lies inside one logical block: one activity bit per
+                    // group, two instructions per element.  (Skipping, per warp, the groups none of its 32 rows needs
+                    // was tried and lost: a warpgroup still waits for its slowest warp, and the branches cost more
+                    // than the exponentials they save.)
 #pragma unroll
-                    for (int i = 0; i < TK; ++i) {
-                        const bool act = ((row_bits >> (i >> p.lgBKV)) & 1u) && (i < n_valid);
-                        r[i] = act ? r[i] : 0xff800000u;
+                    for (int gq = 0; gq < TK / 16; ++gq) {
+                        const bool grp = (row_bits >> ((gq * 16) >> p.lgBKV)) & 1u;
+#pragma unroll
+                        for (int i = gq * 16; i < gq * 16 + 16; ++i) r[i] = (grp && i < n_valid) ? r[i] : 0xff800000u;
                     }
                 }
                 float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
@@ -1857,7 +1899,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x ^ 1]), (gp >> 1) & 1, abortp));
                     if (!ok) break;
                     tc_fence_after();
-#pragma unroll
+#pragma unroll 1  // rare path: kept small
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t o[32];
                         tmem_ld32(t_o + c * 32, o);
@@ -2040,29 +2082,36 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
 static int static_smem_bytes(int kernel) { return (kernel == 2 || kernel == 4) ? 3072 : 1024; }
 
 static int kv_buffers_that_fit(int d, int T_KV, int kernel) {
-    const int q = (kernel == 1 ? 2 : 1) * kTQ * d * 2;
+    const int q = ((kernel == 1 || kernel == 4) ? 2 : 1) * kTQ * d * 2;  // kernel 1: two Q slots; kernel 4: two Q buffers
     const int kv = T_KV * d * 2;
     return (232448 - static_smem_bytes(kernel) - q) / kv;
 }
 
-static void split_stages(int total, int* nk, int* nv) {
-    *nk = total / 2;
-    *nv = total - *nk;  // V is held one step longer than K, it gets the odd buffer
+static void split_stages(int total, int kernel, int* nk, int* nv) {
+    if (kernel == 4) {
+        // a K tile lives for one tile period (load -> its Q K^T), a V tile for about three (load -> its P V): two K
+        // buffers measured as fast as three, so V gets three fifths
+        *nk = total * 2 / 5;
+        if (*nk < 2) *nk = 2;
+    } else {
+        *nk = total / 2;  // V is held one step longer than K, it gets the odd buffer
+    }
+    *nv = total - *nk;
     if (*nk > kMaxStages) *nk = kMaxStages;
     if (*nv > kMaxStages) *nv = kMaxStages;
 }
 
 int attention_max_stages(int d, int T_KV, int kernel) {
     const int nb = kv_buffers_that_fit(d, T_KV, kernel);
-    if (kernel == 1) return nb > 2 * kMaxStages ? 2 * kMaxStages : nb;
+    if (kernel == 1 || kernel == 4) return nb > 2 * kMaxStages ? 2 * kMaxStages : nb;  // total K + V buffers
     const int s = nb / 2;
     return s > kMaxStages ? kMaxStages : s;
 }
 
 int attention_smem_bytes(int d, int T_KV, int stages, int kernel) {
-    const int q = (kernel == 1 ? 2 : 1) * kTQ * d * 2;
+    const int q = ((kernel == 1 || kernel == 4) ? 2 : 1) * kTQ * d * 2;
     const int kv = T_KV * d * 2;
-    int need = q + (kernel == 1 ? stages : 2 * stages) * kv;
+    int need = q + ((kernel == 1 || kernel == 4) ? stages : 2 * stages) * kv;
     // more than half of the SM's shared memory, so exactly one CTA (and one 512-column TMEM allocation) per SM
     if (need < 120 * 1024) need = 120 * 1024;
     return need;
@@ -2092,7 +2141,7 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     p.sK = a.g.sK;
     p.stages = a.stages;
     p.stages_v = a.stages;
-    if (a.kernel == 1) split_stages(a.stages, &p.stages, &p.stages_v);
+    if (a.kernel == 1 || a.kernel == 4) split_stages(a.stages, a.kernel, &p.stages, &p.stages_v);
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)a.d));
     cudaError_t e;
     const int key = a.kernel * 1000 + a.d + a.g.T_KV / 64;  // kernel, d, T_KV

@@ -244,6 +244,20 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t* v) {
                  : "memory");
 }
 
+// Read-only global loads the compiler may neither delay nor duplicate: a prefetch into registers stays where it is
+// written (a plain load that is first used an iteration later tends to be moved next to that use, which puts its
+// latency back on the critical path).
+__device__ __forceinline__ int ldg_pinned_s32(const int* p) {
+    int v;
+    asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ unsigned long long ldg_pinned_u64(const uint64_t* p) {
+    unsigned long long v;
+    asm volatile("ld.global.nc.b64 %0, [%1];" : "=l"(v) : "l"(p));
+    return v;
+}
+
 // Three-input maximum and packed two-lane fp32 arithmetic (sm_100): they halve the number of
 // instructions the softmax loop issues around its exponentials.
 __device__ __forceinline__ float max3(float a, float b, float c) {
