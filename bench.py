@@ -28,7 +28,7 @@ sys.path.insert(0, ROOT)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch on the bench workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists for the workload)
-NCU_TRAFFIC_BYTES = {"mid": 201.9e6}  # 175.8 MB read + 26.1 MB written (profiles/attention_kernel_mid.md, capture B)
+NCU_TRAFFIC_BYTES = {"mid": 199.6e6}  # 174.5 MB read + 25.1 MB written (profiles/attention_kernel_mid.md, capture B)
 
 
 def load_peaks():
@@ -44,7 +44,7 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons while the timed region runs: NVML polled every 5 ms from a thread
+    """Samples SM clocks and throttle reasons while the timed region runs: NVML polled about every millisecond from a thread
     (read-only queries), or, where the NVML binding is missing, `nvidia-smi -lms 100`."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -77,7 +77,7 @@ class ClockSampler:
                 self.power.append(nv.nvmlDeviceGetPowerUsage(handle) / 1000.0)
             except Exception:
                 pass
-            time.sleep(0.005)
+            time.sleep(0.001)
 
     def start(self):
         try:
