@@ -59,18 +59,24 @@ __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __re
         const uint4* words = reinterpret_cast<const uint4*>(base & ~15ull);
         const long long rb = (long long)(base & 15ull) + (long long)row * nKb, re = rb + nKb;
         const long long w0 = rb >> 4, w1 = (re + 15) >> 4;
-        unsigned carry = 0;  // last byte of the previous step (bit 0)
+        // The next step's words are loaded before this step's are processed (two loads in flight per lane).  The last
+        // byte of a step does not know its right neighbour yet: if its left neighbour is inactive it is counted one
+        // step later, by lane 0, once that neighbour (bit 0 of the next step) is known.
+        unsigned carry = 0;  // bits 1:0 = the previous step's last two bytes (bit 1 = the last one)
+        unsigned m_next = row_word_bits(words, w0 + lane, rb, re);
         for (long long w = w0; w < w1; w += 32) {
-            const unsigned m = row_word_bits(words, w + lane, rb, re);
+            const unsigned m = m_next;
+            m_next = (w + 32 < w1) ? row_word_bits(words, w + 32 + lane, rb, re) : 0u;
             // neighbours across lanes: previous lane's bit 15, next lane's bit 0
             unsigned prev15 = __shfl_up_sync(kFull, m >> 15, 1);
             unsigned next0 = __shfl_down_sync(kFull, m & 1u, 1);
-            if (lane == 0) prev15 = carry;
-            if (lane == 31) next0 = (w + 32 < w1) ? (row_word_bits(words, w + 32, rb, re) & 1u) : 0u;
+            if (lane == 0) prev15 = carry >> 1;
+            if (lane == 31) next0 = 0u;
             const unsigned left = ((m << 1) | prev15) & 0xffffu, right = (m >> 1) | (next0 << 15);
             nnz += __popc(m);
             runs += __popc(m & (left | right));
-            carry = __shfl_sync(kFull, m >> 15, 31);
+            if (lane == 0 && carry == 2u && (m & 1u)) ++runs;  // previous step's last byte: active, left inactive, right active
+            carry = __shfl_sync(kFull, (m >> 14) & 3u, 31);
         }
         for (int o = 16; o > 0; o >>= 1) {
             nnz += __shfl_down_sync(kFull, nnz, o);
@@ -167,8 +173,10 @@ __global__ void __launch_bounds__(256) csr_fill_kernel(const uint8_t* __restrict
     const long long rb = (long long)(base & 15ull) + (long long)row * nKb, re = rb + nKb;
     const long long w0 = rb >> 4, w1 = (re + 15) >> 4;
     int32_t out = row_ptr[row];
+    unsigned m_next = row_word_bits(words, w0 + lane, rb, re);
     for (long long w = w0; w < w1; w += 32) {
-        unsigned m = row_word_bits(words, w + lane, rb, re);
+        unsigned m = m_next;  // the next step's words are loaded before this step's are written out
+        m_next = (w + 32 < w1) ? row_word_bits(words, w + 32 + lane, rb, re) : 0u;
         const int cnt = __popc(m);
         int incl = cnt;
         for (int o = 1; o < 32; o <<= 1) {
@@ -203,16 +211,10 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
     extern __shared__ unsigned long long bm[];  // [slots][nKt]: one membership word per 128-row slot
     __shared__ int32_t warp_cnt[8];
     __shared__ int32_t warp_slot_cnt[8];
-    __shared__ int32_t running;
-    __shared__ int32_t running_slots;
     const int trow = blockIdx.x;
     const int h = trow / g.nQt, t = trow % g.nQt;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int i = tid; i < g.nKt * g.slots; i += blockDim.x) bm[i] = 0ull;
-    if (tid == 0) {
-        running = 0;
-        running_slots = 0;
-    }
     __syncthreads();
 
     int32_t cap_begin;
@@ -262,40 +264,47 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
     }
     __syncthreads();
 
-    for (int i0 = 0; i0 < g.nKt; i0 += blockDim.x) {
-        const int i = i0 + tid;
-        const unsigned long long w0 = (i < g.nKt) ? bm[i] : 0ull;
-        const unsigned long long w1 = (i < g.nKt && g.slots == 2) ? bm[g.nKt + i] : 0ull;
+    // Compaction in column order.  Each warp owns a contiguous range of tile columns: it counts its non-zero words,
+    // the eight counts are exchanged once, and the warp walks its range again to write them out (two block
+    // barriers in all, whatever the number of tile columns).
+    const int chunk = ((g.nKt + 255) / 256) * 32;
+    const int c0 = warp * chunk, c1 = min(g.nKt, c0 + chunk);
+    int32_t my_cnt = 0, my_slots = 0;
+    for (int i0 = c0; i0 < c1; i0 += 32) {
+        const int i = i0 + lane;
+        const unsigned long long w0 = (i < c1) ? bm[i] : 0ull;
+        const unsigned long long w1 = (i < c1 && g.slots == 2) ? bm[g.nKt + i] : 0ull;
+        my_cnt += __popc(__ballot_sync(kFull, (w0 | w1) != 0ull));
+        my_slots += __popc(__ballot_sync(kFull, w0 != 0ull)) + __popc(__ballot_sync(kFull, w1 != 0ull));
+    }
+    if (lane == 0) {
+        warp_cnt[warp] = my_cnt;
+        warp_slot_cnt[warp] = my_slots;
+    }
+    __syncthreads();
+    int32_t before = 0, total = 0, total_slots = 0;
+    for (int k = 0; k < 8; ++k) {
+        if (k < warp) before += warp_cnt[k];
+        total += warp_cnt[k];
+        total_slots += warp_slot_cnt[k];
+    }
+    int32_t pos0 = cap_begin + before;
+    for (int i0 = c0; i0 < c1; i0 += 32) {
+        const int i = i0 + lane;
+        const unsigned long long w0 = (i < c1) ? bm[i] : 0ull;
+        const unsigned long long w1 = (i < c1 && g.slots == 2) ? bm[g.nKt + i] : 0ull;
         const bool any = (w0 | w1) != 0ull;
         const unsigned bits = __ballot_sync(kFull, any);
-        const unsigned sbits0 = __ballot_sync(kFull, w0 != 0ull), sbits1 = __ballot_sync(kFull, w1 != 0ull);
-        if (lane == 0) {
-            warp_cnt[warp] = __popc(bits);
-            warp_slot_cnt[warp] = __popc(sbits0) + __popc(sbits1);
-        }
-        __syncthreads();
-        int32_t before = running;
-        int32_t total = 0, total_slots = 0;
-        for (int k = 0; k < 8; ++k) {
-            if (k < warp) before += warp_cnt[k];
-            total += warp_cnt[k];
-            total_slots += warp_slot_cnt[k];
-        }
         if (any) {
-            const int32_t pos = cap_begin + before + __popc(bits & ((1u << lane) - 1u));
+            const int32_t pos = pos0 + __popc(bits & ((1u << lane) - 1u));
             tile_col[pos] = i;
             tile_member[(size_t)pos * g.slots] = w0;
             if (g.slots == 2) tile_member[(size_t)pos * 2 + 1] = w1;
         }
-        __syncthreads();
-        if (tid == 0) {
-            running += total;
-            running_slots += total_slots;
-        }
-        __syncthreads();
+        pos0 += __popc(bits);
     }
     if (tid == 0) {
-        const int32_t cnt = running;
+        const int32_t cnt = total;
         tile_begin[trow] = cap_begin;
         tile_cnt[trow] = cnt;
         int32_t P = 1;
@@ -308,7 +317,7 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
         }
         if (cnt) {
             atomicAdd(&counters->ntiles, (unsigned long long)cnt);
-            atomicAdd(&counters->nslot_tiles, (unsigned long long)running_slots);
+            atomicAdd(&counters->nslot_tiles, (unsigned long long)total_slots);
         }
     }
 }
@@ -342,7 +351,7 @@ __device__ __forceinline__ int32_t block_excl_scan(int32_t v, int32_t* warp_buf,
     return before + incl - v;
 }
 
-__global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, int rank_warps, int key_cap,
+__global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, int rank_warps_max, int key_cap, int no_split,
                                                          const int32_t* __restrict__ tile_begin,
                                                          const int32_t* __restrict__ tile_cnt,
                                                          const int32_t* __restrict__ row_parts,
@@ -376,11 +385,17 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
     int32_t run_items = 0, run_split = 0, run_slots = 0;
     for (int r0 = row0; r0 < row1; r0 += blockDim.x) {
         const int r = r0 + tid;
-        const int32_t P = (r < row1) ? row_parts[r] : 0;
-        int32_t tot_i, tot_s, tot_w;
-        const int32_t off_i = block_excl_scan(P, warp_buf, &tot_i);
-        const int32_t off_s = block_excl_scan(P > 1 ? 1 : 0, warp_buf, &tot_s);
-        const int32_t off_w = block_excl_scan(P > 1 ? P : 0, warp_buf, &tot_w);
+        int32_t P, tot_i, tot_s = 0, tot_w = 0, off_i, off_s = 0, off_w = 0;
+        if (no_split) {  // the plan never splits a row: one item per row, no scans needed
+            P = (r < row1) ? 1 : 0;
+            off_i = tid;
+            tot_i = min((int)blockDim.x, row1 - r0);
+        } else {
+            P = (r < row1) ? row_parts[r] : 0;
+            off_i = block_excl_scan(P, warp_buf, &tot_i);
+            off_s = block_excl_scan(P > 1 ? 1 : 0, warp_buf, &tot_s);
+            off_w = block_excl_scan(P > 1 ? P : 0, warp_buf, &tot_w);
+        }
         if (r < row1) {
             const int32_t tb = tile_begin[r], cnt = tile_cnt[r];
             const int32_t slot = slot_base + run_slots + off_w;
@@ -388,8 +403,9 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
                 WorkItem it;
                 it.head = r / g.nQt;
                 it.q_tile = r % g.nQt;
-                it.tile_begin = tb + (int32_t)(((int64_t)cnt * p) / P);
-                it.tile_end = tb + (int32_t)(((int64_t)cnt * (p + 1)) / P);
+                // equal contiguous ranges (the 64-bit division only where a row is split)
+                it.tile_begin = (P == 1) ? tb : tb + (int32_t)(((int64_t)cnt * p) / P);
+                it.tile_end = (P == 1) ? tb + cnt : tb + (int32_t)(((int64_t)cnt * (p + 1)) / P);
                 it.part = p;
                 it.nparts = P;
                 it.ws_slot = (P > 1) ? (slot + p) * g.slots : -1;  // 128-row workspace slots
@@ -397,7 +413,6 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
                 const int32_t li = run_items + off_i + p;
                 items_tmp[item_base + li] = it;
                 key[li] = it.ntiles;
-                atomicAdd(&bins[it.ntiles], 1);
             }
             if (P > 1) {
                 for (int sl = 0; sl < g.slots; ++sl) {
@@ -416,6 +431,15 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
     }
     __syncthreads();
     const int32_t n_items = run_items;
+    // histogram of item lengths; lanes of a warp that hold the same length add once (rows of one mask tend to have
+    // similar lengths, and one shared-memory atomic per item on a handful of addresses serialises the CTA)
+    for (int i0 = 0; i0 < n_items; i0 += blockDim.x) {
+        const int i = i0 + tid;
+        const int32_t k = (i < n_items) ? key[i] : -1 - (tid & 31);
+        const unsigned peers = __match_any_sync(kFull, k);
+        if (i < n_items && (peers >> (tid & 31)) <= 1u) atomicAdd(&bins[k], __popc(peers));
+    }
+    __syncthreads();
 
     // ---- B: bucket starts, longest first ----
     if (tid < 32) {
@@ -435,6 +459,9 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
     __syncthreads();
 
     // ---- C1: stable rank ----
+    // per-warp histograms cost rank_warps * nbins shared-memory words to clear and scan: worth it from a few hundred
+    // items per warp on
+    const int rank_warps = min(rank_warps_max, n_items / 256);
     if (rank_warps >= 2) {
         // The group's items are cut into `rank_warps` contiguous chunks, one per warp: per-warp histograms, then for
         // every length the warps' counts are turned into start offsets (bucket start + counts of the earlier chunks),
@@ -445,8 +472,15 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
         for (int i = tid; i < rank_warps * nbins; i += blockDim.x) whist[i] = 0;
         __syncthreads();
         const int c0 = warp * chunk, c1 = min(n_items, c0 + chunk);
-        if (warp < rank_warps)
-            for (int i = c0 + lane; i < c1; i += 32) atomicAdd(&whist[warp * nbins + key[i]], 1);
+        if (warp < rank_warps) {
+            for (int i0 = c0; i0 < c1; i0 += 32) {
+                const int i = i0 + lane;
+                const int32_t k = (i < c1) ? key[i] : -1 - lane;
+                const unsigned peers = __match_any_sync(kFull, k);
+                if (i < c1 && (peers >> lane) <= 1u) whist[warp * nbins + k] += __popc(peers);  // this warp's own row
+                __syncwarp();
+            }
+        }
         __syncthreads();
         for (int b = tid; b < nbins; b += blockDim.x) {
             int32_t run = bins[b];
@@ -574,8 +608,9 @@ cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const i
         attr_bytes = smem;
     }
     const int grid = (order == BSA_ORDER_GLOBAL_LPT) ? 1 : g.H;
-    organize_kernel<<<grid, 1024, smem, stream>>>(g, order, rank_warps, (int)organize_key_cap(g, order, split_pmax), tile_begin,
-                                                   tile_cnt, row_parts, head_counts, items_tmp, items, split_rows, counters);
+    organize_kernel<<<grid, 1024, smem, stream>>>(g, order, rank_warps, (int)organize_key_cap(g, order, split_pmax),
+                                                   split_pmax <= 1 ? 1 : 0, tile_begin, tile_cnt, row_parts, head_counts,
+                                                   items_tmp, items, split_rows, counters);
     count_launch();
     return cudaGetLastError();
 }
