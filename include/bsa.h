@@ -44,7 +44,7 @@ typedef enum {
 /* Mapping of one dimension of the logical geometry onto the physical tile (Section 4.2). */
 enum { BSA_MAP_DIRECT = 0, BSA_MAP_COARSENED = 1, BSA_MAP_REFINED = 2 };
 /* Traversal order of the work queue (Section 4.3). */
-enum { BSA_ORDER_HEAD_MAJOR_LPT = 0, BSA_ORDER_GLOBAL_LPT = 1 };
+enum { BSA_ORDER_HEAD_MAJOR_LPT = 0, BSA_ORDER_GLOBAL_LPT = 1, BSA_ORDER_NATURAL = 2 /* row-major, unsorted: ablation baseline */ };
 
 /* One catalog entry: a physical plan P = <g_Q, g_KV, sigma, e> (Section 4.1).  g_Q and g_KV follow
  * from (B_Q, B_KV) and the tile shape; sigma = {order, split_tau, split_pmax, stages}; e = kernel. */

@@ -29,6 +29,7 @@ using namespace ptx;
 #ifdef BSA_TRACE
 __device__ long long g_trace[12][4096];  // producer, Q K^T (or single) issuer, softmax warps 0-7, P V issuer (role 6 in the 7-warp kernel)
 __device__ long long g_trace_aux[12][4];  // last tile's stamps inside softmax_tile, per warp
+__device__ long long g_cta_times[2][4096];  // %globaltimer at entry and exit of every CTA of the ping-pong kernel
 #define BSA_TRACE_DECL(n) int n = 0
 #define BSA_TRACE_POINT(role, n, tag)                                              \
     do {                                                                           \
@@ -1380,6 +1381,9 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     __shared__ uint32_t abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef BSA_TRACE
+    if (tid == 0 && blockIdx.x < 4096) g_cta_times[0][blockIdx.x] = (long long)globaltimer_ns();
+#endif
     if (smem_u32(smem) & 1023u) {  // never expected; fail with a status instead of corrupting tiles
         if (tid == 0) atomicExch(&p.counters->status, (int)BSA_ERR_CUDA);
         return;
@@ -1943,6 +1947,9 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     __syncthreads();
     if (tid == 0 && abort_flag) atomicExch(&p.counters->status, (int)BSA_ERR_DEVICE_TIMEOUT);
     if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+#ifdef BSA_TRACE
+    if (tid == 0 && blockIdx.x < 4096) g_cta_times[1][blockIdx.x] = (long long)globaltimer_ns();
+#endif
 }
 
 // ------------------------------------------------------------------------------------------
@@ -2119,6 +2126,8 @@ int attention_smem_bytes(int d, int T_KV, int stages, int kernel) {
 
 #ifdef BSA_TRACE
 extern "C" __attribute__((visibility("default"))) int bsa_debug_trace_copy(long long* host, int role) {
+    if (role >= 100)  // 100 / 101: CTA entry / exit times
+        return (int)cudaMemcpyFromSymbol(host, g_cta_times, sizeof(long long) * 4096, sizeof(long long) * 4096 * (role - 100));
     return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * 4096, sizeof(long long) * 4096 * role);
 }
 #endif

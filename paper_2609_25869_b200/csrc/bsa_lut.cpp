@@ -52,6 +52,8 @@ static const bsa_plan_desc_t kCatalog[] = {
     {26, 128, 64, 0, 0, 1, BSA_ORDER_GLOBAL_LPT, 4, "q128k64_pp_global"},
     {27, 128, 64, 0, 4, 8, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k64_pp_split4x8"},
     {28, 128, 64, 0, 2, 16, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k64_pp_split2x16"},
+    // work items in row-major order, not sorted by length: the baseline of the task-organisation ablation (Section 4.3)
+    {29, 128, 128, 0, 0, 1, BSA_ORDER_NATURAL, 4, "q128k128_pp_natural"},
 };
 static const int kCatalogSize = (int)(sizeof(kCatalog) / sizeof(kCatalog[0]));
 static const int64_t kDefaultWorkspace = 2ll << 30;

@@ -431,6 +431,15 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
     }
     __syncthreads();
     const int32_t n_items = run_items;
+    if (order == BSA_ORDER_NATURAL) {  // unsorted: the items stay in (head, q_tile, part) order
+        for (int i = tid; i < n_items; i += blockDim.x) items[item_base + i] = items_tmp[item_base + i];
+        if (tid == 0 && grp == gridDim.x - 1) {
+            counters->nitems = item_base + n_items;
+            counters->nsplit_rows = (split_base + run_split) * g.slots;
+            counters->nslots = slot_base + run_slots;
+        }
+        return;
+    }
     // histogram of item lengths; lanes of a warp that hold the same length add once (rows of one mask tend to have
     // similar lengths, and one shared-memory atomic per item on a handful of addresses serialises the CTA)
     for (int i0 = 0; i0 < n_items; i0 += blockDim.x) {

@@ -1,0 +1,145 @@
+"""Quality of the shipped plan table on requests it was not compiled from (paper Section 6.4 "selection regret",
+Table 7 cold / warm / amortized request cost).
+
+For every evaluation request (the five named configurations and the first requests of the dynamic-request sweep,
+all with seeds disjoint from the profiling corpus of ``lut_build.py``): every eligible catalog plan is validated and
+timed exactly as in Algorithm 1 (median of 5 forwards after 3 warm-ups, L2 flushed), the plan the table selects for
+the request is looked up through ``bsa_plan_create``, and
+
+    regret           = latency(selected plan) / latency(fastest eligible plan)
+    speedup vs base  = latency(base plan of the request key) / latency(selected plan)
+    cold / warm / A4 = plan create + forward, forward alone on the prepared plan, (create + 4 forwards) / 4
+
+are reported per request and summarised (geometric mean, P95, P99, share within 3 %, win / tie / loss with a 3 % band).
+
+    python -m paper_2609_25869_b200.regret --sweep-requests 16
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import statistics
+import sys
+
+
+def _gm(xs):
+    return math.exp(sum(math.log(x) for x in xs) / len(xs)) if xs else float("nan")
+
+
+def _pct(xs, p):
+    xs = sorted(xs)
+    if not xs:
+        return float("nan")
+    k = min(len(xs) - 1, max(0, int(math.ceil(p / 100.0 * len(xs))) - 1))
+    return xs[k]
+
+
+def summarise(rows):
+    """rows: dicts with t_selected, t_best, t_base (ms).  Pure host logic (unit-tested on the CPU)."""
+    reg = [r["t_selected"] / r["t_best"] for r in rows]
+    spd = [r["t_base"] / r["t_selected"] for r in rows]
+    win = sum(1 for s in spd if s > 1.03)
+    loss = sum(1 for s in spd if s < 1.0 / 1.03)
+    return {"n": len(rows), "regret_gm": _gm(reg), "regret_p95": _pct(reg, 95), "regret_p99": _pct(reg, 99),
+            "regret_max": max(reg) if reg else float("nan"),
+            "within_3pct": sum(1 for x in reg if x <= 1.03) / max(1, len(reg)),
+            "speedup_vs_base_gm": _gm(spd), "win": win, "tie": len(rows) - win - loss, "loss": loss}
+
+
+def organisation_ablation(rows):
+    """Task-organisation ablation (Section 4.3, the paper's Table 5) on the requests whose geometry the 128x128 tile
+    covers directly: the same kernel and tiles, work items unsorted (O0), longest-first inside each head or over all
+    heads (O1), and the better of those with Split-K also allowed (O2).  Speedups over O0, geometric means."""
+    o1h, o1g, o1, o2 = [], [], [], []
+    for r in rows:
+        t = r.get("lat_by_plan", {})
+        if r["key"][:2] != (128, 128) or "q128k128_pp_natural" not in t:
+            continue
+        t0 = t["q128k128_pp_natural"]
+        h, g = t.get("q128k128_pp"), t.get("q128k128_pp_global")
+        if h is None or g is None:
+            continue
+        o1h.append(t0 / h)
+        o1g.append(t0 / g)
+        o1.append(t0 / min(h, g))
+        o2.append(t0 / min(h, g, t.get("q128k128_pp_split4x8", float("inf"))))
+    return {"n": len(o1), "O1_head_major": _gm(o1h), "O1_global": _gm(o1g), "O1_best_order": _gm(o1), "O2_with_split_k": _gm(o2),
+            "O1_best_order_min_max": (min(o1), max(o1)) if o1 else None}
+
+
+def evaluate(reqs, log=print):
+    import torch
+    from . import bsa
+    from .lut_build import profile
+    cat = bsa.catalog()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    rows = []
+    for req in reqs:
+        cases, lat, _, base = profile([req], log=lambda *a, **k: None)
+        key = (req.B_Q, req.B_KV, req.d)
+        mine = {p: t for (c, p), t in lat.items() if c == req.name}
+        if not mine:
+            continue
+        mask = torch.from_numpy(req.mask).cuda()
+        q, k, v = (t.cuda() for t in req.qkv())
+        O = torch.empty_like(q)
+        L = torch.empty((req.H, req.N), dtype=torch.float32, device="cuda")
+        cold = []
+        sel = None
+        for it in range(6):
+            flush.fill_(it)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            plan = bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d)
+            plan.forward(q, k, v, O, L)
+            b.record()
+            b.synchronize()
+            inf = plan.info()
+            sel = inf["plan"]["plan_id"]
+            plan.destroy()
+            if it >= 2:
+                cold.append(a.elapsed_time(b))
+        if sel not in mine:  # the selected plan failed validation on this request: counts as the slowest plan
+            mine[sel] = max(mine.values())
+        best = min(mine, key=lambda p: (mine[p], p))
+        t_cold = statistics.median(cold)
+        row = {"name": req.name, "key": key, "density": inf["density"], "skew": inf["skew"], "lut_hit": inf["lut_hit"],
+               "selected": cat[sel]["name"], "best": cat[best]["name"], "t_selected": mine[sel], "t_best": mine[best],
+               "t_base": mine.get(base[key], float("nan")), "t_cold": t_cold,
+               "t_a4": (t_cold - mine[sel]) / 4.0 + mine[sel], "n_eligible": len(mine),
+               "lat_by_plan": {cat[p]["name"]: t for p, t in mine.items()}}
+        rows.append(row)
+        log(f"{req.name:12s} B={key[:2]} d={key[2]} dens={row['density']:.3f} skew={row['skew']:.1f} hit={row['lut_hit']} "
+            f"selected {row['selected']:22s} {row['t_selected']*1e3:9.0f} us | best {row['best']:22s} {row['t_best']*1e3:9.0f} us "
+            f"| regret {row['t_selected']/row['t_best']:.3f} | base/selected {row['t_base']/row['t_selected']:.3f} "
+            f"| cold {t_cold*1e3:9.0f} us, A4 {row['t_a4']*1e3:9.0f} us")
+    return rows
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--sweep-requests", type=int, default=16)
+    ap.add_argument("--json", default="")
+    args = ap.parse_args(argv)
+    from . import inputs as I
+    reqs = [I.CONFIGS[n]() for n in ("tiny", "mid", "hunyuan", "stress_a", "stress_b")]
+    for r in range(args.sweep_requests):
+        q = I.config_sweep(r)
+        q.name = f"sweep{r}"
+        reqs.append(q)
+    rows = evaluate(reqs)
+    s = summarise(rows)
+    print(json.dumps(s))
+    print("task organisation ablation:", json.dumps(organisation_ablation(rows)))
+    cold = _gm([r["t_cold"] / r["t_selected"] for r in rows])
+    a4 = _gm([r["t_a4"] / r["t_selected"] for r in rows])
+    print(f"cold request / warm forward, geometric mean: {cold:.3f}; four-pass amortized / warm: {a4:.3f}")
+    if args.json:
+        with open(args.json, "w") as f:
+            json.dump({"rows": rows, "summary": s}, f, indent=1, default=str)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

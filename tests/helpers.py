@@ -71,6 +71,17 @@ def check_plan_structure(req, plan, heads=None):
         assert te - tb == nt and 0 <= part < nparts
         seen.setdefault((h, qt), []).append((part, tb, te, nparts, slot))
     assert len(seen) == req.H * inf["nQt"]
+    # order of the list (Section 4.3): longest first, ties in (head, q_tile, part) order - inside each head
+    # (order 0), over all heads (order 1), or plain row-major (order 2)
+    order = inf["plan"]["order"]
+    rows = [tuple(int(x) for x in it) for it in items]
+    if order == 0:
+        want = sorted(rows, key=lambda r: (r[0], -r[7], r[1], r[4]))
+    elif order == 1:
+        want = sorted(rows, key=lambda r: (-r[7], r[0], r[1], r[4]))
+    else:
+        want = sorted(rows, key=lambda r: (r[0], r[1], r[4]))
+    assert rows == want, "work items are not in the plan's order"
     nsplit = 0
     for (h, qt), parts in seen.items():
         parts.sort()

@@ -18,13 +18,13 @@ def _sample(req, per_head, seed=77, heads=None):
 
 
 # ---------------------------------------------------------------- the five configurations
-@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28])
+@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29])
 def test_tiny_full_oracle_every_plan(plan_id):
     res = Hh.run_request(I.config_tiny(), plan_id=plan_id)
     assert res["pairs"] == res["info"]["nnz_blocks"] * 64 * 64
 
 
-@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 10, 12, 14, 16, 18, 20, 22, 24, 25, 26])
+@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 10, 12, 14, 16, 18, 20, 22, 24, 25, 26, 29])
 def test_mid_full_oracle(plan_id):
     """-1 is the configuration bench.py times (the plan the shipped table selects); every row is compared."""
     Hh.run_request(I.config_mid(), plan_id=plan_id)
@@ -223,6 +223,32 @@ def test_request_from_host_buffers_matches_device_path():
     inf = bsa.request_host(req.mask, req.B_Q, req.B_KV, req.N, req.H, req.d, q, k, v, O, LSE)
     assert inf["device_status"] == 0
     Hh.compare_with_oracle(req, O, LSE, (q, k, v))
+
+
+@pytest.mark.parametrize("plan_id", [22, 27])
+def test_forward_replays_from_a_cuda_graph(plan_id):
+    """bsa_forward only launches kernels (no allocation, no synchronisation): it can be captured into a CUDA graph
+    and replayed, with and without Split-K, and the replay gives the bits of the direct call."""
+    req = I.config_tiny()
+    mask, q, k, v, _ = Hh.to_dev(req, None)
+    with bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=plan_id) as plan:
+        O0, L0 = plan.forward(q, k, v)  # also sets the kernels' shared-memory attributes before the capture
+        torch.cuda.synchronize()
+        O = torch.zeros_like(O0)
+        L = torch.zeros_like(L0)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                plan.forward(q, k, v, O, L, stream=side)
+        for _ in range(3):
+            O.zero_()
+            L.zero_()
+            graph.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(O, O0) and torch.equal(L, L0)
+        assert plan.info()["device_status"] == 0
 
 
 def test_launch_counter_counts_our_kernels():

@@ -163,3 +163,17 @@ def test_offline_table_compilation_matches_algorithm_1(tmp_path):
     bsa.lut_load(path)
     assert bsa.lib().bsa_lut_num_regimes() == len(got)
     bsa.lut_clear()
+
+
+def test_regret_summary_statistics():
+    """Selection-regret summary (host arithmetic only): geometric mean, percentiles, 3 % band for win/tie/loss."""
+    from paper_2609_25869_b200.regret import summarise
+    rows = [{"t_selected": 1.00, "t_best": 1.00, "t_base": 1.50},   # regret 1.00, speedup 1.50 -> win
+            {"t_selected": 2.04, "t_best": 2.00, "t_base": 2.04},   # regret 1.02, speedup 1.00 -> tie
+            {"t_selected": 1.10, "t_best": 1.00, "t_base": 1.00},   # regret 1.10, speedup 0.909 -> loss
+            {"t_selected": 4.00, "t_best": 4.00, "t_base": 4.10}]   # regret 1.00, speedup 1.025 -> tie
+    s = summarise(rows)
+    assert s["n"] == 4 and (s["win"], s["tie"], s["loss"]) == (1, 2, 1)
+    assert abs(s["regret_gm"] - (1.0 * 1.02 * 1.10 * 1.0) ** 0.25) < 1e-12
+    assert s["regret_max"] == 1.10 and s["regret_p95"] == 1.10 and abs(s["within_3pct"] - 0.75) < 1e-12
+    assert abs(s["speedup_vs_base_gm"] - (1.5 * 1.0 * (1 / 1.1) * 1.025) ** 0.25) < 1e-12
