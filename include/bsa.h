@@ -44,7 +44,13 @@ typedef enum {
 /* Mapping of one dimension of the logical geometry onto the physical tile (Section 4.2). */
 enum { BSA_MAP_DIRECT = 0, BSA_MAP_COARSENED = 1, BSA_MAP_REFINED = 2 };
 /* Traversal order of the work queue (Section 4.3). */
-enum { BSA_ORDER_HEAD_MAJOR_LPT = 0, BSA_ORDER_GLOBAL_LPT = 1, BSA_ORDER_NATURAL = 2 /* row-major, unsorted: ablation baseline */ };
+enum {
+    BSA_ORDER_HEAD_MAJOR_LPT = 0,     /* longest first inside each head                                         */
+    BSA_ORDER_GLOBAL_LPT = 1,         /* longest first over all heads                                           */
+    BSA_ORDER_NATURAL = 2,            /* row-major, unsorted (baseline of the task-organisation ablation)       */
+    BSA_ORDER_HEAD_MAJOR_BUCKETS = 3, /* by half-octave length bucket inside each head, row-major inside a bucket */
+    BSA_ORDER_GLOBAL_BUCKETS = 4      /* the same over all heads                                                */
+};
 
 /* One catalog entry: a physical plan P = <g_Q, g_KV, sigma, e> (Section 4.1).  g_Q and g_KV follow
  * from (B_Q, B_KV) and the tile shape; sigma = {order, split_tau, split_pmax, stages}; e = kernel. */
@@ -125,6 +131,17 @@ BSA_API bsa_status_t bsa_plan_create(const uint8_t* mask_dev, int B_Q, int B_KV,
 BSA_API bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int B_KV, int64_t N, int heads, int d,
                                 const bsa_options_t* options /* may be NULL */, void* stream,
                                 bsa_plan_t** out_plan);
+
+/* The same for a bit-packed mask (the paper does not fix a mask format, Section 2.1 only defines M; this variant has
+ * no counterpart there).  Row (h, qb) starts at mask_bits_dev + (h * nQb + qb) * row_stride_bytes; block column c of
+ * the row is bit (c & 7) of its byte c >> 3 (1 = active; numpy.packbits(..., bitorder="little")).  Bits at or beyond
+ * nKb and the padding bytes of a row are ignored.  mask_bits_dev must be 4-byte aligned and row_stride_bytes a
+ * multiple of 4 that holds nKb bits, else INVALID_ARG (GPU untouched).  Device memory, borrowed for the call.  The
+ * planner then reads one eighth of the byte format's mask traffic; everything downstream is identical, and so is
+ * every output (the GPU tests compare the two plans' exported structures and outputs bit for bit). */
+BSA_API bsa_status_t bsa_plan_create_packed(const uint8_t* mask_bits_dev, int64_t row_stride_bytes, int B_Q, int B_KV,
+                                    int64_t N, int heads, int d, const bsa_options_t* options /* may be NULL */,
+                                    void* stream, bsa_plan_t** out_plan);
 
 /* ---------------------------------------------------------------------------------------------
  * bsa_forward -- execute the plan's native kernels (Section 4: main attention kernel, then the

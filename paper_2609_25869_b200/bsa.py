@@ -74,6 +74,7 @@ def lib() -> ctypes.CDLL:
     vp, i32, i64, f64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_double
     L.bsa_plan_create.argtypes = [vp, i32, i32, i64, i32, i32, ctypes.POINTER(vp)]
     L.bsa_plan_create_ex.argtypes = [vp, i32, i32, i64, i32, i32, ctypes.POINTER(Options), vp, ctypes.POINTER(vp)]
+    L.bsa_plan_create_packed.argtypes = [vp, i64, i32, i32, i64, i32, i32, ctypes.POINTER(Options), vp, ctypes.POINTER(vp)]
     L.bsa_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.bsa_plan_destroy.argtypes = [vp]
     L.bsa_request_host.argtypes = [vp, i32, i32, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.POINTER(Options),
@@ -209,6 +210,34 @@ def plan_create(mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: 
     opt = Options(plan_id, 0, max_workspace_bytes)
     _check(lib().bsa_plan_create_ex(mask.data_ptr(), B_Q, B_KV, N, heads, d, ctypes.byref(opt), _stream_ptr(stream),
                                     ctypes.byref(h)), "bsa_plan_create")
+    return Plan(h.value)
+
+
+def pack_mask(mask):
+    """Bit-pack a uint8/bool mask tensor ``[heads, nQb, nKb]`` (CUDA or CPU) into the layout ``plan_create_packed``
+    reads: little-endian bits, rows padded to a multiple of 4 bytes.  Returns ``(packed uint8 tensor, row stride)``.
+    A convenience for callers and tests (plain torch ops, not part of the timed path)."""
+    import torch
+    h, nq, nk = mask.shape
+    stride = ((nk + 31) // 32) * 4
+    m = (mask != 0).to(torch.uint8)
+    pad = stride * 8 - nk
+    if pad:
+        m = torch.nn.functional.pad(m, (0, pad))
+    w = torch.tensor([1, 2, 4, 8, 16, 32, 64, 128], dtype=torch.uint8, device=m.device)
+    packed = (m.view(h, nq, stride, 8) * w).sum(dim=-1, dtype=torch.int32).to(torch.uint8).contiguous()
+    return packed, stride
+
+
+def plan_create_packed(mask_bits, row_stride: int, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1,
+                       max_workspace_bytes: int = 0, stream=None) -> Plan:
+    """``bsa_plan_create_packed``: ``mask_bits`` is a uint8 CUDA tensor of bit-packed rows (see ``pack_mask``)."""
+    import torch
+    assert mask_bits.is_cuda and mask_bits.is_contiguous() and mask_bits.dtype == torch.uint8
+    h = ctypes.c_void_p()
+    opt = Options(plan_id, 0, max_workspace_bytes)
+    _check(lib().bsa_plan_create_packed(mask_bits.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
+                                        _stream_ptr(stream), ctypes.byref(h)), "bsa_plan_create_packed")
     return Plan(h.value)
 
 

@@ -111,10 +111,16 @@ static void free_plan(bsa_plan* p) {
         }                                \
     } while (0)
 
-extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int B_KV, int64_t N, int heads, int d,
-                                           const bsa_options_t* options, void* stream_v, bsa_plan_t** out_plan) {
+// `packed_stride` = 0: one byte per logical block; > 0: bit-packed rows of that many bytes (bsa_plan_create_packed)
+static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, int B_Q, int B_KV, int64_t N, int heads,
+                                int d, const bsa_options_t* options, void* stream_v, bsa_plan_t** out_plan) {
     bsa_status_t vs = validate(mask_dev, B_Q, B_KV, N, heads, d, out_plan);
     if (vs != BSA_OK) return vs;
+    if (packed_stride > 0) {
+        const int64_t nKb64 = (N + B_KV - 1) / B_KV;
+        if (packed_stride % 4 != 0 || packed_stride * 8 < nKb64 || (reinterpret_cast<uintptr_t>(mask_dev) & 3u))
+            return BSA_ERR_INVALID_ARG;
+    }
     *out_plan = nullptr;
     const double t0 = now_us();
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
@@ -158,7 +164,12 @@ extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int
     p->counters = reinterpret_cast<PlanCountersDev*>(p->arena1 + o_cnt);
     p->head_counts = reinterpret_cast<int32_t*>(p->arena1 + o_hc);
     BSA_CUDA(cudaMemsetAsync(p->arena1 + o_zero, 0, a1_bytes - o_zero, stream), "memset");
-    BSA_CUDA(launch_mask_row_stats(mask_dev, nrows, nKb, p->row_nnz, p->stats, stream), "mask_row_stats");
+    const uint32_t* mask_words = reinterpret_cast<const uint32_t*>(mask_dev);
+    if (packed_stride > 0)
+        BSA_CUDA(launch_mask_row_stats_packed(mask_words, packed_stride / 4, nrows, nKb, p->row_nnz, p->stats, stream),
+                 "mask_row_stats_packed");
+    else
+        BSA_CUDA(launch_mask_row_stats(mask_dev, nrows, nKb, p->row_nnz, p->stats, stream), "mask_row_stats");
     const double t1 = now_us();
 
     // ---- lines 3-5: only the scalars cross to the host ----
@@ -230,7 +241,11 @@ extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int
         BSA_CUDA(cudaMallocAsync(&p->ws_O, (size_t)p->ws_bytes, stream), "workspace");
         p->ws_LSE = p->ws_O + (size_t)p->max_items * g.T_Q * d;
     }
-    BSA_CUDA(launch_csr_fill(mask_dev, nrows, nKb, p->row_ptr, p->col_idx, stream), "csr_fill");
+    if (packed_stride > 0)
+        BSA_CUDA(launch_csr_fill_packed(mask_words, packed_stride / 4, nrows, nKb, p->row_ptr, p->col_idx, stream),
+                 "csr_fill_packed");
+    else
+        BSA_CUDA(launch_csr_fill(mask_dev, nrows, nKb, p->row_ptr, p->col_idx, stream), "csr_fill");
     BSA_CUDA(launch_tile_map(g, p->row_ptr, p->col_idx, p->desc.split_tau, pmax, p->tile_begin, p->tile_cnt,
                              p->row_parts, p->tile_col, p->tile_member, p->head_counts, p->counters, stream),
              "tile_map");
@@ -245,6 +260,18 @@ extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int
     p->us_total = (float)(t4 - t0);
     *out_plan = p;
     return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_plan_create_ex(const uint8_t* mask_dev, int B_Q, int B_KV, int64_t N, int heads, int d,
+                                           const bsa_options_t* options, void* stream_v, bsa_plan_t** out_plan) {
+    return create_impl(mask_dev, 0, B_Q, B_KV, N, heads, d, options, stream_v, out_plan);
+}
+
+extern "C" bsa_status_t bsa_plan_create_packed(const uint8_t* mask_bits_dev, int64_t row_stride_bytes, int B_Q, int B_KV,
+                                               int64_t N, int heads, int d, const bsa_options_t* options, void* stream_v,
+                                               bsa_plan_t** out_plan) {
+    if (row_stride_bytes <= 0) return BSA_ERR_INVALID_ARG;
+    return create_impl(mask_bits_dev, row_stride_bytes, B_Q, B_KV, N, heads, d, options, stream_v, out_plan);
 }
 
 extern "C" bsa_status_t bsa_plan_create(const uint8_t* mask_dev, int B_Q, int B_KV, int64_t N, int heads, int d,

@@ -62,6 +62,10 @@ struct MapGeom {
 cudaError_t launch_mask_row_stats(const uint8_t* mask, int nrows, int nKb, int32_t* row_nnz, MaskStatsDev* stats,
                                   cudaStream_t stream);
 cudaError_t launch_row_scan(const int32_t* row_nnz, int nrows, int32_t* row_ptr, cudaStream_t stream);
+cudaError_t launch_mask_row_stats_packed(const uint32_t* mask, long long stride_words, int nrows, int nKb,
+                                         int32_t* row_nnz, MaskStatsDev* stats, cudaStream_t stream);
+cudaError_t launch_csr_fill_packed(const uint32_t* mask, long long stride_words, int nrows, int nKb,
+                                   const int32_t* row_ptr, int32_t* col_idx, cudaStream_t stream);
 cudaError_t launch_csr_fill(const uint8_t* mask, int nrows, int nKb, const int32_t* row_ptr, int32_t* col_idx,
                             cudaStream_t stream);
 cudaError_t launch_tile_map(const MapGeom& g, const int32_t* row_ptr, const int32_t* col_idx, int split_tau,

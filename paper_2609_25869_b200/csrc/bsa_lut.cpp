@@ -54,6 +54,12 @@ static const bsa_plan_desc_t kCatalog[] = {
     {28, 128, 64, 0, 2, 16, BSA_ORDER_HEAD_MAJOR_LPT, 4, "q128k64_pp_split2x16"},
     // work items in row-major order, not sorted by length: the baseline of the task-organisation ablation (Section 4.3)
     {29, 128, 128, 0, 0, 1, BSA_ORDER_NATURAL, 4, "q128k128_pp_natural"},
+    // longest first by half-octave length bucket, row-major inside a bucket (balance without giving up the K/V
+    // tiles that neighbouring Q tiles share)
+    {30, 128, 128, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_BUCKETS, 4, "q128k128_pp_hb"},
+    {31, 128, 128, 0, 0, 1, BSA_ORDER_GLOBAL_BUCKETS, 4, "q128k128_pp_gb"},
+    {32, 128, 64, 0, 0, 1, BSA_ORDER_NATURAL, 4, "q128k64_pp_natural"},
+    {33, 128, 64, 0, 0, 1, BSA_ORDER_GLOBAL_BUCKETS, 4, "q128k64_pp_gb"},
 };
 static const int kCatalogSize = (int)(sizeof(kCatalog) / sizeof(kCatalog[0]));
 static const int64_t kDefaultWorkspace = 2ll << 30;

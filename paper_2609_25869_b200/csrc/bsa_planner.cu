@@ -107,6 +107,101 @@ __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __re
 }
 
 // ------------------------------------------------------------------------------------------
+// The same two mask passes for a bit-packed mask: bit (c & 7) of byte c >> 3 of a row is block column c; rows start
+// every `stride_words` 32-bit words (4-byte aligned).  One 32-bit word (32 blocks) per lane and step; bits at or
+// beyond nKb are ignored.  The mask traffic is one eighth of the byte format's.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned packed_row_word(const uint32_t* __restrict__ row, int w, int nwords, int nKb) {
+    if (w >= nwords) return 0u;
+    unsigned m = __ldg(row + w);
+    const int valid = nKb - w * 32;
+    if (valid < 32) m &= (1u << valid) - 1u;
+    return m;
+}
+
+__global__ void __launch_bounds__(256) mask_row_stats_packed_kernel(const uint32_t* __restrict__ mask, long long stride_words,
+                                                                     int nrows, int nKb, int32_t* __restrict__ row_nnz,
+                                                                     MaskStatsDev* stats) {
+    __shared__ unsigned s_nnz[8], s_runs[8];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + warp;
+    unsigned nnz = 0, runs = 0;
+    if (row < nrows) {
+        const uint32_t* r = mask + (long long)row * stride_words;
+        const int nwords = (nKb + 31) >> 5;
+        unsigned carry = 0;  // bits 1:0 = the previous step's last two blocks (bit 1 = the last one)
+        unsigned m_next = packed_row_word(r, lane, nwords, nKb);
+        for (int w = 0; w < nwords; w += 32) {
+            const unsigned m = m_next;
+            m_next = (w + 32 < nwords) ? packed_row_word(r, w + 32 + lane, nwords, nKb) : 0u;
+            unsigned prev31 = __shfl_up_sync(kFull, m >> 31, 1);
+            unsigned next0 = __shfl_down_sync(kFull, m & 1u, 1);
+            if (lane == 0) prev31 = carry >> 1;
+            if (lane == 31) next0 = 0u;
+            const unsigned left = (m << 1) | prev31, right = (m >> 1) | (next0 << 31);
+            nnz += __popc(m);
+            runs += __popc(m & (left | right));
+            if (lane == 0 && carry == 2u && (m & 1u)) ++runs;  // see mask_row_stats_kernel
+            carry = __shfl_sync(kFull, m >> 30, 31);
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            nnz += __shfl_down_sync(kFull, nnz, o);
+            runs += __shfl_down_sync(kFull, runs, o);
+        }
+        if (lane == 0) row_nnz[row] = (int32_t)nnz;
+    }
+    if (lane == 0) {
+        s_nnz[warp] = nnz;
+        s_runs[warp] = runs;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long tn = 0, tr = 0;
+        unsigned mx = 0;
+        for (int w = 0; w < 8; ++w) {
+            tn += s_nnz[w];
+            tr += s_runs[w];
+            mx = max(mx, s_nnz[w]);
+        }
+        if (tn) {
+            atomicAdd(&stats->nnz, tn);
+            atomicAdd(&stats->in_runs, tr);
+            atomicMax(&stats->max_row_nnz, mx);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) csr_fill_packed_kernel(const uint32_t* __restrict__ mask, long long stride_words,
+                                                               int nrows, int nKb, const int32_t* __restrict__ row_ptr,
+                                                               int32_t* __restrict__ col_idx) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + warp;
+    if (row >= nrows) return;
+    const uint32_t* r = mask + (long long)row * stride_words;
+    const int nwords = (nKb + 31) >> 5;
+    int32_t out = row_ptr[row];
+    unsigned m_next = packed_row_word(r, lane, nwords, nKb);
+    for (int w = 0; w < nwords; w += 32) {
+        unsigned m = m_next;
+        m_next = (w + 32 < nwords) ? packed_row_word(r, w + 32 + lane, nwords, nKb) : 0u;
+        const int cnt = __popc(m);
+        int incl = cnt;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int x = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl += x;
+        }
+        int pos = out + incl - cnt;
+        const int col0 = (w + lane) * 32;
+        while (m) {
+            const int b = __ffs(m) - 1;
+            col_idx[pos++] = col0 + b;
+            m &= m - 1;
+        }
+        out += __shfl_sync(kFull, incl, 31);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // row_scan: exclusive scan of row_nnz by one CTA (rows are few: heads * query blocks).
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) row_scan_kernel(const int32_t* __restrict__ row_nnz, int nrows,
@@ -331,6 +426,18 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
 //      (stable: ties keep (head, q_tile, part) order), then all threads scatter.
 // Shared memory: bins [nKt + 2] then one int per item of the group.
 // ------------------------------------------------------------------------------------------
+// Histogram size of the sort: one bin per item length, and at least the 64 half-octave buckets.
+__host__ __device__ __forceinline__ int organize_bins(const MapGeom& g) { return g.nKt + 2 > 64 ? g.nKt + 2 : 64; }
+
+// Half-octave bucket of an item length (0, 1, 2, 3, 4-5, 6-7, 8-11, 12-15, ...): the bucketed orders sort by it, so
+// items of similar length keep their row-major order, and with it the K/V tiles neighbouring Q tiles share.
+__host__ __device__ __forceinline__ int32_t length_bucket(int32_t n) {
+    if (n <= 1) return n < 0 ? 0 : n;
+    int lz = 0;
+    while ((n >> (lz + 1)) != 0) ++lz;  // floor(log2 n), n >= 2
+    return 2 * lz + ((n >> (lz - 1)) & 1);
+}
+
 __device__ __forceinline__ int32_t block_excl_scan(int32_t v, int32_t* warp_buf, int32_t* total_out) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
     int32_t incl = v;
@@ -360,13 +467,15 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
                                                          SplitRow* __restrict__ split_rows, PlanCountersDev* counters) {
     extern __shared__ int32_t sm[];
     __shared__ int32_t warp_buf[32];
-    const int nbins = g.nKt + 2;
+    const int nbins = organize_bins(g);
+    const bool bucketed = (order == BSA_ORDER_HEAD_MAJOR_BUCKETS || order == BSA_ORDER_GLOBAL_BUCKETS);
+    const bool global_group = (order == BSA_ORDER_GLOBAL_LPT || order == BSA_ORDER_GLOBAL_BUCKETS);
     int32_t* bins = sm;            // [nbins]
     int32_t* key = sm + nbins;     // [items of the group]: length, then rank
     const int tid = threadIdx.x;
     const int grp = blockIdx.x;
     int row0, row1, item_base = 0, split_base = 0, slot_base = 0;
-    if (order == BSA_ORDER_GLOBAL_LPT) {
+    if (global_group) {
         row0 = 0;
         row1 = g.H * g.nQt;
     } else {
@@ -412,7 +521,7 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
                 it.ntiles = it.tile_end - it.tile_begin;
                 const int32_t li = run_items + off_i + p;
                 items_tmp[item_base + li] = it;
-                key[li] = it.ntiles;
+                key[li] = bucketed ? length_bucket(it.ntiles) : it.ntiles;
             }
             if (P > 1) {
                 for (int sl = 0; sl < g.slots; ++sl) {
@@ -537,7 +646,7 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
     for (int i = tid; i < n_items; i += blockDim.x) items[item_base + key[i]] = items_tmp[item_base + i];
 
     if (tid == 0) {
-        if (order == BSA_ORDER_GLOBAL_LPT) {
+        if (global_group) {
             counters->nitems = n_items;
             counters->nsplit_rows = run_split * g.slots;
             counters->nslots = run_slots;
@@ -554,6 +663,20 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
 cudaError_t launch_mask_row_stats(const uint8_t* mask, int nrows, int nKb, int32_t* row_nnz, MaskStatsDev* stats,
                                   cudaStream_t stream) {
     mask_row_stats_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, nrows, nKb, row_nnz, stats);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mask_row_stats_packed(const uint32_t* mask, long long stride_words, int nrows, int nKb,
+                                         int32_t* row_nnz, MaskStatsDev* stats, cudaStream_t stream) {
+    mask_row_stats_packed_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, stride_words, nrows, nKb, row_nnz, stats);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_csr_fill_packed(const uint32_t* mask, long long stride_words, int nrows, int nKb,
+                                   const int32_t* row_ptr, int32_t* col_idx, cudaStream_t stream) {
+    csr_fill_packed_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, stride_words, nrows, nKb, row_ptr, col_idx);
     count_launch();
     return cudaGetLastError();
 }
@@ -588,13 +711,14 @@ cudaError_t launch_tile_map(const MapGeom& g, const int32_t* row_ptr, const int3
 }
 
 static size_t organize_key_cap(const MapGeom& g, int order, int split_pmax) {
-    const size_t rows = (order == BSA_ORDER_GLOBAL_LPT) ? (size_t)g.H * g.nQt : (size_t)g.nQt;
+    const bool global_group = (order == BSA_ORDER_GLOBAL_LPT || order == BSA_ORDER_GLOBAL_BUCKETS);
+    const size_t rows = global_group ? (size_t)g.H * g.nQt : (size_t)g.nQt;
     return rows * (size_t)(split_pmax < 1 ? 1 : split_pmax);
 }
 
 // Minimum (one ranking warp): length histogram + one key per item of a group.
 size_t organize_smem_bytes(const MapGeom& g, int order, int split_pmax) {
-    return ((size_t)g.nKt + 2 + organize_key_cap(g, order, split_pmax)) * sizeof(int32_t);
+    return ((size_t)organize_bins(g) + organize_key_cap(g, order, split_pmax)) * sizeof(int32_t);
 }
 
 cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const int32_t* tile_begin,
@@ -604,7 +728,7 @@ cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const i
     // the caller checked organize_smem_bytes() against the device limit when it chose `order`; whatever shared
     // memory is left up to 200 KB holds per-warp histograms for the parallel ranking (up to one per warp)
     const size_t base = organize_smem_bytes(g, order, split_pmax);
-    const size_t per_warp = ((size_t)g.nKt + 2) * sizeof(int32_t);
+    const size_t per_warp = (size_t)organize_bins(g) * sizeof(int32_t);
     const size_t budget = 200 * 1024;
     int rank_warps = base < budget ? (int)((budget - base) / per_warp) : 0;
     if (rank_warps > 32) rank_warps = 32;
@@ -616,7 +740,7 @@ cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const i
         if (e != cudaSuccess) return e;
         attr_bytes = smem;
     }
-    const int grid = (order == BSA_ORDER_GLOBAL_LPT) ? 1 : g.H;
+    const int grid = (order == BSA_ORDER_GLOBAL_LPT || order == BSA_ORDER_GLOBAL_BUCKETS) ? 1 : g.H;
     organize_kernel<<<grid, 1024, smem, stream>>>(g, order, rank_warps, (int)organize_key_cap(g, order, split_pmax),
                                                    split_pmax <= 1 ? 1 : 0, tile_begin, tile_cnt, row_parts, head_counts,
                                                    items_tmp, items, split_rows, counters);

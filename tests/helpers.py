@@ -75,12 +75,20 @@ def check_plan_structure(req, plan, heads=None):
     # (order 0), over all heads (order 1), or plain row-major (order 2)
     order = inf["plan"]["order"]
     rows = [tuple(int(x) for x in it) for it in items]
+
+    def bucket(n):  # half-octaves: 0, 1, 2, 3, 4-5, 6-7, 8-11, 12-15, ...
+        return n if n <= 1 else 2 * (n.bit_length() - 1) + ((n >> (n.bit_length() - 2)) & 1)
+
     if order == 0:
         want = sorted(rows, key=lambda r: (r[0], -r[7], r[1], r[4]))
     elif order == 1:
         want = sorted(rows, key=lambda r: (-r[7], r[0], r[1], r[4]))
-    else:
+    elif order == 2:
         want = sorted(rows, key=lambda r: (r[0], r[1], r[4]))
+    elif order == 3:
+        want = sorted(rows, key=lambda r: (r[0], -bucket(r[7]), r[1], r[4]))
+    else:
+        want = sorted(rows, key=lambda r: (-bucket(r[7]), r[0], r[1], r[4]))
     assert rows == want, "work items are not in the plan's order"
     nsplit = 0
     for (h, qt), parts in seen.items():

@@ -18,13 +18,13 @@ def _sample(req, per_head, seed=77, heads=None):
 
 
 # ---------------------------------------------------------------- the five configurations
-@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29])
+@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 5, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29, 30, 31, 32, 33])
 def test_tiny_full_oracle_every_plan(plan_id):
     res = Hh.run_request(I.config_tiny(), plan_id=plan_id)
     assert res["pairs"] == res["info"]["nnz_blocks"] * 64 * 64
 
 
-@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 10, 12, 14, 16, 18, 20, 22, 24, 25, 26, 29])
+@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 10, 12, 14, 16, 18, 20, 22, 24, 25, 26, 29, 30, 31])
 def test_mid_full_oracle(plan_id):
     """-1 is the configuration bench.py times (the plan the shipped table selects); every row is compared."""
     Hh.run_request(I.config_mid(), plan_id=plan_id)
@@ -249,6 +249,35 @@ def test_forward_replays_from_a_cuda_graph(plan_id):
             torch.cuda.synchronize()
             assert torch.equal(O, O0) and torch.equal(L, L0)
         assert plan.info()["device_status"] == 0
+
+
+@pytest.mark.parametrize("B_Q,B_KV,N,d,plan_id", [(16, 16, 1000, 64, 22), (32, 64, 4100, 128, 23), (128, 128, 16384, 128, -1),
+                                                  (16, 32, 40000, 64, 25), (256, 16, 9000, 128, 1), (64, 64, 130, 64, 27)])
+def test_bit_packed_mask_gives_the_same_plan_and_output(B_Q, B_KV, N, d, plan_id):
+    """bsa_plan_create_packed reads the mask as bits: statistics, block-CSR, tiles, work items and the forward's output
+    are those of the byte-mask plan, bit for bit (row lengths that are not multiples of 8 or 32 blocks included)."""
+    H = 3
+    M = I.random_mask(11, H, I.cdiv(N, B_Q), I.cdiv(N, B_KV), 0.3)
+    M[1, 2, :] = 0
+    req = I.Request("packed", H, N, d, B_Q, B_KV, M, qkv_seed=9)
+    mask, q, k, v, _ = Hh.to_dev(req, None)
+    bits, stride = bsa.pack_mask(mask)
+    with bsa.plan_create(mask, B_Q, B_KV, N, H, d, plan_id=plan_id) as pa, \
+            bsa.plan_create_packed(bits, stride, B_Q, B_KV, N, H, d, plan_id=plan_id) as pb:
+        ia, ib = pa.info(), pb.info()
+        for key in ("nnz_blocks", "blocks_in_runs", "max_row_nnz", "density", "run_coverage", "skew", "ntiles", "nitems"):
+            assert ia[key] == ib[key], key
+        assert ia["plan"]["plan_id"] == ib["plan"]["plan_id"]
+        for x, y in zip(pa.export_csr(), pb.export_csr()):
+            assert np.array_equal(x, y)
+        for h in range(H):
+            for x, y in zip(pa.export_tiles(h), pb.export_tiles(h)):
+                assert np.array_equal(x, y)
+        assert np.array_equal(pa.export_items(), pb.export_items())
+        Oa, La = pa.forward(q, k, v)
+        Ob, Lb = pb.forward(q, k, v)
+        torch.cuda.synchronize()
+        assert torch.equal(Oa, Ob) and torch.equal(La, Lb)
 
 
 def test_launch_counter_counts_our_kernels():

@@ -1,9 +1,11 @@
 """CPU-only tests: the C-ABI library loads and exports what include/bsa.h declares, the catalog and
 eligibility rules, and the plan-table lookup (Algorithm 2) against the oracle's restatement of it."""
+import ctypes
 import os
 import re
 import subprocess
 
+import numpy as np
 import pytest
 
 from oracle import oracle
@@ -177,3 +179,27 @@ def test_regret_summary_statistics():
     assert abs(s["regret_gm"] - (1.0 * 1.02 * 1.10 * 1.0) ** 0.25) < 1e-12
     assert s["regret_max"] == 1.10 and s["regret_p95"] == 1.10 and abs(s["within_3pct"] - 0.75) < 1e-12
     assert abs(s["speedup_vs_base_gm"] - (1.5 * 1.0 * (1 / 1.1) * 1.025) ** 0.25) < 1e-12
+
+
+def test_pack_mask_matches_numpy_packbits():
+    """The binding's bit-packing helper: little-endian bits, rows padded to a multiple of 4 bytes."""
+    import torch
+    rng = np.random.default_rng(3)
+    for nk in (1, 7, 8, 31, 32, 33, 100):
+        m = (rng.random((2, 5, nk)) < 0.4).astype(np.uint8)
+        packed, stride = bsa.pack_mask(torch.from_numpy(m))
+        assert stride % 4 == 0 and stride * 8 >= nk and packed.shape == (2, 5, stride)
+        ref = np.packbits(m, axis=2, bitorder="little")
+        got = packed.numpy()
+        assert np.array_equal(got[:, :, : ref.shape[2]], ref) and not got[:, :, ref.shape[2]:].any()
+
+
+def test_packed_create_rejects_bad_layouts_without_a_gpu():
+    h = ctypes.c_void_p()
+    L = bsa.lib()
+    fake = ctypes.c_void_p(0x1000)  # never dereferenced: the checks come first
+    assert L.bsa_plan_create_packed(fake, 6, 128, 128, 1024, 1, 128, None, None, ctypes.byref(h)) == 1   # stride % 4
+    assert L.bsa_plan_create_packed(fake, 0, 128, 128, 1024, 1, 128, None, None, ctypes.byref(h)) == 1   # stride <= 0
+    assert L.bsa_plan_create_packed(fake, 4, 16, 16, 1024, 1, 128, None, None, ctypes.byref(h)) == 1     # 64 blocks > 32 bits
+    assert L.bsa_plan_create_packed(ctypes.c_void_p(0x1002), 8, 16, 16, 1024, 1, 128, None, None, ctypes.byref(h)) == 1
+    assert L.bsa_plan_create_packed(None, 8, 16, 16, 1024, 1, 128, None, None, ctypes.byref(h)) == 1
