@@ -1349,6 +1349,19 @@ __device__ __forceinline__ ItemSpan load_item_span(const WorkItem* items, int id
     return r;
 }
 
+// Slot and phase of a shared-memory ring, advanced once per tile (the single-thread roles sit on the path of every
+// tile: no division by the ring depth there).
+struct RingPos {
+    int stage = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void advance(int depth) {
+        if (++stage == depth) {
+            stage = 0;
+            phase ^= 1u;
+        }
+    }
+};
+
 struct __align__(8) PpBarriers {
     uint64_t q_full[2], q_empty[2], o_free, o_full, e_ready, e_taken;
     uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
@@ -1525,6 +1538,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             // while K slots are free, and a new item's first Q K^T does not wait for its Q tile.
             uint32_t g = 0, itq = 0;  // itq: Q tiles issued (buffer itq & 1)
             uint32_t seq = 0;          // non-empty items entered
+            RingPos ring;              // K ring position of tile g
             bool ok = true;
             BSA_TRACE_DECL(tn);
             int pq_row0 = 0, pq_row1 = 0, pq_row2 = 0, pq_head0 = 0, pq_head1 = 0, pq_head2 = 0;
@@ -1568,11 +1582,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (!ok) break;
                 ++seq;
                 int col_next = p.tile_col[it.tile_begin];
-                for (int j = it.tile_begin; j < it.tile_end && ok; ++j, ++g) {
+                for (int j = it.tile_begin; j < it.tile_end && ok; ++j, ++g, ring.advance(NSK)) {
                     const int col_cur = col_next;
                     if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
-                    const int stage = g % NSK;
-                    const uint32_t ph = (g / NSK) & 1;
+                    const int stage = ring.stage;
+                    const uint32_t ph = ring.phase;
                     while (ok && npend > 0 &&
                            (pq_need0 <= (int)g - NSK ||
                             mbar_test_wait(smem_u32(&bars.q_empty[itq & 1]), ((itq >> 1) & 1) ^ 1)))
@@ -1601,6 +1615,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         } else if (warp == 11 && lane == 0) {
             // =========================== V producer ===========================
             uint32_t g = 0;
+            RingPos ring;  // V ring position of tile g
             bool ok = true;
             WorkItem it_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);
             for (int kr = 0; kr < n_rounds && ok; ++kr) {
@@ -1608,11 +1623,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 it_next = load_item(p.items, cta_item_index(kr + 1, blockIdx.x, gridDim.x), n_items);
                 if (it.ntiles <= 0) continue;
                 int col_next = p.tile_col[it.tile_begin];
-                for (int j = it.tile_begin; j < it.tile_end; ++j, ++g) {
+                for (int j = it.tile_begin; j < it.tile_end; ++j, ++g, ring.advance(NSV)) {
                     const int col_cur = col_next;
                     if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
-                    const int stage = g % NSV;
-                    const uint32_t ph = (g / NSV) & 1;
+                    const int stage = ring.stage;
+                    const uint32_t ph = ring.phase;
                     ok = mbar_wait(smem_u32(&bars.v_empty[stage]), ph ^ 1, abortp);
                     if (!ok) break;
                     mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), KV_TILE);
@@ -1630,6 +1645,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
             const uint64_t descQ0 = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
             const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
+            RingPos ring;  // K ring position of the tile being issued
             uint32_t itq = 0, g = 0;
             bool ok = true;
             BSA_TRACE_DECL(tn);
@@ -1642,10 +1658,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 ok = mbar_wait(smem_u32(&bars.q_full[qb]), (itq >> 1) & 1, abortp);
                 if (!ok) break;
                 const uint64_t descQ = descQ0 + (uint64_t)((qb * NSUB * Q_SUB) >> 4);
-                for (int j = 0; j < n; ++j) {
+                for (int j = 0; j < n; ++j, ring.advance(NSK)) {
                     const uint32_t gs = g + j;
-                    const int stage = gs % NSK;
-                    const uint32_t ph = (gs / NSK) & 1, sb = gs & 1;
+                    const int stage = ring.stage;
+                    const uint32_t ph = ring.phase, sb = gs & 1;
                     // K tile present, and S[sb] read into registers by the softmax of tile gs-2
                     if (gs >= 2)
                         ok = mbar_wait2(smem_u32(&bars.s_free[sb]), ((gs >> 1) - 1) & 1, smem_u32(&bars.k_full[stage]), ph, abortp);
@@ -1673,6 +1689,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             // =========================== P V issuer ===========================
             constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
             const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
+            RingPos ring;  // V ring position of the tile being issued
             uint32_t itq = 0, g = 0;
             bool ok = true;
             BSA_TRACE_DECL(tn);
@@ -1681,10 +1698,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const int n = n_next;
                 n_next = load_item(p.items, cta_item_index(kr + 1, blockIdx.x, gridDim.x), n_items).ntiles;
                 if (n <= 0) continue;
-                for (int j = 0; j < n; ++j) {
+                for (int j = 0; j < n; ++j, ring.advance(NSV)) {
                     const uint32_t gp = g + j;
-                    const int stage = gp % NSV;
-                    const uint32_t ph = (gp / NSV) & 1, sb = gp & 1;
+                    const int stage = ring.stage;
+                    const uint32_t ph = ring.phase, sb = gp & 1;
                     // V tile present (normally long before), accumulator drained by the epilogue (first tile of an
                     // item), and last the P tile, which is the one this thread normally waits for
                     if (j == 0) {
