@@ -1549,9 +1549,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const uint32_t b = itq & 1;
                 if (!mbar_wait(smem_u32(&bars.q_empty[b]), ((itq >> 1) & 1) ^ 1, abortp)) return false;
                 mbar_arrive_expect_tx(smem_u32(&bars.q_full[b]), NSUB * Q_SUB);
-                for (int s = 0; s < NSUB; ++s)
-                    tma_load_3d(smem_u32(sQ + b * NSUB * Q_SUB + s * Q_SUB), &tmQ, smem_u32(&bars.q_full[b]), s * 64, pq_row0,
-                                pq_head0);
+                tma_load_4d(smem_u32(sQ + b * NSUB * Q_SUB), &tmQ, smem_u32(&bars.q_full[b]), 0, pq_row0, 0, pq_head0);
                 ++itq;
                 pq_row0 = pq_row1; pq_head0 = pq_head1; pq_need0 = pq_need1;
                 pq_row1 = pq_row2; pq_head1 = pq_head2; pq_need1 = pq_need2;
@@ -1597,9 +1595,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     if (!ok) break;
                     BSA_TRACE_POINT(0, tn, 20);
                     mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), KV_TILE);
-                    for (int s = 0; s < NSUB; ++s)
-                        tma_load_3d(smem_u32(sK + stage * KV_TILE + s * KV_SUB), &tmK, smem_u32(&bars.k_full[stage]),
-                                    s * 64, col_cur * TK, it.head);
+                    tma_load_4d(smem_u32(sK + stage * KV_TILE), &tmK, smem_u32(&bars.k_full[stage]), 0, col_cur * TK, 0, it.head);
                     BSA_TRACE_POINT(0, tn, 21);
 #ifdef BSA_TRACE_KLAT
                     mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
@@ -1631,9 +1627,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     ok = mbar_wait(smem_u32(&bars.v_empty[stage]), ph ^ 1, abortp);
                     if (!ok) break;
                     mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), KV_TILE);
-                    for (int s = 0; s < NSUB; ++s)
-                        tma_load_3d(smem_u32(sV + stage * KV_TILE + s * KV_SUB), &tmV, smem_u32(&bars.v_full[stage]),
-                                    s * 64, col_cur * TK, it.head);
+                    tma_load_4d(smem_u32(sV + stage * KV_TILE), &tmV, smem_u32(&bars.v_full[stage]), 0, col_cur * TK, 0, it.head);
                 }
             }
             if (!ok) {
@@ -2055,11 +2049,29 @@ bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, i
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same tensor as {64 columns, N rows, d/64 column groups, heads}; box = {64, rows, d/64, 1}: one copy lands all
+// 64-column sub-tiles of a row block back to back (the [sub-tile][row][64] layout the MMA descriptors address).
+bool encode_map4(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows) {
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[4] = {64, (cuuint64_t)N, (cuuint64_t)(d / 64), (cuuint64_t)heads};
+    cuuint64_t strides[3] = {(cuuint64_t)d * 2, 128, (cuuint64_t)N * (cuuint64_t)d * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, (cuuint32_t)(d / 64), 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int D, int TK, int KERNEL>
 cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t stream, const char** err) {
     CUtensorMap tq, tk, tv;
-    if (!encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ) || !encode_map(&tk, a.K, a.g.N, a.g.H, D, TK) ||
-        !encode_map(&tv, a.V, a.g.N, a.g.H, D, TK)) {
+    const bool ok_maps = (KERNEL == 4)
+                             ? (encode_map4(&tq, a.Q, a.g.N, a.g.H, D, kTQ) && encode_map4(&tk, a.K, a.g.N, a.g.H, D, TK) &&
+                                encode_map4(&tv, a.V, a.g.N, a.g.H, D, TK))
+                             : (encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ) && encode_map(&tk, a.K, a.g.N, a.g.H, D, TK) &&
+                                encode_map(&tv, a.V, a.g.N, a.g.H, D, TK));
+    if (!ok_maps) {
         *err = "cuTensorMapEncodeTiled failed";
         return cudaErrorInvalidValue;
     }
