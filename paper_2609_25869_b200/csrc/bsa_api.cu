@@ -461,23 +461,37 @@ extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int 
     const size_t lbytes = (size_t)heads * (size_t)N * 4;
     const size_t o_m = 0, o_q = align_up(mbytes), o_k = o_q + align_up(tbytes), o_v = o_k + align_up(tbytes),
                  o_o = o_v + align_up(tbytes), o_l = o_o + align_up(tbytes), total = o_l + align_up(lbytes);
-    cudaStream_t s = nullptr;
+    // Two streams kept per host thread: the mask goes first on `s` and the plan is created behind it, while Q, K and V
+    // travel on `s2`; the forward waits for them.  Planning (statistics copy, lookup, preparation kernels) thus
+    // overlaps the 3 x heads x N x d x 2 bytes of input copies instead of following them.
+    static thread_local cudaStream_t s = nullptr, s2 = nullptr;
+    static thread_local cudaEvent_t inputs_ready = nullptr;
+    cudaError_t e = cudaSuccess;
+    if (!s) e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
+    if (e == cudaSuccess && !s2) e = cudaStreamCreateWithFlags(&s2, cudaStreamNonBlocking);
+    if (e == cudaSuccess && !inputs_ready) e = cudaEventCreateWithFlags(&inputs_ready, cudaEventDisableTiming);
+    if (e != cudaSuccess) { set_cuda_err(e, "request streams"); return BSA_ERR_CUDA; }
     uint8_t* buf = nullptr;
-    cudaError_t e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
-    if (e != cudaSuccess) { set_cuda_err(e, "stream"); return BSA_ERR_CUDA; }
     bsa_status_t st = BSA_OK;
     bsa_plan_t* plan = nullptr;
     e = cudaMallocAsync(&buf, total, s);
-    if (e != cudaSuccess) { set_cuda_err(e, "request buffers"); cudaStreamDestroy(s); return BSA_ERR_OOM; }
+    if (e != cudaSuccess) { set_cuda_err(e, "request buffers"); return BSA_ERR_OOM; }
     e = cudaMemcpyAsync(buf + o_m, mask_host, mbytes, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_q, Q_host, tbytes, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_k, K_host, tbytes, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_v, V_host, tbytes, cudaMemcpyHostToDevice, s);
+    // the buffer exists once `s` reaches this point: order the other stream behind it
+    if (e == cudaSuccess) e = cudaEventRecord(inputs_ready, s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s2, inputs_ready, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_q, Q_host, tbytes, cudaMemcpyHostToDevice, s2);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_k, K_host, tbytes, cudaMemcpyHostToDevice, s2);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_v, V_host, tbytes, cudaMemcpyHostToDevice, s2);
+    if (e == cudaSuccess) e = cudaEventRecord(inputs_ready, s2);
     if (e == cudaSuccess) {
         st = bsa_plan_create_ex(buf + o_m, B_Q, B_KV, N, heads, d, options, s, &plan);
-        if (st == BSA_OK)
-            st = bsa_forward(plan, buf + o_q, buf + o_k, buf + o_v, buf + o_o, reinterpret_cast<float*>(buf + o_l), s);
         if (st == BSA_OK) {
+            e = cudaStreamWaitEvent(s, inputs_ready, 0);
+            if (e == cudaSuccess)
+                st = bsa_forward(plan, buf + o_q, buf + o_k, buf + o_v, buf + o_o, reinterpret_cast<float*>(buf + o_l), s);
+        }
+        if (st == BSA_OK && e == cudaSuccess) {
             e = cudaMemcpyAsync(O_host, buf + o_o, tbytes, cudaMemcpyDeviceToHost, s);
             if (e == cudaSuccess) e = cudaMemcpyAsync(LSE_host, buf + o_l, lbytes, cudaMemcpyDeviceToHost, s);
             if (e == cudaSuccess) e = cudaStreamSynchronize(s);
@@ -490,9 +504,9 @@ extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int 
         if (info_out) *info_out = info;
     }
     if (plan) bsa_plan_destroy(plan);
+    cudaStreamSynchronize(s2);  // on an error path the copies may still be in flight
     cudaFreeAsync(buf, s);
     cudaStreamSynchronize(s);
-    cudaStreamDestroy(s);
     if (e != cudaSuccess) { set_cuda_err(e, "request"); return BSA_ERR_CUDA; }
     return st;
 }
