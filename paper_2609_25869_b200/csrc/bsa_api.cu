@@ -164,25 +164,50 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     p->counters = reinterpret_cast<PlanCountersDev*>(p->arena1 + o_cnt);
     p->head_counts = reinterpret_cast<int32_t*>(p->arena1 + o_hc);
     BSA_CUDA(cudaMemsetAsync(p->arena1 + o_zero, 0, a1_bytes - o_zero, stream), "memset");
+    // ---- lines 3-5: only the scalars cross to the host.  The statistics kernel's last CTA posts them into pinned
+    // host memory and the host polls for the sequence number (a few microseconds less than a copy command and an
+    // event); if nothing arrives within a millisecond the host falls back to that copy.
+    static thread_local MaskStatsHost* posted = nullptr;
+    static thread_local unsigned post_seq = 0;
+    if (!posted) {
+        BSA_CUDA(cudaMallocHost(&posted, sizeof(MaskStatsHost)), "pinned stats");
+        memset(posted, 0, sizeof *posted);
+    }
+    const unsigned seq = ++post_seq ? post_seq : ++post_seq;  // never 0
     const uint32_t* mask_words = reinterpret_cast<const uint32_t*>(mask_dev);
     if (packed_stride > 0)
-        BSA_CUDA(launch_mask_row_stats_packed(mask_words, packed_stride / 4, nrows, nKb, p->row_nnz, p->stats, stream),
+        BSA_CUDA(launch_mask_row_stats_packed(mask_words, packed_stride / 4, nrows, nKb, p->row_nnz, p->stats, stream, posted,
+                                              seq),
                  "mask_row_stats_packed");
     else
-        BSA_CUDA(launch_mask_row_stats(mask_dev, nrows, nKb, p->row_nnz, p->stats, stream), "mask_row_stats");
+        BSA_CUDA(launch_mask_row_stats(mask_dev, nrows, nKb, p->row_nnz, p->stats, stream, posted, seq), "mask_row_stats");
     const double t1 = now_us();
-
-    // ---- lines 3-5: only the scalars cross to the host ----
-    static thread_local MaskStatsDev* pinned = nullptr;
-    if (!pinned) BSA_CUDA(cudaMallocHost(&pinned, sizeof(MaskStatsDev)), "pinned stats");
-    static thread_local cudaEvent_t stats_copied = nullptr;
-    if (!stats_copied) BSA_CUDA(cudaEventCreateWithFlags(&stats_copied, cudaEventDisableTiming), "stats event");
-    BSA_CUDA(cudaMemcpyAsync(pinned, p->stats, sizeof(MaskStatsDev), cudaMemcpyDeviceToHost, stream), "stats copy");
-    BSA_CUDA(cudaEventRecord(stats_copied, stream), "stats event record");
     // the row-pointer scan needs nothing from the host: it runs while the host waits for the scalars
     BSA_CUDA(launch_row_scan(p->row_nnz, nrows, p->row_ptr, stream), "row_scan");
-    BSA_CUDA(cudaEventSynchronize(stats_copied), "stats sync");
-    p->hstats = *pinned;
+    {
+        volatile unsigned* flag = &posted->seq;
+        const double t_poll = now_us();
+        bool arrived = true;
+        while (*flag != seq) {
+            if (now_us() - t_poll > 1000.0) {
+                arrived = false;
+                break;
+            }
+        }
+        if (arrived) {
+            std::atomic_thread_fence(std::memory_order_acquire);
+            p->hstats.nnz = posted->nnz;
+            p->hstats.in_runs = posted->in_runs;
+            p->hstats.max_row_nnz = posted->max_row_nnz;
+            p->hstats.blocks_done = 0;
+        } else {
+            static thread_local MaskStatsDev* pinned = nullptr;
+            if (!pinned) BSA_CUDA(cudaMallocHost(&pinned, sizeof(MaskStatsDev)), "pinned stats copy");
+            BSA_CUDA(cudaMemcpyAsync(pinned, p->stats, sizeof(MaskStatsDev), cudaMemcpyDeviceToHost, stream), "stats copy");
+            BSA_CUDA(cudaStreamSynchronize(stream), "stats sync");
+            p->hstats = *pinned;
+        }
+    }
     const double t2 = now_us();
 
     // ---- lines 6-19: regime lookup, ranked fallback, eligibility ----

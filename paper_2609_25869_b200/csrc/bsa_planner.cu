@@ -43,12 +43,27 @@ __device__ __forceinline__ unsigned row_word_bits(const uint4* __restrict__ word
     return bits & keep;
 }
 
+// Called by thread 0 of every CTA of a statistics kernel after it has added its share: the CTA that finds itself last
+// copies the totals into pinned host memory, so the host can read them without a copy command or an event.
+__device__ __forceinline__ void post_stats_if_last(MaskStatsDev* stats, MaskStatsHost* post, unsigned seq) {
+    if (!post) return;
+    __threadfence();
+    if (atomicAdd(&stats->blocks_done, 1u) != gridDim.x - 1) return;
+    __threadfence();
+    post->nnz = atomicAdd(&stats->nnz, 0ull);
+    post->in_runs = atomicAdd(&stats->in_runs, 0ull);
+    post->max_row_nnz = atomicMax(&stats->max_row_nnz, 0u);
+    __threadfence_system();
+    *reinterpret_cast<volatile unsigned*>(&post->seq) = seq;
+}
+
 // ------------------------------------------------------------------------------------------
 // mask_row_stats: one warp per (head, query-block) row.
 // A block counts towards run coverage iff its left or right neighbour in the same row is active.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __restrict__ mask, int nrows, int nKb,
-                                                              int32_t* __restrict__ row_nnz, MaskStatsDev* stats) {
+                                                              int32_t* __restrict__ row_nnz, MaskStatsDev* stats,
+                                                              MaskStatsHost* post, unsigned seq) {
     __shared__ unsigned s_nnz[8], s_runs[8], s_max[8];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row = blockIdx.x * 8 + warp;
@@ -103,6 +118,7 @@ __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __re
             atomicAdd(&stats->in_runs, tr);
             atomicMax(&stats->max_row_nnz, mx);
         }
+        post_stats_if_last(stats, post, seq);
     }
 }
 
@@ -121,7 +137,7 @@ __device__ __forceinline__ unsigned packed_row_word(const uint32_t* __restrict__
 
 __global__ void __launch_bounds__(256) mask_row_stats_packed_kernel(const uint32_t* __restrict__ mask, long long stride_words,
                                                                      int nrows, int nKb, int32_t* __restrict__ row_nnz,
-                                                                     MaskStatsDev* stats) {
+                                                                     MaskStatsDev* stats, MaskStatsHost* post, unsigned seq) {
     __shared__ unsigned s_nnz[8], s_runs[8];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row = blockIdx.x * 8 + warp;
@@ -168,6 +184,7 @@ __global__ void __launch_bounds__(256) mask_row_stats_packed_kernel(const uint32
             atomicAdd(&stats->in_runs, tr);
             atomicMax(&stats->max_row_nnz, mx);
         }
+        post_stats_if_last(stats, post, seq);
     }
 }
 
@@ -661,15 +678,17 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
 }  // namespace
 
 cudaError_t launch_mask_row_stats(const uint8_t* mask, int nrows, int nKb, int32_t* row_nnz, MaskStatsDev* stats,
-                                  cudaStream_t stream) {
-    mask_row_stats_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, nrows, nKb, row_nnz, stats);
+                                  cudaStream_t stream, MaskStatsHost* post, unsigned seq) {
+    mask_row_stats_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, nrows, nKb, row_nnz, stats, post, seq);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_mask_row_stats_packed(const uint32_t* mask, long long stride_words, int nrows, int nKb,
-                                         int32_t* row_nnz, MaskStatsDev* stats, cudaStream_t stream) {
-    mask_row_stats_packed_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, stride_words, nrows, nKb, row_nnz, stats);
+                                         int32_t* row_nnz, MaskStatsDev* stats, cudaStream_t stream, MaskStatsHost* post,
+                                         unsigned seq) {
+    mask_row_stats_packed_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, stride_words, nrows, nKb, row_nnz, stats, post,
+                                                                        seq);
     count_launch();
     return cudaGetLastError();
 }
