@@ -160,8 +160,45 @@ BSA_API bsa_status_t bsa_plan_create_packed(const uint8_t* mask_bits_dev, int64_
 BSA_API bsa_status_t bsa_forward(const bsa_plan_t* plan, const void* Q_dev, const void* K_dev, const void* V_dev,
                          void* O_dev, float* LSE_dev, void* stream);
 
-/* Frees the plan and every device buffer it owns.  Synchronises with the plan's create stream. */
+/* Lets go of the plan.  A plan from bsa_plan_create* is freed with every device buffer it owns, and the call
+ * synchronises with the plan's create stream.  A plan from bsa_plan_cache_get is shared: the call only drops the
+ * caller's hold (no synchronisation) unless it was the last one. */
 BSA_API bsa_status_t bsa_plan_destroy(bsa_plan_t* plan);
+
+/* ---------------------------------------------------------------------------------------------
+ * Plan cache -- the warm path of Section 5.2 / Section 6.5: while the mask stays the same across
+ * layers or denoising steps, the prepared plan is reused and only the attention kernels run.  The
+ * paper leaves the reuse to the caller; this cache recognises a repeated mask by itself.
+ *
+ * bsa_plan_cache_get runs the mask-statistics kernel (as bsa_plan_create does), which here also sums
+ * a 128-bit position-salted fingerprint of the activity pattern, and looks up
+ * (fingerprint, B_Q, B_KV, N, heads, d, mask format and alignment, options, device, plan-table
+ * generation).  Hit: the prepared plan is returned (*out_hit = 1), nothing else is launched; if the
+ * plan was prepared on another stream, `stream` is first made to wait for that preparation.  Miss:
+ * the plan is prepared exactly as by bsa_plan_create_ex / bsa_plan_create_packed, kept in the cache
+ * and returned (*out_hit = 0); beyond `capacity` plans the least recently used one is dropped.
+ * Two different masks collide only if both 64-bit sums agree (no comparison of the masks follows).
+ *
+ *   row_stride_bytes : 0 = one byte per logical block (as bsa_plan_create); > 0 = bit-packed rows
+ *                      (as bsa_plan_create_packed).  mask_dev is device memory, borrowed for the call.
+ *   out_plan         : shared with the cache and with every other caller that got the same plan;
+ *                      give it back with bsa_plan_destroy.  Forwards on one plan must be
+ *                      stream-ordered (they share the Split-K workspace).
+ *   out_hit          : may be NULL.
+ * bsa_lut_load, bsa_lut_clear and bsa_force_plan start a new generation: plans selected before are
+ * not returned afterwards.  All four calls are thread-safe.  bsa_plan_cache_destroy drops the
+ * cache's holds (plans still held by callers stay valid) and synchronises with the create streams
+ * of the plans it frees.  Errors: as bsa_plan_create_ex; INVALID_ARG for a null cache, capacity < 1
+ * or a negative stride.
+ */
+typedef struct bsa_plan_cache bsa_plan_cache_t;
+BSA_API bsa_status_t bsa_plan_cache_create(int capacity, bsa_plan_cache_t** out_cache);
+BSA_API bsa_status_t bsa_plan_cache_get(bsa_plan_cache_t* cache, const uint8_t* mask_dev, int64_t row_stride_bytes, int B_Q,
+                                int B_KV, int64_t N, int heads, int d, const bsa_options_t* options /* may be NULL */,
+                                void* stream, bsa_plan_t** out_plan, int* out_hit);
+BSA_API bsa_status_t bsa_plan_cache_stats(bsa_plan_cache_t* cache, int64_t* hits, int64_t* misses, int64_t* evictions,
+                                  int32_t* entries);
+BSA_API bsa_status_t bsa_plan_cache_destroy(bsa_plan_cache_t* cache);
 
 /* ---------------------------------------------------------------------------------------------
  * bsa_request_host -- one complete request from HOST buffers: copies mask, Q, K, V to the device,

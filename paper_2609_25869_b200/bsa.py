@@ -75,6 +75,12 @@ def lib() -> ctypes.CDLL:
     L.bsa_plan_create.argtypes = [vp, i32, i32, i64, i32, i32, ctypes.POINTER(vp)]
     L.bsa_plan_create_ex.argtypes = [vp, i32, i32, i64, i32, i32, ctypes.POINTER(Options), vp, ctypes.POINTER(vp)]
     L.bsa_plan_create_packed.argtypes = [vp, i64, i32, i32, i64, i32, i32, ctypes.POINTER(Options), vp, ctypes.POINTER(vp)]
+    L.bsa_plan_cache_create.argtypes = [i32, ctypes.POINTER(vp)]
+    L.bsa_plan_cache_get.argtypes = [vp, vp, i64, i32, i32, i64, i32, i32, ctypes.POINTER(Options), vp, ctypes.POINTER(vp),
+                                     ctypes.POINTER(i32)]
+    L.bsa_plan_cache_stats.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i64),
+                                       ctypes.POINTER(ctypes.c_int32)]
+    L.bsa_plan_cache_destroy.argtypes = [vp]
     L.bsa_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.bsa_plan_destroy.argtypes = [vp]
     L.bsa_request_host.argtypes = [vp, i32, i32, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.POINTER(Options),
@@ -239,6 +245,46 @@ def plan_create_packed(mask_bits, row_stride: int, B_Q: int, B_KV: int, N: int, 
     _check(lib().bsa_plan_create_packed(mask_bits.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
                                         _stream_ptr(stream), ctypes.byref(h)), "bsa_plan_create_packed")
     return Plan(h.value)
+
+
+class PlanCache:
+    """``bsa_plan_cache_*``: prepared plans keyed by a fingerprint of the mask's activity pattern (warm path)."""
+
+    def __init__(self, capacity: int = 64):
+        h = ctypes.c_void_p()
+        _check(lib().bsa_plan_cache_create(capacity, ctypes.byref(h)), "bsa_plan_cache_create")
+        self._h = h.value
+
+    def get(self, mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1, max_workspace_bytes: int = 0,
+            stream=None, row_stride: int = 0):
+        """``bsa_plan_cache_get``: returns ``(plan, hit)``.  ``row_stride`` > 0: ``mask`` is bit-packed (``pack_mask``).
+        The plan is shared with the cache; ``plan.destroy()`` only gives it back."""
+        import torch
+        assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool)
+        h = ctypes.c_void_p()
+        hit = ctypes.c_int(0)
+        opt = Options(plan_id, 0, max_workspace_bytes)
+        _check(lib().bsa_plan_cache_get(self._h, mask.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
+                                        _stream_ptr(stream), ctypes.byref(h), ctypes.byref(hit)), "bsa_plan_cache_get")
+        return Plan(h.value), bool(hit.value)
+
+    def stats(self) -> Dict:
+        a, b, c = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+        n = ctypes.c_int32()
+        _check(lib().bsa_plan_cache_stats(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(n)),
+               "bsa_plan_cache_stats")
+        return {"hits": a.value, "misses": b.value, "evictions": c.value, "entries": n.value}
+
+    def destroy(self):
+        if self._h:
+            _check(lib().bsa_plan_cache_destroy(self._h), "bsa_plan_cache_destroy")
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
 
 def request_host(mask: np.ndarray, B_Q: int, B_KV: int, N: int, heads: int, d: int, Q, K, V, O, LSE,

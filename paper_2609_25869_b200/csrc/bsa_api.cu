@@ -5,7 +5,10 @@
 #include <time.h>
 
 #include <atomic>
+#include <list>
+#include <mutex>
 #include <new>
+#include <unordered_map>
 
 #include "bsa_common.h"
 
@@ -28,6 +31,8 @@ int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, d
 int catalog_size();
 
 static std::atomic<long long> g_launches{0};
+// bumped whenever the plan table or the forced plan changes: cached plans selected before that are not reused
+static std::atomic<unsigned> g_select_generation{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 static thread_local char g_cuda_err[256] = "";
@@ -83,6 +88,31 @@ struct bsa_plan {
     int lut_hit;
     int32_t buckets[4];
     float us_mask_state, us_stats_sync, us_lookup, us_launch_prep, us_total;
+    // sharing (plan cache): the plan is freed when the last holder lets go; `ready` (cached plans only) is recorded
+    // behind the preparation kernels so that a later request on another stream can wait for them
+    std::atomic<int> refs;
+    cudaEvent_t ready;
+};
+
+// ---- plan cache (warm path of Section 5.2: a prepared plan is reused while the mask stays the same) ----
+namespace {
+struct CacheKey {
+    uint64_t hash[2];
+    int64_t N, packed_stride, max_ws;
+    int32_t B_Q, B_KV, heads, d, align, force, device;
+    uint32_t generation;
+    bool operator==(const CacheKey& o) const { return memcmp(this, &o, sizeof *this) == 0; }
+};
+struct CacheKeyHash {
+    size_t operator()(const CacheKey& k) const { return (size_t)(k.hash[0] ^ (k.hash[1] * 0x9E3779B97F4A7C15ull)); }
+};
+}  // namespace
+struct bsa_plan_cache {
+    std::mutex mu;
+    int capacity;
+    std::list<std::pair<CacheKey, bsa_plan*>> lru;  // most recently used first
+    std::unordered_map<CacheKey, std::list<std::pair<CacheKey, bsa_plan*>>::iterator, CacheKeyHash> index;
+    int64_t hits, misses, evictions;
 };
 
 static bsa_status_t validate(const void* mask, int B_Q, int B_KV, int64_t N, int heads, int d, void* out) {
@@ -95,6 +125,7 @@ static bsa_status_t validate(const void* mask, int B_Q, int B_KV, int64_t N, int
 
 static void free_plan(bsa_plan* p) {
     if (!p) return;
+    if (p->ready) cudaEventDestroy(p->ready);
     if (p->arena1) cudaFreeAsync(p->arena1, p->stream);
     if (p->arena2) cudaFreeAsync(p->arena2, p->stream);
     if (p->ws_O) cudaFreeAsync(p->ws_O, p->stream);
@@ -111,9 +142,18 @@ static void free_plan(bsa_plan* p) {
         }                                \
     } while (0)
 
-// `packed_stride` = 0: one byte per logical block; > 0: bit-packed rows of that many bytes (bsa_plan_create_packed)
+// one holder lets go of the plan; the last one frees it (stream-ordered on the plan's create stream, no wait)
+static bool release_plan(bsa_plan* p) {
+    if (p->refs.fetch_sub(1, std::memory_order_acq_rel) > 1) return false;
+    free_plan(p);
+    return true;
+}
+
+// `packed_stride` = 0: one byte per logical block; > 0: bit-packed rows of that many bytes (bsa_plan_create_packed).
+// `cache` (may be null): look the mask up after the statistics have arrived and reuse the prepared plan on a hit.
 static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, int B_Q, int B_KV, int64_t N, int heads,
-                                int d, const bsa_options_t* options, void* stream_v, bsa_plan_t** out_plan) {
+                                int d, const bsa_options_t* options, void* stream_v, bsa_plan_t** out_plan,
+                                bsa_plan_cache* cache = nullptr, int* cache_hit = nullptr) {
     bsa_status_t vs = validate(mask_dev, B_Q, B_KV, N, heads, d, out_plan);
     if (vs != BSA_OK) return vs;
     if (packed_stride > 0) {
@@ -126,7 +166,8 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
     bsa_plan* p = new (std::nothrow) bsa_plan();
     if (!p) return BSA_ERR_OOM;
-    memset(p, 0, sizeof *p);
+    memset(static_cast<void*>(p), 0, sizeof *p);
+    p->refs.store(1, std::memory_order_relaxed);
     p->stream = stream;
     p->d = d;
     BSA_CUDA(cudaGetDevice(&p->device), "cudaGetDevice");
@@ -177,10 +218,11 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     const uint32_t* mask_words = reinterpret_cast<const uint32_t*>(mask_dev);
     if (packed_stride > 0)
         BSA_CUDA(launch_mask_row_stats_packed(mask_words, packed_stride / 4, nrows, nKb, p->row_nnz, p->stats, stream, posted,
-                                              seq),
+                                              seq, cache != nullptr),
                  "mask_row_stats_packed");
     else
-        BSA_CUDA(launch_mask_row_stats(mask_dev, nrows, nKb, p->row_nnz, p->stats, stream, posted, seq), "mask_row_stats");
+        BSA_CUDA(launch_mask_row_stats(mask_dev, nrows, nKb, p->row_nnz, p->stats, stream, posted, seq, cache != nullptr),
+                 "mask_row_stats");
     const double t1 = now_us();
     // the row-pointer scan needs nothing from the host: it runs while the host waits for the scalars
     BSA_CUDA(launch_row_scan(p->row_nnz, nrows, p->row_ptr, stream), "row_scan");
@@ -200,6 +242,8 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
             p->hstats.in_runs = posted->in_runs;
             p->hstats.max_row_nnz = posted->max_row_nnz;
             p->hstats.blocks_done = 0;
+            p->hstats.hash[0] = posted->hash[0];
+            p->hstats.hash[1] = posted->hash[1];
         } else {
             static thread_local MaskStatsDev* pinned = nullptr;
             if (!pinned) BSA_CUDA(cudaMallocHost(&pinned, sizeof(MaskStatsDev)), "pinned stats copy");
@@ -210,14 +254,55 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     }
     const double t2 = now_us();
 
+    const int64_t max_ws = options ? options->max_workspace_bytes : 0;
+    int forced = (options && options->force_plan_id >= 0) ? options->force_plan_id : get_force_plan();
+    CacheKey key;
+    if (cache) {
+        // ---- warm path: the same activity pattern, request key and selection inputs give the same plan ----
+        memset(&key, 0, sizeof key);
+        key.hash[0] = p->hstats.hash[0];
+        key.hash[1] = p->hstats.hash[1];
+        key.N = N; key.packed_stride = packed_stride; key.max_ws = max_ws;
+        key.B_Q = B_Q; key.B_KV = B_KV; key.heads = heads; key.d = d;
+        key.align = packed_stride > 0 ? 0 : (int32_t)(reinterpret_cast<uintptr_t>(mask_dev) & 15u);
+        key.force = forced; key.device = p->device;
+        key.generation = g_select_generation.load(std::memory_order_relaxed);
+        bsa_plan* found = nullptr;
+        {
+            std::lock_guard<std::mutex> lock(cache->mu);
+            auto it = cache->index.find(key);
+            if (it != cache->index.end()) {
+                cache->lru.splice(cache->lru.begin(), cache->lru, it->second);
+                found = it->second->second;
+                found->refs.fetch_add(1, std::memory_order_relaxed);
+                ++cache->hits;
+            } else {
+                ++cache->misses;
+            }
+        }
+        if (found) {
+            free_plan(p);  // only the first arena exists; its kernels are stream-ordered before the free
+            p = nullptr;
+            if (found->stream != stream) {
+                cudaError_t e = cudaStreamWaitEvent(stream, found->ready, 0);
+                if (e != cudaSuccess) {
+                    set_cuda_err(e, "cache wait");
+                    release_plan(found);
+                    return BSA_ERR_CUDA;
+                }
+            }
+            if (cache_hit) *cache_hit = 1;
+            *out_plan = found;
+            return BSA_OK;
+        }
+    }
+
     // ---- lines 6-19: regime lookup, ranked fallback, eligibility ----
     const double total_blocks = (double)nrows * nKb;
     const double nnz = (double)p->hstats.nnz;
     const double density = total_blocks > 0 ? nnz / total_blocks : 0.0;
     const double run_cov = nnz > 0 ? (double)p->hstats.in_runs / nnz : 0.0;
     const double skew = nnz > 0 ? (double)p->hstats.max_row_nnz / (nnz / (double)nrows) : 0.0;
-    const int64_t max_ws = options ? options->max_workspace_bytes : 0;
-    int forced = (options && options->force_plan_id >= 0) ? options->force_plan_id : get_force_plan();
     int plan_id;
     if (forced >= 0) {
         plan_id = plan_eligible(forced, B_Q, B_KV, N, heads, d, max_ws) ? forced : -1;
@@ -283,7 +368,82 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     p->us_lookup = (float)(t3 - t2);
     p->us_launch_prep = (float)(t4 - t3);
     p->us_total = (float)(t4 - t0);
+    if (cache) {
+        BSA_CUDA(cudaEventCreateWithFlags(&p->ready, cudaEventDisableTiming), "cache event");
+        BSA_CUDA(cudaEventRecord(p->ready, stream), "cache event record");
+        p->refs.store(2, std::memory_order_relaxed);  // the cache and the caller
+        bsa_plan* dropped[2] = {nullptr, nullptr};
+        {
+            std::lock_guard<std::mutex> lock(cache->mu);
+            auto it = cache->index.find(key);
+            if (it != cache->index.end()) {  // another thread prepared the same mask meanwhile: the newer plan stays
+                dropped[0] = it->second->second;
+                cache->lru.erase(it->second);
+                cache->index.erase(it);
+            }
+            cache->lru.emplace_front(key, p);
+            cache->index[key] = cache->lru.begin();
+            if ((int)cache->lru.size() > cache->capacity) {
+                dropped[1] = cache->lru.back().second;
+                cache->index.erase(cache->lru.back().first);
+                cache->lru.pop_back();
+                ++cache->evictions;
+            }
+        }
+        for (bsa_plan* q : dropped)
+            if (q) release_plan(q);
+        if (cache_hit) *cache_hit = 0;
+    }
     *out_plan = p;
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_plan_cache_create(int capacity, bsa_plan_cache_t** out_cache) {
+    if (!out_cache || capacity < 1) return BSA_ERR_INVALID_ARG;
+    bsa_plan_cache* c = new (std::nothrow) bsa_plan_cache();
+    if (!c) return BSA_ERR_OOM;
+    c->capacity = capacity;
+    c->hits = c->misses = c->evictions = 0;
+    *out_cache = c;
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_plan_cache_get(bsa_plan_cache_t* cache, const uint8_t* mask_dev, int64_t row_stride_bytes, int B_Q,
+                                           int B_KV, int64_t N, int heads, int d, const bsa_options_t* options,
+                                           void* stream_v, bsa_plan_t** out_plan, int* out_hit) {
+    if (!cache || row_stride_bytes < 0) return BSA_ERR_INVALID_ARG;
+    int hit = 0;
+    bsa_status_t st = create_impl(mask_dev, row_stride_bytes, B_Q, B_KV, N, heads, d, options, stream_v, out_plan, cache, &hit);
+    if (st == BSA_OK && out_hit) *out_hit = hit;
+    return st;
+}
+
+extern "C" bsa_status_t bsa_plan_cache_stats(bsa_plan_cache_t* cache, int64_t* hits, int64_t* misses, int64_t* evictions,
+                                             int32_t* entries) {
+    if (!cache) return BSA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(cache->mu);
+    if (hits) *hits = cache->hits;
+    if (misses) *misses = cache->misses;
+    if (evictions) *evictions = cache->evictions;
+    if (entries) *entries = (int32_t)cache->lru.size();
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_plan_cache_destroy(bsa_plan_cache_t* cache) {
+    if (!cache) return BSA_ERR_INVALID_ARG;
+    cudaError_t e = cudaSuccess;
+    for (auto& kv : cache->lru) {
+        cudaStream_t s = kv.second->stream;
+        if (release_plan(kv.second)) {
+            cudaError_t e1 = cudaStreamSynchronize(s);
+            if (e == cudaSuccess) e = e1;
+        }
+    }
+    delete cache;
+    if (e != cudaSuccess) {
+        set_cuda_err(e, "cache destroy sync");
+        return BSA_ERR_CUDA;
+    }
     return BSA_OK;
 }
 
@@ -341,7 +501,7 @@ extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const vo
 extern "C" bsa_status_t bsa_plan_destroy(bsa_plan_t* p) {
     if (!p) return BSA_ERR_INVALID_ARG;
     cudaStream_t s = p->stream;
-    free_plan(p);
+    if (!release_plan(p)) return BSA_OK;  // a plan cache (or another request that got it from there) still holds it
     cudaError_t e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
         set_cuda_err(e, "destroy sync");
@@ -548,8 +708,14 @@ extern "C" int bsa_plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int 
 }
 extern "C" int bsa_base_plan(int B_Q, int B_KV, int d) { return base_plan(B_Q, B_KV, d); }
 extern "C" uint64_t bsa_catalog_hash(void) { return catalog_hash(); }
-extern "C" bsa_status_t bsa_lut_load(const char* path) { return lut_load(path); }
-extern "C" void bsa_lut_clear(void) { lut_clear(); }
+extern "C" bsa_status_t bsa_lut_load(const char* path) {
+    g_select_generation.fetch_add(1, std::memory_order_relaxed);
+    return lut_load(path);
+}
+extern "C" void bsa_lut_clear(void) {
+    g_select_generation.fetch_add(1, std::memory_order_relaxed);
+    lut_clear();
+}
 extern "C" int bsa_lut_num_regimes(void) { return lut_num_regimes(); }
 extern "C" int bsa_lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_coverage,
                               double skew, int64_t max_ws, int* hit_out) {
@@ -558,7 +724,10 @@ extern "C" int bsa_lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, do
 extern "C" void bsa_lut_buckets(int64_t N, double density, double skew, double run_coverage, int32_t out[4]) {
     lut_buckets(N, density, skew, run_coverage, out);
 }
-extern "C" void bsa_force_plan(int plan_id) { set_force_plan(plan_id); }
+extern "C" void bsa_force_plan(int plan_id) {
+    g_select_generation.fetch_add(1, std::memory_order_relaxed);
+    set_force_plan(plan_id);
+}
 
 extern "C" const char* bsa_status_string(bsa_status_t s) {
     switch (s) {

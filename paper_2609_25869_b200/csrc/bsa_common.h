@@ -36,11 +36,13 @@ struct MaskStatsDev {
     unsigned long long in_runs;
     unsigned int max_row_nnz;
     unsigned int blocks_done;  // CTAs of the statistics kernel that have added their share (starts at zero)
+    unsigned long long hash[2];  // 128-bit fingerprint of the activity pattern (only when asked for, else 0)
 };
 // The statistics as the kernel's last CTA posts them into pinned host memory; `seq` is written last.
 struct MaskStatsHost {
     unsigned long long nnz;
     unsigned long long in_runs;
+    unsigned long long hash[2];
     unsigned int max_row_nnz;
     unsigned int seq;
 };
@@ -66,13 +68,15 @@ struct MapGeom {
 };
 
 // ---- planner entry points (bsa_planner.cu); all launch on `stream`, none synchronises -------
-// `post` (may be null): pinned host memory the last CTA writes the totals to, tagged with `seq`
+// `post` (may be null): pinned host memory the last CTA writes the totals to, tagged with `seq`.
+// `with_hash`: also accumulate the 128-bit fingerprint of the activity pattern (the plan cache's key).
 cudaError_t launch_mask_row_stats(const uint8_t* mask, int nrows, int nKb, int32_t* row_nnz, MaskStatsDev* stats,
-                                  cudaStream_t stream, MaskStatsHost* post = nullptr, unsigned seq = 0);
+                                  cudaStream_t stream, MaskStatsHost* post = nullptr, unsigned seq = 0,
+                                  bool with_hash = false);
 cudaError_t launch_row_scan(const int32_t* row_nnz, int nrows, int32_t* row_ptr, cudaStream_t stream);
 cudaError_t launch_mask_row_stats_packed(const uint32_t* mask, long long stride_words, int nrows, int nKb,
                                          int32_t* row_nnz, MaskStatsDev* stats, cudaStream_t stream,
-                                         MaskStatsHost* post = nullptr, unsigned seq = 0);
+                                         MaskStatsHost* post = nullptr, unsigned seq = 0, bool with_hash = false);
 cudaError_t launch_csr_fill_packed(const uint32_t* mask, long long stride_words, int nrows, int nKb,
                                    const int32_t* row_ptr, int32_t* col_idx, cudaStream_t stream);
 cudaError_t launch_csr_fill(const uint8_t* mask, int nrows, int nKb, const int32_t* row_ptr, int32_t* col_idx,

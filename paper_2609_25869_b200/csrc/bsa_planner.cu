@@ -52,15 +52,51 @@ __device__ __forceinline__ void post_stats_if_last(MaskStatsDev* stats, MaskStat
     __threadfence();
     post->nnz = atomicAdd(&stats->nnz, 0ull);
     post->in_runs = atomicAdd(&stats->in_runs, 0ull);
+    post->hash[0] = atomicAdd(&stats->hash[0], 0ull);
+    post->hash[1] = atomicAdd(&stats->hash[1], 0ull);
     post->max_row_nnz = atomicMax(&stats->max_row_nnz, 0u);
     __threadfence_system();
     *reinterpret_cast<volatile unsigned*>(&post->seq) = seq;
 }
 
+// Fingerprint of the activity pattern, for the plan cache: every non-empty word of a row (its activity bits `m`, at
+// word position `pos` of row `row`) is mixed with its position by two different 64-bit finalisers, and the two
+// results are summed over the mask modulo 2^64 (a sum, so that warps and CTAs can add their shares in any order).
+__device__ __forceinline__ unsigned long long mix64(unsigned long long x, unsigned long long c1, unsigned long long c2) {
+    x ^= x >> 33;
+    x *= c1;
+    x ^= x >> 29;
+    x *= c2;
+    x ^= x >> 32;
+    return x;
+}
+struct MaskHash {
+    unsigned long long a = 0, b = 0;
+    __device__ __forceinline__ void add(unsigned m, int row, long long pos) {
+        if (!m) return;
+        const unsigned long long where = ((unsigned long long)(unsigned)row << 32) | (unsigned long long)(unsigned)pos;
+        const unsigned long long x = where * 0x9E3779B97F4A7C15ull + (unsigned long long)m * 0xC2B2AE3D27D4EB4Full + 1ull;
+        a += mix64(x, 0xFF51AFD7ED558CCDull, 0xC4CEB9FE1A85EC53ull);
+        b += mix64(x ^ 0x5851F42D4C957F2Dull, 0xBF58476D1CE4E5B9ull, 0x94D049BB133111EBull);
+    }
+    // adds the warp's total to the two global sums
+    __device__ __forceinline__ void flush(MaskStatsDev* stats, int lane) {
+        for (int o = 16; o > 0; o >>= 1) {
+            a += __shfl_down_sync(kFull, a, o);
+            b += __shfl_down_sync(kFull, b, o);
+        }
+        if (lane == 0 && (a | b)) {
+            atomicAdd(&stats->hash[0], a);
+            atomicAdd(&stats->hash[1], b);
+        }
+    }
+};
+
 // ------------------------------------------------------------------------------------------
 // mask_row_stats: one warp per (head, query-block) row.
 // A block counts towards run coverage iff its left or right neighbour in the same row is active.
 // ------------------------------------------------------------------------------------------
+template <bool HASH>
 __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __restrict__ mask, int nrows, int nKb,
                                                               int32_t* __restrict__ row_nnz, MaskStatsDev* stats,
                                                               MaskStatsHost* post, unsigned seq) {
@@ -79,8 +115,10 @@ __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __re
         // step later, by lane 0, once that neighbour (bit 0 of the next step) is known.
         unsigned carry = 0;  // bits 1:0 = the previous step's last two bytes (bit 1 = the last one)
         unsigned m_next = row_word_bits(words, w0 + lane, rb, re);
+        MaskHash hash;
         for (long long w = w0; w < w1; w += 32) {
             const unsigned m = m_next;
+            if (HASH) hash.add(m, row, w - w0 + lane);
             m_next = (w + 32 < w1) ? row_word_bits(words, w + 32 + lane, rb, re) : 0u;
             // neighbours across lanes: previous lane's bit 15, next lane's bit 0
             unsigned prev15 = __shfl_up_sync(kFull, m >> 15, 1);
@@ -98,6 +136,7 @@ __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __re
             runs += __shfl_down_sync(kFull, runs, o);
         }
         if (lane == 0) row_nnz[row] = (int32_t)nnz;
+        if (HASH) hash.flush(stats, lane);
     }
     if (lane == 0) {
         s_nnz[warp] = nnz;
@@ -135,6 +174,7 @@ __device__ __forceinline__ unsigned packed_row_word(const uint32_t* __restrict__
     return m;
 }
 
+template <bool HASH>
 __global__ void __launch_bounds__(256) mask_row_stats_packed_kernel(const uint32_t* __restrict__ mask, long long stride_words,
                                                                      int nrows, int nKb, int32_t* __restrict__ row_nnz,
                                                                      MaskStatsDev* stats, MaskStatsHost* post, unsigned seq) {
@@ -147,8 +187,10 @@ __global__ void __launch_bounds__(256) mask_row_stats_packed_kernel(const uint32
         const int nwords = (nKb + 31) >> 5;
         unsigned carry = 0;  // bits 1:0 = the previous step's last two blocks (bit 1 = the last one)
         unsigned m_next = packed_row_word(r, lane, nwords, nKb);
+        MaskHash hash;
         for (int w = 0; w < nwords; w += 32) {
             const unsigned m = m_next;
+            if (HASH) hash.add(m, row, w + lane);
             m_next = (w + 32 < nwords) ? packed_row_word(r, w + 32 + lane, nwords, nKb) : 0u;
             unsigned prev31 = __shfl_up_sync(kFull, m >> 31, 1);
             unsigned next0 = __shfl_down_sync(kFull, m & 1u, 1);
@@ -165,6 +207,7 @@ __global__ void __launch_bounds__(256) mask_row_stats_packed_kernel(const uint32
             runs += __shfl_down_sync(kFull, runs, o);
         }
         if (lane == 0) row_nnz[row] = (int32_t)nnz;
+        if (HASH) hash.flush(stats, lane);
     }
     if (lane == 0) {
         s_nnz[warp] = nnz;
@@ -678,17 +721,24 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
 }  // namespace
 
 cudaError_t launch_mask_row_stats(const uint8_t* mask, int nrows, int nKb, int32_t* row_nnz, MaskStatsDev* stats,
-                                  cudaStream_t stream, MaskStatsHost* post, unsigned seq) {
-    mask_row_stats_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, nrows, nKb, row_nnz, stats, post, seq);
+                                  cudaStream_t stream, MaskStatsHost* post, unsigned seq, bool with_hash) {
+    if (with_hash)
+        mask_row_stats_kernel<true><<<(nrows + 7) / 8, 256, 0, stream>>>(mask, nrows, nKb, row_nnz, stats, post, seq);
+    else
+        mask_row_stats_kernel<false><<<(nrows + 7) / 8, 256, 0, stream>>>(mask, nrows, nKb, row_nnz, stats, post, seq);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_mask_row_stats_packed(const uint32_t* mask, long long stride_words, int nrows, int nKb,
                                          int32_t* row_nnz, MaskStatsDev* stats, cudaStream_t stream, MaskStatsHost* post,
-                                         unsigned seq) {
-    mask_row_stats_packed_kernel<<<(nrows + 7) / 8, 256, 0, stream>>>(mask, stride_words, nrows, nKb, row_nnz, stats, post,
-                                                                        seq);
+                                         unsigned seq, bool with_hash) {
+    if (with_hash)
+        mask_row_stats_packed_kernel<true>
+            <<<(nrows + 7) / 8, 256, 0, stream>>>(mask, stride_words, nrows, nKb, row_nnz, stats, post, seq);
+    else
+        mask_row_stats_packed_kernel<false>
+            <<<(nrows + 7) / 8, 256, 0, stream>>>(mask, stride_words, nrows, nKb, row_nnz, stats, post, seq);
     count_launch();
     return cudaGetLastError();
 }

@@ -280,6 +280,121 @@ def test_bit_packed_mask_gives_the_same_plan_and_output(B_Q, B_KV, N, d, plan_id
         assert torch.equal(Oa, Ob) and torch.equal(La, Lb)
 
 
+def test_plan_cache_reuses_the_plan_of_a_repeated_mask():
+    """Warm path: the second request with the same mask gets the SAME prepared plan (one statistics kernel and one
+    row scan launched, nothing else), its output matches the oracle and an uncached plan bit for bit; any change of
+    the activity pattern (one block more, one block moved along its row, two rows exchanged) misses."""
+    req = I.config_tiny()
+    mask, q, k, v, qkv_cpu = Hh.to_dev(req)
+    cache = bsa.PlanCache(capacity=8)
+    args = (req.B_Q, req.B_KV, req.N, req.H, req.d)
+    p0, hit0 = cache.get(mask, *args)
+    n0 = bsa.kernel_launch_count()
+    p1, hit1 = cache.get(mask.clone(), *args)       # another buffer, the same pattern
+    n1 = bsa.kernel_launch_count()
+    assert (hit0, hit1) == (False, True) and p0._h.value == p1._h.value
+    assert n1 - n0 == 2
+    O1, L1 = p1.forward(q, k, v)
+    torch.cuda.synchronize()
+    Hh.compare_with_oracle(req, O1, L1, qkv_cpu)
+    Hh.check_plan_structure(req, p1)
+    with bsa.plan_create(mask, *args) as fresh:
+        O2, L2 = fresh.forward(q, k, v)
+        torch.cuda.synchronize()
+        assert torch.equal(O1, O2) and torch.equal(L1, L2)
+    # a mask given as other non-zero byte values is the same activity pattern
+    p2, hit2 = cache.get(mask * 7, *args)
+    assert hit2 and p2._h.value == p0._h.value
+    # changed patterns
+    M = req.mask.copy()
+    h, r = 1, 3
+    c_off = int(np.flatnonzero(M[h, r] == 0)[0])
+    c_on = int(np.flatnonzero(M[h, r])[0])
+    more = M.copy(); more[h, r, c_off] = 1
+    moved = more.copy(); moved[h, r, c_on] = 0          # same count as M, one block at another column
+    swapped = M.copy(); swapped[h, [r, r + 1]] = swapped[h, [r + 1, r]]
+    assert not np.array_equal(swapped, M)
+    for variant in (more, moved, swapped):
+        pv, hitv = cache.get(torch.from_numpy(variant).cuda(), *args)
+        assert not hitv and pv._h.value != p0._h.value
+        rv = I.Request("variant", req.H, req.N, req.d, req.B_Q, req.B_KV, variant, qkv_seed=req.qkv_seed)
+        Hh.check_plan_structure(rv, pv)
+        Ov, Lv = pv.forward(q, k, v)
+        torch.cuda.synchronize()
+        Hh.compare_with_oracle(rv, Ov, Lv, qkv_cpu)
+        pv.destroy()
+    # the request key is part of the cache key: another forced plan, or the bit-packed form, is prepared anew
+    p3, hit3 = cache.get(mask, *args, plan_id=2)
+    bits, stride = bsa.pack_mask(mask)
+    p4, hit4 = cache.get(bits, *args, row_stride=stride)
+    p5, hit5 = cache.get(bits.clone(), *args, row_stride=stride)
+    assert not hit3 and not hit4 and hit5 and p4._h.value == p5._h.value
+    O4, L4 = p5.forward(q, k, v)
+    torch.cuda.synchronize()
+    assert torch.equal(O4, O1) and torch.equal(L4, L1)
+    st = cache.stats()
+    assert st == {"hits": 3, "misses": 6, "evictions": 0, "entries": 6}
+    for p in (p0, p1, p2, p3, p4, p5):
+        p.destroy()
+    cache.destroy()
+
+
+def test_plan_cache_evicts_the_least_recently_used_plan_and_plans_outlive_it():
+    req = I.config_tiny()
+    _, q, k, v, qkv_cpu = Hh.to_dev(req)
+    args = (req.B_Q, req.B_KV, req.N, req.H, req.d)
+    masks = []
+    for s in range(3):
+        masks.append(I.random_mask(100 + s, req.H, req.nQb, req.nKb, 0.25))
+    dev = [torch.from_numpy(m).cuda() for m in masks]
+    cache = bsa.PlanCache(capacity=2)
+    pa, _ = cache.get(dev[0], *args)
+    pb, _ = cache.get(dev[1], *args)
+    pa2, hit = cache.get(dev[0], *args)            # 0 becomes the most recent
+    assert hit
+    pc, _ = cache.get(dev[2], *args)               # evicts 1
+    assert cache.stats()["evictions"] == 1 and cache.stats()["entries"] == 2
+    _, hit_b = cache.get(dev[1], *args)            # prepared again, evicts 0
+    _, hit_a = cache.get(dev[0], *args)
+    assert not hit_b and not hit_a
+    # pb was evicted while held: it is still a complete plan
+    rb = I.Request("evicted", req.H, req.N, req.d, req.B_Q, req.B_KV, masks[1], qkv_seed=req.qkv_seed)
+    Ob, Lb = pb.forward(q, k, v)
+    torch.cuda.synchronize()
+    Hh.compare_with_oracle(rb, Ob, Lb, qkv_cpu)
+    # plans outlive the cache itself
+    cache.destroy()
+    ra = I.Request("kept", req.H, req.N, req.d, req.B_Q, req.B_KV, masks[0], qkv_seed=req.qkv_seed)
+    Oa, La = pa.forward(q, k, v)
+    torch.cuda.synchronize()
+    Hh.compare_with_oracle(ra, Oa, La, qkv_cpu)
+    for p in (pa, pa2, pb, pc):
+        p.destroy()
+
+
+def test_plan_cache_hit_on_another_stream_waits_for_the_preparation():
+    req = I.config_mid()
+    mask, q, k, v, _ = Hh.to_dev(req)
+    args = (req.B_Q, req.B_KV, req.N, req.H, req.d)
+    cache = bsa.PlanCache(capacity=2)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    p0, _ = cache.get(mask, *args, stream=s1)
+    p1, hit = cache.get(mask, *args, stream=s2)    # the preparation on s1 may still be running
+    assert hit
+    with torch.cuda.stream(s2):
+        O1 = torch.empty_like(q)
+        L1 = torch.empty(q.shape[:2], dtype=torch.float32, device="cuda")
+        p1.forward(q, k, v, O1, L1, stream=s2)
+    torch.cuda.synchronize()
+    with bsa.plan_create(mask, *args) as fresh:
+        O2, L2 = fresh.forward(q, k, v)
+        torch.cuda.synchronize()
+    assert torch.equal(O1, O2) and torch.equal(L1, L2)
+    p0.destroy(); p1.destroy()
+    cache.destroy()
+
+
 def test_launch_counter_counts_our_kernels():
     req = I.config_tiny()
     mask, q, k, v, _ = Hh.to_dev(req)

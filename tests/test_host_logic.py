@@ -203,3 +203,27 @@ def test_packed_create_rejects_bad_layouts_without_a_gpu():
     assert L.bsa_plan_create_packed(fake, 4, 16, 16, 1024, 1, 128, None, None, ctypes.byref(h)) == 1     # 64 blocks > 32 bits
     assert L.bsa_plan_create_packed(ctypes.c_void_p(0x1002), 8, 16, 16, 1024, 1, 128, None, None, ctypes.byref(h)) == 1
     assert L.bsa_plan_create_packed(None, 8, 16, 16, 1024, 1, 128, None, None, ctypes.byref(h)) == 1
+
+
+def test_plan_cache_host_calls_without_a_gpu():
+    """The cache itself is host state: it is created, read and destroyed without a device, and bad arguments are
+    refused before anything touches one."""
+    L = bsa.lib()
+    c = ctypes.c_void_p()
+    assert L.bsa_plan_cache_create(0, ctypes.byref(c)) == 1
+    assert L.bsa_plan_cache_create(4, None) == 1
+    assert L.bsa_plan_cache_create(4, ctypes.byref(c)) == 0 and c.value
+    hits, misses, ev = ctypes.c_int64(-1), ctypes.c_int64(-1), ctypes.c_int64(-1)
+    n = ctypes.c_int32(-1)
+    assert L.bsa_plan_cache_stats(c, ctypes.byref(hits), ctypes.byref(misses), ctypes.byref(ev), ctypes.byref(n)) == 0
+    assert (hits.value, misses.value, ev.value, n.value) == (0, 0, 0, 0)
+    h = ctypes.c_void_p()
+    fake = ctypes.c_void_p(0x1000)  # never dereferenced: the checks come first
+    assert L.bsa_plan_cache_get(None, fake, 0, 128, 128, 1024, 1, 128, None, None, ctypes.byref(h), None) == 1
+    assert L.bsa_plan_cache_get(c, fake, -4, 128, 128, 1024, 1, 128, None, None, ctypes.byref(h), None) == 1
+    assert L.bsa_plan_cache_get(c, None, 0, 128, 128, 1024, 1, 128, None, None, ctypes.byref(h), None) == 1
+    assert L.bsa_plan_cache_get(c, fake, 6, 128, 128, 1024, 1, 128, None, None, ctypes.byref(h), None) == 1   # stride % 4
+    assert L.bsa_plan_cache_get(c, fake, 0, 128, 128, 1024, 1, 96, None, None, ctypes.byref(h), None) == 2    # d unsupported
+    assert L.bsa_plan_cache_stats(None, None, None, None, None) == 1
+    assert L.bsa_plan_cache_destroy(c) == 0
+    assert L.bsa_plan_cache_destroy(None) == 1
