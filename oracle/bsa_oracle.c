@@ -20,6 +20,9 @@
  *  - N need not be a multiple of the block sizes: the last block is ragged and
  *    keys >= N do not exist.
  *
+ * Section 2.1 gives Q as N_q x d and K, V as N_kv x d: the number of query
+ * tokens (N) and of key tokens (N_kv) are separate arguments.
+ *
  * Inputs are bf16 bit patterns (the same rounded values the GPU sees),
  * widened exactly to double.
  */
@@ -48,18 +51,18 @@ int bsa_oracle_num_threads(void) {
 
 /*
  * Evaluate n_sel query blocks.  Selected block s is (sel_head[s], sel_qblock[s]);
- * its rows are tokens sel_qblock[s]*B_Q ... (+B_Q-1), clipped to N.
+ * its rows are tokens sel_qblock[s]*B_Q ... (+B_Q-1), clipped to N; keys are tokens 0 ... N_kv-1.
  * row_step > 1 evaluates only every row_step-th row of each block (rows are
  * independent; used to bound oracle time on very dense requests); rows not
  * evaluated are left untouched in the outputs.
  *
  * mask : uint8 [H][nQb][nKb], nonzero = active
- * Q,K,V: bf16 bits [H][N][d]
+ * Q    : bf16 bits [H][N][d]        K,V: bf16 bits [H][N_kv][d]
  * O    : double [n_sel][B_Q][d]     LSE: double [n_sel][B_Q]
  * pairs_out (optional): number of active token pairs evaluated.
  * Returns 0, or -1 on allocation failure.
  */
-int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int B_KV, int64_t N, int d,
+int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int B_KV, int64_t N, int64_t N_kv, int d,
                       const uint16_t* Q, const uint16_t* K, const uint16_t* V,
                       int n_sel, const int32_t* sel_head, const int32_t* sel_qblock, int row_step,
                       double* O, double* LSE, int64_t* pairs_out) {
@@ -70,7 +73,7 @@ int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int
     if (row_step < 1) row_step = 1;
 #pragma omp parallel reduction(+ : pairs_total)
     {
-        double* s = (double*)malloc(sizeof(double) * (size_t)(N > 0 ? N : 1));
+        double* s = (double*)malloc(sizeof(double) * (size_t)(N_kv > 0 ? N_kv : 1));
         double* q = (double*)malloc(sizeof(double) * (size_t)d);
         double* acc = (double*)malloc(sizeof(double) * (size_t)d);
         if (!s || !q || !acc) {
@@ -82,8 +85,8 @@ int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int
                 const int h = sel_head[sidx];
                 const int bi = sel_qblock[sidx];
                 const uint8_t* mrow = mask + ((size_t)h * nQb + bi) * nKb;
-                const uint16_t* Kh = K + (size_t)h * N * d;
-                const uint16_t* Vh = V + (size_t)h * N * d;
+                const uint16_t* Kh = K + (size_t)h * N_kv * d;
+                const uint16_t* Vh = V + (size_t)h * N_kv * d;
                 for (int r = 0; r < B_Q; r += row_step) {
                     const int64_t i = (int64_t)bi * B_Q + r;
                     if (i >= N) break;
@@ -96,7 +99,7 @@ int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int
                     for (int bj = 0; bj < nKb; ++bj) {
                         if (!mrow[bj]) continue;
                         int64_t j0 = (int64_t)bj * B_KV, j1 = j0 + B_KV;
-                        if (j1 > N) j1 = N;
+                        if (j1 > N_kv) j1 = N_kv;
                         for (int64_t j = j0; j < j1; ++j) {
                             const uint16_t* kj = Kh + (size_t)j * d;
                             double dot = 0.0;
@@ -118,7 +121,7 @@ int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int
                     for (int bj = 0; bj < nKb; ++bj) {
                         if (!mrow[bj]) continue;
                         int64_t j0 = (int64_t)bj * B_KV, j1 = j0 + B_KV;
-                        if (j1 > N) j1 = N;
+                        if (j1 > N_kv) j1 = N_kv;
                         for (int64_t j = j0; j < j1; ++j) {
                             const double p = exp(s[j] - m);
                             l += p;

@@ -68,7 +68,7 @@ def _load():
         lib.bsa_oracle_blocks.restype = ctypes.c_int
         lib.bsa_oracle_blocks.argtypes = [
             ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
-            ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
+            ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
             ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         lib.bsa_oracle_num_threads.restype = ctypes.c_int
         _lib = lib
@@ -88,26 +88,28 @@ def cdiv(a: int, b: int) -> int:
 # --------------------------------------------------------------------------
 def attention_blocks(mask: np.ndarray, B_Q: int, B_KV: int, N: int, d: int,
                      Qb: np.ndarray, Kb: np.ndarray, Vb: np.ndarray,
-                     sel: Sequence[Tuple[int, int]], row_step: int = 1):
+                     sel: Sequence[Tuple[int, int]], row_step: int = 1, N_kv: Optional[int] = None):
     """Masked attention (Eq. 1) on selected (head, query-block) pairs.
 
-    ``Qb/Kb/Vb`` are uint16 bf16 bit patterns ``[H, N, d]``.  Returns
+    ``Qb`` is ``[H, N, d]`` and ``Kb/Vb`` are ``[H, N_kv, d]`` uint16 bf16 bit patterns (Section 2.1: N_q query
+    and N_kv key tokens; ``N_kv`` defaults to ``N``).  Returns
     ``(O [n_sel, B_Q, d] float64, LSE [n_sel, B_Q] float64, active_pairs)``;
     rows at or beyond N, and rows skipped by ``row_step``, are NaN.
     """
     lib = _load()
     mask = np.ascontiguousarray(mask, dtype=np.uint8)
     H, nQb, nKb = mask.shape
-    assert nQb == cdiv(N, B_Q) and nKb == cdiv(N, B_KV)
-    for a in (Qb, Kb, Vb):
-        assert a.dtype == np.uint16 and a.shape == (H, N, d) and a.flags.c_contiguous
+    N_kv = N if N_kv is None else N_kv
+    assert nQb == cdiv(N, B_Q) and nKb == cdiv(N_kv, B_KV)
+    for a, n_tok in ((Qb, N), (Kb, N_kv), (Vb, N_kv)):
+        assert a.dtype == np.uint16 and a.shape == (H, n_tok, d) and a.flags.c_contiguous
     sel_h = np.ascontiguousarray([s[0] for s in sel], dtype=np.int32)
     sel_b = np.ascontiguousarray([s[1] for s in sel], dtype=np.int32)
     n = len(sel_h)
     O = np.full((n, B_Q, d), np.nan, dtype=np.float64)
     LSE = np.full((n, B_Q), np.nan, dtype=np.float64)
     pairs = ctypes.c_int64(0)
-    rc = lib.bsa_oracle_blocks(mask.ctypes.data, H, nQb, nKb, B_Q, B_KV, N, d, Qb.ctypes.data, Kb.ctypes.data,
+    rc = lib.bsa_oracle_blocks(mask.ctypes.data, H, nQb, nKb, B_Q, B_KV, N, N_kv, d, Qb.ctypes.data, Kb.ctypes.data,
                                Vb.ctypes.data, n, sel_h.ctypes.data, sel_b.ctypes.data, row_step,
                                O.ctypes.data, LSE.ctypes.data, ctypes.byref(pairs))
     if rc != 0:
@@ -115,11 +117,11 @@ def attention_blocks(mask: np.ndarray, B_Q: int, B_KV: int, N: int, d: int,
     return O, LSE, int(pairs.value)
 
 
-def attention_full(mask, B_Q, B_KV, N, d, Qb, Kb, Vb):
+def attention_full(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, N_kv=None):
     """Eq. 1 on every row.  Returns ``O [H, N, d]`` and ``LSE [H, N]`` (float64)."""
     H, nQb, _ = mask.shape
     sel = [(h, i) for h in range(H) for i in range(nQb)]
-    O, LSE, pairs = attention_blocks(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, sel)
+    O, LSE, pairs = attention_blocks(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, sel, N_kv=N_kv)
     O = O.reshape(H, nQb * B_Q, d)[:, :N]
     LSE = LSE.reshape(H, nQb * B_Q)[:, :N]
     return np.ascontiguousarray(O), np.ascontiguousarray(LSE), pairs
@@ -129,19 +131,19 @@ def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
     return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
-def expand_mask(mask_h: np.ndarray, B_Q: int, B_KV: int, N: int) -> np.ndarray:
-    """E(M) of one head as an explicit ``[N, N]`` boolean matrix (Section 2.1)."""
-    return np.repeat(np.repeat(mask_h != 0, B_Q, axis=0), B_KV, axis=1)[:N, :N]
+def expand_mask(mask_h: np.ndarray, B_Q: int, B_KV: int, N: int, N_kv=None) -> np.ndarray:
+    """E(M) of one head as an explicit ``[N, N_kv]`` boolean matrix (Section 2.1)."""
+    return np.repeat(np.repeat(mask_h != 0, B_Q, axis=0), B_KV, axis=1)[:N, :(N if N_kv is None else N_kv)]
 
 
-def attention_bruteforce(mask, B_Q, B_KV, N, d, Qb, Kb, Vb):
+def attention_bruteforce(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, N_kv=None):
     """Eq. 1 through an explicit token-pair matrix, one row at a time (tiny inputs)."""
     H = mask.shape[0]
     Q, K, V = (bf16_bits_to_f64(x) for x in (Qb, Kb, Vb))
     O = np.zeros((H, N, d))
     LSE = np.full((H, N), -np.inf)
     for h in range(H):
-        E = expand_mask(mask[h], B_Q, B_KV, N)
+        E = expand_mask(mask[h], B_Q, B_KV, N, N_kv)
         for i in range(N):
             J = np.nonzero(E[i])[0]
             if J.size == 0:
@@ -158,11 +160,11 @@ def attention_bruteforce(mask, B_Q, B_KV, N, d, Qb, Kb, Vb):
 # --------------------------------------------------------------------------
 # Section 2.3 accounting
 # --------------------------------------------------------------------------
-def active_pairs(mask: np.ndarray, B_Q: int, B_KV: int, N: int) -> int:
+def active_pairs(mask: np.ndarray, B_Q: int, B_KV: int, N: int, N_kv=None) -> int:
     """Number of in-range token pairs in E(M), all heads."""
     H, nQb, nKb = mask.shape
     rq = np.minimum(B_Q, N - np.arange(nQb) * B_Q).astype(np.int64)
-    ck = np.minimum(B_KV, N - np.arange(nKb) * B_KV).astype(np.int64)
+    ck = np.minimum(B_KV, (N if N_kv is None else N_kv) - np.arange(nKb) * B_KV).astype(np.int64)
     return int(((mask != 0).astype(np.int64) * rq[None, :, None] * ck[None, None, :]).sum())
 
 

@@ -40,6 +40,41 @@ def test_all_ones_mask_is_dense_softmax_attention():
     np.testing.assert_allclose(LSE, ref_L.numpy(), rtol=0, atol=1e-12)
 
 
+def test_dense_softmax_with_more_keys_than_queries_and_fewer():
+    """Section 2.1: Q is N_q x d, K and V are N_kv x d.  With every block active the result is the textbook
+    softmax(Q K^T / sqrt(d)) V of the rectangular score matrix (ragged last blocks on both sides)."""
+    H, d, B_Q, B_KV = 2, 32, 32, 64
+    for N_q, N_kv in ((70, 200), (200, 70)):
+        q, _, _ = I.make_qkv(21, H, N_q, d)
+        _, k, v = I.make_qkv(22, H, N_kv, d)
+        M = np.ones((H, I.cdiv(N_q, B_Q), I.cdiv(N_kv, B_KV)), dtype=np.uint8)
+        O, LSE, pairs = oracle.attention_full(M, B_Q, B_KV, N_q, d, I.bf16_bits(q), I.bf16_bits(k), I.bf16_bits(v),
+                                              N_kv=N_kv)
+        q64, k64, v64 = (t.to(torch.float64) for t in (q, k, v))
+        s = q64 @ k64.transpose(1, 2) / math.sqrt(d)
+        assert pairs == H * N_q * N_kv == oracle.active_pairs(M, B_Q, B_KV, N_q, N_kv)
+        assert O.shape == (H, N_q, d)
+        np.testing.assert_allclose(O, (torch.softmax(s, dim=-1) @ v64).numpy(), rtol=0, atol=1e-12)
+        np.testing.assert_allclose(LSE, torch.logsumexp(s, dim=-1).numpy(), rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("B_Q,B_KV,N_q,N_kv", [(16, 32, 50, 130), (64, 16, 130, 40)])
+def test_bruteforce_token_pair_matrix_rectangular(B_Q, B_KV, N_q, N_kv):
+    H, d = 2, 16
+    q, _, _ = I.make_qkv(31, H, N_q, d)
+    _, k, v = I.make_qkv(32, H, N_kv, d)
+    Qb, Kb, Vb = I.bf16_bits(q), I.bf16_bits(k), I.bf16_bits(v)
+    M = I.random_mask(9, H, I.cdiv(N_q, B_Q), I.cdiv(N_kv, B_KV), 0.4, empty_rows=0.2)
+    O, LSE, pairs = oracle.attention_full(M, B_Q, B_KV, N_q, d, Qb, Kb, Vb, N_kv=N_kv)
+    bO, bL = oracle.attention_bruteforce(M, B_Q, B_KV, N_q, d, Qb, Kb, Vb, N_kv=N_kv)
+    np.testing.assert_allclose(O, bO, rtol=0, atol=1e-13)
+    assert np.array_equal(np.isneginf(LSE), np.isneginf(bL))
+    fin = np.isfinite(bL)
+    np.testing.assert_allclose(LSE[fin], bL[fin], rtol=0, atol=1e-13)
+    E = sum(int(oracle.expand_mask(M[h], B_Q, B_KV, N_q, N_kv).sum()) for h in range(H))
+    assert pairs == E == oracle.active_pairs(M, B_Q, B_KV, N_q, N_kv)
+
+
 def test_hand_computed_two_keys():
     # d = 4, one query q = (2,0,0,0), keys k0 = (2,0,0,0), k1 = (-2,0,0,0): scores 4/2 = 2 and -2.
     N, d = 2, 4
