@@ -70,6 +70,9 @@ typedef struct bsa_options {
                                      eligibility); -1: Algorithm 2                                   */
     int32_t reserved0;
     int64_t max_workspace_bytes;  /* Split-K workspace the request may bind; <= 0: library default   */
+    int64_t N_kv;                 /* key/value tokens per head (Section 2.1: K, V are N_kv x d); <= 0: N_kv = N.
+                                     The mask then has ceil(N_kv / B_KV) block columns, K and V are
+                                     [heads, N_kv, d]; Q, O and LSE keep N rows.                      */
 } bsa_options_t;
 
 /* Scalar mask statistics s_A(M) (Section 5.1) and what launch preparation produced. */
@@ -99,6 +102,7 @@ typedef struct bsa_plan_info {
     float us_launch_prep;         /* CSR fill, tile mapping, task organisation (launch + allocs)    */
     float us_total;
     int32_t device_status;        /* 0, or BSA_ERR_DEVICE_TIMEOUT if any forward hit a bounded wait  */
+    int64_t N_kv;                 /* key/value tokens per head (= N unless the options said otherwise) */
 } bsa_plan_info_t;
 
 /* ---------------------------------------------------------------------------------------------

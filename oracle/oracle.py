@@ -239,7 +239,7 @@ def refine_columns(c: int, ratio: int) -> List[int]:
 # plan coverage: does a set of physical tiles preserve E(M)?
 # --------------------------------------------------------------------------
 def coverage_counts(H: int, N: int, B_Q: int, B_KV: int, T_Q: int, T_KV: int,
-                    tiles: Dict[int, Tuple[np.ndarray, np.ndarray, np.ndarray]]) -> np.ndarray:
+                    tiles: Dict[int, Tuple[np.ndarray, np.ndarray, np.ndarray]], N_kv=None) -> np.ndarray:
     """Count how many tiles cover each cell, honouring membership bits.
 
     A cell is ``min(B_Q,T_Q) x min(B_KV,T_KV)`` tokens; every block and every
@@ -248,11 +248,11 @@ def coverage_counts(H: int, N: int, B_Q: int, B_KV: int, T_Q: int, T_KV: int,
     with tile_row_ptr relative to that head's arrays.  Membership bit
     ``a * sK + b`` (``sQ = max(1, T_Q // B_Q)``, ``sK = max(1, T_KV // B_KV)``,
     ``a < sQ``, ``b < sK``) says logical sub-block (a, b) of the tile is active;
-    bits of sub-blocks that start at or beyond N must be clear.
+    bits of sub-blocks that start at or beyond N (rows) or N_kv (columns, default N) must be clear.
     Returns int32 ``[H, nCq, nCk]``.
     """
     cq, ck = min(B_Q, T_Q), min(B_KV, T_KV)
-    nCq, nCk = cdiv(N, cq), cdiv(N, ck)
+    nCq, nCk = cdiv(N, cq), cdiv(N if N_kv is None else N_kv, ck)
     sQ, sK = max(1, T_Q // B_Q), max(1, T_KV // B_KV)
     cells_q, cells_k = T_Q // cq, T_KV // ck  # cells per tile edge
     cover = np.zeros((H, nCq, nCk), dtype=np.int32)
@@ -277,10 +277,10 @@ def coverage_counts(H: int, N: int, B_Q: int, B_KV: int, T_Q: int, T_KV: int,
     return cover
 
 
-def expected_cell_cover(mask: np.ndarray, N: int, B_Q: int, B_KV: int, T_Q: int, T_KV: int) -> np.ndarray:
+def expected_cell_cover(mask: np.ndarray, N: int, B_Q: int, B_KV: int, T_Q: int, T_KV: int, N_kv=None) -> np.ndarray:
     """E(M) at cell granularity: 1 on cells of active blocks, else 0."""
     cq, ck = min(B_Q, T_Q), min(B_KV, T_KV)
-    nCq, nCk = cdiv(N, cq), cdiv(N, ck)
+    nCq, nCk = cdiv(N, cq), cdiv(N if N_kv is None else N_kv, ck)
     e = np.repeat(np.repeat((mask != 0).astype(np.int32), B_Q // cq, axis=1), B_KV // ck, axis=2)
     return np.ascontiguousarray(e[:, :nCq, :nCk])
 

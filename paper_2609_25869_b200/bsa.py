@@ -30,7 +30,7 @@ class PlanDesc(ctypes.Structure):
 
 class Options(ctypes.Structure):
     _fields_ = [("force_plan_id", ctypes.c_int32), ("reserved0", ctypes.c_int32),
-                ("max_workspace_bytes", ctypes.c_int64)]
+                ("max_workspace_bytes", ctypes.c_int64), ("N_kv", ctypes.c_int64)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -45,7 +45,8 @@ class PlanInfo(ctypes.Structure):
                 ("ntiles", ctypes.c_int64), ("nitems", ctypes.c_int64), ("nsplit_rows", ctypes.c_int64),
                 ("workspace_bytes", ctypes.c_int64), ("covered_pairs", ctypes.c_int64),
                 ("us_mask_state", ctypes.c_float), ("us_stats_sync", ctypes.c_float), ("us_lookup", ctypes.c_float),
-                ("us_launch_prep", ctypes.c_float), ("us_total", ctypes.c_float), ("device_status", ctypes.c_int32)]
+                ("us_launch_prep", ctypes.c_float), ("us_total", ctypes.c_float), ("device_status", ctypes.c_int32),
+                ("N_kv", ctypes.c_int64)]
 
     def as_dict(self) -> Dict:
         out = {}
@@ -208,12 +209,13 @@ class Plan:
 
 
 def plan_create(mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1,
-                max_workspace_bytes: int = 0, stream=None) -> Plan:
-    """``bsa_plan_create_ex``: ``mask`` is a uint8/bool CUDA tensor ``[heads, nQb, nKb]``."""
+                max_workspace_bytes: int = 0, stream=None, N_kv: int = 0) -> Plan:
+    """``bsa_plan_create_ex``: ``mask`` is a uint8/bool CUDA tensor ``[heads, nQb, nKb]``; ``N_kv`` > 0 gives K and V
+    that many tokens per head (Q, O, LSE keep ``N``)."""
     import torch
     assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool)
     h = ctypes.c_void_p()
-    opt = Options(plan_id, 0, max_workspace_bytes)
+    opt = Options(plan_id, 0, max_workspace_bytes, N_kv)
     _check(lib().bsa_plan_create_ex(mask.data_ptr(), B_Q, B_KV, N, heads, d, ctypes.byref(opt), _stream_ptr(stream),
                                     ctypes.byref(h)), "bsa_plan_create")
     return Plan(h.value)
@@ -236,12 +238,12 @@ def pack_mask(mask):
 
 
 def plan_create_packed(mask_bits, row_stride: int, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1,
-                       max_workspace_bytes: int = 0, stream=None) -> Plan:
+                       max_workspace_bytes: int = 0, stream=None, N_kv: int = 0) -> Plan:
     """``bsa_plan_create_packed``: ``mask_bits`` is a uint8 CUDA tensor of bit-packed rows (see ``pack_mask``)."""
     import torch
     assert mask_bits.is_cuda and mask_bits.is_contiguous() and mask_bits.dtype == torch.uint8
     h = ctypes.c_void_p()
-    opt = Options(plan_id, 0, max_workspace_bytes)
+    opt = Options(plan_id, 0, max_workspace_bytes, N_kv)
     _check(lib().bsa_plan_create_packed(mask_bits.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
                                         _stream_ptr(stream), ctypes.byref(h)), "bsa_plan_create_packed")
     return Plan(h.value)
@@ -256,14 +258,14 @@ class PlanCache:
         self._h = h.value
 
     def get(self, mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1, max_workspace_bytes: int = 0,
-            stream=None, row_stride: int = 0):
+            stream=None, row_stride: int = 0, N_kv: int = 0):
         """``bsa_plan_cache_get``: returns ``(plan, hit)``.  ``row_stride`` > 0: ``mask`` is bit-packed (``pack_mask``).
         The plan is shared with the cache; ``plan.destroy()`` only gives it back."""
         import torch
         assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool)
         h = ctypes.c_void_p()
         hit = ctypes.c_int(0)
-        opt = Options(plan_id, 0, max_workspace_bytes)
+        opt = Options(plan_id, 0, max_workspace_bytes, N_kv)
         _check(lib().bsa_plan_cache_get(self._h, mask.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
                                         _stream_ptr(stream), ctypes.byref(h), ctypes.byref(hit)), "bsa_plan_cache_get")
         return Plan(h.value), bool(hit.value)
@@ -288,12 +290,12 @@ class PlanCache:
 
 
 def request_host(mask: np.ndarray, B_Q: int, B_KV: int, N: int, heads: int, d: int, Q, K, V, O, LSE,
-                 plan_id: int = -1) -> Dict:
+                 plan_id: int = -1, N_kv: int = 0) -> Dict:
     """``bsa_request_host``: all arguments are HOST buffers (torch CPU tensors or numpy arrays)."""
     def ptr(x):
         return x.data_ptr() if hasattr(x, "data_ptr") else x.ctypes.data
     inf = PlanInfo()
-    opt = Options(plan_id, 0, 0)
+    opt = Options(plan_id, 0, 0, N_kv)
     _check(lib().bsa_request_host(ptr(mask), B_Q, B_KV, N, heads, d, ptr(Q), ptr(K), ptr(V), ptr(O), ptr(LSE),
                                   ctypes.byref(opt), ctypes.byref(inf)), "bsa_request_host")
     return inf.as_dict()

@@ -15,9 +15,9 @@
 namespace bsa {
 // bsa_lut.cpp
 const bsa_plan_desc_t* catalog_entry(int plan_id);
-bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int heads, MapGeom* g);
+bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int64_t N_kv, int heads, MapGeom* g);
 int64_t plan_workspace_bytes(const bsa_plan_desc_t& P, int64_t N, int heads, int d);
-bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws);
+bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws, int64_t N_kv = 0);
 int base_plan(int B_Q, int B_KV, int d);
 uint64_t catalog_hash();
 void lut_buckets(int64_t N, double density, double skew, double run_cov, int32_t out[4]);
@@ -27,7 +27,7 @@ bsa_status_t lut_load(const char* path);
 void set_force_plan(int id);
 int get_force_plan();
 int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_cov, double skew,
-               int64_t max_ws, int* hit_out, int32_t buckets_out[4]);
+               int64_t max_ws, int* hit_out, int32_t buckets_out[4], int64_t N_kv = 0);
 int catalog_size();
 
 static std::atomic<long long> g_launches{0};
@@ -98,7 +98,7 @@ struct bsa_plan {
 namespace {
 struct CacheKey {
     uint64_t hash[2];
-    int64_t N, packed_stride, max_ws;
+    int64_t N, N_kv, packed_stride, max_ws;
     int32_t B_Q, B_KV, heads, d, align, force, device;
     uint32_t generation;
     bool operator==(const CacheKey& o) const { return memcmp(this, &o, sizeof *this) == 0; }
@@ -121,6 +121,10 @@ static bsa_status_t validate(const void* mask, int B_Q, int B_KV, int64_t N, int
     if (!(d == 64 || d == 128) || !p2(B_Q) || !p2(B_KV)) return BSA_ERR_UNSUPPORTED;
     if (N > (1ll << 30)) return BSA_ERR_UNSUPPORTED;
     return BSA_OK;
+}
+// key/value tokens per head of a request: the options' N_kv, else N
+static int64_t request_n_kv(const bsa_options_t* options, int64_t N) {
+    return (options && options->N_kv > 0) ? options->N_kv : N;
 }
 
 static void free_plan(bsa_plan* p) {
@@ -156,8 +160,10 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
                                 bsa_plan_cache* cache = nullptr, int* cache_hit = nullptr) {
     bsa_status_t vs = validate(mask_dev, B_Q, B_KV, N, heads, d, out_plan);
     if (vs != BSA_OK) return vs;
+    const int64_t N_kv = request_n_kv(options, N);
+    if (N_kv > (1ll << 30)) return BSA_ERR_UNSUPPORTED;
     if (packed_stride > 0) {
-        const int64_t nKb64 = (N + B_KV - 1) / B_KV;
+        const int64_t nKb64 = (N_kv + B_KV - 1) / B_KV;
         if (packed_stride % 4 != 0 || packed_stride * 8 < nKb64 || (reinterpret_cast<uintptr_t>(mask_dev) & 3u))
             return BSA_ERR_INVALID_ARG;
     }
@@ -188,7 +194,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
         }
     }
 
-    const int nQb = (int)((N + B_Q - 1) / B_Q), nKb = (int)((N + B_KV - 1) / B_KV);
+    const int nQb = (int)((N + B_Q - 1) / B_Q), nKb = (int)((N_kv + B_KV - 1) / B_KV);
     const int64_t nrows64 = (int64_t)heads * nQb;
     if (nrows64 >= (1ll << 31) - 8) { delete p; return BSA_ERR_UNSUPPORTED; }
     const int nrows = (int)nrows64;
@@ -262,7 +268,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
         memset(&key, 0, sizeof key);
         key.hash[0] = p->hstats.hash[0];
         key.hash[1] = p->hstats.hash[1];
-        key.N = N; key.packed_stride = packed_stride; key.max_ws = max_ws;
+        key.N = N; key.N_kv = N_kv; key.packed_stride = packed_stride; key.max_ws = max_ws;
         key.B_Q = B_Q; key.B_KV = B_KV; key.heads = heads; key.d = d;
         key.align = packed_stride > 0 ? 0 : (int32_t)(reinterpret_cast<uintptr_t>(mask_dev) & 15u);
         key.force = forced; key.device = p->device;
@@ -305,15 +311,15 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     const double skew = nnz > 0 ? (double)p->hstats.max_row_nnz / (nnz / (double)nrows) : 0.0;
     int plan_id;
     if (forced >= 0) {
-        plan_id = plan_eligible(forced, B_Q, B_KV, N, heads, d, max_ws) ? forced : -1;
+        plan_id = plan_eligible(forced, B_Q, B_KV, N, heads, d, max_ws, N_kv) ? forced : -1;
         lut_buckets(N, density, skew, run_cov, p->buckets);
         p->lut_hit = 0;
     } else {
-        plan_id = lut_select(B_Q, B_KV, N, heads, d, density, run_cov, skew, max_ws, &p->lut_hit, p->buckets);
+        plan_id = lut_select(B_Q, B_KV, N, heads, d, density, run_cov, skew, max_ws, &p->lut_hit, p->buckets, N_kv);
     }
     if (plan_id < 0) { free_plan(p); return BSA_ERR_NO_ELIGIBLE_PLAN; }
     p->desc = *catalog_entry(plan_id);
-    make_geom(p->desc, B_Q, B_KV, N, heads, &p->g);
+    make_geom(p->desc, B_Q, B_KV, N, N_kv, heads, &p->g);
     p->stages = p->desc.stages > 0 ? p->desc.stages : attention_max_stages(d, p->desc.T_KV, p->desc.kernel);
     const double t3 = now_us();
 
@@ -524,7 +530,7 @@ extern "C" bsa_status_t bsa_plan_get_info(const bsa_plan_t* p, bsa_plan_info_t* 
     const MapGeom& g = p->g;
     info->map_q = g.sQ > 1 ? BSA_MAP_COARSENED : (g.rq > 1 ? BSA_MAP_REFINED : BSA_MAP_DIRECT);
     info->map_kv = g.sK > 1 ? BSA_MAP_COARSENED : (g.rk > 1 ? BSA_MAP_REFINED : BSA_MAP_DIRECT);
-    info->heads = g.H; info->d = p->d; info->B_Q = g.B_Q; info->B_KV = g.B_KV; info->N = g.N;
+    info->heads = g.H; info->d = p->d; info->B_Q = g.B_Q; info->B_KV = g.B_KV; info->N = g.N; info->N_kv = g.N_kv;
     info->nQb = g.nQb; info->nKb = g.nKb; info->nQt = g.nQt; info->nKt = g.nKt;
     info->member_bits = g.sQ128 * g.sK;
     info->member_words = g.slots;
@@ -640,12 +646,15 @@ extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int 
     bsa_plan_t* dummy = nullptr;
     bsa_status_t vs = validate(mask_host, B_Q, B_KV, N, heads, d, &dummy);
     if (vs != BSA_OK) return vs;
-    const size_t nQb = (size_t)((N + B_Q - 1) / B_Q), nKb = (size_t)((N + B_KV - 1) / B_KV);
+    const int64_t N_kv = request_n_kv(options, N);
+    if (N_kv > (1ll << 30)) return BSA_ERR_UNSUPPORTED;
+    const size_t nQb = (size_t)((N + B_Q - 1) / B_Q), nKb = (size_t)((N_kv + B_KV - 1) / B_KV);
     const size_t mbytes = (size_t)heads * nQb * nKb;
-    const size_t tbytes = (size_t)heads * (size_t)N * d * 2;
+    const size_t tbytes = (size_t)heads * (size_t)N * d * 2;      // Q, O
+    const size_t kbytes = (size_t)heads * (size_t)N_kv * d * 2;   // K, V
     const size_t lbytes = (size_t)heads * (size_t)N * 4;
-    const size_t o_m = 0, o_q = align_up(mbytes), o_k = o_q + align_up(tbytes), o_v = o_k + align_up(tbytes),
-                 o_o = o_v + align_up(tbytes), o_l = o_o + align_up(tbytes), total = o_l + align_up(lbytes);
+    const size_t o_m = 0, o_q = align_up(mbytes), o_k = o_q + align_up(tbytes), o_v = o_k + align_up(kbytes),
+                 o_o = o_v + align_up(kbytes), o_l = o_o + align_up(tbytes), total = o_l + align_up(lbytes);
     // Two streams kept per host thread: the mask goes first on `s` and the plan is created behind it, while Q, K and V
     // travel on `s2`; the forward waits for them.  Planning (statistics copy, lookup, preparation kernels) thus
     // overlaps the 3 x heads x N x d x 2 bytes of input copies instead of following them.
@@ -666,8 +675,8 @@ extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int 
     if (e == cudaSuccess) e = cudaEventRecord(inputs_ready, s);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(s2, inputs_ready, 0);
     if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_q, Q_host, tbytes, cudaMemcpyHostToDevice, s2);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_k, K_host, tbytes, cudaMemcpyHostToDevice, s2);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_v, V_host, tbytes, cudaMemcpyHostToDevice, s2);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_k, K_host, kbytes, cudaMemcpyHostToDevice, s2);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_v, V_host, kbytes, cudaMemcpyHostToDevice, s2);
     if (e == cudaSuccess) e = cudaEventRecord(inputs_ready, s2);
     if (e == cudaSuccess) {
         st = bsa_plan_create_ex(buf + o_m, B_Q, B_KV, N, heads, d, options, s, &plan);

@@ -59,7 +59,8 @@ struct AttnParams {
     float* ws_O;
     float* ws_LSE;
     unsigned long long full_member;
-    int32_t N;
+    int32_t N;    // query tokens per head
+    int32_t Nkv;  // key/value tokens per head
     int32_t lgBQ;   // log2(B_Q) when B_Q < 128, else 31 (row >> 31 == 0)
     int32_t lgBKV;  // log2(B_KV) when B_KV < T_KV, else 31
     int32_t sK;     // logical KV sub-blocks per tile
@@ -435,9 +436,9 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     col_next = p.tile_col[it.tile_begin + j + 1];
                     member_next = p.tile_member[it.tile_begin + j + 1];
                 }
-                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
+                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.Nkv);
                 const uint32_t row_bits = (uint32_t)((member >> ((tid >> p.lgBQ) * p.sK)) & sub_mask);
-                const int n_valid = p.N - kv0;  // columns >= n_valid do not exist
+                const int n_valid = p.Nkv - kv0;  // columns >= n_valid do not exist
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[sb]), (gs >> 1) & 1, abortp));
                 if (!ok) break;
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 10);
@@ -800,9 +801,9 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
                     member_next = p.tile_member[(size_t)(it.tile_begin + j + 1) * 2 + x];
                 }
                 if (member == 0ull) continue;
-                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
+                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.Nkv);
                 const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
-                const int n_valid = p.N - kv0;
+                const int n_valid = p.Nkv - kv0;
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), cnt & 1, abortp));
                 if (!ok) break;
                 tc_fence_after();
@@ -1141,9 +1142,9 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     col_next = p.tile_col[it.tile_begin + j + 1];
                     member_next = p.tile_member[it.tile_begin + j + 1];
                 }
-                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
+                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.Nkv);
                 const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
-                const int n_valid = p.N - kv0;
+                const int n_valid = p.Nkv - kv0;
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[sb]), (gs >> 1) & 1, abortp));
                 if (!ok) break;
                 tc_fence_after();
@@ -1802,9 +1803,9 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     col_next = ldg_pinned_s32(p.tile_col + it.tile_begin + j + 2);
                     member_next = ldg_pinned_u64(p.tile_member + it.tile_begin + j + 2);
                 }
-                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.N);
+                const bool need_mask = (member != p.full_member) || (kv0 + TK > p.Nkv);
                 const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
-                const int n_valid = p.N - kv0;
+                const int n_valid = p.Nkv - kv0;
                 if (lane == 0 && j == j0) BSA_TRACE_POINT(2 + warp, tn, 35);
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), (gs >> 1) & 1, abortp));
                 if (!ok) break;
@@ -2067,10 +2068,10 @@ template <int D, int TK, int KERNEL>
 cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t stream, const char** err) {
     CUtensorMap tq, tk, tv;
     const bool ok_maps = (KERNEL == 4)
-                             ? (encode_map4(&tq, a.Q, a.g.N, a.g.H, D, kTQ) && encode_map4(&tk, a.K, a.g.N, a.g.H, D, TK) &&
-                                encode_map4(&tv, a.V, a.g.N, a.g.H, D, TK))
-                             : (encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ) && encode_map(&tk, a.K, a.g.N, a.g.H, D, TK) &&
-                                encode_map(&tv, a.V, a.g.N, a.g.H, D, TK));
+                             ? (encode_map4(&tq, a.Q, a.g.N, a.g.H, D, kTQ) && encode_map4(&tk, a.K, a.g.N_kv, a.g.H, D, TK) &&
+                                encode_map4(&tv, a.V, a.g.N_kv, a.g.H, D, TK))
+                             : (encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ) && encode_map(&tk, a.K, a.g.N_kv, a.g.H, D, TK) &&
+                                encode_map(&tv, a.V, a.g.N_kv, a.g.H, D, TK));
     if (!ok_maps) {
         *err = "cuTensorMapEncodeTiled failed";
         return cudaErrorInvalidValue;
@@ -2174,6 +2175,7 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     const int bits = a.g.sQ128 * a.g.sK;
     p.full_member = (bits >= 64) ? ~0ull : ((1ull << bits) - 1ull);
     p.N = (int32_t)a.g.N;
+    p.Nkv = (int32_t)a.g.N_kv;
     p.lgBQ = (a.g.sQ128 > 1) ? a.g.lgBQ : 31;
     p.lgBKV = (a.g.sK > 1) ? a.g.lgBKV : 31;
     p.sK = a.g.sK;

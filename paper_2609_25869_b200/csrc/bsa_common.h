@@ -64,7 +64,8 @@ struct MapGeom {
     int32_t sQ, rq;  // logical rows per tile row (coarsened) / tile rows per logical row (refined)
     int32_t sK, rk;  // same for columns
     int32_t lgBQ, lgBKV, lgSK;
-    int64_t N;
+    int64_t N;     // query tokens per head (rows of Q, O, LSE)
+    int64_t N_kv;  // key/value tokens per head (rows of K, V; columns of the score matrix)
 };
 
 // ---- planner entry points (bsa_planner.cu); all launch on `stream`, none synchronises -------

@@ -78,9 +78,10 @@ int ilog2(int v) {
     return l;
 }
 
-bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int heads, MapGeom* g) {
+bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int64_t N_kv, int heads, MapGeom* g) {
     g->H = heads;
     g->N = N;
+    g->N_kv = N_kv;
     g->B_Q = B_Q;
     g->B_KV = B_KV;
     g->T_Q = P.T_Q;
@@ -88,9 +89,9 @@ bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int heads
     g->slots = P.T_Q / kTQ;
     g->sQ128 = B_Q < kTQ ? kTQ / B_Q : 1;
     g->nQb = (int)((N + B_Q - 1) / B_Q);
-    g->nKb = (int)((N + B_KV - 1) / B_KV);
+    g->nKb = (int)((N_kv + B_KV - 1) / B_KV);
     g->nQt = (int)((N + P.T_Q - 1) / P.T_Q);
-    g->nKt = (int)((N + P.T_KV - 1) / P.T_KV);
+    g->nKt = (int)((N_kv + P.T_KV - 1) / P.T_KV);
     g->sQ = B_Q < P.T_Q ? P.T_Q / B_Q : 1;
     g->rq = B_Q > P.T_Q ? B_Q / P.T_Q : 1;
     g->sK = B_KV < P.T_KV ? P.T_KV / B_KV : 1;
@@ -108,14 +109,16 @@ int64_t plan_workspace_bytes(const bsa_plan_desc_t& P, int64_t N, int heads, int
 }
 
 // Eligible(P, R), Section 4.4: logical geometry, tensor properties, metadata format, workspace.
-bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws) {
+bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws, int64_t N_kv = 0) {
     const bsa_plan_desc_t* P = catalog_entry(plan_id);
     if (!P) return false;
     if (!(d == 64 || d == 128)) return false;
     if (!pow2_in(B_Q, 16, 256) || !pow2_in(B_KV, 16, 256)) return false;
     if (N <= 0 || heads <= 0 || N > (1ll << 30)) return false;
     MapGeom g;
-    make_geom(*P, B_Q, B_KV, N, heads, &g);
+    if (N_kv <= 0) N_kv = N;
+    if (N_kv > (1ll << 30)) return false;
+    make_geom(*P, B_Q, B_KV, N, N_kv, heads, &g);
     if (g.sQ128 * g.sK > 64) return false;  // one 64-bit membership word per 128-row slot
     if (P->split_pmax > 32) return false;   // the merge kernel keeps up to 32 partial LSEs in registers
     const int max_st = attention_max_stages(d, P->T_KV, P->kernel);
@@ -257,7 +260,7 @@ int get_force_plan() { return g_force_plan; }
 
 // Algorithm 2, lines 6-19: z = <k, u, s>; r = rho(z); ranked list or base plan; first eligible.
 int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_cov, double skew,
-               int64_t max_ws, int* hit_out, int32_t buckets_out[4]) {
+               int64_t max_ws, int* hit_out, int32_t buckets_out[4], int64_t N_kv = 0) {
     int32_t b[4];
     lut_buckets(N, density, skew, run_cov, b);
     if (buckets_out) memcpy(buckets_out, b, sizeof b);
@@ -279,7 +282,7 @@ int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, d
     if (!hit) ranked.push_back(base_plan(B_Q, B_KV, d));
     if (hit_out) *hit_out = hit ? 1 : 0;
     for (int id : ranked)
-        if (plan_eligible(id, B_Q, B_KV, N, heads, d, max_ws)) return id;
+        if (plan_eligible(id, B_Q, B_KV, N, heads, d, max_ws, N_kv)) return id;
     return -1;
 }
 

@@ -106,6 +106,11 @@ class Request:
     mask: np.ndarray  # uint8 [H, nQb, nKb]
     qkv_seed: int
     note: str = ""
+    N_kv: int = 0  # key/value tokens per head; 0 = N (self-attention, every workload of the paper)
+
+    @property
+    def n_kv(self) -> int:
+        return self.N_kv if self.N_kv > 0 else self.N
 
     @property
     def nQb(self) -> int:
@@ -113,10 +118,14 @@ class Request:
 
     @property
     def nKb(self) -> int:
-        return cdiv(self.N, self.B_KV)
+        return cdiv(self.n_kv, self.B_KV)
 
     def qkv(self):
-        return make_qkv(self.qkv_seed, self.H, self.N, self.d)
+        if self.n_kv == self.N:
+            return make_qkv(self.qkv_seed, self.H, self.N, self.d)
+        q, _, _ = make_qkv(self.qkv_seed, self.H, self.N, self.d)
+        _, k, v = make_qkv(self.qkv_seed + 7777, self.H, self.n_kv, self.d)
+        return q, k, v
 
 
 # --------------------------------------------------------------------------

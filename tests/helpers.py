@@ -56,8 +56,8 @@ def check_plan_structure(req, plan, heads=None):
             mem = [int(a) | (int(b) << bits) for a, b in tm]
         tiles[h] = (trp, tc, mem)
         ntiles += len(tc)
-    cover = oracle.coverage_counts(req.H, req.N, req.B_Q, req.B_KV, T_Q, T_KV, tiles)
-    expect = oracle.expected_cell_cover(req.mask, req.N, req.B_Q, req.B_KV, T_Q, T_KV)
+    cover = oracle.coverage_counts(req.H, req.N, req.B_Q, req.B_KV, T_Q, T_KV, tiles, N_kv=req.n_kv)
+    expect = oracle.expected_cell_cover(req.mask, req.N, req.B_Q, req.B_KV, T_Q, T_KV, N_kv=req.n_kv)
     for h in hs:
         assert np.array_equal(cover[h], expect[h]), f"tile plan does not cover E(M) exactly (head {h})"
     if heads is None:
@@ -114,7 +114,8 @@ def compare_with_oracle(req, O, LSE, qkv_cpu, sel=None, row_step=1, guards=True)
     assert not O[row_empty].any(), "O must be exactly zero on rows with no active block"
     if sel is None:
         sel = [(h, b) for h in range(req.H) for b in range(req.nQb)]
-    oO, oL, pairs = oracle.attention_blocks(req.mask, req.B_Q, req.B_KV, req.N, req.d, Qb, Kb, Vb, sel, row_step)
+    oO, oL, pairs = oracle.attention_blocks(req.mask, req.B_Q, req.B_KV, req.N, req.d, Qb, Kb, Vb, sel, row_step,
+                                            N_kv=req.n_kv)
     dO, dL = [], []
     for n, (h, b) in enumerate(sel):
         r0 = b * req.B_Q
@@ -137,7 +138,7 @@ def compare_with_oracle(req, O, LSE, qkv_cpu, sel=None, row_step=1, guards=True)
 
 def run_request(req, plan_id=-1, qkv=None, sel=None, row_step=1, structure=True, heads=None, guards=True):
     mask, q, k, v, qkv_cpu = to_dev(req, qkv)
-    with bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=plan_id) as plan:
+    with bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=plan_id, N_kv=req.N_kv) as plan:
         O, LSE = plan.forward(q, k, v)
         torch.cuda.synchronize()
         inf = plan.info()
