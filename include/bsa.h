@@ -109,17 +109,18 @@ typedef struct bsa_plan_info {
  * bsa_plan_create -- online plan selection and launch preparation (Section 5.2, Algorithm 2).
  *
  * Builds the shared mask state mu(M) on the GPU (block-CSR offsets, active KV column indices and
- * the scalar statistics), copies only the scalars to the host (the one synchronisation of the
+ * the scalar statistics), passes only the scalars to the host (the one synchronisation of the
  * call), looks up the regime in the loaded plan table, takes the first eligible plan of its
  * ranking (base plan on a miss), then derives that plan's metadata on the GPU: physical tile
  * lists with membership bits (Direct / Coarsened / Refined mapping, Section 4.2), work items per Q
  * tile row, Split-K partitions of heavy rows, longest-first order (Section 4.3).
  *
- *   mask_dev : uint8 [heads, ceil(N/B_Q), ceil(N/B_KV)], row-major, nonzero = active block.
+ *   mask_dev : uint8 [heads, ceil(N/B_Q), ceil(N_kv/B_KV)], row-major, nonzero = active block.
  *              Borrowed: read by kernels this call submits to `stream`; it may be freed or
  *              overwritten by work ordered after the call on that stream (or after a stream sync).
  *   B_Q,B_KV : logical block geometry, powers of two in [16, 256].
- *   N        : tokens per head (N_q = N_kv = N); need not be a multiple of the block sizes.
+ *   N        : query tokens per head, N_q of Section 2.1; need not be a multiple of the block sizes.
+ *              The key/value token count N_kv equals N unless options->N_kv says otherwise (_ex variants).
  *   heads    : independent (batch x head) problems.
  *   d        : head dimension, 64 or 128.  Scale is 1/sqrt(d); attention is non-causal.
  *   out_plan : receives the plan; the plan owns its device buffers (CSR, tile lists, work items,
@@ -151,7 +152,8 @@ BSA_API bsa_status_t bsa_plan_create_packed(const uint8_t* mask_bits_dev, int64_
  * bsa_forward -- execute the plan's native kernels (Section 4: main attention kernel, then the
  * Split-K reduction kernel when the plan has partitions).
  *
- *   Q,K,V : bf16 [heads, N, d], d contiguous, 16-byte aligned base, device memory, borrowed.
+ *   Q     : bf16 [heads, N, d], d contiguous, 16-byte aligned base, device memory, borrowed.
+ *   K,V   : bf16 [heads, N_kv, d], the same (N_kv = N unless the plan was created with options->N_kv).
  *   O     : bf16 [heads, N, d], written for every row; rows with no active block get 0.
  *   LSE   : fp32 [heads, N], natural-log log-sum-exp of the scaled scores over E(M); -inf for rows
  *           with no active block.
