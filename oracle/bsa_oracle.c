@@ -24,7 +24,8 @@
  * tokens (N) and of key tokens (N_kv) are separate arguments.
  *
  * Inputs are bf16 bit patterns (the same rounded values the GPU sees),
- * widened exactly to double.
+ * widened exactly to double; with fp16 != 0 they are IEEE half bit patterns
+ * instead (the tensor type is a request property, Section 4.4).
  */
 #include <math.h>
 #include <stdint.h>
@@ -40,6 +41,18 @@ static inline double bf16_to_double(uint16_t b) {
     memcpy(&f, &u, sizeof f);
     return (double)f;
 }
+
+/* IEEE 754 binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits. */
+static inline double f16_to_double(uint16_t h) {
+    const int sign = h >> 15, e = (h >> 10) & 31, m = h & 1023;
+    double v;
+    if (e == 0) v = ldexp((double)m, -24);                 /* zero and subnormals: m * 2^-24 */
+    else if (e == 31) v = m ? NAN : INFINITY;
+    else v = ldexp((double)(1024 + m), e - 25);            /* (1 + m/1024) * 2^(e-15) */
+    return sign ? -v : v;
+}
+
+static inline double in_to_double(uint16_t b, int fp16) { return fp16 ? f16_to_double(b) : bf16_to_double(b); }
 
 int bsa_oracle_num_threads(void) {
 #ifdef _OPENMP
@@ -57,12 +70,13 @@ int bsa_oracle_num_threads(void) {
  * evaluated are left untouched in the outputs.
  *
  * mask : uint8 [H][nQb][nKb], nonzero = active
- * Q    : bf16 bits [H][N][d]        K,V: bf16 bits [H][N_kv][d]
+ * Q    : bf16 (or fp16) bits [H][N][d]        K,V: the same, [H][N_kv][d]
  * O    : double [n_sel][B_Q][d]     LSE: double [n_sel][B_Q]
  * pairs_out (optional): number of active token pairs evaluated.
  * Returns 0, or -1 on allocation failure.
  */
 int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int B_KV, int64_t N, int64_t N_kv, int d,
+                      int fp16,
                       const uint16_t* Q, const uint16_t* K, const uint16_t* V,
                       int n_sel, const int32_t* sel_head, const int32_t* sel_qblock, int row_step,
                       double* O, double* LSE, int64_t* pairs_out) {
@@ -92,7 +106,7 @@ int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int
                     if (i >= N) break;
                     double* o_out = O + ((size_t)sidx * B_Q + r) * d;
                     const uint16_t* qi = Q + ((size_t)h * N + i) * d;
-                    for (int c = 0; c < d; ++c) q[c] = bf16_to_double(qi[c]);
+                    for (int c = 0; c < d; ++c) q[c] = in_to_double(qi[c], fp16);
                     /* scores over the reachable keys J(h,i) */
                     int64_t cnt = 0;
                     double m = -INFINITY;
@@ -103,7 +117,7 @@ int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int
                         for (int64_t j = j0; j < j1; ++j) {
                             const uint16_t* kj = Kh + (size_t)j * d;
                             double dot = 0.0;
-                            for (int c = 0; c < d; ++c) dot += q[c] * bf16_to_double(kj[c]);
+                            for (int c = 0; c < d; ++c) dot += q[c] * in_to_double(kj[c], fp16);
                             dot *= inv_sqrt_d;
                             s[j] = dot;
                             if (dot > m) m = dot;
@@ -126,7 +140,7 @@ int bsa_oracle_blocks(const uint8_t* mask, int H, int nQb, int nKb, int B_Q, int
                             const double p = exp(s[j] - m);
                             l += p;
                             const uint16_t* vj = Vh + (size_t)j * d;
-                            for (int c = 0; c < d; ++c) acc[c] += p * bf16_to_double(vj[c]);
+                            for (int c = 0; c < d; ++c) acc[c] += p * in_to_double(vj[c], fp16);
                         }
                     }
                     for (int c = 0; c < d; ++c) o_out[c] = acc[c] / l;

@@ -68,7 +68,7 @@ def _load():
         lib.bsa_oracle_blocks.restype = ctypes.c_int
         lib.bsa_oracle_blocks.argtypes = [
             ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64,
-            ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
+            ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
             ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         lib.bsa_oracle_num_threads.restype = ctypes.c_int
         _lib = lib
@@ -88,11 +88,12 @@ def cdiv(a: int, b: int) -> int:
 # --------------------------------------------------------------------------
 def attention_blocks(mask: np.ndarray, B_Q: int, B_KV: int, N: int, d: int,
                      Qb: np.ndarray, Kb: np.ndarray, Vb: np.ndarray,
-                     sel: Sequence[Tuple[int, int]], row_step: int = 1, N_kv: Optional[int] = None):
+                     sel: Sequence[Tuple[int, int]], row_step: int = 1, N_kv: Optional[int] = None,
+                     dtype: str = "bf16"):
     """Masked attention (Eq. 1) on selected (head, query-block) pairs.
 
     ``Qb`` is ``[H, N, d]`` and ``Kb/Vb`` are ``[H, N_kv, d]`` uint16 bf16 bit patterns (Section 2.1: N_q query
-    and N_kv key tokens; ``N_kv`` defaults to ``N``).  Returns
+    and N_kv key tokens; ``N_kv`` defaults to ``N``), or IEEE half bit patterns with ``dtype="fp16"``.  Returns
     ``(O [n_sel, B_Q, d] float64, LSE [n_sel, B_Q] float64, active_pairs)``;
     rows at or beyond N, and rows skipped by ``row_step``, are NaN.
     """
@@ -109,7 +110,8 @@ def attention_blocks(mask: np.ndarray, B_Q: int, B_KV: int, N: int, d: int,
     O = np.full((n, B_Q, d), np.nan, dtype=np.float64)
     LSE = np.full((n, B_Q), np.nan, dtype=np.float64)
     pairs = ctypes.c_int64(0)
-    rc = lib.bsa_oracle_blocks(mask.ctypes.data, H, nQb, nKb, B_Q, B_KV, N, N_kv, d, Qb.ctypes.data, Kb.ctypes.data,
+    assert dtype in ("bf16", "fp16")
+    rc = lib.bsa_oracle_blocks(mask.ctypes.data, H, nQb, nKb, B_Q, B_KV, N, N_kv, d, int(dtype == "fp16"), Qb.ctypes.data, Kb.ctypes.data,
                                Vb.ctypes.data, n, sel_h.ctypes.data, sel_b.ctypes.data, row_step,
                                O.ctypes.data, LSE.ctypes.data, ctypes.byref(pairs))
     if rc != 0:
@@ -117,11 +119,11 @@ def attention_blocks(mask: np.ndarray, B_Q: int, B_KV: int, N: int, d: int,
     return O, LSE, int(pairs.value)
 
 
-def attention_full(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, N_kv=None):
+def attention_full(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, N_kv=None, dtype="bf16"):
     """Eq. 1 on every row.  Returns ``O [H, N, d]`` and ``LSE [H, N]`` (float64)."""
     H, nQb, _ = mask.shape
     sel = [(h, i) for h in range(H) for i in range(nQb)]
-    O, LSE, pairs = attention_blocks(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, sel, N_kv=N_kv)
+    O, LSE, pairs = attention_blocks(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, sel, N_kv=N_kv, dtype=dtype)
     O = O.reshape(H, nQb * B_Q, d)[:, :N]
     LSE = LSE.reshape(H, nQb * B_Q)[:, :N]
     return np.ascontiguousarray(O), np.ascontiguousarray(LSE), pairs
@@ -131,15 +133,20 @@ def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
     return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
+def bits_to_f64(b: np.ndarray, dtype: str = "bf16") -> np.ndarray:
+    """16-bit patterns to float64: bf16, or IEEE half through numpy's own float16."""
+    return np.ascontiguousarray(b).view(np.float16).astype(np.float64) if dtype == "fp16" else bf16_bits_to_f64(b)
+
+
 def expand_mask(mask_h: np.ndarray, B_Q: int, B_KV: int, N: int, N_kv=None) -> np.ndarray:
     """E(M) of one head as an explicit ``[N, N_kv]`` boolean matrix (Section 2.1)."""
     return np.repeat(np.repeat(mask_h != 0, B_Q, axis=0), B_KV, axis=1)[:N, :(N if N_kv is None else N_kv)]
 
 
-def attention_bruteforce(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, N_kv=None):
+def attention_bruteforce(mask, B_Q, B_KV, N, d, Qb, Kb, Vb, N_kv=None, dtype="bf16"):
     """Eq. 1 through an explicit token-pair matrix, one row at a time (tiny inputs)."""
     H = mask.shape[0]
-    Q, K, V = (bf16_bits_to_f64(x) for x in (Qb, Kb, Vb))
+    Q, K, V = (bits_to_f64(x, dtype) for x in (Qb, Kb, Vb))
     O = np.zeros((H, N, d))
     LSE = np.full((H, N), -np.inf)
     for h in range(H):

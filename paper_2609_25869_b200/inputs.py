@@ -67,13 +67,14 @@ def uniform01(seed: int, stream: int, *idx: np.ndarray) -> np.ndarray:
 # --------------------------------------------------------------------------
 # Q / K / V
 # --------------------------------------------------------------------------
-def make_qkv(seed: int, H: int, N: int, d: int):
-    """i.i.d. N(0,1) rounded to bf16 (round-to-nearest-even).
+def make_qkv(seed: int, H: int, N: int, d: int, dtype: str = "bf16"):
+    """i.i.d. N(0,1) rounded to bf16 (round-to-nearest-even), or to IEEE half with ``dtype="fp16"``.
 
-    Returns three ``torch.bfloat16`` CPU tensors of shape ``[H, N, d]``.  The
+    Returns three ``torch.bfloat16`` (``torch.float16``) CPU tensors of shape ``[H, N, d]``.  The
     oracle always consumes these same rounded values (as raw 16-bit patterns).
     """
     import torch
+    tdt = {"bf16": torch.bfloat16, "fp16": torch.float16}[dtype]
 
     out = []
     for t in range(3):
@@ -81,12 +82,12 @@ def make_qkv(seed: int, H: int, N: int, d: int):
         g.manual_seed((seed * 1000003 + t * 7919 + 12345) & 0x7FFFFFFFFFFFFFFF)
         x = torch.empty((H, N, d), dtype=torch.float32)
         x.normal_(0.0, 1.0, generator=g)
-        out.append(x.to(torch.bfloat16))
+        out.append(x.to(tdt))
     return tuple(out)
 
 
 def bf16_bits(t) -> np.ndarray:
-    """torch.bfloat16 CPU tensor -> numpy uint16 view of the same bytes."""
+    """torch.bfloat16 (or float16) CPU tensor -> numpy uint16 view of the same bytes."""
     import torch
 
     return t.contiguous().view(torch.int16).numpy().view(np.uint16)
@@ -107,6 +108,7 @@ class Request:
     qkv_seed: int
     note: str = ""
     N_kv: int = 0  # key/value tokens per head; 0 = N (self-attention, every workload of the paper)
+    dtype: str = "bf16"  # element type of Q, K, V, O ("fp16": IEEE half)
 
     @property
     def n_kv(self) -> int:
@@ -122,9 +124,9 @@ class Request:
 
     def qkv(self):
         if self.n_kv == self.N:
-            return make_qkv(self.qkv_seed, self.H, self.N, self.d)
-        q, _, _ = make_qkv(self.qkv_seed, self.H, self.N, self.d)
-        _, k, v = make_qkv(self.qkv_seed + 7777, self.H, self.n_kv, self.d)
+            return make_qkv(self.qkv_seed, self.H, self.N, self.d, self.dtype)
+        q, _, _ = make_qkv(self.qkv_seed, self.H, self.N, self.d, self.dtype)
+        _, k, v = make_qkv(self.qkv_seed + 7777, self.H, self.n_kv, self.d, self.dtype)
         return q, k, v
 
 

@@ -75,6 +75,34 @@ def test_bruteforce_token_pair_matrix_rectangular(B_Q, B_KV, N_q, N_kv):
     assert pairs == E == oracle.active_pairs(M, B_Q, B_KV, N_q, N_kv)
 
 
+def test_half_precision_inputs_dense_softmax_and_bruteforce():
+    """Tensor type as a request property (Section 4.4): IEEE half inputs, widened exactly.  Dense mask against
+    torch's softmax on torch's own half -> double conversion (normal, subnormal and zero values included), and a
+    sparse mask against the brute force, which converts through numpy's float16."""
+    H, N, d, B = 2, 96, 32, 32
+    q, k, v = I.make_qkv(51, H, N, d, dtype="fp16")
+    assert q.dtype == torch.float16
+    k[0, 0, :4] = torch.tensor([6e-8, -3e-6, 0.0, 65504.0 / 4096], dtype=torch.float16)  # subnormals, zero
+    q[0, 1, :4] = torch.tensor([5.96e-8, 1e-7, -0.0, 2.0], dtype=torch.float16)
+    Qb, Kb, Vb = I.bf16_bits(q), I.bf16_bits(k), I.bf16_bits(v)
+    M = np.ones((H, N // B, N // B), dtype=np.uint8)
+    O, LSE, _ = oracle.attention_full(M, B, B, N, d, Qb, Kb, Vb, dtype="fp16")
+    q64, k64, v64 = (t.to(torch.float64) for t in (q, k, v))
+    s = q64 @ k64.transpose(1, 2) / math.sqrt(d)
+    np.testing.assert_allclose(O, (torch.softmax(s, dim=-1) @ v64).numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(LSE, torch.logsumexp(s, dim=-1).numpy(), rtol=0, atol=1e-12)
+    # the same bits read as bf16 are other numbers: the flag matters
+    O_b, _, _ = oracle.attention_full(M, B, B, N, d, Qb, Kb, Vb)
+    assert np.abs(O_b - O).max() > 1e-3
+    Ms = I.random_mask(3, H, N // B, N // B, 0.5, empty_rows=0.3)
+    O, LSE, _ = oracle.attention_full(Ms, B, B, N, d, Qb, Kb, Vb, dtype="fp16")
+    bO, bL = oracle.attention_bruteforce(Ms, B, B, N, d, Qb, Kb, Vb, dtype="fp16")
+    np.testing.assert_allclose(O, bO, rtol=0, atol=1e-13)
+    fin = np.isfinite(bL)
+    assert np.array_equal(np.isfinite(LSE), fin)
+    np.testing.assert_allclose(LSE[fin], bL[fin], rtol=0, atol=1e-13)
+
+
 def test_hand_computed_two_keys():
     # d = 4, one query q = (2,0,0,0), keys k0 = (2,0,0,0), k1 = (-2,0,0,0): scores 4/2 = 2 and -2.
     N, d = 2, 4
