@@ -65,10 +65,15 @@ typedef struct bsa_plan_desc {
     char name[48];
 } bsa_plan_desc_t;
 
+/* Element type of Q, K, V and O (a tensor property x of the request, Section 4.4).  Scores, softmax state and the
+ * output accumulator are fp32 either way; P is rounded to the same 16-bit type for the second product.  Half inputs
+ * are served by the plans of the ping-pong kernel only (the others are not eligible for such a request). */
+enum { BSA_DTYPE_BF16 = 0, BSA_DTYPE_FP16 = 1 };
+
 typedef struct bsa_options {
     int32_t force_plan_id;        /* >= 0: skip the lookup and use this catalog entry (still checked for
                                      eligibility); -1: Algorithm 2                                   */
-    int32_t reserved0;
+    int32_t dtype;                /* BSA_DTYPE_*: element type of Q, K, V and O (tensor property x)   */
     int64_t max_workspace_bytes;  /* Split-K workspace the request may bind; <= 0: library default   */
     int64_t N_kv;                 /* key/value tokens per head (Section 2.1: K, V are N_kv x d); <= 0: N_kv = N.
                                      The mask then has ceil(N_kv / B_KV) block columns, K and V are
@@ -103,6 +108,8 @@ typedef struct bsa_plan_info {
     float us_total;
     int32_t device_status;        /* 0, or BSA_ERR_DEVICE_TIMEOUT if any forward hit a bounded wait  */
     int64_t N_kv;                 /* key/value tokens per head (= N unless the options said otherwise) */
+    int32_t dtype;                /* BSA_DTYPE_* of the request                                        */
+    int32_t reserved1;
 } bsa_plan_info_t;
 
 /* ---------------------------------------------------------------------------------------------
@@ -152,9 +159,10 @@ BSA_API bsa_status_t bsa_plan_create_packed(const uint8_t* mask_bits_dev, int64_
  * bsa_forward -- execute the plan's native kernels (Section 4: main attention kernel, then the
  * Split-K reduction kernel when the plan has partitions).
  *
- *   Q     : bf16 [heads, N, d], d contiguous, 16-byte aligned base, device memory, borrowed.
- *   K,V   : bf16 [heads, N_kv, d], the same (N_kv = N unless the plan was created with options->N_kv).
- *   O     : bf16 [heads, N, d], written for every row; rows with no active block get 0.
+ *   Q     : bf16 (fp16 if the plan was created with options->dtype = BSA_DTYPE_FP16) [heads, N, d], d contiguous,
+ *           16-byte aligned base, device memory, borrowed.
+ *   K,V   : the same type, [heads, N_kv, d] (N_kv = N unless the plan was created with options->N_kv).
+ *   O     : the same type, [heads, N, d], written for every row; rows with no active block get 0.
  *   LSE   : fp32 [heads, N], natural-log log-sum-exp of the scaled scores over E(M); -inf for rows
  *           with no active block.
  *

@@ -28,8 +28,11 @@ class PlanDesc(ctypes.Structure):
                 ("order", ctypes.c_int32), ("kernel", ctypes.c_int32), ("name", ctypes.c_char * 48)]
 
 
+DTYPES = {"bf16": 0, "fp16": 1}  # BSA_DTYPE_*
+
+
 class Options(ctypes.Structure):
-    _fields_ = [("force_plan_id", ctypes.c_int32), ("reserved0", ctypes.c_int32),
+    _fields_ = [("force_plan_id", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("max_workspace_bytes", ctypes.c_int64), ("N_kv", ctypes.c_int64)]
 
 
@@ -46,7 +49,7 @@ class PlanInfo(ctypes.Structure):
                 ("workspace_bytes", ctypes.c_int64), ("covered_pairs", ctypes.c_int64),
                 ("us_mask_state", ctypes.c_float), ("us_stats_sync", ctypes.c_float), ("us_lookup", ctypes.c_float),
                 ("us_launch_prep", ctypes.c_float), ("us_total", ctypes.c_float), ("device_status", ctypes.c_int32),
-                ("N_kv", ctypes.c_int64)]
+                ("N_kv", ctypes.c_int64), ("dtype", ctypes.c_int32), ("reserved1", ctypes.c_int32)]
 
     def as_dict(self) -> Dict:
         out = {}
@@ -153,8 +156,8 @@ class Plan:
     def forward(self, Q, K, V, O=None, LSE=None, stream=None):
         """``bsa_forward``: Q, K, V are bf16 CUDA tensors ``[heads, N, d]``; returns ``(O, LSE)``."""
         import torch
-        assert Q.is_cuda and Q.dtype == torch.bfloat16 and Q.is_contiguous()
-        assert K.is_contiguous() and V.is_contiguous() and K.dtype == V.dtype == torch.bfloat16
+        assert Q.is_cuda and Q.dtype in (torch.bfloat16, torch.float16) and Q.is_contiguous()  # as the plan's dtype
+        assert K.is_contiguous() and V.is_contiguous() and K.dtype == V.dtype == Q.dtype
         if O is None:
             O = torch.empty_like(Q)
         if LSE is None:
@@ -209,13 +212,13 @@ class Plan:
 
 
 def plan_create(mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1,
-                max_workspace_bytes: int = 0, stream=None, N_kv: int = 0) -> Plan:
+                max_workspace_bytes: int = 0, stream=None, N_kv: int = 0, dtype: str = "bf16") -> Plan:
     """``bsa_plan_create_ex``: ``mask`` is a uint8/bool CUDA tensor ``[heads, nQb, nKb]``; ``N_kv`` > 0 gives K and V
-    that many tokens per head (Q, O, LSE keep ``N``)."""
+    that many tokens per head (Q, O, LSE keep ``N``); ``dtype`` "fp16" prepares the plan for half tensors."""
     import torch
     assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool)
     h = ctypes.c_void_p()
-    opt = Options(plan_id, 0, max_workspace_bytes, N_kv)
+    opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv)
     _check(lib().bsa_plan_create_ex(mask.data_ptr(), B_Q, B_KV, N, heads, d, ctypes.byref(opt), _stream_ptr(stream),
                                     ctypes.byref(h)), "bsa_plan_create")
     return Plan(h.value)
@@ -238,12 +241,12 @@ def pack_mask(mask):
 
 
 def plan_create_packed(mask_bits, row_stride: int, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1,
-                       max_workspace_bytes: int = 0, stream=None, N_kv: int = 0) -> Plan:
+                       max_workspace_bytes: int = 0, stream=None, N_kv: int = 0, dtype: str = "bf16") -> Plan:
     """``bsa_plan_create_packed``: ``mask_bits`` is a uint8 CUDA tensor of bit-packed rows (see ``pack_mask``)."""
     import torch
     assert mask_bits.is_cuda and mask_bits.is_contiguous() and mask_bits.dtype == torch.uint8
     h = ctypes.c_void_p()
-    opt = Options(plan_id, 0, max_workspace_bytes, N_kv)
+    opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv)
     _check(lib().bsa_plan_create_packed(mask_bits.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
                                         _stream_ptr(stream), ctypes.byref(h)), "bsa_plan_create_packed")
     return Plan(h.value)
@@ -258,14 +261,14 @@ class PlanCache:
         self._h = h.value
 
     def get(self, mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1, max_workspace_bytes: int = 0,
-            stream=None, row_stride: int = 0, N_kv: int = 0):
+            stream=None, row_stride: int = 0, N_kv: int = 0, dtype: str = "bf16"):
         """``bsa_plan_cache_get``: returns ``(plan, hit)``.  ``row_stride`` > 0: ``mask`` is bit-packed (``pack_mask``).
         The plan is shared with the cache; ``plan.destroy()`` only gives it back."""
         import torch
         assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool)
         h = ctypes.c_void_p()
         hit = ctypes.c_int(0)
-        opt = Options(plan_id, 0, max_workspace_bytes, N_kv)
+        opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv)
         _check(lib().bsa_plan_cache_get(self._h, mask.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
                                         _stream_ptr(stream), ctypes.byref(h), ctypes.byref(hit)), "bsa_plan_cache_get")
         return Plan(h.value), bool(hit.value)
@@ -290,12 +293,12 @@ class PlanCache:
 
 
 def request_host(mask: np.ndarray, B_Q: int, B_KV: int, N: int, heads: int, d: int, Q, K, V, O, LSE,
-                 plan_id: int = -1, N_kv: int = 0) -> Dict:
+                 plan_id: int = -1, N_kv: int = 0, dtype: str = "bf16") -> Dict:
     """``bsa_request_host``: all arguments are HOST buffers (torch CPU tensors or numpy arrays)."""
     def ptr(x):
         return x.data_ptr() if hasattr(x, "data_ptr") else x.ctypes.data
     inf = PlanInfo()
-    opt = Options(plan_id, 0, 0, N_kv)
+    opt = Options(plan_id, DTYPES[dtype], 0, N_kv)
     _check(lib().bsa_request_host(ptr(mask), B_Q, B_KV, N, heads, d, ptr(Q), ptr(K), ptr(V), ptr(O), ptr(LSE),
                                   ctypes.byref(opt), ctypes.byref(inf)), "bsa_request_host")
     return inf.as_dict()

@@ -17,7 +17,8 @@ namespace bsa {
 const bsa_plan_desc_t* catalog_entry(int plan_id);
 bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int64_t N_kv, int heads, MapGeom* g);
 int64_t plan_workspace_bytes(const bsa_plan_desc_t& P, int64_t N, int heads, int d);
-bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws, int64_t N_kv = 0);
+bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws, int64_t N_kv = 0,
+                   int dtype = BSA_DTYPE_BF16);
 int base_plan(int B_Q, int B_KV, int d);
 uint64_t catalog_hash();
 void lut_buckets(int64_t N, double density, double skew, double run_cov, int32_t out[4]);
@@ -27,7 +28,7 @@ bsa_status_t lut_load(const char* path);
 void set_force_plan(int id);
 int get_force_plan();
 int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_cov, double skew,
-               int64_t max_ws, int* hit_out, int32_t buckets_out[4], int64_t N_kv = 0);
+               int64_t max_ws, int* hit_out, int32_t buckets_out[4], int64_t N_kv = 0, int dtype = BSA_DTYPE_BF16);
 int catalog_size();
 
 static std::atomic<long long> g_launches{0};
@@ -55,6 +56,7 @@ struct bsa_plan {
     bsa_plan_desc_t desc;
     MapGeom g;
     int d;
+    int dtype;  // BSA_DTYPE_*
     int stages;
     cudaStream_t stream;
     int device;
@@ -99,7 +101,7 @@ namespace {
 struct CacheKey {
     uint64_t hash[2];
     int64_t N, N_kv, packed_stride, max_ws;
-    int32_t B_Q, B_KV, heads, d, align, force, device;
+    int32_t B_Q, B_KV, heads, d, align, force, device, dtype;
     uint32_t generation;
     bool operator==(const CacheKey& o) const { return memcmp(this, &o, sizeof *this) == 0; }
 };
@@ -162,6 +164,8 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     if (vs != BSA_OK) return vs;
     const int64_t N_kv = request_n_kv(options, N);
     if (N_kv > (1ll << 30)) return BSA_ERR_UNSUPPORTED;
+    const int dtype = options ? options->dtype : BSA_DTYPE_BF16;
+    if (dtype != BSA_DTYPE_BF16 && dtype != BSA_DTYPE_FP16) return BSA_ERR_UNSUPPORTED;
     if (packed_stride > 0) {
         const int64_t nKb64 = (N_kv + B_KV - 1) / B_KV;
         if (packed_stride % 4 != 0 || packed_stride * 8 < nKb64 || (reinterpret_cast<uintptr_t>(mask_dev) & 3u))
@@ -176,6 +180,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     p->refs.store(1, std::memory_order_relaxed);
     p->stream = stream;
     p->d = d;
+    p->dtype = dtype;
     BSA_CUDA(cudaGetDevice(&p->device), "cudaGetDevice");
     BSA_CUDA(cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, p->device), "device attribute");
     {
@@ -271,7 +276,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
         key.N = N; key.N_kv = N_kv; key.packed_stride = packed_stride; key.max_ws = max_ws;
         key.B_Q = B_Q; key.B_KV = B_KV; key.heads = heads; key.d = d;
         key.align = packed_stride > 0 ? 0 : (int32_t)(reinterpret_cast<uintptr_t>(mask_dev) & 15u);
-        key.force = forced; key.device = p->device;
+        key.force = forced; key.device = p->device; key.dtype = dtype;
         key.generation = g_select_generation.load(std::memory_order_relaxed);
         bsa_plan* found = nullptr;
         {
@@ -311,11 +316,11 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     const double skew = nnz > 0 ? (double)p->hstats.max_row_nnz / (nnz / (double)nrows) : 0.0;
     int plan_id;
     if (forced >= 0) {
-        plan_id = plan_eligible(forced, B_Q, B_KV, N, heads, d, max_ws, N_kv) ? forced : -1;
+        plan_id = plan_eligible(forced, B_Q, B_KV, N, heads, d, max_ws, N_kv, dtype) ? forced : -1;
         lut_buckets(N, density, skew, run_cov, p->buckets);
         p->lut_hit = 0;
     } else {
-        plan_id = lut_select(B_Q, B_KV, N, heads, d, density, run_cov, skew, max_ws, &p->lut_hit, p->buckets, N_kv);
+        plan_id = lut_select(B_Q, B_KV, N, heads, d, density, run_cov, skew, max_ws, &p->lut_hit, p->buckets, N_kv, dtype);
     }
     if (plan_id < 0) { free_plan(p); return BSA_ERR_NO_ELIGIBLE_PLAN; }
     p->desc = *catalog_entry(plan_id);
@@ -495,6 +500,7 @@ extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const vo
     a.max_items = (int32_t)(p->max_items < (1 << 30) ? p->max_items : (1 << 30));
     a.max_split_rows = p->g.H * p->g.nQt * p->g.slots;
     a.num_sms = p->num_sms;
+    a.f16 = p->dtype == BSA_DTYPE_FP16;
     const char* detail = "launch";
     cudaError_t e = launch_forward(a, reinterpret_cast<cudaStream_t>(stream_v), &detail);
     if (e != cudaSuccess) {
@@ -530,7 +536,7 @@ extern "C" bsa_status_t bsa_plan_get_info(const bsa_plan_t* p, bsa_plan_info_t* 
     const MapGeom& g = p->g;
     info->map_q = g.sQ > 1 ? BSA_MAP_COARSENED : (g.rq > 1 ? BSA_MAP_REFINED : BSA_MAP_DIRECT);
     info->map_kv = g.sK > 1 ? BSA_MAP_COARSENED : (g.rk > 1 ? BSA_MAP_REFINED : BSA_MAP_DIRECT);
-    info->heads = g.H; info->d = p->d; info->B_Q = g.B_Q; info->B_KV = g.B_KV; info->N = g.N; info->N_kv = g.N_kv;
+    info->heads = g.H; info->d = p->d; info->B_Q = g.B_Q; info->B_KV = g.B_KV; info->N = g.N; info->N_kv = g.N_kv; info->dtype = p->dtype;
     info->nQb = g.nQb; info->nKb = g.nKb; info->nQt = g.nQt; info->nKt = g.nKt;
     info->member_bits = g.sQ128 * g.sK;
     info->member_words = g.slots;

@@ -1369,7 +1369,7 @@ struct __align__(8) PpBarriers {
     uint64_t s_full[2], s_free[2], p_ready[2], pv_done[2];
 };
 
-template <int D, int TK>
+template <int D, int TK, bool F16>
 __global__ void __launch_bounds__(kPpThreads, 1)
 bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                         const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
@@ -1505,7 +1505,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                             uint32_t v[8];
 #pragma unroll
                             for (int e = 0; e < 8; ++e)
-                                v[e] = pack_bf16x2(__uint_as_float(o[q * 16 + 2 * e]) * inv_l,
+                                v[e] = pack_16x2<F16>(__uint_as_float(o[q * 16 + 2 * e]) * inv_l,
                                                    __uint_as_float(o[q * 16 + 2 * e + 1]) * inv_l);
                             st_global_v8(orow + c * 32 + q * 16, v);
                         }
@@ -1637,7 +1637,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             }
         } else if (warp == 9 && lane == 0) {
             // =========================== Q K^T issuer ===========================
-            constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
+            constexpr uint32_t idesc_qk = make_idesc_f32(kTQ, TK, 0, 0, F16);
             const uint64_t descQ0 = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
             const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
             RingPos ring;  // K ring position of the tile being issued
@@ -1682,7 +1682,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             }
         } else if (warp == 10 && lane == 0) {
             // =========================== P V issuer ===========================
-            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            constexpr uint32_t idesc_pv = make_idesc_f32(kTQ, D, 0, 1, F16);
             const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
             RingPos ring;  // V ring position of the tile being issued
             uint32_t itq = 0, g = 0;
@@ -1892,8 +1892,8 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
                     sum01 = add_f32x2(sum01, pack_f32x2(p0, p1));
                     sum23 = add_f32x2(sum23, pack_f32x2(p2, p3));
-                    r[i / 2] = pack_bf16x2(p0, p1);
-                    r[i / 2 + 1] = pack_bf16x2(p2, p3);
+                    r[i / 2] = pack_16x2<F16>(p0, p1);
+                    r[i / 2 + 1] = pack_16x2<F16>(p2, p3);
                     if (kStoreInLoop && (i & 31) == 28) tmem_st16(t_p + (i >> 5) * 16, &r[(i >> 5) * 16]);
                 }
                 float s0, s1, s2, s3;
@@ -1974,8 +1974,9 @@ template <int D>
 __global__ void __launch_bounds__(256) bsa_merge_kernel(const SplitRow* __restrict__ split_rows,
                                                          const PlanCountersDev* __restrict__ counters,
                                                          const float* __restrict__ ws_O, const float* __restrict__ ws_LSE,
-                                                         __nv_bfloat16* __restrict__ O, float* __restrict__ LSE, int N) {
-    constexpr int GROUPS = D / 8;                   // 8 output columns (16 bytes of bf16) per thread
+                                                         __nv_bfloat16* __restrict__ O, float* __restrict__ LSE, int N,
+                                                         int f16) {
+    constexpr int GROUPS = D / 8;                   // 8 output columns (16 bytes of bf16 or fp16) per thread
     constexpr int CHUNKS = kTQ * GROUPS / 256;      // CTAs' worth of work per merged 128-row tile
     const int n_units = counters->nsplit_rows * CHUNKS;
     for (int cu = blockIdx.x; cu < n_units; cu += gridDim.x) {
@@ -2009,10 +2010,17 @@ __global__ void __launch_bounds__(256) bsa_merge_kernel(const SplitRow* __restri
         }
         const float inv = (tot > 0.f) ? 1.f / tot : 0.f;
         uint4 v;
-        v.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-        v.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
-        v.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
-        v.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+        if (f16) {
+            v.x = pack_f16x2(acc[0] * inv, acc[1] * inv);
+            v.y = pack_f16x2(acc[2] * inv, acc[3] * inv);
+            v.z = pack_f16x2(acc[4] * inv, acc[5] * inv);
+            v.w = pack_f16x2(acc[6] * inv, acc[7] * inv);
+        } else {
+            v.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+            v.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+            v.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
+            v.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+        }
         *reinterpret_cast<uint4*>(O + ((size_t)s.head * N + row) * D + gcol) = v;
         if (gcol == 0) LSE[(size_t)s.head * N + row] = (tot > 0.f) ? m_use + logf(tot) : -INFINITY;
     }
@@ -2052,14 +2060,15 @@ bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, i
 
 // The same tensor as {64 columns, N rows, d/64 column groups, heads}; box = {64, rows, d/64, 1}: one copy lands all
 // 64-column sub-tiles of a row block back to back (the [sub-tile][row][64] layout the MMA descriptors address).
-bool encode_map4(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows) {
+bool encode_map4(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows, bool f16 = false) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
     cuuint64_t dims[4] = {64, (cuuint64_t)N, (cuuint64_t)(d / 64), (cuuint64_t)heads};
     cuuint64_t strides[3] = {(cuuint64_t)d * 2, 128, (cuuint64_t)N * (cuuint64_t)d * 2};
     cuuint32_t box[4] = {64, (cuuint32_t)box_rows, (cuuint32_t)(d / 64), 1};
     cuuint32_t es[4] = {1, 1, 1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+    return enc(m, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+               strides, box, es,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -2068,8 +2077,9 @@ template <int D, int TK, int KERNEL>
 cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t stream, const char** err) {
     CUtensorMap tq, tk, tv;
     const bool ok_maps = (KERNEL == 4)
-                             ? (encode_map4(&tq, a.Q, a.g.N, a.g.H, D, kTQ) && encode_map4(&tk, a.K, a.g.N_kv, a.g.H, D, TK) &&
-                                encode_map4(&tv, a.V, a.g.N_kv, a.g.H, D, TK))
+                             ? (encode_map4(&tq, a.Q, a.g.N, a.g.H, D, kTQ, a.f16) &&
+                                encode_map4(&tk, a.K, a.g.N_kv, a.g.H, D, TK, a.f16) &&
+                                encode_map4(&tv, a.V, a.g.N_kv, a.g.H, D, TK, a.f16))
                              : (encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ) && encode_map(&tk, a.K, a.g.N_kv, a.g.H, D, TK) &&
                                 encode_map(&tv, a.V, a.g.N_kv, a.g.H, D, TK));
     if (!ok_maps) {
@@ -2077,6 +2087,10 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
         return cudaErrorInvalidValue;
     }
     const int smem = attention_smem_bytes(D, TK, a.stages, KERNEL);
+    if (a.f16 && KERNEL != 4) {  // only the ping-pong kernel is instantiated for half inputs (eligibility says so too)
+        *err = "fp16 inputs need a ping-pong-kernel plan";
+        return cudaErrorInvalidValue;
+    }
     static int attr_bytes = 0;  // per instantiation; grows to the largest request seen
     if (smem > attr_bytes) {
         cudaError_t e;
@@ -2088,8 +2102,11 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
             e = cudaFuncSetAttribute(bsa_attention_pair_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         else if (KERNEL == 2)
             e = cudaFuncSetAttribute(bsa_attention_cs_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        else
-            e = cudaFuncSetAttribute(bsa_attention_pp_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        else {
+            e = cudaFuncSetAttribute(bsa_attention_pp_kernel<D, TK, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(bsa_attention_pp_kernel<D, TK, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        }
         if (e != cudaSuccess) {
             *err = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
@@ -2107,7 +2124,8 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
     else if (KERNEL == 2)
         bsa_attention_cs_kernel<D, TK><<<grid, kCsThreads, smem, stream>>>(tq, tk, tv, p);
     else
-        bsa_attention_pp_kernel<D, TK><<<grid, kPpThreads, smem, stream>>>(tq, tk, tv, p);
+        (a.f16 ? bsa_attention_pp_kernel<D, TK, true> : bsa_attention_pp_kernel<D, TK, false>)
+            <<<grid, kPpThreads, smem, stream>>>(tq, tk, tv, p);
     count_launch();
     return cudaGetLastError();
 }
@@ -2217,10 +2235,10 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
         if (grid < 1) grid = 1;
         if (a.d == 128)
             bsa_merge_kernel<128><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
-                                                            reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N);
+                                                            reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16);
         else
             bsa_merge_kernel<64><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
-                                                           reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N);
+                                                           reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16);
         count_launch();
         e = cudaGetLastError();
     }

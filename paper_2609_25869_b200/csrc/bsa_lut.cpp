@@ -109,9 +109,12 @@ int64_t plan_workspace_bytes(const bsa_plan_desc_t& P, int64_t N, int heads, int
 }
 
 // Eligible(P, R), Section 4.4: logical geometry, tensor properties, metadata format, workspace.
-bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws, int64_t N_kv = 0) {
+bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws, int64_t N_kv = 0,
+                   int dtype = BSA_DTYPE_BF16) {
     const bsa_plan_desc_t* P = catalog_entry(plan_id);
     if (!P) return false;
+    if (dtype != BSA_DTYPE_BF16 && dtype != BSA_DTYPE_FP16) return false;
+    if (dtype == BSA_DTYPE_FP16 && P->kernel != 4) return false;  // tensor property: only the ping-pong kernel takes half
     if (!(d == 64 || d == 128)) return false;
     if (!pow2_in(B_Q, 16, 256) || !pow2_in(B_KV, 16, 256)) return false;
     if (N <= 0 || heads <= 0 || N > (1ll << 30)) return false;
@@ -260,7 +263,7 @@ int get_force_plan() { return g_force_plan; }
 
 // Algorithm 2, lines 6-19: z = <k, u, s>; r = rho(z); ranked list or base plan; first eligible.
 int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_cov, double skew,
-               int64_t max_ws, int* hit_out, int32_t buckets_out[4], int64_t N_kv = 0) {
+               int64_t max_ws, int* hit_out, int32_t buckets_out[4], int64_t N_kv = 0, int dtype = BSA_DTYPE_BF16) {
     int32_t b[4];
     lut_buckets(N, density, skew, run_cov, b);
     if (buckets_out) memcpy(buckets_out, b, sizeof b);
@@ -282,7 +285,7 @@ int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, d
     if (!hit) ranked.push_back(base_plan(B_Q, B_KV, d));
     if (hit_out) *hit_out = hit ? 1 : 0;
     for (int id : ranked)
-        if (plan_eligible(id, B_Q, B_KV, N, heads, d, max_ws, N_kv)) return id;
+        if (plan_eligible(id, B_Q, B_KV, N, heads, d, max_ws, N_kv, dtype)) return id;
     return -1;
 }
 

@@ -164,14 +164,18 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uin
 }
 // Instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation.
 // b_mn_major = 1 when B is stored with its N dimension contiguous (V in PV).
-__host__ __device__ constexpr uint32_t make_idesc_bf16_f32(int M, int N, int a_mn_major, int b_mn_major) {
+// `f16` = true: A and B are IEEE half (format code 0) instead of bf16 (format code 1).
+__host__ __device__ constexpr uint32_t make_idesc_f32(int M, int N, int a_mn_major, int b_mn_major, bool f16) {
     return (1u << 4)                        // D format: f32
-           | (1u << 7)                      // A format: bf16
-           | (1u << 10)                     // B format: bf16
+           | ((f16 ? 0u : 1u) << 7)         // A format
+           | ((f16 ? 0u : 1u) << 10)        // B format
            | (uint32_t(a_mn_major) << 15)   // A major
            | (uint32_t(b_mn_major) << 16)   // B major
            | (uint32_t(N >> 3) << 17)       // N / 8
            | (uint32_t(M >> 4) << 24);      // M / 16
+}
+__host__ __device__ constexpr uint32_t make_idesc_bf16_f32(int M, int N, int a_mn_major, int b_mn_major) {
+    return make_idesc_f32(M, N, a_mn_major, b_mn_major, false);
 }
 
 // ---------------------------------------------------------------- tcgen05: MMA (one thread issues)
@@ -298,6 +302,16 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// two fp32 values to the 16-bit input/output type of a kernel instantiation
+template <bool F16>
+__device__ __forceinline__ uint32_t pack_16x2(float lo, float hi) {
+    return F16 ? pack_f16x2(lo, hi) : pack_bf16x2(lo, hi);
 }
 
 }  // namespace ptx

@@ -115,7 +115,7 @@ def compare_with_oracle(req, O, LSE, qkv_cpu, sel=None, row_step=1, guards=True)
     if sel is None:
         sel = [(h, b) for h in range(req.H) for b in range(req.nQb)]
     oO, oL, pairs = oracle.attention_blocks(req.mask, req.B_Q, req.B_KV, req.N, req.d, Qb, Kb, Vb, sel, row_step,
-                                            N_kv=req.n_kv)
+                                            N_kv=req.n_kv, dtype=req.dtype)
     dO, dL = [], []
     for n, (h, b) in enumerate(sel):
         r0 = b * req.B_Q
@@ -138,7 +138,8 @@ def compare_with_oracle(req, O, LSE, qkv_cpu, sel=None, row_step=1, guards=True)
 
 def run_request(req, plan_id=-1, qkv=None, sel=None, row_step=1, structure=True, heads=None, guards=True):
     mask, q, k, v, qkv_cpu = to_dev(req, qkv)
-    with bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=plan_id, N_kv=req.N_kv) as plan:
+    with bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=plan_id, N_kv=req.N_kv,
+                         dtype=req.dtype) as plan:
         O, LSE = plan.forward(q, k, v)
         torch.cuda.synchronize()
         inf = plan.info()
