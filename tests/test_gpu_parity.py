@@ -377,6 +377,47 @@ def test_half_precision_mid_and_ineligible_plans():
         assert not torch.equal(Oh.view(torch.int16), Ob.view(torch.int16))
 
 
+# ---------------------------------------------------------------- seeded random requests
+def _random_request(n):
+    """Request n of a seeded family: geometry, token counts (ragged, N_q != N_kv in a third of the cases), head
+    dimension, element type, mask structure (Bernoulli, runs, banded, with empty rows) and plan all follow from n."""
+    r = np.random.RandomState(1000 + n)
+    B_Q, B_KV = (int(2 ** r.randint(4, 9)) for _ in range(2))
+    d = int(r.choice([64, 128]))
+    dtype = "fp16" if r.rand() < 0.3 else "bf16"
+    H = int(r.randint(1, 5))
+    N = int(r.randint(1, 5000))
+    N_kv = int(r.randint(1, 5000)) if r.rand() < 0.35 else 0
+    nQb, nKb = I.cdiv(N, B_Q), I.cdiv(N_kv or N, B_KV)
+    kind = r.randint(0, 3)
+    if kind == 0:
+        M = I.random_mask(n, H, nQb, nKb, float(r.choice([0.05, 0.3, 0.7, 1.0])), empty_rows=float(r.choice([0.0, 0.2])))
+    elif kind == 1:   # a band around the (scaled) diagonal plus a few full columns
+        i, j = np.meshgrid(np.arange(nQb), np.arange(nKb), indexing="ij")
+        band = np.abs(i * nKb - j * nQb) <= int(r.randint(1, 4)) * max(nQb, nKb)
+        M = np.repeat(band[None], H, axis=0).astype(np.uint8)
+        M[:, :, r.randint(0, nKb, size=2)] = 1
+    else:             # contiguous runs
+        M = np.zeros((H, nQb, nKb), dtype=np.uint8)
+        for h in range(H):
+            for q in range(nQb):
+                for _ in range(int(r.randint(0, 4))):
+                    a = int(r.randint(0, nKb))
+                    M[h, q, a:a + int(r.randint(1, 9))] = 1
+    cat = bsa.catalog()
+    ok = [c["plan_id"] for c in cat if (dtype == "bf16" or c["kernel"] == 4) and
+          bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d)]
+    plan_id = -1 if r.rand() < 0.3 else int(r.choice(ok))
+    return I.Request(f"random{n}", H, N, d, B_Q, B_KV, M, qkv_seed=300 + n, N_kv=N_kv, dtype=dtype), plan_id
+
+
+@pytest.mark.parametrize("n", range(96))
+def test_random_requests_match_the_oracle(n):
+    req, plan_id = _random_request(n)
+    nsel = min(req.nQb, max(1, 600 // req.B_Q))
+    Hh.run_request(req, plan_id=plan_id, sel=_sample(req, nsel), guards=False)
+
+
 def test_plan_cache_reuses_the_plan_of_a_repeated_mask():
     """Warm path: the second request with the same mask gets the SAME prepared plan (one statistics kernel and one
     row scan launched, nothing else), its output matches the oracle and an uncached plan bit for bit; any change of
