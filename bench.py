@@ -291,6 +291,8 @@ def main():
     ap.add_argument("--extra", default="", help="comma list of extra workloads reported under 'others'")
     ap.add_argument("--sweep-requests", type=int, default=50)
     ap.add_argument("--sweep-heads", type=int, default=24)
+    ap.add_argument("--shard-heads", action="store_true",
+                    help="strong scaling: ONE request, its heads split over the ranks (no collective on the data path)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -323,8 +325,17 @@ def main():
         torch.cuda.synchronize()
 
     def bench_workload(name, steps, warmup, with_e2e):
-        req = make_request(name, rank)
+        req = make_request(name, 0 if args.shard_heads else rank)
         q, k, v = req.qkv()
+        if args.shard_heads:  # every rank builds the same request and keeps its own contiguous range of heads
+            import dataclasses
+            from paper_2609_25869_b200 import shard
+            lo, hi = shard.head_range(req.H, rank, world)
+            if hi == lo:
+                raise SystemExit(f"--shard-heads: {req.H} heads cannot feed {world} ranks")
+            q, k, v = (t[lo:hi].contiguous() for t in (q, k, v))
+            req = dataclasses.replace(req, H=hi - lo, mask=req.mask[lo:hi].copy(),
+                                      note=req.note + f"; heads {lo}-{hi - 1} of {req.H} on this rank")
         mask_d = torch.from_numpy(req.mask).cuda()
         qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
         O = torch.empty_like(qd)
@@ -442,7 +453,8 @@ def main():
         "metric": "effective TFLOP/s on active blocks (4*d flops per active token pair), whole request: "
                   "plan create + forward",
         "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "strong" if args.shard_heads else "weak",
+        "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic", "config": workload_config(req, args.workload),
         "clocks": r["clocks"],
         "e2e": {"value": world * r["flops"] / e2e_s / 1e12, "unit": "TFLOP/s",

@@ -36,6 +36,45 @@ def _rank_main(rank, world, port, q):
     dist.destroy_process_group()
 
 
+def _shard_rank_main(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    from paper_2609_25869_b200 import shard
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    H = 5  # uneven: rank 0 gets 3 heads, rank 1 gets 2
+    lo, hi = shard.head_range(H, rank, world)
+    full = torch.arange(H * 4 * 3, dtype=torch.float32).reshape(H, 4, 3)
+    got = shard.all_gather_heads(full[lo:hi].clone(), H, dist)
+    q.put((rank, (lo, hi), bool(torch.equal(got, full))))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_head_sharding_ranges_and_gather_with_gloo():
+    """Head-sharded driver, host side: ranges partition the heads for every (H, world), and the padded all-gather
+    puts uneven shards back together on both ranks."""
+    sys.path.insert(0, ROOT)
+    from paper_2609_25869_b200 import shard
+    for H in range(0, 40):
+        for world in range(1, 10):
+            rs = shard.head_ranges(H, world)
+            assert rs[0][0] == 0 and rs[-1][1] == H
+            assert all(a[1] == b[0] for a, b in zip(rs[:-1], rs[1:]))
+            sizes = [hi - lo for lo, hi in rs]
+            assert max(sizes) - min(sizes) <= 1 and sizes == sorted(sizes, reverse=True)
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 31500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_shard_rank_main, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res == [(0, (0, 3), True), (1, (3, 5), True)]
+
+
 def test_two_rank_aggregation_with_gloo():
     ctx = mp.get_context("spawn")
     q = ctx.Queue()

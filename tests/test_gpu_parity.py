@@ -377,6 +377,30 @@ def test_half_precision_mid_and_ineligible_plans():
         assert not torch.equal(Oh.view(torch.int16), Ob.view(torch.int16))
 
 
+def test_head_sharded_forward_equals_the_unsharded_one():
+    """Heads are independent: three ranks' worth of head ranges, run one after the other on this GPU through the
+    sharded driver, give the same bits as the whole request under the same plan."""
+    from paper_2609_25869_b200 import shard
+    req = I.config_tiny()
+    H = 5
+    M = I.random_mask(71, H, req.nQb, req.nKb, 0.3, empty_rows=0.1)
+    req = I.Request("sharded", H, req.N, req.d, req.B_Q, req.B_KV, M, qkv_seed=29)
+    mask, q, k, v, qkv_cpu = Hh.to_dev(req)
+    with bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, H, req.d, plan_id=22) as plan:
+        O, LSE = plan.forward(q, k, v)
+        torch.cuda.synchronize()
+    Hh.compare_with_oracle(req, O, LSE, qkv_cpu)
+    parts = []
+    for lo, hi in shard.head_ranges(H, 3):
+        Ol, Ll, info = shard.forward_local(mask[lo:hi].contiguous(), q[lo:hi].contiguous(), k[lo:hi].contiguous(),
+                                           v[lo:hi].contiguous(), req.B_Q, req.B_KV, req.N, req.d, plan_id=22)
+        assert info["heads"] == hi - lo
+        parts.append((Ol, Ll))
+    assert torch.equal(torch.cat([p[0] for p in parts]), O) and torch.equal(torch.cat([p[1] for p in parts]), LSE)
+    E, L0, none = shard.forward_local(mask[:0], q[:0], k[:0], v[:0], req.B_Q, req.B_KV, req.N, req.d)
+    assert E.shape[0] == 0 and L0.shape == (0, req.N) and none is None
+
+
 # ---------------------------------------------------------------- seeded random requests
 def _random_request(n):
     """Request n of a seeded family: geometry, token counts (ragged, N_q != N_kv in a third of the cases), head
