@@ -69,6 +69,11 @@ typedef struct bsa_plan_desc {
  * output accumulator are fp32 either way; P is rounded to the same 16-bit type for the second product.  Half inputs
  * are served by the plans of the ping-pong kernel only (the others are not eligible for such a request). */
 enum { BSA_DTYPE_BF16 = 0, BSA_DTYPE_FP16 = 1 };
+/* Storage layout of Q, K, V and O (another tensor property of the request, Section 3 / Section 4.4):
+ * [heads][N][d] (head-major, the default) or [N][heads][d] (token-major, what a fused QKV projection of a
+ * [batch, sequence, heads, d] model leaves behind).  Only strides change (tensor maps and output addressing); every
+ * catalog plan serves both.  LSE is [heads][N] either way. */
+enum { BSA_LAYOUT_HND = 0, BSA_LAYOUT_NHD = 1 };
 
 typedef struct bsa_options {
     int32_t force_plan_id;        /* >= 0: skip the lookup and use this catalog entry (still checked for
@@ -78,6 +83,8 @@ typedef struct bsa_options {
     int64_t N_kv;                 /* key/value tokens per head (Section 2.1: K, V are N_kv x d); <= 0: N_kv = N.
                                      The mask then has ceil(N_kv / B_KV) block columns, K and V are
                                      [heads, N_kv, d]; Q, O and LSE keep N rows.                      */
+    int32_t layout;               /* BSA_LAYOUT_*                                                     */
+    int32_t reserved2;
 } bsa_options_t;
 
 /* Scalar mask statistics s_A(M) (Section 5.1) and what launch preparation produced. */
@@ -109,7 +116,7 @@ typedef struct bsa_plan_info {
     int32_t device_status;        /* 0, or BSA_ERR_DEVICE_TIMEOUT if any forward hit a bounded wait  */
     int64_t N_kv;                 /* key/value tokens per head (= N unless the options said otherwise) */
     int32_t dtype;                /* BSA_DTYPE_* of the request                                        */
-    int32_t reserved1;
+    int32_t layout;               /* BSA_LAYOUT_* of the request                                       */
 } bsa_plan_info_t;
 
 /* ---------------------------------------------------------------------------------------------

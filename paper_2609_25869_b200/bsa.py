@@ -29,11 +29,13 @@ class PlanDesc(ctypes.Structure):
 
 
 DTYPES = {"bf16": 0, "fp16": 1}  # BSA_DTYPE_*
+LAYOUTS = {"hnd": 0, "nhd": 1}   # BSA_LAYOUT_*: [heads, N, d] or [N, heads, d]
 
 
 class Options(ctypes.Structure):
     _fields_ = [("force_plan_id", ctypes.c_int32), ("dtype", ctypes.c_int32),
-                ("max_workspace_bytes", ctypes.c_int64), ("N_kv", ctypes.c_int64)]
+                ("max_workspace_bytes", ctypes.c_int64), ("N_kv", ctypes.c_int64),
+                ("layout", ctypes.c_int32), ("reserved2", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -49,7 +51,7 @@ class PlanInfo(ctypes.Structure):
                 ("workspace_bytes", ctypes.c_int64), ("covered_pairs", ctypes.c_int64),
                 ("us_mask_state", ctypes.c_float), ("us_stats_sync", ctypes.c_float), ("us_lookup", ctypes.c_float),
                 ("us_launch_prep", ctypes.c_float), ("us_total", ctypes.c_float), ("device_status", ctypes.c_int32),
-                ("N_kv", ctypes.c_int64), ("dtype", ctypes.c_int32), ("reserved1", ctypes.c_int32)]
+                ("N_kv", ctypes.c_int64), ("dtype", ctypes.c_int32), ("layout", ctypes.c_int32)]
 
     def as_dict(self) -> Dict:
         out = {}
@@ -150,8 +152,9 @@ def _stream_ptr(stream) -> Optional[int]:
 class Plan:
     """Handle of a prepared plan (``bsa_plan_create`` ... ``bsa_plan_destroy``)."""
 
-    def __init__(self, handle: int):
+    def __init__(self, handle: int, layout: str = "hnd"):
         self._h = ctypes.c_void_p(handle)
+        self.layout = layout
 
     def forward(self, Q, K, V, O=None, LSE=None, stream=None):
         """``bsa_forward``: Q, K, V are bf16 CUDA tensors ``[heads, N, d]``; returns ``(O, LSE)``."""
@@ -160,8 +163,9 @@ class Plan:
         assert K.is_contiguous() and V.is_contiguous() and K.dtype == V.dtype == Q.dtype
         if O is None:
             O = torch.empty_like(Q)
-        if LSE is None:
-            LSE = torch.empty(Q.shape[:2], dtype=torch.float32, device=Q.device)
+        if LSE is None:  # [heads, N] whatever the layout of Q
+            hn = Q.shape[:2] if self.layout == "hnd" else (Q.shape[1], Q.shape[0])
+            LSE = torch.empty(hn, dtype=torch.float32, device=Q.device)
         _check(lib().bsa_forward(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
                                  _stream_ptr(stream)), "bsa_forward")
         return O, LSE
@@ -212,16 +216,17 @@ class Plan:
 
 
 def plan_create(mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1,
-                max_workspace_bytes: int = 0, stream=None, N_kv: int = 0, dtype: str = "bf16") -> Plan:
+                max_workspace_bytes: int = 0, stream=None, N_kv: int = 0, dtype: str = "bf16",
+                layout: str = "hnd") -> Plan:
     """``bsa_plan_create_ex``: ``mask`` is a uint8/bool CUDA tensor ``[heads, nQb, nKb]``; ``N_kv`` > 0 gives K and V
     that many tokens per head (Q, O, LSE keep ``N``); ``dtype`` "fp16" prepares the plan for half tensors."""
     import torch
     assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool)
     h = ctypes.c_void_p()
-    opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv)
+    opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv, LAYOUTS[layout], 0)
     _check(lib().bsa_plan_create_ex(mask.data_ptr(), B_Q, B_KV, N, heads, d, ctypes.byref(opt), _stream_ptr(stream),
                                     ctypes.byref(h)), "bsa_plan_create")
-    return Plan(h.value)
+    return Plan(h.value, layout)
 
 
 def pack_mask(mask):
@@ -241,15 +246,16 @@ def pack_mask(mask):
 
 
 def plan_create_packed(mask_bits, row_stride: int, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1,
-                       max_workspace_bytes: int = 0, stream=None, N_kv: int = 0, dtype: str = "bf16") -> Plan:
+                       max_workspace_bytes: int = 0, stream=None, N_kv: int = 0, dtype: str = "bf16",
+                       layout: str = "hnd") -> Plan:
     """``bsa_plan_create_packed``: ``mask_bits`` is a uint8 CUDA tensor of bit-packed rows (see ``pack_mask``)."""
     import torch
     assert mask_bits.is_cuda and mask_bits.is_contiguous() and mask_bits.dtype == torch.uint8
     h = ctypes.c_void_p()
-    opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv)
+    opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv, LAYOUTS[layout], 0)
     _check(lib().bsa_plan_create_packed(mask_bits.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
                                         _stream_ptr(stream), ctypes.byref(h)), "bsa_plan_create_packed")
-    return Plan(h.value)
+    return Plan(h.value, layout)
 
 
 class PlanCache:
@@ -261,17 +267,17 @@ class PlanCache:
         self._h = h.value
 
     def get(self, mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1, max_workspace_bytes: int = 0,
-            stream=None, row_stride: int = 0, N_kv: int = 0, dtype: str = "bf16"):
+            stream=None, row_stride: int = 0, N_kv: int = 0, dtype: str = "bf16", layout: str = "hnd"):
         """``bsa_plan_cache_get``: returns ``(plan, hit)``.  ``row_stride`` > 0: ``mask`` is bit-packed (``pack_mask``).
         The plan is shared with the cache; ``plan.destroy()`` only gives it back."""
         import torch
         assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool)
         h = ctypes.c_void_p()
         hit = ctypes.c_int(0)
-        opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv)
+        opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv, LAYOUTS[layout], 0)
         _check(lib().bsa_plan_cache_get(self._h, mask.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
                                         _stream_ptr(stream), ctypes.byref(h), ctypes.byref(hit)), "bsa_plan_cache_get")
-        return Plan(h.value), bool(hit.value)
+        return Plan(h.value, layout), bool(hit.value)
 
     def stats(self) -> Dict:
         a, b, c = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
@@ -293,12 +299,12 @@ class PlanCache:
 
 
 def request_host(mask: np.ndarray, B_Q: int, B_KV: int, N: int, heads: int, d: int, Q, K, V, O, LSE,
-                 plan_id: int = -1, N_kv: int = 0, dtype: str = "bf16") -> Dict:
+                 plan_id: int = -1, N_kv: int = 0, dtype: str = "bf16", layout: str = "hnd") -> Dict:
     """``bsa_request_host``: all arguments are HOST buffers (torch CPU tensors or numpy arrays)."""
     def ptr(x):
         return x.data_ptr() if hasattr(x, "data_ptr") else x.ctypes.data
     inf = PlanInfo()
-    opt = Options(plan_id, DTYPES[dtype], 0, N_kv)
+    opt = Options(plan_id, DTYPES[dtype], 0, N_kv, LAYOUTS[layout], 0)
     _check(lib().bsa_request_host(ptr(mask), B_Q, B_KV, N, heads, d, ptr(Q), ptr(K), ptr(V), ptr(O), ptr(LSE),
                                   ctypes.byref(opt), ctypes.byref(inf)), "bsa_request_host")
     return inf.as_dict()

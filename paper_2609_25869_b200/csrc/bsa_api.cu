@@ -57,6 +57,7 @@ struct bsa_plan {
     MapGeom g;
     int d;
     int dtype;  // BSA_DTYPE_*
+    int layout;  // BSA_LAYOUT_*
     int stages;
     cudaStream_t stream;
     int device;
@@ -101,7 +102,7 @@ namespace {
 struct CacheKey {
     uint64_t hash[2];
     int64_t N, N_kv, packed_stride, max_ws;
-    int32_t B_Q, B_KV, heads, d, align, force, device, dtype;
+    int32_t B_Q, B_KV, heads, d, align, force, device, dtype, layout, pad;
     uint32_t generation;
     bool operator==(const CacheKey& o) const { return memcmp(this, &o, sizeof *this) == 0; }
 };
@@ -166,6 +167,8 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     if (N_kv > (1ll << 30)) return BSA_ERR_UNSUPPORTED;
     const int dtype = options ? options->dtype : BSA_DTYPE_BF16;
     if (dtype != BSA_DTYPE_BF16 && dtype != BSA_DTYPE_FP16) return BSA_ERR_UNSUPPORTED;
+    const int layout = options ? options->layout : BSA_LAYOUT_HND;
+    if (layout != BSA_LAYOUT_HND && layout != BSA_LAYOUT_NHD) return BSA_ERR_UNSUPPORTED;
     if (packed_stride > 0) {
         const int64_t nKb64 = (N_kv + B_KV - 1) / B_KV;
         if (packed_stride % 4 != 0 || packed_stride * 8 < nKb64 || (reinterpret_cast<uintptr_t>(mask_dev) & 3u))
@@ -181,6 +184,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     p->stream = stream;
     p->d = d;
     p->dtype = dtype;
+    p->layout = layout;
     BSA_CUDA(cudaGetDevice(&p->device), "cudaGetDevice");
     BSA_CUDA(cudaDeviceGetAttribute(&p->num_sms, cudaDevAttrMultiProcessorCount, p->device), "device attribute");
     {
@@ -276,7 +280,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
         key.N = N; key.N_kv = N_kv; key.packed_stride = packed_stride; key.max_ws = max_ws;
         key.B_Q = B_Q; key.B_KV = B_KV; key.heads = heads; key.d = d;
         key.align = packed_stride > 0 ? 0 : (int32_t)(reinterpret_cast<uintptr_t>(mask_dev) & 15u);
-        key.force = forced; key.device = p->device; key.dtype = dtype;
+        key.force = forced; key.device = p->device; key.dtype = dtype; key.layout = layout;
         key.generation = g_select_generation.load(std::memory_order_relaxed);
         bsa_plan* found = nullptr;
         {
@@ -501,6 +505,7 @@ extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const vo
     a.max_split_rows = p->g.H * p->g.nQt * p->g.slots;
     a.num_sms = p->num_sms;
     a.f16 = p->dtype == BSA_DTYPE_FP16;
+    a.nhd = p->layout == BSA_LAYOUT_NHD;
     const char* detail = "launch";
     cudaError_t e = launch_forward(a, reinterpret_cast<cudaStream_t>(stream_v), &detail);
     if (e != cudaSuccess) {
@@ -536,7 +541,7 @@ extern "C" bsa_status_t bsa_plan_get_info(const bsa_plan_t* p, bsa_plan_info_t* 
     const MapGeom& g = p->g;
     info->map_q = g.sQ > 1 ? BSA_MAP_COARSENED : (g.rq > 1 ? BSA_MAP_REFINED : BSA_MAP_DIRECT);
     info->map_kv = g.sK > 1 ? BSA_MAP_COARSENED : (g.rk > 1 ? BSA_MAP_REFINED : BSA_MAP_DIRECT);
-    info->heads = g.H; info->d = p->d; info->B_Q = g.B_Q; info->B_KV = g.B_KV; info->N = g.N; info->N_kv = g.N_kv; info->dtype = p->dtype;
+    info->heads = g.H; info->d = p->d; info->B_Q = g.B_Q; info->B_KV = g.B_KV; info->N = g.N; info->N_kv = g.N_kv; info->dtype = p->dtype; info->layout = p->layout;
     info->nQb = g.nQb; info->nKb = g.nKb; info->nQt = g.nQt; info->nKt = g.nKt;
     info->member_bits = g.sQ128 * g.sK;
     info->member_words = g.slots;

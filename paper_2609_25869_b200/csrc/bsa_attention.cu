@@ -59,6 +59,7 @@ struct AttnParams {
     float* ws_O;
     float* ws_LSE;
     unsigned long long full_member;
+    int64_t o_head, o_row;  // element strides of O (and of Q) between heads and between token rows
     int32_t N;    // query tokens per head
     int32_t Nkv;  // key/value tokens per head
     int32_t lgBQ;   // log2(B_Q) when B_Q < 128, else 31 (row >> 31 == 0)
@@ -418,7 +419,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             if (it.ntiles == 0) {
                 // no physical tile touches this Q tile row: O = 0, LSE = -inf
                 if (row_ok) {
-                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D);
+                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.o_head + (size_t)row * p.o_row));
 #pragma unroll
                     for (int c = 0; c < D / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
                     p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
@@ -488,7 +489,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 const float lse = (l > 0.f) ? fmaf(m_ref, 0.6931471805599453f, logf(l)) : -INFINITY;
                 const uint32_t t_o = tmem + lane_base + kColO;
                 if (it.nparts == 1) {
-                    __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D;
+                    __nv_bfloat16* orow = p.O + ((size_t)it.head * p.o_head + (size_t)row * p.o_row);
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t r[32];
@@ -835,7 +836,7 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
                 // no tile of this item reaches this slot's rows: O = 0, LSE = -inf (or an empty partial state)
                 if (it.nparts == 1) {
                     if (row_ok) {
-                        uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D);
+                        uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.o_head + (size_t)row * p.o_row));
 #pragma unroll
                         for (int c = 0; c < D / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
                         p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
@@ -854,7 +855,7 @@ bsa_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_
             const float inv_l = (l > 0.f) ? 1.f / l : 0.f;
             const float lse = (l > 0.f) ? fmaf(m_ref, 0.6931471805599453f, logf(l)) : -INFINITY;
             if (it.nparts == 1) {
-                __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D;
+                __nv_bfloat16* orow = p.O + ((size_t)it.head * p.o_head + (size_t)row * p.o_row);
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t r[32];
@@ -1124,7 +1125,7 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             const bool row_ok = row < p.N;
             if (it.ntiles == 0) {
                 if (row_ok) {
-                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D + half * DC);
+                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.o_head + (size_t)row * p.o_row) + half * DC);
 #pragma unroll
                     for (int c = 0; c < DC / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
                     if (half == 0) p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
@@ -1240,7 +1241,7 @@ bsa_attention_cs_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const float lse = (l_tot > 0.f) ? fmaf(m_ref, 0.6931471805599453f, logf(l_tot)) : -INFINITY;
                 const uint32_t t_o = tmem + lane_base + kColO + half * DC;
                 if (it.nparts == 1) {
-                    __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D + half * DC;
+                    __nv_bfloat16* orow = p.O + ((size_t)it.head * p.o_head + (size_t)row * p.o_row) + half * DC;
 #pragma unroll
                     for (int c = 0; c < DC / 32; ++c) {
                         uint32_t o[32];
@@ -1463,7 +1464,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             if (it.ntiles < 0) continue;  // past the end of the list
             if (it.ntiles == 0) {  // no active column: zero output, LSE = -inf
                 if (row_ok) {
-                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.N + row) * D);
+                    uint4* o = reinterpret_cast<uint4*>(p.O + ((size_t)it.head * p.o_head + (size_t)row * p.o_row));
 #pragma unroll
                     for (int c = 0; c < D / 8; ++c) o[c] = make_uint4(0, 0, 0, 0);
                     p.LSE[(size_t)it.head * p.N + row] = -INFINITY;
@@ -1483,7 +1484,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             tc_fence_after();
             if (lane == 0) BSA_TRACE_POINT(11, tn, 31);
             ++itn;
-            __nv_bfloat16* orow = p.O + ((size_t)it.head * p.N + row) * D;
+            __nv_bfloat16* orow = p.O + ((size_t)it.head * p.o_head + (size_t)row * p.o_row);
             float* wrow = p.ws_O + ((size_t)it.ws_slot * kTQ + tw) * D;
 #pragma unroll 1  // once per item: a rolled loop keeps the kernel's code small
             for (int c = 0; c < D / 32; ++c) {
@@ -1975,7 +1976,7 @@ __global__ void __launch_bounds__(256) bsa_merge_kernel(const SplitRow* __restri
                                                          const PlanCountersDev* __restrict__ counters,
                                                          const float* __restrict__ ws_O, const float* __restrict__ ws_LSE,
                                                          __nv_bfloat16* __restrict__ O, float* __restrict__ LSE, int N,
-                                                         int f16) {
+                                                         int f16, long long o_head, long long o_row) {
     constexpr int GROUPS = D / 8;                   // 8 output columns (16 bytes of bf16 or fp16) per thread
     constexpr int CHUNKS = kTQ * GROUPS / 256;      // CTAs' worth of work per merged 128-row tile
     const int n_units = counters->nsplit_rows * CHUNKS;
@@ -2021,7 +2022,7 @@ __global__ void __launch_bounds__(256) bsa_merge_kernel(const SplitRow* __restri
             v.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
             v.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
         }
-        *reinterpret_cast<uint4*>(O + ((size_t)s.head * N + row) * D + gcol) = v;
+        *reinterpret_cast<uint4*>(O + ((size_t)s.head * o_head + (size_t)row * o_row) + gcol) = v;
         if (gcol == 0) LSE[(size_t)s.head * N + row] = (tot > 0.f) ? m_use + logf(tot) : -INFINITY;
     }
 }
@@ -2046,11 +2047,16 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // bf16 [heads][N][d] viewed as a 3-D tensor {d, N, heads}; box = {64, rows, 1}; rows beyond N read as zero.
-bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows) {
+// `nhd`: the tensor is stored [N][heads][d] instead (token-major); only the two byte strides change.
+bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows, bool nhd) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
     cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)heads};
     cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)N * (cuuint64_t)d * 2};
+    if (nhd) {
+        strides[0] = (cuuint64_t)heads * (cuuint64_t)d * 2;
+        strides[1] = (cuuint64_t)d * 2;
+    }
     cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t es[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
@@ -2060,11 +2066,15 @@ bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, i
 
 // The same tensor as {64 columns, N rows, d/64 column groups, heads}; box = {64, rows, d/64, 1}: one copy lands all
 // 64-column sub-tiles of a row block back to back (the [sub-tile][row][64] layout the MMA descriptors address).
-bool encode_map4(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows, bool f16 = false) {
+bool encode_map4(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows, bool f16, bool nhd) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
     cuuint64_t dims[4] = {64, (cuuint64_t)N, (cuuint64_t)(d / 64), (cuuint64_t)heads};
     cuuint64_t strides[3] = {(cuuint64_t)d * 2, 128, (cuuint64_t)N * (cuuint64_t)d * 2};
+    if (nhd) {
+        strides[0] = (cuuint64_t)heads * (cuuint64_t)d * 2;
+        strides[2] = (cuuint64_t)d * 2;
+    }
     cuuint32_t box[4] = {64, (cuuint32_t)box_rows, (cuuint32_t)(d / 64), 1};
     cuuint32_t es[4] = {1, 1, 1, 1};
     return enc(m, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
@@ -2077,11 +2087,12 @@ template <int D, int TK, int KERNEL>
 cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t stream, const char** err) {
     CUtensorMap tq, tk, tv;
     const bool ok_maps = (KERNEL == 4)
-                             ? (encode_map4(&tq, a.Q, a.g.N, a.g.H, D, kTQ, a.f16) &&
-                                encode_map4(&tk, a.K, a.g.N_kv, a.g.H, D, TK, a.f16) &&
-                                encode_map4(&tv, a.V, a.g.N_kv, a.g.H, D, TK, a.f16))
-                             : (encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ) && encode_map(&tk, a.K, a.g.N_kv, a.g.H, D, TK) &&
-                                encode_map(&tv, a.V, a.g.N_kv, a.g.H, D, TK));
+                             ? (encode_map4(&tq, a.Q, a.g.N, a.g.H, D, kTQ, a.f16, a.nhd) &&
+                                encode_map4(&tk, a.K, a.g.N_kv, a.g.H, D, TK, a.f16, a.nhd) &&
+                                encode_map4(&tv, a.V, a.g.N_kv, a.g.H, D, TK, a.f16, a.nhd))
+                             : (encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ, a.nhd) &&
+                                encode_map(&tk, a.K, a.g.N_kv, a.g.H, D, TK, a.nhd) &&
+                                encode_map(&tv, a.V, a.g.N_kv, a.g.H, D, TK, a.nhd));
     if (!ok_maps) {
         *err = "cuTensorMapEncodeTiled failed";
         return cudaErrorInvalidValue;
@@ -2194,6 +2205,8 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     p.full_member = (bits >= 64) ? ~0ull : ((1ull << bits) - 1ull);
     p.N = (int32_t)a.g.N;
     p.Nkv = (int32_t)a.g.N_kv;
+    p.o_head = a.nhd ? (int64_t)a.d : (int64_t)a.g.N * a.d;
+    p.o_row = a.nhd ? (int64_t)a.g.H * a.d : (int64_t)a.d;
     p.lgBQ = (a.g.sQ128 > 1) ? a.g.lgBQ : 31;
     p.lgBKV = (a.g.sK > 1) ? a.g.lgBKV : 31;
     p.sK = a.g.sK;
@@ -2235,10 +2248,10 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
         if (grid < 1) grid = 1;
         if (a.d == 128)
             bsa_merge_kernel<128><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
-                                                            reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16);
+                                                            reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16, p.o_head, p.o_row);
         else
             bsa_merge_kernel<64><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
-                                                           reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16);
+                                                           reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16, p.o_head, p.o_row);
         count_launch();
         e = cudaGetLastError();
     }

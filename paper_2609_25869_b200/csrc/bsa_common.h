@@ -114,6 +114,7 @@ struct ForwardArgs {
     int32_t max_split_rows;  // host-side upper bound
     int32_t num_sms;
     int32_t f16;             // 1: Q, K, V, O are IEEE half (ping-pong-kernel plans only); 0: bf16
+    int32_t nhd;             // 1: Q, K, V, O are stored [N][heads][d] (token-major); 0: [heads][N][d]
 };
 cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char** err_detail);
 // `stages` counts K buffers plus V buffers for the paired kernel (kernel 1), K = V ring depth for kernel 0

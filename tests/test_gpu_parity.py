@@ -377,6 +377,61 @@ def test_half_precision_mid_and_ineligible_plans():
         assert not torch.equal(Oh.view(torch.int16), Ob.view(torch.int16))
 
 
+# ---------------------------------------------------------------- token-major layout [N, heads, d]
+@pytest.mark.parametrize("B_Q,B_KV,N,N_kv,d,dtype", [(64, 64, 2048, 0, 64, "bf16"), (128, 128, 3000, 0, 128, "bf16"),
+                                                      (32, 64, 1500, 2600, 128, "bf16"), (128, 128, 2500, 0, 128, "fp16")])
+def test_token_major_layout_gives_the_same_output(B_Q, B_KV, N, N_kv, d, dtype):
+    """Q, K, V, O stored [N, heads, d] (the layout is a tensor property of the request): one plan per kernel family
+    and a Split-K plan give, permuted back, the bits of the head-major run; the first is also compared with the oracle."""
+    H = 3
+    M = I.random_mask(81, H, I.cdiv(N, B_Q), I.cdiv(N_kv or N, B_KV), 0.3, empty_rows=0.1)
+    req = I.Request("nhd", H, N, d, B_Q, B_KV, M, qkv_seed=31, N_kv=N_kv, dtype=dtype)
+    mask, q, k, v, qkv_cpu = Hh.to_dev(req)
+    qt, kt, vt = (t.permute(1, 0, 2).contiguous() for t in (q, k, v))
+    cat = bsa.catalog()
+    plans = []
+    for kern in (4, 0, 1, 2, 3):
+        ids = [c["plan_id"] for c in cat if c["kernel"] == kern and c["split_pmax"] == 1 and
+               (dtype == "bf16" or kern == 4) and bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d)]
+        plans += ids[:1]
+    plans += [c["plan_id"] for c in cat if c["split_pmax"] > 1 and (dtype == "bf16" or c["kernel"] == 4) and
+              bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d)][:1]
+    assert len(plans) >= (6 if dtype == "bf16" else 2)
+    for n, pid in enumerate(plans):
+        with bsa.plan_create(mask, B_Q, B_KV, N, H, d, plan_id=pid, N_kv=N_kv, dtype=dtype) as pa, \
+                bsa.plan_create(mask, B_Q, B_KV, N, H, d, plan_id=pid, N_kv=N_kv, dtype=dtype, layout="nhd") as pb:
+            assert pb.info()["layout"] == 1 and pa.info()["layout"] == 0
+            Oa, La = pa.forward(q, k, v)
+            Ob, Lb = pb.forward(qt, kt, vt)
+            torch.cuda.synchronize()
+            assert Ob.shape == (N, H, d) and Lb.shape == (H, N)
+            assert torch.equal(Ob.permute(1, 0, 2), Oa) and torch.equal(La, Lb), pid
+            if n == 0:
+                Hh.compare_with_oracle(req, Ob.permute(1, 0, 2).contiguous(), Lb, qkv_cpu)
+
+
+def test_token_major_layout_from_host_buffers_and_cache_key():
+    req = I.config_tiny()
+    mask, q, k, v, qkv_cpu = Hh.to_dev(req)
+    args = (req.B_Q, req.B_KV, req.N, req.H, req.d)
+    with bsa.plan_create(mask, *args) as plan:
+        O, LSE = plan.forward(q, k, v)
+        torch.cuda.synchronize()
+    qh, kh, vh = (t.permute(1, 0, 2).contiguous() for t in qkv_cpu)
+    Oh = torch.empty_like(qh)
+    Lh = torch.empty((req.H, req.N), dtype=torch.float32)
+    bsa.request_host(req.mask, *args, qh, kh, vh, Oh, Lh, layout="nhd")
+    assert torch.equal(Oh.permute(1, 0, 2), O.cpu()) and torch.equal(Lh, LSE.cpu())
+    cache = bsa.PlanCache(4)
+    p0, h0 = cache.get(mask, *args)
+    p1, h1 = cache.get(mask, *args, layout="nhd")   # another tensor property: another plan
+    p2, h2 = cache.get(mask, *args, layout="nhd")
+    assert (h0, h1, h2) == (False, False, True) and p1._h.value == p2._h.value != p0._h.value
+    for p in (p0, p1, p2):
+        p.destroy()
+    cache.destroy()
+
+
 def test_head_sharded_forward_equals_the_unsharded_one():
     """Heads are independent: three ranks' worth of head ranges, run one after the other on this GPU through the
     sharded driver, give the same bits as the whole request under the same plan."""
