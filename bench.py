@@ -346,8 +346,8 @@ def main():
         flops = 4.0 * req.d * pairs
 
         def step():
-            plan = bsa.plan_create(mask_d, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=args.plan)
-            plan.forward(qd, kd, vd, O, LSE)
+            plan = bsa.plan_create(mask_d, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=args.plan, stream=stream)
+            plan.forward(qd, kd, vd, O, LSE, stream=stream)
             return plan
 
         for _ in range(warmup):

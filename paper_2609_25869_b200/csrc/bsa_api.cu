@@ -209,20 +209,35 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     const int nrows = (int)nrows64;
 
     // ---- Algorithm 2, line 1: shared mask state mu(M), part 1 (row counts + scalar statistics) ----
+    // Small masks: the column indices get room for every block of the mask in this first arena, so that the CSR fill
+    // does not have to wait for the host to learn nnz: it is queued right behind the row scan and runs while the host
+    // waits for the statistics and looks the plan up.
+    const int64_t all_blocks = (int64_t)nrows * nKb;
+    const bool early_fill = !cache && all_blocks <= (1ll << 20);  // (a cache hit would throw the fill away)
     size_t o_nnz = 0, o_ptr = align_up(o_nnz + sizeof(int32_t) * (size_t)nrows);
-    size_t o_zero = align_up(o_ptr + sizeof(int32_t) * ((size_t)nrows + 1));
-    size_t o_stats = o_zero, o_cnt = o_stats + 256, o_hc = o_cnt + 256;
+    size_t o_col_early = align_up(o_ptr + sizeof(int32_t) * ((size_t)nrows + 1));
+    size_t o_zero = early_fill ? align_up(o_col_early + sizeof(int32_t) * (size_t)(all_blocks + 1)) : o_col_early;
+    size_t o_cnt = o_zero, o_hc = o_cnt + 256;
     size_t a1_bytes = align_up(o_hc + sizeof(int32_t) * 3 * (size_t)heads);
     BSA_CUDA(cudaMallocAsync(&p->arena1, a1_bytes, stream), "arena1");
     p->row_nnz = reinterpret_cast<int32_t*>(p->arena1 + o_nnz);
     p->row_ptr = reinterpret_cast<int32_t*>(p->arena1 + o_ptr);
-    p->stats = reinterpret_cast<MaskStatsDev*>(p->arena1 + o_stats);
     p->counters = reinterpret_cast<PlanCountersDev*>(p->arena1 + o_cnt);
     p->head_counts = reinterpret_cast<int32_t*>(p->arena1 + o_hc);
-    BSA_CUDA(cudaMemsetAsync(p->arena1 + o_zero, 0, a1_bytes - o_zero, stream), "memset");
+    // The statistics accumulators live in a small device buffer of this host thread (one per device) that the
+    // statistics kernel itself leaves at zero, so nothing has to be cleared in front of that kernel.  A request that
+    // ended in an error may have left them dirty: then, and at first use, they are cleared here.
+    constexpr int kAccDevices = 64;
+    static thread_local MaskStatsDev* acc_dev[kAccDevices] = {};
+    static thread_local bool acc_clean[kAccDevices] = {};
+    if (p->device < 0 || p->device >= kAccDevices) { free_plan(p); return BSA_ERR_UNSUPPORTED; }
+    if (!acc_dev[p->device]) BSA_CUDA(cudaMalloc(&acc_dev[p->device], 256), "statistics accumulators");
+    p->stats = acc_dev[p->device];
+    if (!acc_clean[p->device]) BSA_CUDA(cudaMemsetAsync(p->stats, 0, 256, stream), "accumulator memset");
+    acc_clean[p->device] = false;  // until this request's totals have arrived
     // ---- lines 3-5: only the scalars cross to the host.  The statistics kernel's last CTA posts them into pinned
     // host memory and the host polls for the sequence number (a few microseconds less than a copy command and an
-    // event); if nothing arrives within a millisecond the host falls back to that copy.
+    // event); if nothing arrives within a millisecond the host waits for the stream instead.
     static thread_local MaskStatsHost* posted = nullptr;
     static thread_local unsigned post_seq = 0;
     if (!posted) {
@@ -239,8 +254,18 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
         BSA_CUDA(launch_mask_row_stats(mask_dev, nrows, nKb, p->row_nnz, p->stats, stream, posted, seq, cache != nullptr),
                  "mask_row_stats");
     const double t1 = now_us();
+    // the counters the later kernels add to (not needed before the statistics have reached the host)
+    BSA_CUDA(cudaMemsetAsync(p->arena1 + o_zero, 0, a1_bytes - o_zero, stream), "memset");
     // the row-pointer scan needs nothing from the host: it runs while the host waits for the scalars
     BSA_CUDA(launch_row_scan(p->row_nnz, nrows, p->row_ptr, stream), "row_scan");
+    if (early_fill) {
+        p->col_idx = reinterpret_cast<int32_t*>(p->arena1 + o_col_early);
+        if (packed_stride > 0)
+            BSA_CUDA(launch_csr_fill_packed(mask_words, packed_stride / 4, nrows, nKb, p->row_ptr, p->col_idx, stream),
+                     "csr_fill_packed");
+        else
+            BSA_CUDA(launch_csr_fill(mask_dev, nrows, nKb, p->row_ptr, p->col_idx, stream), "csr_fill");
+    }
     {
         volatile unsigned* flag = &posted->seq;
         const double t_poll = now_us();
@@ -251,21 +276,22 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
                 break;
             }
         }
-        if (arrived) {
-            std::atomic_thread_fence(std::memory_order_acquire);
-            p->hstats.nnz = posted->nnz;
-            p->hstats.in_runs = posted->in_runs;
-            p->hstats.max_row_nnz = posted->max_row_nnz;
-            p->hstats.blocks_done = 0;
-            p->hstats.hash[0] = posted->hash[0];
-            p->hstats.hash[1] = posted->hash[1];
-        } else {
-            static thread_local MaskStatsDev* pinned = nullptr;
-            if (!pinned) BSA_CUDA(cudaMallocHost(&pinned, sizeof(MaskStatsDev)), "pinned stats copy");
-            BSA_CUDA(cudaMemcpyAsync(pinned, p->stats, sizeof(MaskStatsDev), cudaMemcpyDeviceToHost, stream), "stats copy");
+        if (!arrived) {  // a long queue in front of the kernel: wait for the stream instead of spinning on
             BSA_CUDA(cudaStreamSynchronize(stream), "stats sync");
-            p->hstats = *pinned;
+            if (*flag != seq) {
+                set_cuda_err(cudaErrorUnknown, "statistics were not posted");
+                free_plan(p);
+                return BSA_ERR_CUDA;
+            }
         }
+        std::atomic_thread_fence(std::memory_order_acquire);
+        p->hstats.nnz = posted->nnz;
+        p->hstats.in_runs = posted->in_runs;
+        p->hstats.max_row_nnz = posted->max_row_nnz;
+        p->hstats.blocks_done = 0;
+        p->hstats.hash[0] = posted->hash[0];
+        p->hstats.hash[1] = posted->hash[1];
+        acc_clean[p->device] = true;  // the kernel's last CTA left the accumulators at zero
     }
     const double t2 = now_us();
 
@@ -342,7 +368,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     p->max_items = trows * pmax;
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
-    const size_t o_col = take(sizeof(int32_t) * (size_t)(nnz_i + 1));
+    const size_t o_col = early_fill ? 0 : take(sizeof(int32_t) * (size_t)(nnz_i + 1));
     const size_t o_tb = take(sizeof(int32_t) * (size_t)trows);
     const size_t o_tc = take(sizeof(int32_t) * (size_t)trows);
     const size_t o_rp = take(sizeof(int32_t) * (size_t)trows);
@@ -352,7 +378,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     const size_t o_it1 = take(sizeof(WorkItem) * (size_t)p->max_items);
     const size_t o_sr = take(sizeof(SplitRow) * (size_t)(pmax > 1 ? trows * g.slots : 1));
     BSA_CUDA(cudaMallocAsync(&p->arena2, o, stream), "arena2");
-    p->col_idx = reinterpret_cast<int32_t*>(p->arena2 + o_col);
+    if (!early_fill) p->col_idx = reinterpret_cast<int32_t*>(p->arena2 + o_col);
     p->tile_begin = reinterpret_cast<int32_t*>(p->arena2 + o_tb);
     p->tile_cnt = reinterpret_cast<int32_t*>(p->arena2 + o_tc);
     p->row_parts = reinterpret_cast<int32_t*>(p->arena2 + o_rp);
@@ -366,11 +392,14 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
         BSA_CUDA(cudaMallocAsync(&p->ws_O, (size_t)p->ws_bytes, stream), "workspace");
         p->ws_LSE = p->ws_O + (size_t)p->max_items * g.T_Q * d;
     }
-    if (packed_stride > 0)
+    if (early_fill) {
+        // already queued before the statistics arrived
+    } else if (packed_stride > 0) {
         BSA_CUDA(launch_csr_fill_packed(mask_words, packed_stride / 4, nrows, nKb, p->row_ptr, p->col_idx, stream),
                  "csr_fill_packed");
-    else
+    } else {
         BSA_CUDA(launch_csr_fill(mask_dev, nrows, nKb, p->row_ptr, p->col_idx, stream), "csr_fill");
+    }
     BSA_CUDA(launch_tile_map(g, p->row_ptr, p->col_idx, p->desc.split_tau, pmax, p->tile_begin, p->tile_cnt,
                              p->row_parts, p->tile_col, p->tile_member, p->head_counts, p->counters, stream),
              "tile_map");

@@ -44,17 +44,20 @@ __device__ __forceinline__ unsigned row_word_bits(const uint4* __restrict__ word
 }
 
 // Called by thread 0 of every CTA of a statistics kernel after it has added its share: the CTA that finds itself last
-// copies the totals into pinned host memory, so the host can read them without a copy command or an event.
+// moves the totals into pinned host memory, so the host can read them without a copy command or an event.
 __device__ __forceinline__ void post_stats_if_last(MaskStatsDev* stats, MaskStatsHost* post, unsigned seq) {
     if (!post) return;
     __threadfence();
     if (atomicAdd(&stats->blocks_done, 1u) != gridDim.x - 1) return;
     __threadfence();
-    post->nnz = atomicAdd(&stats->nnz, 0ull);
-    post->in_runs = atomicAdd(&stats->in_runs, 0ull);
-    post->hash[0] = atomicAdd(&stats->hash[0], 0ull);
-    post->hash[1] = atomicAdd(&stats->hash[1], 0ull);
-    post->max_row_nnz = atomicMax(&stats->max_row_nnz, 0u);
+    // the totals are taken out and the accumulators left at zero for the next request that uses them (no memset
+    // in front of the next statistics kernel)
+    post->nnz = atomicExch(&stats->nnz, 0ull);
+    post->in_runs = atomicExch(&stats->in_runs, 0ull);
+    post->hash[0] = atomicExch(&stats->hash[0], 0ull);
+    post->hash[1] = atomicExch(&stats->hash[1], 0ull);
+    post->max_row_nnz = atomicExch(&stats->max_row_nnz, 0u);
+    atomicExch(&stats->blocks_done, 0u);
     __threadfence_system();
     *reinterpret_cast<volatile unsigned*>(&post->seq) = seq;
 }
