@@ -181,6 +181,18 @@ BSA_API bsa_status_t bsa_plan_create_packed(const uint8_t* mask_bits_dev, int64_
 BSA_API bsa_status_t bsa_forward(const bsa_plan_t* plan, const void* Q_dev, const void* K_dev, const void* V_dev,
                          void* O_dev, float* LSE_dev, void* stream);
 
+/* One cold request on device buffers in a single call: bsa_plan_create_ex (row_stride_bytes = 0) or
+ * bsa_plan_create_packed (> 0) followed by bsa_forward on the same stream, arguments as there.  The forward is
+ * queued before the call returns, which saves a caller in an interpreted language the second trip through its
+ * foreign-function layer (on the 200-us Mid request that trip is hidden behind the preparation kernels and the
+ * single call measures the same).  *out_plan receives the plan (reusable
+ * for further forwards; give it back with bsa_plan_destroy); on any error nothing is returned and nothing is kept.
+ * Errors: those of the two calls; the pointer checks of bsa_forward come first (GPU untouched). */
+BSA_API bsa_status_t bsa_request_device(const uint8_t* mask_dev, int64_t row_stride_bytes, int B_Q, int B_KV, int64_t N,
+                                int heads, int d, const void* Q_dev, const void* K_dev, const void* V_dev, void* O_dev,
+                                float* LSE_dev, const bsa_options_t* options /* may be NULL */, void* stream,
+                                bsa_plan_t** out_plan);
+
 /* Lets go of the plan.  A plan from bsa_plan_create* is freed with every device buffer it owns, and the call
  * synchronises with the plan's create stream.  A plan from bsa_plan_cache_get is shared: the call only drops the
  * caller's hold (no synchronisation) unless it was the last one. */

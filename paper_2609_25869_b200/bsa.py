@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
                                        ctypes.POINTER(ctypes.c_int32)]
     L.bsa_plan_cache_destroy.argtypes = [vp]
     L.bsa_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.bsa_request_device.argtypes = [vp, i64, i32, i32, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.POINTER(Options), vp,
+                                     ctypes.POINTER(vp)]
     L.bsa_plan_destroy.argtypes = [vp]
     L.bsa_request_host.argtypes = [vp, i32, i32, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.POINTER(Options),
                                    ctypes.POINTER(PlanInfo)]
@@ -227,6 +229,25 @@ def plan_create(mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: 
     _check(lib().bsa_plan_create_ex(mask.data_ptr(), B_Q, B_KV, N, heads, d, ctypes.byref(opt), _stream_ptr(stream),
                                     ctypes.byref(h)), "bsa_plan_create")
     return Plan(h.value, layout)
+
+
+def request(mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, Q, K, V, O=None, LSE=None, plan_id: int = -1,
+            max_workspace_bytes: int = 0, stream=None, N_kv: int = 0, dtype: str = "bf16", layout: str = "hnd",
+            row_stride: int = 0):
+    """``bsa_request_device``: plan create + forward in one call (CUDA tensors).  Returns ``(plan, O, LSE)``; the plan
+    can run further forwards and is given back with ``plan.destroy()``."""
+    import torch
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None:
+        hn = Q.shape[:2] if layout == "hnd" else (Q.shape[1], Q.shape[0])
+        LSE = torch.empty(hn, dtype=torch.float32, device=Q.device)
+    h = ctypes.c_void_p()
+    opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv, LAYOUTS[layout], 0)
+    _check(lib().bsa_request_device(mask.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, Q.data_ptr(), K.data_ptr(),
+                                    V.data_ptr(), O.data_ptr(), LSE.data_ptr(), ctypes.byref(opt), _stream_ptr(stream),
+                                    ctypes.byref(h)), "bsa_request_device")
+    return Plan(h.value, layout), O, LSE
 
 
 def pack_mask(mask):

@@ -432,6 +432,32 @@ def test_token_major_layout_from_host_buffers_and_cache_key():
     cache.destroy()
 
 
+def test_single_call_request_equals_create_plus_forward():
+    req = I.config_tiny()
+    mask, q, k, v, qkv_cpu = Hh.to_dev(req)
+    args = (req.B_Q, req.B_KV, req.N, req.H, req.d)
+    n0 = bsa.kernel_launch_count()
+    plan, O, LSE = bsa.request(mask, *args, q, k, v, plan_id=2)
+    torch.cuda.synchronize()
+    assert bsa.kernel_launch_count() - n0 == 7       # five planner kernels, attention, Split-K merge
+    Hh.compare_with_oracle(req, O, LSE, qkv_cpu)
+    Hh.check_plan_structure(req, plan)
+    with bsa.plan_create(mask, *args, plan_id=2) as two:
+        O2, L2 = two.forward(q, k, v)
+        O3, L3 = plan.forward(q, k, v)              # the returned plan is an ordinary one
+        torch.cuda.synchronize()
+    assert torch.equal(O, O2) and torch.equal(LSE, L2) and torch.equal(O, O3) and torch.equal(LSE, L3)
+    plan.destroy()
+    bits, stride = bsa.pack_mask(mask)
+    pb, Ob, Lb = bsa.request(bits, *args, q, k, v, plan_id=2, row_stride=stride)
+    torch.cuda.synchronize()
+    assert torch.equal(Ob, O) and torch.equal(Lb, LSE)
+    pb.destroy()
+    with pytest.raises(bsa.BsaError) as e:           # a misaligned tensor is refused before anything is planned
+        bsa.request(mask, *args, q.view(-1)[1:1 + q.numel() - 8].view(-1), k, v, O, LSE)
+    assert e.value.status == 1
+
+
 def test_head_sharded_forward_equals_the_unsharded_one():
     """Heads are independent: three ranks' worth of head ranges, run one after the other on this GPU through the
     sharded driver, give the same bits as the whole request under the same plan."""
