@@ -501,6 +501,14 @@ __host__ __device__ __forceinline__ int32_t length_bucket(int32_t n) {
     return 2 * lz + ((n >> (lz - 1)) & 1);
 }
 
+// Lanes of the warp that hold the same key as this lane (32 shuffles: constant time, unlike match.any).
+__device__ __forceinline__ unsigned warp_peers(int32_t k) {
+    unsigned m = 0;
+#pragma unroll
+    for (int l = 0; l < 32; ++l) m |= (__shfl_sync(kFull, k, l) == k ? 1u : 0u) << l;
+    return m;
+}
+
 __device__ __forceinline__ int32_t block_excl_scan(int32_t v, int32_t* warp_buf, int32_t* total_out) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
     int32_t incl = v;
@@ -612,17 +620,35 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
         }
         return;
     }
-    // histogram of item lengths; lanes of a warp that hold the same length add once (rows of one mask tend to have
-    // similar lengths, and one shared-memory atomic per item on a handful of addresses serialises the CTA)
-    for (int i0 = 0; i0 < n_items; i0 += blockDim.x) {
-        const int i = i0 + tid;
-        const int32_t k = (i < n_items) ? key[i] : -1 - (tid & 31);
-        const unsigned peers = __match_any_sync(kFull, k);
-        if (i < n_items && (peers >> (tid & 31)) <= 1u) atomicAdd(&bins[k], __popc(peers));
+    // ---- B + C1: stable counting sort by length (longest first; ties keep (head, q_tile, part) order) ----
+    // The items are cut into contiguous chunks, one per ranking warp.  Every warp histograms its chunk into a private
+    // row; the column sums give the bucket sizes, their suffix sums the bucket starts (longest first), and within a
+    // bucket the warps' shares follow in chunk order; every warp then ranks its own chunk in order.  Lanes with equal
+    // keys are found with 32 shuffles (warp_peers): `match.any` takes time in proportion to the number of distinct
+    // keys in the warp and made this kernel 16 us long on 1024 items.
+    int rank_warps = min(rank_warps_max, (n_items + 63) / 64);
+    if (rank_warps < 1) rank_warps = 1;
+    const int warp = tid >> 5, lane = tid & 31;
+    int32_t* whist = key + key_cap;  // [rank_warps][nbins]; one warp alone uses `bins` itself
+    int32_t* wb = (rank_warps >= 2) ? whist + warp * nbins : bins;
+    const int chunk = (((n_items + rank_warps - 1) / rank_warps) + 31) & ~31;
+    const int c0 = warp * chunk, c1 = min(n_items, c0 + chunk);
+    if (rank_warps >= 2) {
+        for (int i = tid; i < rank_warps * nbins; i += blockDim.x) whist[i] = 0;
+        __syncthreads();
     }
+    if (warp < rank_warps)
+        for (int i = c0 + lane; i < c1; i += 32) atomicAdd(&wb[key[i]], 1);  // this warp's own row
     __syncthreads();
-
-    // ---- B: bucket starts, longest first ----
+    if (rank_warps >= 2) {
+        for (int b = tid; b < nbins; b += blockDim.x) {
+            int32_t tot = 0;
+            for (int w = 0; w < rank_warps; ++w) tot += whist[w * nbins + b];
+            bins[b] = tot;
+        }
+        __syncthreads();
+    }
+    // bucket starts, longest first
     if (tid < 32) {
         int32_t carry = 0;
         for (int hi = nbins - 1; hi >= 0; hi -= 32) {
@@ -638,31 +664,7 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
         }
     }
     __syncthreads();
-
-    // ---- C1: stable rank ----
-    // per-warp histograms cost rank_warps * nbins shared-memory words to clear and scan: worth it from a few hundred
-    // items per warp on
-    const int rank_warps = min(rank_warps_max, n_items / 256);
     if (rank_warps >= 2) {
-        // The group's items are cut into `rank_warps` contiguous chunks, one per warp: per-warp histograms, then for
-        // every length the warps' counts are turned into start offsets (bucket start + counts of the earlier chunks),
-        // then every warp ranks its own chunk in order.  Same ranks as the one-warp walk below.
-        int32_t* whist = key + key_cap;  // [rank_warps][nbins]
-        const int warp = tid >> 5, lane = tid & 31;
-        const int chunk = (((n_items + rank_warps - 1) / rank_warps) + 31) & ~31;
-        for (int i = tid; i < rank_warps * nbins; i += blockDim.x) whist[i] = 0;
-        __syncthreads();
-        const int c0 = warp * chunk, c1 = min(n_items, c0 + chunk);
-        if (warp < rank_warps) {
-            for (int i0 = c0; i0 < c1; i0 += 32) {
-                const int i = i0 + lane;
-                const int32_t k = (i < c1) ? key[i] : -1 - lane;
-                const unsigned peers = __match_any_sync(kFull, k);
-                if (i < c1 && (peers >> lane) <= 1u) whist[warp * nbins + k] += __popc(peers);  // this warp's own row
-                __syncwarp();
-            }
-        }
-        __syncthreads();
         for (int b = tid; b < nbins; b += blockDim.x) {
             int32_t run = bins[b];
             for (int w = 0; w < rank_warps; ++w) {
@@ -672,33 +674,17 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
             }
         }
         __syncthreads();
-        if (warp < rank_warps) {
-            int32_t* wb = whist + warp * nbins;
-            for (int i0 = c0; i0 < c1; i0 += 32) {
-                const int i = i0 + lane;
-                const bool valid = i < c1;
-                const int32_t k = valid ? key[i] : -1 - lane;  // invalid lanes get unique keys
-                const unsigned peers = __match_any_sync(kFull, k);
-                int32_t rank = 0;
-                if (valid) rank = wb[k] + __popc(peers & ((1u << lane) - 1u));
-                __syncwarp();
-                if (valid && (peers >> lane) <= 1u) wb[k] += __popc(peers);  // highest lane of the peer set
-                __syncwarp();
-                if (valid) key[i] = rank;
-            }
-        }
-    } else if (tid < 32) {
-        for (int i0 = 0; i0 < n_items; i0 += 32) {
-            const int i = i0 + tid;
-            const bool valid = i < n_items;
-            const int32_t k = valid ? key[i] : -1 - tid;  // invalid lanes get unique keys
-            const unsigned peers = __match_any_sync(kFull, k);
+    }
+    if (warp < rank_warps) {
+        for (int i0 = c0; i0 < c1; i0 += 32) {
+            const int i = i0 + lane;
+            const bool valid = i < c1;
+            const int32_t k = valid ? key[i] : -1 - lane;  // invalid lanes get unique keys
+            const unsigned peers = warp_peers(k);
             int32_t rank = 0;
-            if (valid) {
-                rank = bins[k] + __popc(peers & ((1u << tid) - 1u));
-            }
+            if (valid) rank = wb[k] + __popc(peers & ((1u << lane) - 1u));
             __syncwarp();
-            if (valid && (peers >> tid) <= 1u) bins[k] += __popc(peers);  // highest lane of the peer set
+            if (valid && (peers >> lane) <= 1u) wb[k] += __popc(peers);  // highest lane of the peer set
             __syncwarp();
             if (valid) key[i] = rank;
         }
