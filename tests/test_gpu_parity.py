@@ -458,6 +458,55 @@ def test_single_call_request_equals_create_plus_forward():
     assert e.value.status == 1
 
 
+def test_concurrent_requests_from_several_host_threads():
+    """Four host threads, each with its own stream, plan and run different requests at the same time (the binding
+    releases the interpreter lock inside the C calls; the library keeps its per-request host state per thread), some
+    through one shared plan cache: every output equals the one the request gives alone."""
+    import threading
+    reqs = []
+    for t in range(4):
+        r = I.config_tiny(seed=40 + t)
+        reqs.append((r, Hh.to_dev(r)))
+    want = []
+    for r, (mask, q, k, v, _) in reqs:
+        with bsa.plan_create(mask, r.B_Q, r.B_KV, r.N, r.H, r.d) as plan:
+            O, L = plan.forward(q, k, v)
+            torch.cuda.synchronize()
+            want.append((O.clone(), L.clone()))
+    cache = bsa.PlanCache(8)
+    errors = []
+
+    def worker(t):
+        try:
+            r, (mask, q, k, v, _) = reqs[t]
+            st = torch.cuda.Stream()
+            for it in range(25):
+                if it % 2:
+                    plan, _ = cache.get(mask, r.B_Q, r.B_KV, r.N, r.H, r.d, stream=st)
+                else:
+                    plan = bsa.plan_create(mask, r.B_Q, r.B_KV, r.N, r.H, r.d, stream=st)
+                O = torch.empty_like(q)
+                L = torch.empty(q.shape[:2], dtype=torch.float32, device="cuda")
+                plan.forward(q, k, v, O, L, stream=st)
+                st.synchronize()
+                if not (torch.equal(O, want[t][0]) and torch.equal(L, want[t][1])):
+                    errors.append((t, it, "output differs"))
+                plan.destroy()
+        except Exception as e:  # noqa: BLE001 - reported by the main thread
+            errors.append((t, repr(e)))
+
+    torch.cuda.synchronize()
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(4)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    assert not errors, errors[:3]
+    st = cache.stats()
+    assert st["hits"] + st["misses"] == 48 and st["entries"] == 4 and st["misses"] >= 4
+    cache.destroy()
+
+
 def test_head_sharded_forward_equals_the_unsharded_one():
     """Heads are independent: three ranks' worth of head ranges, run one after the other on this GPU through the
     sharded driver, give the same bits as the whole request under the same plan."""
