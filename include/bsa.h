@@ -2,12 +2,19 @@
  * bsa.h -- C ABI of the B200 (sm_100a) forward of dynamic block-sparse attention.
  *
  * A request R = <A, M, B, x> (paper, Section 3 "Online request path" and Section 4.4) supplies a
- * logical block mask M with geometry B = (B_Q, B_KV) and the tensor properties x (here: bf16,
- * head dim d, layout [heads, N, d]).  The library computes masked attention (Section 2.1, Eq. 1)
+ * logical block mask M with geometry B = (B_Q, B_KV) and the tensor properties x (here: bf16 or fp16,
+ * head dim d in {64, 128}, layout [heads, N, d] or [N, heads, d]; bsa_options_t carries the non-default
+ * ones, and N_kv when keys and queries differ in number).  The library computes masked attention
+ * (Section 2.1, Eq. 1)
  *
  *     O_M = softmax(Q K^T / sqrt(d) + B_M) V,   B_M = 0 on E(M), -inf elsewhere,
  *
  * plus the fp32 log-sum-exp of each row, touching only physical tiles that cover active blocks.
+ *
+ * Entry points: bsa_plan_create[_ex|_packed] -> bsa_forward (any number of times) -> bsa_plan_destroy;
+ * bsa_request_device (create + forward in one call); bsa_request_host (the same from host buffers);
+ * bsa_plan_cache_* (prepared plans reused when the mask repeats); bsa_plan_get_info / bsa_plan_export_* (what
+ * was planned); bsa_lut_* / bsa_catalog_* (plan table and catalog); bsa_mask_stats_noalloc.
  *
  * All pointers named *_dev are DEVICE pointers on the current CUDA device; pointers named
  * *_host are HOST pointers.  No function throws; every call returns a status.  `stream` is a
