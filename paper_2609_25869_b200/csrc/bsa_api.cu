@@ -718,50 +718,113 @@ extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int 
     const size_t lbytes = (size_t)heads * (size_t)N * 4;
     const size_t o_m = 0, o_q = align_up(mbytes), o_k = o_q + align_up(tbytes), o_v = o_k + align_up(kbytes),
                  o_o = o_v + align_up(kbytes), o_l = o_o + align_up(tbytes), total = o_l + align_up(lbytes);
-    // Two streams kept per host thread: the mask goes first on `s` and the plan is created behind it, while Q, K and V
-    // travel on `s2`; the forward waits for them.  Planning (statistics copy, lookup, preparation kernels) thus
-    // overlaps the 3 x heads x N x d x 2 bytes of input copies instead of following them.
-    static thread_local cudaStream_t s = nullptr, s2 = nullptr;
-    static thread_local cudaEvent_t inputs_ready = nullptr;
+    // Heads are independent, and with the head-major layout a range of heads is a contiguous slice of every tensor:
+    // the request is cut into up to 8 groups of heads (at least 32 MB of Q, K, V each: with smaller groups the
+    // copies themselves got slower, 43 instead of 53 GB/s) and pipelined over three streams kept per host thread --
+    // inputs of group g+1 travel (s2) while group g is planned and computed (s) and the output of group g-1 travels
+    // back (s3; the link is full duplex).  What is left after the last input byte is one group's forward and its
+    // output copy.  The token-major layout is not cut.
+    const size_t head_in = ((size_t)N + 2 * (size_t)N_kv) * d * 2;
+    int hc = (int)(((size_t)32 << 20) / (head_in ? head_in : 1)) + 1;  // heads per group
+    if (hc < (heads + 7) / 8) hc = (heads + 7) / 8;
+    if (hc > heads || (options && options->layout == BSA_LAYOUT_NHD)) hc = heads;
+    const int G = (heads + hc - 1) / hc;
+    static thread_local cudaStream_t s = nullptr, s2 = nullptr, s3 = nullptr;
+    static thread_local cudaEvent_t buf_ready = nullptr, in_ready[8] = {}, out_ready[8] = {};
     cudaError_t e = cudaSuccess;
     if (!s) e = cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking);
     if (e == cudaSuccess && !s2) e = cudaStreamCreateWithFlags(&s2, cudaStreamNonBlocking);
-    if (e == cudaSuccess && !inputs_ready) e = cudaEventCreateWithFlags(&inputs_ready, cudaEventDisableTiming);
+    if (e == cudaSuccess && !s3) e = cudaStreamCreateWithFlags(&s3, cudaStreamNonBlocking);
+    if (e == cudaSuccess && !buf_ready) e = cudaEventCreateWithFlags(&buf_ready, cudaEventDisableTiming);
+    for (int g = 0; g < 8 && e == cudaSuccess; ++g) {
+        if (!in_ready[g]) e = cudaEventCreateWithFlags(&in_ready[g], cudaEventDisableTiming);
+        if (e == cudaSuccess && !out_ready[g]) e = cudaEventCreateWithFlags(&out_ready[g], cudaEventDisableTiming);
+    }
     if (e != cudaSuccess) { set_cuda_err(e, "request streams"); return BSA_ERR_CUDA; }
     uint8_t* buf = nullptr;
     bsa_status_t st = BSA_OK;
-    bsa_plan_t* plan = nullptr;
+    bsa_plan_t* plans[8] = {};
     e = cudaMallocAsync(&buf, total, s);
     if (e != cudaSuccess) { set_cuda_err(e, "request buffers"); return BSA_ERR_OOM; }
     e = cudaMemcpyAsync(buf + o_m, mask_host, mbytes, cudaMemcpyHostToDevice, s);
-    // the buffer exists once `s` reaches this point: order the other stream behind it
-    if (e == cudaSuccess) e = cudaEventRecord(inputs_ready, s);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(s2, inputs_ready, 0);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_q, Q_host, tbytes, cudaMemcpyHostToDevice, s2);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_k, K_host, kbytes, cudaMemcpyHostToDevice, s2);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_v, V_host, kbytes, cudaMemcpyHostToDevice, s2);
-    if (e == cudaSuccess) e = cudaEventRecord(inputs_ready, s2);
-    if (e == cudaSuccess) {
-        st = bsa_plan_create_ex(buf + o_m, B_Q, B_KV, N, heads, d, options, s, &plan);
-        if (st == BSA_OK) {
-            e = cudaStreamWaitEvent(s, inputs_ready, 0);
-            if (e == cudaSuccess)
-                st = bsa_forward(plan, buf + o_q, buf + o_k, buf + o_v, buf + o_o, reinterpret_cast<float*>(buf + o_l), s);
-        }
-        if (st == BSA_OK && e == cudaSuccess) {
-            e = cudaMemcpyAsync(O_host, buf + o_o, tbytes, cudaMemcpyDeviceToHost, s);
-            if (e == cudaSuccess) e = cudaMemcpyAsync(LSE_host, buf + o_l, lbytes, cudaMemcpyDeviceToHost, s);
-            if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-        }
+    // the buffer exists once `s` reaches this point: order the other streams behind it
+    if (e == cudaSuccess) e = cudaEventRecord(buf_ready, s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s2, buf_ready, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s3, buf_ready, 0);
+    const size_t q_head = (size_t)N * d * 2, k_head = (size_t)N_kv * d * 2, l_head = (size_t)N * 4;
+    for (int g = 0; g < G && e == cudaSuccess; ++g) {  // all input copies are queued first, in group order
+        const size_t h0 = (size_t)g * hc, nh = (size_t)((g + 1) * hc <= heads ? hc : heads - g * hc);
+        e = cudaMemcpyAsync(buf + o_q + h0 * q_head, static_cast<const uint8_t*>(Q_host) + h0 * q_head, nh * q_head,
+                            cudaMemcpyHostToDevice, s2);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(buf + o_k + h0 * k_head, static_cast<const uint8_t*>(K_host) + h0 * k_head, nh * k_head,
+                                cudaMemcpyHostToDevice, s2);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(buf + o_v + h0 * k_head, static_cast<const uint8_t*>(V_host) + h0 * k_head, nh * k_head,
+                                cudaMemcpyHostToDevice, s2);
+        if (e == cudaSuccess) e = cudaEventRecord(in_ready[g], s2);
     }
-    if (st == BSA_OK && e == cudaSuccess && plan) {
-        bsa_plan_info_t info;
-        st = bsa_plan_get_info(plan, &info);
-        if (st == BSA_OK && info.device_status != 0) st = BSA_ERR_DEVICE_TIMEOUT;
-        if (info_out) *info_out = info;
+    for (int g = 0; g < G && e == cudaSuccess && st == BSA_OK; ++g) {
+        const size_t h0 = (size_t)g * hc;
+        const int nh = (g + 1) * hc <= heads ? hc : heads - g * hc;
+        st = bsa_plan_create_ex(buf + o_m + h0 * nQb * nKb, B_Q, B_KV, N, nh, d, options, s, &plans[g]);
+        if (st != BSA_OK) break;
+        e = cudaStreamWaitEvent(s, in_ready[g], 0);
+        if (e != cudaSuccess) break;
+        st = bsa_forward(plans[g], buf + o_q + h0 * q_head, buf + o_k + h0 * k_head, buf + o_v + h0 * k_head,
+                         buf + o_o + h0 * q_head, reinterpret_cast<float*>(buf + o_l + h0 * l_head), s);
+        if (st != BSA_OK) break;
+        e = cudaEventRecord(out_ready[g], s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s3, out_ready[g], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(static_cast<uint8_t*>(O_host) + h0 * q_head, buf + o_o + h0 * q_head, (size_t)nh * q_head,
+                                cudaMemcpyDeviceToHost, s3);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(reinterpret_cast<uint8_t*>(LSE_host) + h0 * l_head, buf + o_l + h0 * l_head,
+                                (size_t)nh * l_head, cudaMemcpyDeviceToHost, s3);
     }
-    if (plan) bsa_plan_destroy(plan);
-    cudaStreamSynchronize(s2);  // on an error path the copies may still be in flight
+    // every stream is drained on every path: copies may still be in flight after an error
+    cudaError_t e3 = cudaStreamSynchronize(s3), e2 = cudaStreamSynchronize(s2), e1 = cudaStreamSynchronize(s);
+    if (e == cudaSuccess) e = e3 != cudaSuccess ? e3 : (e2 != cudaSuccess ? e2 : e1);
+    if (st == BSA_OK && e == cudaSuccess) {
+        // one info for the whole request: counts add up over the groups, the plan is the first group's
+        bsa_plan_info_t tot;
+        memset(&tot, 0, sizeof tot);
+        for (int g = 0; g < G && st == BSA_OK; ++g) {
+            bsa_plan_info_t info;
+            st = bsa_plan_get_info(plans[g], &info);
+            if (st != BSA_OK) break;
+            if (info.device_status != 0) st = BSA_ERR_DEVICE_TIMEOUT;
+            if (g == 0) {
+                tot = info;
+                continue;
+            }
+            tot.heads += info.heads;
+            tot.nnz_blocks += info.nnz_blocks;
+            tot.blocks_in_runs += info.blocks_in_runs;
+            if (info.max_row_nnz > tot.max_row_nnz) tot.max_row_nnz = info.max_row_nnz;
+            tot.ntiles += info.ntiles;
+            tot.nitems += info.nitems;
+            tot.nsplit_rows += info.nsplit_rows;
+            tot.workspace_bytes += info.workspace_bytes;
+            tot.covered_pairs += info.covered_pairs;
+            tot.us_mask_state += info.us_mask_state;
+            tot.us_stats_sync += info.us_stats_sync;
+            tot.us_lookup += info.us_lookup;
+            tot.us_launch_prep += info.us_launch_prep;
+            tot.us_total += info.us_total;
+            tot.device_status |= info.device_status;
+        }
+        if (G > 1) {
+            const double rows = (double)tot.heads * (double)tot.nQb, nnz = (double)tot.nnz_blocks;
+            tot.density = rows > 0 ? nnz / (rows * (double)tot.nKb) : 0.0;
+            tot.run_coverage = nnz > 0 ? (double)tot.blocks_in_runs / nnz : 0.0;
+            tot.skew = nnz > 0 ? (double)tot.max_row_nnz / (nnz / rows) : 0.0;
+        }
+        if (info_out) *info_out = tot;
+    }
+    for (int g = 0; g < G; ++g)
+        if (plans[g]) bsa_plan_destroy(plans[g]);
     cudaFreeAsync(buf, s);
     cudaStreamSynchronize(s);
     if (e != cudaSuccess) { set_cuda_err(e, "request"); return BSA_ERR_CUDA; }

@@ -226,6 +226,29 @@ def test_request_from_host_buffers_matches_device_path():
     Hh.compare_with_oracle(req, O, LSE, (q, k, v))
 
 
+def test_pipelined_request_from_pinned_host_buffers():
+    """The bench's end-to-end path on its own workload: bsa_request_host cuts Mid's 8 heads into 3 groups and
+    pipelines copies in, planning + forward, and copies out.  Outputs against the oracle on sampled query blocks of
+    every head; the aggregated info equals the whole mask's statistics and the sums over heads."""
+    req = I.config_mid()
+    q, k, v = req.qkv()
+    qp, kp, vp = (t.pin_memory() for t in (q, k, v))
+    O = torch.empty_like(q).pin_memory()
+    LSE = torch.empty((req.H, req.N), dtype=torch.float32).pin_memory()
+    mask = torch.from_numpy(req.mask).pin_memory()
+    O.fill_(float("nan"))
+    LSE.fill_(float("nan"))
+    inf = bsa.request_host(mask, req.B_Q, req.B_KV, req.N, req.H, req.d, qp, kp, vp, O, LSE)
+    assert inf["device_status"] == 0 and inf["heads"] == req.H
+    Hh.compare_with_oracle(req, O, LSE, (q, k, v), sel=_sample(req, 16))
+    with bsa.plan_create(torch.from_numpy(req.mask).cuda(), req.B_Q, req.B_KV, req.N, req.H, req.d) as whole:
+        w = whole.info()
+    for key in ("nnz_blocks", "blocks_in_runs", "max_row_nnz", "ntiles", "nitems", "covered_pairs"):
+        assert inf[key] == w[key], key
+    for key in ("density", "run_coverage", "skew"):
+        assert abs(inf[key] - w[key]) < 1e-9, key
+
+
 @pytest.mark.parametrize("plan_id", [22, 27])
 def test_forward_replays_from_a_cuda_graph(plan_id):
     """bsa_forward only launches kernels (no allocation, no synchronisation): it can be captured into a CUDA graph
