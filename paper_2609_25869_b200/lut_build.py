@@ -85,6 +85,10 @@ def corpus(scale: str = "full"):
         reqs.append(r)
     reqs.append(I.config_hunyuan(seed=1020))
     if scale != "quick":
+        # the same shapes with few heads (head bucket <= 4): what a head-sharded or head-pipelined request looks like
+        for n, h in enumerate((1, 2, 3, 4)):
+            reqs.append(I.config_mid(seed=1050 + n, H=h))
+        reqs.append(I.config_hunyuan(seed=1060, H=3))
         k = 0
         for B in I.SWEEP_GEOMETRIES:
             for rho in I.SWEEP_DENSITIES:
