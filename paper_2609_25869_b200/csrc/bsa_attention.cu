@@ -1444,6 +1444,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
     volatile uint32_t* abortp = &abort_flag;
+    // Launched with programmatic stream serialisation, this grid may start while the kernel in front of it (the task
+    // organisation) is still running: everything above touches only this CTA's shared memory, TMEM and the kernel
+    // parameters; nothing below runs before that kernel has completed and its writes are visible.
+    grid_dependency_wait();
     const int n_items = p.counters->nitems;
     const int n_rounds = (n_items + (int)gridDim.x - 1) / (int)gridDim.x;
 
@@ -2134,9 +2138,24 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
         bsa_attention_pair_kernel<D, TK><<<grid, kPairThreads, smem, stream>>>(tq, tk, tv, p);
     else if (KERNEL == 2)
         bsa_attention_cs_kernel<D, TK><<<grid, kCsThreads, smem, stream>>>(tq, tk, tv, p);
-    else
-        (a.f16 ? bsa_attention_pp_kernel<D, TK, true> : bsa_attention_pp_kernel<D, TK, false>)
-            <<<grid, kPpThreads, smem, stream>>>(tq, tk, tv, p);
+    else {
+        // The ping-pong kernel waits for its predecessor itself (grid_dependency_wait), so it may be scheduled while
+        // the task-organisation kernel is still sorting: its launch latency and prologue overlap that kernel.
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3((unsigned)kPpThreads);
+        cfg.dynamicSmemBytes = (size_t)smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t le = a.f16 ? cudaLaunchKernelEx(&cfg, bsa_attention_pp_kernel<D, TK, true>, tq, tk, tv, p)
+                               : cudaLaunchKernelEx(&cfg, bsa_attention_pp_kernel<D, TK, false>, tq, tk, tv, p);
+        count_launch();
+        return le;
+    }
     count_launch();
     return cudaGetLastError();
 }

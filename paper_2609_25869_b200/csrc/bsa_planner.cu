@@ -369,6 +369,7 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
     extern __shared__ unsigned long long bm[];  // [slots][nKt]: one membership word per 128-row slot
     __shared__ int32_t warp_cnt[8];
     __shared__ int32_t warp_slot_cnt[8];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // see organize_kernel
     const int trow = blockIdx.x;
     const int h = trow / g.nQt, t = trow % g.nQt;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -538,6 +539,11 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
                                                          SplitRow* __restrict__ split_rows, PlanCountersDev* counters) {
     extern __shared__ int32_t sm[];
     __shared__ int32_t warp_buf[32];
+    // Programmatic dependent launch along tile map -> organisation -> attention: a grid lets its successor be
+    // scheduled as soon as all of its own CTAs have started, and waits for its predecessor's completion itself before
+    // it reads anything (no-ops in ordinary launches).  The successor's launch latency and prologue then overlap.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int nbins = organize_bins(g);
     const bool bucketed = (order == BSA_ORDER_HEAD_MAJOR_BUCKETS || order == BSA_ORDER_GLOBAL_BUCKETS);
     const bool global_group = (order == BSA_ORDER_GLOBAL_LPT || order == BSA_ORDER_GLOBAL_BUCKETS);
@@ -799,11 +805,21 @@ cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const i
         attr_bytes = smem;
     }
     const int grid = (order == BSA_ORDER_GLOBAL_LPT || order == BSA_ORDER_GLOBAL_BUCKETS) ? 1 : g.H;
-    organize_kernel<<<grid, 1024, smem, stream>>>(g, order, rank_warps, (int)organize_key_cap(g, order, split_pmax),
-                                                   split_pmax <= 1 ? 1 : 0, tile_begin, tile_cnt, row_parts, head_counts,
-                                                   items_tmp, items, split_rows, counters);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(1024);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, organize_kernel, g, order, rank_warps,
+                                             (int)organize_key_cap(g, order, split_pmax), split_pmax <= 1 ? 1 : 0, tile_begin,
+                                             tile_cnt, row_parts, head_counts, items_tmp, items, split_rows, counters);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace bsa

@@ -104,6 +104,13 @@ __device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t parity_a, ui
     return true;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// In a grid launched with programmatic stream serialisation: blocks until the grid in front of it in the stream has
+// completed and its memory is visible (a no-op in an ordinary launch).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next grid in the stream, if it was launched that way, be scheduled from now on.
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- TMA
 __device__ __forceinline__ void prefetch_tensormap(const void* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
