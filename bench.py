@@ -28,7 +28,7 @@ sys.path.insert(0, ROOT)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch on the bench workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists for the workload)
-NCU_TRAFFIC_BYTES = {"mid": 199.6e6}  # 174.5 MB read + 25.1 MB written: one ncu capture of one launch on this workload
+NCU_TRAFFIC_BYTES = {"mid": 206.5e6}  # 179.7 MB read + 26.9 MB written: one ncu capture of one launch on this workload
 
 
 def load_peaks():
