@@ -568,6 +568,11 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
     __syncthreads();
 
     // ---- A: unsorted items ----
+    // One pass and one item per row (the common case of a short list under a plan that never splits): the item stays in
+    // this thread's registers until it is written to its final place, instead of going through `items_tmp`.
+    const bool resident = no_split && (row1 - row0) <= (int)blockDim.x;
+    WorkItem mine;
+    mine.head = mine.q_tile = mine.tile_begin = mine.tile_end = mine.part = mine.nparts = mine.ws_slot = mine.ntiles = 0;
     int32_t run_items = 0, run_split = 0, run_slots = 0;
     for (int r0 = row0; r0 < row1; r0 += blockDim.x) {
         const int r = r0 + tid;
@@ -597,7 +602,10 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
                 it.ws_slot = (P > 1) ? (slot + p) * g.slots : -1;  // 128-row workspace slots
                 it.ntiles = it.tile_end - it.tile_begin;
                 const int32_t li = run_items + off_i + p;
-                items_tmp[item_base + li] = it;
+                if (resident)
+                    mine = it;  // li == tid
+                else
+                    items_tmp[item_base + li] = it;
                 key[li] = bucketed ? length_bucket(it.ntiles) : it.ntiles;
             }
             if (P > 1) {
@@ -618,7 +626,11 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
     __syncthreads();
     const int32_t n_items = run_items;
     if (order == BSA_ORDER_NATURAL) {  // unsorted: the items stay in (head, q_tile, part) order
-        for (int i = tid; i < n_items; i += blockDim.x) items[item_base + i] = items_tmp[item_base + i];
+        if (resident) {
+            if (tid < n_items) items[item_base + tid] = mine;
+        } else {
+            for (int i = tid; i < n_items; i += blockDim.x) items[item_base + i] = items_tmp[item_base + i];
+        }
         if (tid == 0 && grp == gridDim.x - 1) {
             counters->nitems = item_base + n_items;
             counters->nsplit_rows = (split_base + run_split) * g.slots;
@@ -698,7 +710,11 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
     __syncthreads();
 
     // ---- C2: scatter ----
-    for (int i = tid; i < n_items; i += blockDim.x) items[item_base + key[i]] = items_tmp[item_base + i];
+    if (resident) {
+        if (tid < n_items) items[item_base + key[tid]] = mine;
+    } else {
+        for (int i = tid; i < n_items; i += blockDim.x) items[item_base + key[i]] = items_tmp[item_base + i];
+    }
 
     if (tid == 0) {
         if (global_group) {
