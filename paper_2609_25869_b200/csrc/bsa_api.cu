@@ -266,6 +266,22 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
         else
             BSA_CUDA(launch_csr_fill(mask_dev, nrows, nKb, p->row_ptr, p->col_idx, stream), "csr_fill");
     }
+    // While the host would only wait: take the second arena now, at the size the previous request of this shape
+    // needed on this thread plus a quarter (masks of one shape have similar nnz); if this request turns out to need
+    // more, it is freed and taken again at the exact size below.
+    struct LastArena {
+        int B_Q, B_KV, heads, d;
+        int64_t N, N_kv;
+        size_t bytes;
+    };
+    static thread_local LastArena last_arena = {};
+    const bool same_shape = last_arena.bytes && last_arena.B_Q == B_Q && last_arena.B_KV == B_KV &&
+                            last_arena.heads == heads && last_arena.d == d && last_arena.N == N && last_arena.N_kv == N_kv;
+    size_t arena2_have = 0;
+    if (early_fill && same_shape) {
+        arena2_have = last_arena.bytes + last_arena.bytes / 4 + 4096;
+        BSA_CUDA(cudaMallocAsync(&p->arena2, arena2_have, stream), "arena2 (predicted)");
+    }
     {
         volatile unsigned* flag = &posted->seq;
         const double t_poll = now_us();
@@ -377,7 +393,12 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     const size_t o_it0 = take(sizeof(WorkItem) * (size_t)p->max_items);
     const size_t o_it1 = take(sizeof(WorkItem) * (size_t)p->max_items);
     const size_t o_sr = take(sizeof(SplitRow) * (size_t)(pmax > 1 ? trows * g.slots : 1));
-    BSA_CUDA(cudaMallocAsync(&p->arena2, o, stream), "arena2");
+    if (p->arena2 && o > arena2_have) {  // the prediction was too small
+        cudaFreeAsync(p->arena2, stream);
+        p->arena2 = nullptr;
+    }
+    if (!p->arena2) BSA_CUDA(cudaMallocAsync(&p->arena2, o, stream), "arena2");
+    last_arena = LastArena{B_Q, B_KV, heads, d, N, N_kv, o};
     if (!early_fill) p->col_idx = reinterpret_cast<int32_t*>(p->arena2 + o_col);
     p->tile_begin = reinterpret_cast<int32_t*>(p->arena2 + o_tb);
     p->tile_cnt = reinterpret_cast<int32_t*>(p->arena2 + o_tc);
