@@ -398,8 +398,8 @@ def main():
             torch.cuda.synchronize()
             if i >= 3:
                 wev[i - 3][0].record(stream)
-            wp, hit = cache.get(mask_d, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=args.plan)
-            wp.forward(qd, kd, vd, O, LSE)
+            wp, hit = cache.request(mask_d, req.B_Q, req.B_KV, req.N, req.H, req.d, qd, kd, vd, O, LSE, plan_id=args.plan,
+                                    stream=stream)
             if i >= 3:
                 wev[i - 3][1].record(stream)
             hits += int(hit)

@@ -236,6 +236,14 @@ BSA_API bsa_status_t bsa_plan_cache_create(int capacity, bsa_plan_cache_t** out_
 BSA_API bsa_status_t bsa_plan_cache_get(bsa_plan_cache_t* cache, const uint8_t* mask_dev, int64_t row_stride_bytes, int B_Q,
                                 int B_KV, int64_t N, int heads, int d, const bsa_options_t* options /* may be NULL */,
                                 void* stream, bsa_plan_t** out_plan, int* out_hit);
+/* bsa_plan_cache_get followed by bsa_forward on the same stream, in one call (as bsa_request_device is for
+ * bsa_plan_create_ex): on a hit nothing lies between the arrival of the mask fingerprint and the launch of the
+ * attention kernel but the table lookup.  *out_plan as for bsa_plan_cache_get (give it back with bsa_plan_destroy). */
+BSA_API bsa_status_t bsa_plan_cache_request(bsa_plan_cache_t* cache, const uint8_t* mask_dev, int64_t row_stride_bytes,
+                                    int B_Q, int B_KV, int64_t N, int heads, int d, const void* Q_dev, const void* K_dev,
+                                    const void* V_dev, void* O_dev, float* LSE_dev,
+                                    const bsa_options_t* options /* may be NULL */, void* stream, bsa_plan_t** out_plan,
+                                    int* out_hit);
 BSA_API bsa_status_t bsa_plan_cache_stats(bsa_plan_cache_t* cache, int64_t* hits, int64_t* misses, int64_t* evictions,
                                   int32_t* entries);
 BSA_API bsa_status_t bsa_plan_cache_destroy(bsa_plan_cache_t* cache);

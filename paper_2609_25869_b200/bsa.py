@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
     L.bsa_plan_cache_create.argtypes = [i32, ctypes.POINTER(vp)]
     L.bsa_plan_cache_get.argtypes = [vp, vp, i64, i32, i32, i64, i32, i32, ctypes.POINTER(Options), vp, ctypes.POINTER(vp),
                                      ctypes.POINTER(i32)]
+    L.bsa_plan_cache_request.argtypes = [vp, vp, i64, i32, i32, i64, i32, i32, vp, vp, vp, vp, vp, ctypes.POINTER(Options),
+                                         vp, ctypes.POINTER(vp), ctypes.POINTER(i32)]
     L.bsa_plan_cache_stats.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i64),
                                        ctypes.POINTER(ctypes.c_int32)]
     L.bsa_plan_cache_destroy.argtypes = [vp]
@@ -298,6 +300,19 @@ class PlanCache:
         opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv, LAYOUTS[layout], 0)
         _check(lib().bsa_plan_cache_get(self._h, mask.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, ctypes.byref(opt),
                                         _stream_ptr(stream), ctypes.byref(h), ctypes.byref(hit)), "bsa_plan_cache_get")
+        return Plan(h.value, layout), bool(hit.value)
+
+    def request(self, mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, Q, K, V, O, LSE, plan_id: int = -1,
+                max_workspace_bytes: int = 0, stream=None, row_stride: int = 0, N_kv: int = 0, dtype: str = "bf16",
+                layout: str = "hnd"):
+        """``bsa_plan_cache_request``: ``get`` + ``forward`` in one call; returns ``(plan, hit)``."""
+        h = ctypes.c_void_p()
+        hit = ctypes.c_int(0)
+        opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv, LAYOUTS[layout], 0)
+        _check(lib().bsa_plan_cache_request(self._h, mask.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, Q.data_ptr(),
+                                            K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), ctypes.byref(opt),
+                                            _stream_ptr(stream), ctypes.byref(h), ctypes.byref(hit)),
+               "bsa_plan_cache_request")
         return Plan(h.value, layout), bool(hit.value)
 
     def stats(self) -> Dict:

@@ -483,6 +483,31 @@ extern "C" bsa_status_t bsa_plan_cache_get(bsa_plan_cache_t* cache, const uint8_
     return st;
 }
 
+extern "C" bsa_status_t bsa_plan_cache_request(bsa_plan_cache_t* cache, const uint8_t* mask_dev, int64_t row_stride_bytes,
+                                               int B_Q, int B_KV, int64_t N, int heads, int d, const void* Q, const void* K,
+                                               const void* V, void* O, float* LSE, const bsa_options_t* options,
+                                               void* stream_v, bsa_plan_t** out_plan, int* out_hit) {
+    if (!cache || !out_plan || row_stride_bytes < 0) return BSA_ERR_INVALID_ARG;
+    *out_plan = nullptr;
+    if (!Q || !K || !V || !O || !LSE) return BSA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V) |
+         reinterpret_cast<uintptr_t>(O)) & 15)
+        return BSA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(LSE) & 3) return BSA_ERR_INVALID_ARG;
+    bsa_plan_t* plan = nullptr;
+    int hit = 0;
+    bsa_status_t st = create_impl(mask_dev, row_stride_bytes, B_Q, B_KV, N, heads, d, options, stream_v, &plan, cache, &hit);
+    if (st != BSA_OK) return st;
+    st = bsa_forward(plan, Q, K, V, O, LSE, stream_v);
+    if (st != BSA_OK) {
+        bsa_plan_destroy(plan);
+        return st;
+    }
+    if (out_hit) *out_hit = hit;
+    *out_plan = plan;
+    return BSA_OK;
+}
+
 extern "C" bsa_status_t bsa_plan_cache_stats(bsa_plan_cache_t* cache, int64_t* hits, int64_t* misses, int64_t* evictions,
                                              int32_t* entries) {
     if (!cache) return BSA_ERR_INVALID_ARG;

@@ -649,7 +649,15 @@ def test_plan_cache_reuses_the_plan_of_a_repeated_mask():
     assert torch.equal(O4, O1) and torch.equal(L4, L1)
     st = cache.stats()
     assert st == {"hits": 3, "misses": 6, "evictions": 0, "entries": 6}
-    for p in (p0, p1, p2, p3, p4, p5):
+    # get + forward in one call
+    O6 = torch.empty_like(q)
+    L6 = torch.empty_like(L1)
+    n0 = bsa.kernel_launch_count()
+    p6, hit6 = cache.request(mask, *args, q, k, v, O6, L6)
+    torch.cuda.synchronize()
+    assert hit6 and p6._h.value == p0._h.value and bsa.kernel_launch_count() - n0 == 2 + 2   # + attention and merge
+    assert torch.equal(O6, O1) and torch.equal(L6, L1)
+    for p in (p0, p1, p2, p3, p4, p5, p6):
         p.destroy()
     cache.destroy()
 
