@@ -593,6 +593,23 @@ def test_random_requests_match_the_oracle(n):
     req, plan_id = _random_request(n)
     nsel = min(req.nQb, max(1, 600 // req.B_Q))
     Hh.run_request(req, plan_id=plan_id, sel=_sample(req, nsel), guards=False)
+    if n % 3:
+        return
+    # every third request also in the token-major layout, from a bit-packed mask and through the single-call entry
+    # point: the same bits as the plain path
+    mask, q, k, v, _ = Hh.to_dev(req)
+    kw = dict(plan_id=plan_id, N_kv=req.N_kv, dtype=req.dtype)
+    args = (req.B_Q, req.B_KV, req.N, req.H, req.d)
+    with bsa.plan_create(mask, *args, **kw) as plain:
+        O, L = plain.forward(q, k, v)
+        torch.cuda.synchronize()
+    bits, stride = bsa.pack_mask(mask)
+    qt, kt, vt = (t.permute(1, 0, 2).contiguous() for t in (q, k, v))
+    pt, Ot, Lt = bsa.request(bits, *args, qt, kt, vt, layout="nhd", row_stride=stride, **kw)
+    torch.cuda.synchronize()
+    assert pt.info()["device_status"] == 0
+    pt.destroy()
+    assert torch.equal(Ot.permute(1, 0, 2), O) and torch.equal(Lt, L)
 
 
 def test_plan_cache_reuses_the_plan_of_a_repeated_mask():
