@@ -202,11 +202,15 @@ BSA_API bsa_status_t bsa_request_device(const uint8_t* mask_dev, int64_t row_str
 
 /* Lets go of the plan.  A plan from bsa_plan_create* is freed with every device buffer it owns, and the call
  * synchronises with the plan's create stream.  A plan from bsa_plan_cache_get is shared: the call only drops the
- * caller's hold (no synchronisation) unless it was the last one. */
+ * caller's hold (no synchronisation) unless it was the last one.
+ * The buffers go back to the memory pool in the create stream's order.  Forwards submitted to OTHER streams are
+ * covered: every such bsa_forward leaves an event behind it that the free waits for, so the plan may be destroyed
+ * (or evicted from a cache) right after the call returns.  The one exception is a forward recorded into a CUDA
+ * graph: keep the plan alive until the last replay of that graph has completed. */
 BSA_API bsa_status_t bsa_plan_destroy(bsa_plan_t* plan);
 
 /* ---------------------------------------------------------------------------------------------
- * Plan cache -- the warm path of Section 5.2 / Section 6.5: while the mask stays the same across
+ * Plan cache -- the warm path of Section 5.2 (measured in Section 7.4, Table 7): while the mask stays the same across
  * layers or denoising steps, the prepared plan is reused and only the attention kernels run.  The
  * paper leaves the reuse to the caller; this cache recognises a repeated mask by itself.
  *
@@ -218,6 +222,10 @@ BSA_API bsa_status_t bsa_plan_destroy(bsa_plan_t* plan);
  * the plan is prepared exactly as by bsa_plan_create_ex / bsa_plan_create_packed, kept in the cache
  * and returned (*out_hit = 0); beyond `capacity` plans the least recently used one is dropped.
  * Two different masks collide only if both 64-bit sums agree (no comparison of the masks follows).
+ * A collision would hand back the plan of the OTHER mask: the forward would then attend over that
+ * mask's blocks and return a wrong O and LSE without any error.  For masks that differ by accident the
+ * chance is about 2^-128 per pair; a caller that must rule it out (masks chosen by an adversary) uses
+ * bsa_plan_create* and keeps the plans itself.
  *
  *   row_stride_bytes : 0 = one byte per logical block (as bsa_plan_create); > 0 = bit-packed rows
  *                      (as bsa_plan_create_packed).  mask_dev is device memory, borrowed for the call.
@@ -284,10 +292,18 @@ BSA_API bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int B_K
  *   BSA_ERR_UNSUPPORTED before anything is launched.
  *
  * The first call on a device resolves the array's device address (cudaGetSymbolAddress) with that
- * device current; make that first call before starting any stream capture.  All calls on a device
- * share the one array, which still holds the previous call's data: the accumulators are cleared
- * on `stream` at the start of every call.  Two calls whose GPU work overlaps (different streams, or
- * different host threads) race on the array and give wrong results: keep them stream-ordered.
+ * device current.  Under CUDA's default lazy module loading that first call is also when the driver
+ * loads the library's module onto the device and reserves the array (and the module's code) there,
+ * so it is the one call that can still fail for lack of device memory (BSA_ERR_CUDA).  Make it once
+ * per device at start-up: before the host hands the device's memory to its own pool, and before any
+ * stream capture.  Later calls on that device touch neither the allocator nor the module loader
+ * (the GPU test checks that the driver's free-memory figure does not move across them).  Host
+ * threads that make their first call on a device concurrently all resolve and store the same
+ * address; that is harmless.
+ * All calls on a device share the one array, which still holds the previous call's data: the
+ * accumulators are cleared on `stream` at the start of every call.  Two calls whose GPU work
+ * overlaps (different streams, or different host threads) race on the array and give wrong results:
+ * keep them stream-ordered.
  * Errors: INVALID_ARG (null pointers, non-positive sizes), UNSUPPORTED (too many rows), CUDA.
  */
 #define BSA_NOALLOC_MAX_ROWS (1 << 20)
@@ -327,6 +343,10 @@ BSA_API int bsa_catalog_size(void);
 BSA_API bsa_status_t bsa_catalog_get(int index, bsa_plan_desc_t* out);
 /* Eligible(P, R) (Section 4.4): geometry, head dim, membership format and workspace. */
 BSA_API int bsa_plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_workspace_bytes);
+/* The same with every request property eligibility looks at: N_kv (<= 0: N_kv = N) and the element type
+ * (BSA_DTYPE_*).  bsa_plan_eligible is this call with N_kv = N and bf16. */
+BSA_API int bsa_plan_eligible_ex(int plan_id, int B_Q, int B_KV, int64_t N, int64_t N_kv, int heads, int d, int dtype,
+                                 int64_t max_workspace_bytes);
 /* Base plan of a request key (eligible for every request with that key). */
 BSA_API int bsa_base_plan(int B_Q, int B_KV, int d);
 /* Hash of the catalog contents; a plan table built for another catalog is rejected. */
@@ -348,6 +368,21 @@ BSA_API void bsa_lut_buckets(int64_t N, double density, double skew, double run_
 /* Process-wide default used when options->force_plan_id is not given: >= 0 forces a plan,
  * -1 restores Algorithm 2. */
 BSA_API void bsa_force_plan(int plan_id);
+
+/* ---------------------------------------------------------------------------------------------
+ * Test hooks for the give-up path of the kernels' bounded waits (no counterpart in the paper).
+ * Every wait inside the attention kernels (on a copy, an MMA, another warp) has a limit in SM clock
+ * cycles; when it runs out the CTA records BSA_ERR_DEVICE_TIMEOUT in the plan's device_status, lets
+ * its copies in flight land, frees its tensor memory and returns.  Both settings are per device
+ * (the current one), apply to forwards launched afterwards, and synchronise the device.
+ *   bsa_debug_set_wait_limit(cycles)   : the limit; <= 0 restores the default (2e9 cycles, about 1 s).
+ *   bsa_debug_withhold_arrival(on)     : while on, the ping-pong kernel's V producer leaves out the
+ *                                        copy of each CTA's first tile and the arrival announcing it,
+ *                                        so the waits behind it run out.  Nothing faults; O and LSE
+ *                                        of such a forward are undefined.
+ */
+BSA_API bsa_status_t bsa_debug_set_wait_limit(long long cycles);
+BSA_API bsa_status_t bsa_debug_withhold_arrival(int on);
 
 BSA_API const char* bsa_status_string(bsa_status_t s);
 BSA_API const char* bsa_last_cuda_error(void);

@@ -103,6 +103,9 @@ def lib() -> ctypes.CDLL:
     L.bsa_catalog_size.restype = i32
     L.bsa_catalog_get.argtypes = [i32, ctypes.POINTER(PlanDesc)]
     L.bsa_plan_eligible.argtypes = [i32, i32, i32, i64, i32, i32, i64]
+    L.bsa_plan_eligible_ex.argtypes = [i32, i32, i32, i64, i64, i32, i32, i32, i64]
+    L.bsa_debug_set_wait_limit.argtypes = [ctypes.c_longlong]
+    L.bsa_debug_withhold_arrival.argtypes = [i32]
     L.bsa_base_plan.argtypes = [i32, i32, i32]
     L.bsa_catalog_hash.restype = ctypes.c_uint64
     L.bsa_lut_load.argtypes = [ctypes.c_char_p]
@@ -373,8 +376,19 @@ def catalog() -> List[Dict]:
     return out
 
 
-def plan_eligible(plan_id, B_Q, B_KV, N, heads, d, max_workspace_bytes=0) -> bool:
-    return bool(lib().bsa_plan_eligible(plan_id, B_Q, B_KV, N, heads, d, max_workspace_bytes))
+def plan_eligible(plan_id, B_Q, B_KV, N, heads, d, max_workspace_bytes=0, N_kv=0, dtype="bf16") -> bool:
+    """``bsa_plan_eligible_ex``: Eligible(P, R) for the request's geometry, token counts, head dim and element type."""
+    return bool(lib().bsa_plan_eligible_ex(plan_id, B_Q, B_KV, N, N_kv, heads, d, DTYPES[dtype], max_workspace_bytes))
+
+
+def debug_set_wait_limit(cycles: int):
+    """``bsa_debug_set_wait_limit`` (test hook): limit of the kernels' bounded waits in SM cycles; <= 0 = default."""
+    _check(lib().bsa_debug_set_wait_limit(cycles), "bsa_debug_set_wait_limit")
+
+
+def debug_withhold_arrival(on: bool):
+    """``bsa_debug_withhold_arrival`` (test hook): make the next forwards' first V tile never arrive."""
+    _check(lib().bsa_debug_withhold_arrival(1 if on else 0), "bsa_debug_withhold_arrival")
 
 
 def lut_load(path: str):

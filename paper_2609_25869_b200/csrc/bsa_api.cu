@@ -95,6 +95,10 @@ struct bsa_plan {
     // behind the preparation kernels so that a later request on another stream can wait for them
     std::atomic<int> refs;
     cudaEvent_t ready;
+    // Recorded behind every forward that was submitted to a stream other than the plan's own (created at the first
+    // such forward): the plan's buffers go back to the pool in the create stream's order, so that stream waits for
+    // this event first.  Forwards on one plan are stream-ordered among themselves, so the latest record covers all.
+    std::atomic<cudaEvent_t> last_use;
 };
 
 // ---- plan cache (warm path of Section 5.2: a prepared plan is reused while the mask stays the same) ----
@@ -133,6 +137,11 @@ static int64_t request_n_kv(const bsa_options_t* options, int64_t N) {
 static void free_plan(bsa_plan* p) {
     if (!p) return;
     if (p->ready) cudaEventDestroy(p->ready);
+    if (cudaEvent_t lu = p->last_use.load(std::memory_order_acquire)) {
+        // a forward on another stream may still be reading the arenas and the workspace
+        cudaStreamWaitEvent(p->stream, lu, 0);
+        cudaEventDestroy(lu);
+    }
     if (p->arena1) cudaFreeAsync(p->arena1, p->stream);
     if (p->arena2) cudaFreeAsync(p->arena2, p->stream);
     if (p->ws_O) cudaFreeAsync(p->ws_O, p->stream);
@@ -181,6 +190,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     if (!p) return BSA_ERR_OOM;
     memset(static_cast<void*>(p), 0, sizeof *p);
     p->refs.store(1, std::memory_order_relaxed);
+    p->last_use.store(nullptr, std::memory_order_relaxed);
     p->stream = stream;
     p->d = d;
     p->dtype = dtype;
@@ -227,7 +237,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     // The statistics accumulators live in a small device buffer of this host thread (one per device) that the
     // statistics kernel itself leaves at zero, so nothing has to be cleared in front of that kernel.  A request that
     // ended in an error may have left them dirty: then, and at first use, they are cleared here.
-    constexpr int kAccDevices = 64;
+    constexpr int kAccDevices = kMaxDevices;
     static thread_local MaskStatsDev* acc_dev[kAccDevices] = {};
     static thread_local bool acc_clean[kAccDevices] = {};
     if (p->device < 0 || p->device >= kAccDevices) { free_plan(p); return BSA_ERR_UNSUPPORTED; }
@@ -579,13 +589,40 @@ extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const vo
     a.max_items = (int32_t)(p->max_items < (1 << 30) ? p->max_items : (1 << 30));
     a.max_split_rows = p->g.H * p->g.nQt * p->g.slots;
     a.num_sms = p->num_sms;
+    a.device = p->device;
     a.f16 = p->dtype == BSA_DTYPE_FP16;
     a.nhd = p->layout == BSA_LAYOUT_NHD;
     const char* detail = "launch";
-    cudaError_t e = launch_forward(a, reinterpret_cast<cudaStream_t>(stream_v), &detail);
+    cudaStream_t fstream = reinterpret_cast<cudaStream_t>(stream_v);
+    cudaError_t e = launch_forward(a, fstream, &detail);
     if (e != cudaSuccess) {
         set_cuda_err(e, detail);
         return BSA_ERR_CUDA;
+    }
+    if (fstream != p->stream) {
+        // The plan's memory is freed in the create stream's order: leave a marker behind this forward that the free
+        // waits for.  Not while `stream` is being captured (an event recorded into a graph cannot be waited for from
+        // outside it): whoever replays a captured forward keeps the plan alive until the replays are done.
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(fstream, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusNone) {
+            bsa_plan* mp = const_cast<bsa_plan*>(p);
+            cudaEvent_t lu = mp->last_use.load(std::memory_order_acquire);
+            if (!lu) {
+                cudaEvent_t fresh = nullptr;
+                e = cudaEventCreateWithFlags(&fresh, cudaEventDisableTiming);
+                if (e != cudaSuccess) {
+                    set_cuda_err(e, "last-use event");
+                    return BSA_ERR_CUDA;
+                }
+                if (mp->last_use.compare_exchange_strong(lu, fresh, std::memory_order_acq_rel)) lu = fresh;
+                else cudaEventDestroy(fresh);  // another thread was first; `lu` now holds its event
+            }
+            e = cudaEventRecord(lu, fstream);
+            if (e != cudaSuccess) {
+                set_cuda_err(e, "last-use record");
+                return BSA_ERR_CUDA;
+            }
+        }
     }
     return BSA_OK;
 }
@@ -886,6 +923,10 @@ extern "C" bsa_status_t bsa_catalog_get(int index, bsa_plan_desc_t* out) {
 }
 extern "C" int bsa_plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, int64_t max_ws) {
     return plan_eligible(plan_id, B_Q, B_KV, N, heads, d, max_ws) ? 1 : 0;
+}
+extern "C" int bsa_plan_eligible_ex(int plan_id, int B_Q, int B_KV, int64_t N, int64_t N_kv, int heads, int d, int dtype,
+                                    int64_t max_ws) {
+    return plan_eligible(plan_id, B_Q, B_KV, N, heads, d, max_ws, N_kv, dtype) ? 1 : 0;
 }
 extern "C" int bsa_base_plan(int B_Q, int B_KV, int d) { return base_plan(B_Q, B_KV, d); }
 extern "C" uint64_t bsa_catalog_hash(void) { return catalog_hash(); }

@@ -16,6 +16,8 @@
 #include <cuda_bf16.h>
 #include <math.h>
 
+#include <atomic>
+
 #include "bsa_common.h"
 #include "sm100_ptx.cuh"
 
@@ -39,6 +41,12 @@ __device__ long long g_cta_times[2][4096];  // %globaltimer at entry and exit of
 #define BSA_TRACE_DECL(n)
 #define BSA_TRACE_POINT(role, n, tag)
 #endif
+
+// Test hook (bsa_debug_withhold_arrival): while non-zero, the V producer of the ping-pong kernel leaves out the copy
+// of the first tile of its CTA together with the arrival that would announce it.  Nothing is in flight for that slot,
+// so nothing can fault; the waits that depend on the tile simply run out, which is how the give-up path (status word,
+// copies in flight allowed to land, TMEM freed, kernel returns) is exercised without a protocol error.
+__device__ int g_withhold_arrival = 0;
 
 namespace {
 
@@ -1500,9 +1508,6 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     mbar_arrive(smem_u32(&bars.o_free));
                     if (lane == 0) BSA_TRACE_POINT(11, tn, 33);
                 }
-#ifdef BSA_ABL_NOSTORE
-                if (inv_l == 12345.f)
-#endif
                 if (it.nparts == 1) {
                     if (row_ok) {  // 32-byte stores: every thread fills whole 32-byte sectors of its own row
 #pragma unroll
@@ -1603,10 +1608,6 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), KV_TILE);
                     tma_load_4d(smem_u32(sK + stage * KV_TILE), &tmK, smem_u32(&bars.k_full[stage]), 0, col_cur * TK, 0, it.head);
                     BSA_TRACE_POINT(0, tn, 21);
-#ifdef BSA_TRACE_KLAT
-                    mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
-                    BSA_TRACE_POINT(0, tn, 23);
-#endif
                 }
             }
             while (ok && npend > 0) ok = issue_q();
@@ -1619,6 +1620,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             uint32_t g = 0;
             RingPos ring;  // V ring position of tile g
             bool ok = true;
+            const bool withhold = *reinterpret_cast<volatile int*>(&g_withhold_arrival) != 0;  // test hook, see above
             WorkItem it_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items);
             for (int kr = 0; kr < n_rounds && ok; ++kr) {
                 const WorkItem it = it_next;
@@ -1630,6 +1632,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     if (j + 1 < it.tile_end) col_next = p.tile_col[j + 1];
                     const int stage = ring.stage;
                     const uint32_t ph = ring.phase;
+                    if (withhold && g == 0) continue;  // this tile never arrives
                     ok = mbar_wait(smem_u32(&bars.v_empty[stage]), ph ^ 1, abortp);
                     if (!ok) break;
                     mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), KV_TILE);
@@ -1758,7 +1761,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                         if (*abortp) return false;
                         const long long now = clock64();
                         if (t0 == 0) t0 = now;
-                        if (now - t0 > 4000000000ll) {
+                        if (now - t0 > *reinterpret_cast<volatile long long*>(&g_wait_limit_cycles)) {
                             *abortp = 1;
                             return false;
                         }
@@ -2106,8 +2109,11 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
         *err = "fp16 inputs need a ping-pong-kernel plan";
         return cudaErrorInvalidValue;
     }
-    static int attr_bytes = 0;  // per instantiation; grows to the largest request seen
-    if (smem > attr_bytes) {
+    // largest size already allowed, per instantiation and per device (the attribute belongs to the device's copy of
+    // the kernel); concurrent first calls may both set it, which is harmless
+    static std::atomic<int> attr_bytes_dev[kMaxDevices];
+    const int dev = (a.device >= 0 && a.device < kMaxDevices) ? a.device : 0;
+    if (smem > attr_bytes_dev[dev].load(std::memory_order_relaxed)) {
         cudaError_t e;
         if (KERNEL == 0)
             e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -2126,7 +2132,7 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
             *err = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
         }
-        attr_bytes = smem;
+        attr_bytes_dev[dev].store(smem, std::memory_order_relaxed);
     }
     int grid = a.num_sms < a.max_items ? a.num_sms : a.max_items;
     if (grid < 1) grid = 1;
@@ -2209,6 +2215,16 @@ extern "C" __attribute__((visibility("default"))) int bsa_debug_trace_copy(long 
     return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(long long) * 4096, sizeof(long long) * 4096 * role);
 }
 #endif
+
+// Test hooks: the limit of the bounded device waits, and the withheld arrival described at g_withhold_arrival.
+extern "C" __attribute__((visibility("default"))) bsa_status_t bsa_debug_set_wait_limit(long long cycles) {
+    const long long v = cycles > 0 ? cycles : 2000000000ll;
+    return cudaMemcpyToSymbol(ptx::g_wait_limit_cycles, &v, sizeof v) == cudaSuccess ? BSA_OK : BSA_ERR_CUDA;
+}
+extern "C" __attribute__((visibility("default"))) bsa_status_t bsa_debug_withhold_arrival(int on) {
+    const int v = on ? 1 : 0;
+    return cudaMemcpyToSymbol(g_withhold_arrival, &v, sizeof v) == cudaSuccess ? BSA_OK : BSA_ERR_CUDA;
+}
 
 cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char** err_detail) {
     AttnParams p;

@@ -7,6 +7,7 @@
 
 namespace bsa {
 
+constexpr int kMaxDevices = 64;  // per-device host state (accumulators, kernel attributes) is kept for this many GPUs
 constexpr int kTQ = 128;  // physical Q tile height of every catalog kernel (one MMA M=128 per CTA)
 
 // One unit of work for a persistent CTA: one Q tile row of one head, restricted to the KV tiles
@@ -113,6 +114,7 @@ struct ForwardArgs {
     int32_t max_items;       // host-side upper bound of the item count
     int32_t max_split_rows;  // host-side upper bound
     int32_t num_sms;
+    int32_t device;          // CUDA device the plan lives on
     int32_t f16;             // 1: Q, K, V, O are IEEE half (ping-pong-kernel plans only); 0: bf16
     int32_t nhd;             // 1: Q, K, V, O are stored [N][heads][d] (token-major); 0: [heads][N][d]
 };

@@ -7,6 +7,8 @@
 // call that can fail late) is not acceptable.  For them this file offers the mask-state statistics
 // kernel with its scratch (one counter per mask row plus the three accumulators) in a fixed
 // device-resident array that lives as long as the library is loaded.
+#include <atomic>
+
 #include "bsa_common.h"
 
 namespace bsa {
@@ -19,8 +21,9 @@ constexpr size_t kScratchBytes = kAccumBytes + sizeof(int32_t) * (size_t)BSA_NOA
 // In HOST code this name is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
-constexpr int kMaxDevices = 64;
-unsigned char* g_scratch_addr[kMaxDevices] = {};  // device address of the array, per device
+// Device address of the array, per device.  Host threads that make their first call on a device at the same time
+// all resolve the same address and store the same value.
+std::atomic<unsigned char*> g_scratch_addr[kMaxDevices];
 
 // Copies the accumulators to the caller's buffer and counts rows without any active block.
 __global__ void __launch_bounds__(256) noalloc_finalize_kernel(const MaskStatsDev* stats, const int32_t* row_nnz,
@@ -54,13 +57,16 @@ extern "C" bsa_status_t bsa_mask_stats_noalloc(const uint8_t* mask_dev, int head
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_v);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BSA_ERR_CUDA;
-    if (!g_scratch_addr[dev]) {
-        // set-up, once per device, with that device current: resolve the array's device address
+    unsigned char* base = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!base) {
+        // Set-up, once per device, with that device current: resolve the array's device address.  With CUDA's lazy
+        // module loading this is also the moment the driver loads this file's module onto the device and reserves
+        // the array there, which is why it can still fail, and why it belongs at start-up.
         void* addr = nullptr;
         if (cudaGetSymbolAddress(&addr, g_noalloc_scratch) != cudaSuccess || !addr) return BSA_ERR_CUDA;
-        g_scratch_addr[dev] = static_cast<unsigned char*>(addr);
+        base = static_cast<unsigned char*>(addr);
+        g_scratch_addr[dev].store(base, std::memory_order_release);
     }
-    unsigned char* base = g_scratch_addr[dev];
     MaskStatsDev* stats = reinterpret_cast<MaskStatsDev*>(base);
     int32_t* row_nnz = reinterpret_cast<int32_t*>(base + kAccumBytes);
     // the array keeps the previous call's contents: the accumulators must start at zero

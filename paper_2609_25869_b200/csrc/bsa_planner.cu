@@ -814,11 +814,9 @@ cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const i
     if (rank_warps > 32) rank_warps = 32;
     if (rank_warps < 2) rank_warps = 0;
     const size_t smem = base + (size_t)rank_warps * per_warp;
-    static size_t attr_bytes = 48 * 1024;
-    if (smem > attr_bytes) {
+    if (smem > 48 * 1024) {  // the attribute is per device: set it whenever the default limit does not do
         cudaError_t e = cudaFuncSetAttribute(organize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attr_bytes = smem;
     }
     const int grid = (order == BSA_ORDER_GLOBAL_LPT || order == BSA_ORDER_GLOBAL_BUCKETS) ? 1 : g.H;
     cudaLaunchConfig_t cfg = {};

@@ -43,9 +43,6 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-#ifdef BSA_ABL_NOLOAD
-    bytes = 0;
-#endif
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
@@ -71,10 +68,15 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// Limit of every bounded wait in SM clock cycles: about one second at 1.9 GHz.  The waits are for events inside one
+// CTA (a copy landing, an MMA completing, another warp's arrival), microseconds apart in a healthy run; the limit is
+// only there so that a protocol error ends in a status word instead of a hung GPU.  A device variable, so that a test
+// can shorten it (bsa_debug_set_wait_limit) and watch a wait run out.
+__device__ long long g_wait_limit_cycles = 2000000000ll;
+
 // Bounded wait.  `abort_flag` is a CTA-wide shared word: once any role gives up it is set, and
-// every other wait returns false promptly.  The limit is about 2 s of SM clock cycles; the clock is
-// consulted only every 64 failed polls (each poll already suspends the thread for a while), and the
-// slow %globaltimer is never read on this path.
+// every other wait returns false promptly.  The clock is consulted only every 64 failed polls (each
+// poll already suspends the thread for a while), and the slow %globaltimer is never read on this path.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = 0;
@@ -85,7 +87,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            if (now - t0 > 4000000000ll) {
+            if (now - t0 > *reinterpret_cast<volatile long long*>(&g_wait_limit_cycles)) {
                 *abort_flag = 1;
                 return false;
             }
@@ -118,9 +120,6 @@ __device__ __forceinline__ void prefetch_tensormap(const void* tmap) {
 // 3-D tiled load global -> shared, completion counted in bytes on an mbarrier.
 // c0 is the innermost coordinate: c0 * element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2) {
-#ifdef BSA_ABL_NOLOAD
-    if (c1 != 0x7fffffff) return;
-#endif
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
@@ -129,9 +128,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint
 // 4-D tiled load: used with the tensor viewed as {64 columns, rows, d/64 column groups, heads}, so that one
 // instruction brings all 64-column sub-tiles of a row block (c0 * element size must be a multiple of 16 bytes).
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2, int c3) {
-#ifdef BSA_ABL_NOLOAD
-    if (c1 != 0x7fffffff) return;
-#endif
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
@@ -188,9 +184,6 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16_f32(int M, int N, int a_m
 // ---------------------------------------------------------------- tcgen05: MMA (one thread issues)
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-#ifdef BSA_ABL_NOQK
-    if (idesc != 0xffffffffu) return;
-#endif
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
@@ -199,9 +192,6 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_
 }
 // D[tmem] (+)= A[tmem] * B[smem]
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-#ifdef BSA_ABL_NOPV
-    if (idesc != 0xffffffffu) return;
-#endif
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"

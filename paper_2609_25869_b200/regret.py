@@ -1,4 +1,4 @@
-"""Quality of the shipped plan table on requests it was not compiled from (paper Section 6.4 "selection regret",
+"""Quality of the shipped plan table on requests it was not compiled from (paper Section 7.4 "selection regret",
 Table 7 cold / warm / amortized request cost).
 
 For every evaluation request (the five named configurations and the first requests of the dynamic-request sweep,
