@@ -255,12 +255,18 @@ def sweep_block(gen, n_requests: int, heads: int, peaks):
         mask = torch.from_numpy(req.mask).cuda()
         flush.fill_(i & 0xFF)
         torch.cuda.synchronize()
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         t0 = time.perf_counter()
+        e0.record()
         plan = bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d)
+        e1.record()  # behind the plan's last preparation kernel: the plan is ready on the GPU when this event is
         t1 = time.perf_counter()
         plan.forward(q, k, v, O, L)
+        e2.record()
         torch.cuda.synchronize()
         t2 = time.perf_counter()
+        planning_us = e0.elapsed_time(e1) * 1e3
+        cold_forward_us = e1.elapsed_time(e2) * 1e3
         for _ in range(3):
             plan.forward(q, k, v, O, L)
         ts = []
@@ -281,14 +287,14 @@ def sweep_block(gen, n_requests: int, heads: int, peaks):
         rows.append({"r": r, "B": [req.B_Q, req.B_KV], "density": round(inf["density"], 4), "skew": round(inf["skew"], 2),
                      "plan": inf["plan"]["name"], "lut_hit": inf["lut_hit"], "cold_request_us": round(cold_us, 1),
                      "plan_create_us": round((t1 - t0) * 1e6, 1), "lookup_us": round(inf["us_lookup"], 2),
-                     "planning_us": round(max(0.0, cold_us - kern_ms * 1e3), 1),
+                     "planning_us": round(planning_us, 1), "cold_forward_us": round(cold_forward_us, 1),
                      "warm_forward_us": round(kern_ms * 1e3, 1), "destroy_us": round((t4 - t3) * 1e6, 1),
                      "tflops_warm": round(4.0 * req.d * pairs / (kern_ms * 1e-3) / 1e12, 1),
                      "covered_over_active": round(inf["covered_pairs"] / max(1, pairs), 3)})
         del mask
     cold = sorted(x["cold_request_us"] for x in rows)
     warm = sorted(x["warm_forward_us"] for x in rows)
-    frac = [x["planning_us"] / x["cold_request_us"] for x in rows]
+    frac = [x["planning_us"] / (x["planning_us"] + x["cold_forward_us"]) for x in rows]
 
     def pct(xs, p):
         return xs[min(len(xs) - 1, int(round(p * (len(xs) - 1))))]
@@ -300,8 +306,10 @@ def sweep_block(gen, n_requests: int, heads: int, peaks):
     by_geom = {}
     for x in rows:
         by_geom.setdefault("%dx%d" % tuple(x["B"]), []).append(x["tflops_warm"])
-    return {"protocol": "50 cold unique requests (new mask each): host clock around plan create + forward + sync; then median of 5 "
-                        "warm forwards after 3 warm-ups; one untimed request sizes the memory pool first",
+    return {"protocol": "cold unique requests (new mask each): host clock around plan create + forward + sync; CUDA events split "
+                        "it into planning (request start until the plan's last preparation kernel has finished, the host's "
+                        "wait for the statistics and the lookup included) and the cold forward; then median of 5 warm "
+                        "forwards after 3 warm-ups; one untimed request sizes the memory pool first",
             "workload": f"{len(rows)} requests, heads={heads} N=75600 d=128, B and density drawn per request",
             "cold_request_us": {"mean": statistics.mean(cold), "gm": gm(cold), "p50": pct(cold, 0.5), "p95": pct(cold, 0.95),
                                 "max": cold[-1]},
@@ -311,6 +319,7 @@ def sweep_block(gen, n_requests: int, heads: int, peaks):
             "plan_create_host_us": {"mean": statistics.mean(x["plan_create_us"] for x in rows),
                                     "max": max(x["plan_create_us"] for x in rows)},
             "lookup_us_mean": statistics.mean(x["lookup_us"] for x in rows),
+            "planning_us": {"mean": statistics.mean(x["planning_us"] for x in rows), "max": max(x["planning_us"] for x in rows)},
             "planning_fraction": {"mean": statistics.mean(frac), "max": max(frac)},
             "destroy_us_mean": statistics.mean(x["destroy_us"] for x in rows),
             "tflops_warm_mean": statistics.mean(x["tflops_warm"] for x in rows),
@@ -434,8 +443,10 @@ def main():
         pairs = count_active_pairs(req)
         flops = 4.0 * req.d * pairs
 
-        def step():
+        def step(ready=None):
             plan = bsa.plan_create(mask_d, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=args.plan, stream=stream)
+            if ready is not None:
+                ready.record(stream)  # behind the plan's last preparation kernel
             plan.forward(qd, kd, vd, O, LSE, stream=stream)
             return plan
 
@@ -445,7 +456,7 @@ def main():
         sampler = ClockSampler(local_rank)
         sampler.start()
         launches0 = bsa.kernel_launch_count()
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        ev = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(2)) for _ in range(steps)]
         host_us, destroy_us = [], []
         plan = None
         for i in range(steps):
@@ -465,6 +476,20 @@ def main():
         launches = bsa.kernel_launch_count() - launches0
         step_ms = [a.elapsed_time(b) for a, b in ev]
         info = plan.info()
+        # Planning share: a few more requests with an event between create and forward (request start -> the plan's
+        # last preparation kernel finished, the host's wait for the statistics and the lookup included).  Kept out of
+        # the timed steps: an event in front of the attention kernel takes away its dependent-launch overlap.
+        plan_ms = []
+        for i in range(min(steps, 5)):
+            flush.fill_(i & 0xFF)
+            torch.cuda.synchronize()
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            p2 = step(c)
+            c.synchronize()
+            plan_ms.append(a.elapsed_time(c))
+            torch.cuda.synchronize()
+            p2.destroy()
         # forward only (warm plan): the attention kernel (+ merge) timed alone, L2 flushed in between
         kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
         for _ in range(3):
@@ -479,6 +504,7 @@ def main():
         k_ms = [a.elapsed_time(b) for a, b in kev]
         res = {"req": req, "pairs": pairs, "flops": flops, "step_ms": sum(step_ms) / len(step_ms),
                "step_ms_median": statistics.median(step_ms), "host_us": statistics.median(host_us),
+               "planning_ms": sum(plan_ms) / len(plan_ms),
                "destroy_us": statistics.median(destroy_us) if destroy_us else None,
                "kernel_ms": sum(k_ms) / len(k_ms), "kernel_ms_median": statistics.median(k_ms), "info": info,
                "launches": launches, "clocks": clocks, "qkv": (q, k, v)}
@@ -503,6 +529,24 @@ def main():
         if cl.get("sm_mhz"):
             res["back_to_back"]["frac_of_tensor_issue_at_clock"] = flops / (
                 bb_ms * 1e-3 * cl["sm_mhz"] * 1e6 * num_sms * TENSOR_FLOP_PER_CLK_PER_SM)
+        if info["plan"]["split_pmax"] > 1 and info["nsplit_rows"] > 0:
+            # the Split-K reduction kernel alone (HBM-bound), over the partials the forwards above left behind
+            mev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+            for i in range(steps):
+                flush.fill_(i & 0xFF)
+                mev[i][0].record(stream)
+                plan.merge_only(O, LSE, stream=stream)
+                mev[i][1].record(stream)
+            torch.cuda.synchronize()
+            m_ms = statistics.mean(a.elapsed_time(b) for a, b in mev)
+            rows_total = req.H * info["nQt"] * info["member_words"]
+            parts = info["nitems"] * info["member_words"] - (rows_total - info["nsplit_rows"])  # 128-row partial slots merged
+            rd = parts * 128 * (req.d + 1) * 4
+            wr = info["nsplit_rows"] * 128 * (2 * req.d + 4)
+            res["merge"] = {"kernel": "bsa_merge_kernel<D>", "launch_ms": m_ms, "merged_tile_rows": info["nsplit_rows"],
+                            "partials": parts, "algorithmic_bytes": rd + wr, "bound": "hbm",
+                            "achieved": (rd + wr) / (m_ms * 1e-3) / 1e9, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                            "frac": (rd + wr) / (m_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         if primary:
             # warm request: the mask repeats, the plan cache recognises it (statistics kernel with the mask
             # fingerprint) and only the forward follows.  Reported beside the cold request; `value` stays the cold one.
@@ -597,12 +641,14 @@ def main():
                     "us_plan_create_host": inf["us_total"], "us_plan_destroy_host": r["destroy_us"],
                     "us_mask_state": inf["us_mask_state"], "us_stats_sync": inf["us_stats_sync"],
                     "us_lookup": inf["us_lookup"], "us_launch_prep": inf["us_launch_prep"],
-                    "planning_fraction": max(0.0, 1.0 - kernel_ms / step_ms),
+                    "us_planning_gpu": r["planning_ms"] * 1e3, "planning_fraction": r["planning_ms"] / r["step_ms"],
                     "plan": inf["plan"]["name"], "lut_hit": inf["lut_hit"], "lut_regimes": lut_regimes,
                     "ntiles": inf["ntiles"],
                     "nitems": inf["nitems"], "active_pairs": r["pairs"], "covered_pairs": inf["covered_pairs"],
                     "density": inf["density"]},
     }
+    if "merge" in r:
+        line["merge"] = r["merge"]
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         nb = req.H * req.nQb if args.workload in ("tiny", "mid") else 2048
         pairs, dt, nsel, thr = oracle_sample(req, r["qkv"], nb)
@@ -620,7 +666,7 @@ def main():
                             "kernel_tflops": kt, "kernel_ms": o["kernel_ms"], "request_ms": o["step_ms"],
                             "request_tflops": o["flops"] / (o["step_ms"] * 1e-3) / 1e12,
                             "frac_of_burst": kt / peaks["bf16_tflops"],
-                            "planning_fraction": max(0.0, 1.0 - o["kernel_ms"] / o["step_ms"]),
+                            "planning_fraction": o["planning_ms"] / o["step_ms"],
                             "covered_over_active": oi["covered_pairs"] / max(1, o["pairs"]),
                             "plan": oi["plan"]["name"], "us_plan_create_host": oi["us_total"], "us_lookup": oi["us_lookup"],
                             "sm_mhz": o["clocks"].get("sm_mhz"), "back_to_back": o["back_to_back"]}

@@ -357,6 +357,11 @@ BSA_API uint64_t bsa_catalog_hash(void);
 BSA_API bsa_status_t bsa_lut_load(const char* path);
 BSA_API void bsa_lut_clear(void);
 BSA_API int bsa_lut_num_regimes(void);
+/* Request keys for which the loaded table holds a learned second-stage partition (Section 5.1: thresholds learned by
+ * a decision tree over log2 N, heads, density, skew and run coverage; its leaves are the regimes).  Such a key is
+ * looked up in its tree; the other keys use the regimes of the fixed bucket edges.  In bsa_plan_info_t a tree lookup
+ * shows as lut_hit = 1 with (leaf index + 1) << 8 added to regime_bucket[3]. */
+BSA_API int bsa_lut_num_trees(void);
 /* Regime lookup + ranked fallback only (no GPU): returns the plan id Algorithm 2 selects for these
  * request scalars, or -1 for no-eligible-plan.  *hit_out (optional) = 1 if the regime was found. */
 BSA_API int bsa_lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_coverage,
@@ -382,6 +387,10 @@ BSA_API void bsa_force_plan(int plan_id);
  *                                        of such a forward are undefined.
  */
 BSA_API bsa_status_t bsa_debug_set_wait_limit(long long cycles);
+/* Measurement hook: launches the Split-K reduction kernel of a plan alone on `stream`, over the partial results the
+ * plan's last forward left in its workspace (so it can be timed by itself; O_dev and LSE_dev are written as by that
+ * forward).  UNSUPPORTED for a plan without Split-K partitions. */
+BSA_API bsa_status_t bsa_debug_merge_only(const bsa_plan_t* plan, void* O_dev, float* LSE_dev, void* stream);
 BSA_API bsa_status_t bsa_debug_withhold_arrival(int on);
 
 BSA_API const char* bsa_status_string(bsa_status_t s);

@@ -106,6 +106,7 @@ def lib() -> ctypes.CDLL:
     L.bsa_plan_eligible_ex.argtypes = [i32, i32, i32, i64, i64, i32, i32, i32, i64]
     L.bsa_debug_set_wait_limit.argtypes = [ctypes.c_longlong]
     L.bsa_debug_withhold_arrival.argtypes = [i32]
+    L.bsa_debug_merge_only.argtypes = [vp, vp, vp, vp]
     L.bsa_base_plan.argtypes = [i32, i32, i32]
     L.bsa_catalog_hash.restype = ctypes.c_uint64
     L.bsa_lut_load.argtypes = [ctypes.c_char_p]
@@ -176,6 +177,10 @@ class Plan:
         _check(lib().bsa_forward(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
                                  _stream_ptr(stream)), "bsa_forward")
         return O, LSE
+
+    def merge_only(self, O, LSE, stream=None):
+        """``bsa_debug_merge_only`` (measurement hook): the Split-K reduction kernel alone, over the last forward's partials."""
+        _check(lib().bsa_debug_merge_only(self._h, O.data_ptr(), LSE.data_ptr(), _stream_ptr(stream)), "bsa_debug_merge_only")
 
     def info(self) -> Dict:
         inf = PlanInfo()

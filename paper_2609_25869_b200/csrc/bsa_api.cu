@@ -24,6 +24,7 @@ uint64_t catalog_hash();
 void lut_buckets(int64_t N, double density, double skew, double run_cov, int32_t out[4]);
 void lut_clear();
 int lut_num_regimes();
+int lut_num_trees();
 bsa_status_t lut_load(const char* path);
 void set_force_plan(int id);
 int get_force_plan();
@@ -564,14 +565,8 @@ extern "C" bsa_status_t bsa_plan_create(const uint8_t* mask_dev, int B_Q, int B_
     return bsa_plan_create_ex(mask_dev, B_Q, B_KV, N, heads, d, nullptr, nullptr, out_plan);
 }
 
-extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const void* K, const void* V, void* O,
-                                    float* LSE, void* stream_v) {
-    if (!p || !Q || !K || !V || !O || !LSE) return BSA_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V) |
-         reinterpret_cast<uintptr_t>(O)) & 15)
-        return BSA_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(LSE) & 3) return BSA_ERR_INVALID_ARG;
-    ForwardArgs a;
+static void fill_forward_args(const bsa_plan_t* p, const void* Q, const void* K, const void* V, void* O, float* LSE,
+                              ForwardArgs& a) {
     memset(&a, 0, sizeof a);
     a.Q = Q; a.K = K; a.V = V; a.O = O; a.LSE = LSE;
     a.items = p->items;
@@ -592,6 +587,30 @@ extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const vo
     a.device = p->device;
     a.f16 = p->dtype == BSA_DTYPE_FP16;
     a.nhd = p->layout == BSA_LAYOUT_NHD;
+}
+
+extern "C" bsa_status_t bsa_debug_merge_only(const bsa_plan_t* p, void* O, float* LSE, void* stream_v) {
+    if (!p || !O || !LSE) return BSA_ERR_INVALID_ARG;
+    if (p->desc.split_pmax <= 1) return BSA_ERR_UNSUPPORTED;
+    ForwardArgs a;
+    fill_forward_args(p, nullptr, nullptr, nullptr, O, LSE, a);
+    cudaError_t e = launch_merge(a, reinterpret_cast<cudaStream_t>(stream_v));
+    if (e != cudaSuccess) {
+        set_cuda_err(e, "merge launch");
+        return BSA_ERR_CUDA;
+    }
+    return BSA_OK;
+}
+
+extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const void* K, const void* V, void* O,
+                                    float* LSE, void* stream_v) {
+    if (!p || !Q || !K || !V || !O || !LSE) return BSA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V) |
+         reinterpret_cast<uintptr_t>(O)) & 15)
+        return BSA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(LSE) & 3) return BSA_ERR_INVALID_ARG;
+    ForwardArgs a;
+    fill_forward_args(p, Q, K, V, O, LSE, a);
     const char* detail = "launch";
     cudaStream_t fstream = reinterpret_cast<cudaStream_t>(stream_v);
     cudaError_t e = launch_forward(a, fstream, &detail);
@@ -939,6 +958,7 @@ extern "C" void bsa_lut_clear(void) {
     lut_clear();
 }
 extern "C" int bsa_lut_num_regimes(void) { return lut_num_regimes(); }
+extern "C" int bsa_lut_num_trees(void) { return lut_num_trees(); }
 extern "C" int bsa_lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, double run_coverage,
                               double skew, int64_t max_ws, int* hit_out) {
     return lut_select(B_Q, B_KV, N, heads, d, density, run_coverage, skew, max_ws, hit_out, nullptr);

@@ -2276,21 +2276,26 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
         return cudaErrorInvalidValue;
     }
     if (e != cudaSuccess) return e;
-    if (a.has_split) {
-        // one CTA per 256 (row, 8-column) units of a merged tile, grid-strided beyond 8 waves
-        const long long want = (long long)a.max_split_rows * (kTQ * (a.d / 8) / 256);
-        int grid = want < 8ll * a.num_sms ? (int)want : 8 * a.num_sms;
-        if (grid < 1) grid = 1;
-        if (a.d == 128)
-            bsa_merge_kernel<128><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
-                                                            reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16, p.o_head, p.o_row);
-        else
-            bsa_merge_kernel<64><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
-                                                           reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16, p.o_head, p.o_row);
-        count_launch();
-        e = cudaGetLastError();
-    }
+    if (a.has_split) e = launch_merge(a, stream);
     return e;
+}
+
+// Split-K reduction alone (also the merge-only test hook: the workspace then holds an earlier forward's partials).
+cudaError_t launch_merge(const ForwardArgs& a, cudaStream_t stream) {
+    const long long o_head = a.nhd ? (long long)a.d : (long long)a.g.N * a.d;
+    const long long o_row = a.nhd ? (long long)a.g.H * a.d : (long long)a.d;
+    // one CTA per 256 (row, 8-column) units of a merged tile, grid-strided beyond 8 waves
+    const long long want = (long long)a.max_split_rows * (kTQ * (a.d / 8) / 256);
+    int grid = want < 8ll * a.num_sms ? (int)want : 8 * a.num_sms;
+    if (grid < 1) grid = 1;
+    if (a.d == 128)
+        bsa_merge_kernel<128><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
+                                                        reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16, o_head, o_row);
+    else
+        bsa_merge_kernel<64><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
+                                                       reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16, o_head, o_row);
+    count_launch();
+    return cudaGetLastError();
 }
 
 }  // namespace bsa

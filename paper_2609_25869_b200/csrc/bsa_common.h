@@ -119,6 +119,7 @@ struct ForwardArgs {
     int32_t nhd;             // 1: Q, K, V, O are stored [N][heads][d] (token-major); 0: [heads][N][d]
 };
 cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char** err_detail);
+cudaError_t launch_merge(const ForwardArgs& a, cudaStream_t stream);  // the Split-K reduction kernel alone
 // `stages` counts K buffers plus V buffers for the paired kernel (kernel 1), K = V ring depth for kernel 0
 int attention_max_stages(int d, int T_KV, int kernel);
 int attention_smem_bytes(int d, int T_KV, int stages, int kernel);

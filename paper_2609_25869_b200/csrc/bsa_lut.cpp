@@ -187,6 +187,37 @@ struct RegimeKey {
 };
 static std::map<RegimeKey, std::vector<int>> g_table;
 static std::mutex g_mu;
+
+// Learned second-stage partition (Section 5.1: "thresholds learned by a decision tree, whose leaves define the finer
+// partitions"): one binary tree per request key over the continuous request features
+//   0: log2 N    1: heads    2: active-block density    3: row-nnz skew    4: active-block-run coverage.
+// An inner node sends a request left when feature < threshold; a leaf holds a ranking.  A key with a tree is looked up
+// in the tree; keys without one use the fixed-edge regimes above.
+struct TreeNode {
+    int feature;        // -1: leaf
+    double threshold;
+    int left, right;
+    std::vector<int> ranked;
+};
+struct TreeKey {
+    int B_Q, B_KV, d;
+    bool operator<(const TreeKey& o) const { return memcmp(this, &o, sizeof(TreeKey)) < 0; }
+};
+static std::map<TreeKey, std::vector<TreeNode>> g_trees;
+constexpr int kTreeFeatures = 5;
+constexpr int kTreeMaxNodes = 4096;
+
+// Leaf of the key's tree these features fall into, or -1 (no tree for the key, or a malformed one).
+static int tree_leaf(const std::vector<TreeNode>& t, const double f[kTreeFeatures]) {
+    int n = 0;
+    for (int steps = 0; steps < kTreeMaxNodes; ++steps) {
+        if (n < 0 || n >= (int)t.size()) return -1;
+        const TreeNode& nd = t[n];
+        if (nd.feature < 0) return n;
+        n = (f[nd.feature] < nd.threshold) ? nd.left : nd.right;
+    }
+    return -1;
+}
 static int g_force_plan = -1;
 
 static int head_bucket(int heads) { return heads <= 4 ? 0 : (heads <= 16 ? 1 : 2); }
@@ -194,6 +225,12 @@ static int head_bucket(int heads) { return heads <= 4 ? 0 : (heads <= 16 ? 1 : 2
 void lut_clear() {
     std::lock_guard<std::mutex> lk(g_mu);
     g_table.clear();
+    g_trees.clear();
+}
+
+int lut_num_trees() {
+    std::lock_guard<std::mutex> lk(g_mu);
+    return (int)g_trees.size();
 }
 
 int lut_num_regimes() {
@@ -202,10 +239,13 @@ int lut_num_regimes() {
 }
 
 // File format (text, one record per line):
-//   BSA_LUT 1
+//   BSA_LUT 1 | 2
 //   catalog <hex hash>
 //   gpu <free text>
 //   regime B_Q B_KV d nb hb db sb rb : id id id ...
+//   (version 2 only) tree B_Q B_KV d <number of nodes>, followed by that many lines, node 0 the root:
+//     node <index> split <feature> <threshold> <left> <right>
+//     node <index> leaf : id id id ...
 bsa_status_t lut_load(const char* path) {
     lut_clear();
     if (!path) return BSA_ERR_INVALID_ARG;
@@ -213,14 +253,54 @@ bsa_status_t lut_load(const char* path) {
     if (!f) return BSA_ERR_LUT;
     char line[1024];
     bool header = false, hash_ok = false;
+    int version = 0;
     std::map<RegimeKey, std::vector<int>> table;
+    std::map<TreeKey, std::vector<TreeNode>> trees;
+    std::vector<TreeNode>* cur_tree = nullptr;  // tree whose node lines are being read
+    int nodes_left = 0;
     bsa_status_t st = BSA_OK;
+    auto parse_ids = [&](const char* q, std::vector<int>* ids) {
+        char* end = nullptr;
+        while (true) {
+            long v = strtol(q, &end, 10);
+            if (end == q) break;
+            if (v < 0 || v >= kCatalogSize) return false;
+            ids->push_back((int)v);
+            q = end;
+        }
+        return !ids->empty();
+    };
     while (fgets(line, sizeof line, f)) {
         if (line[0] == '#' || line[0] == '\n') continue;
+        if (nodes_left > 0 && strncmp(line, "node", 4)) { st = BSA_ERR_LUT; break; }  // a tree's nodes follow its header
         if (!strncmp(line, "BSA_LUT", 7)) {
-            int ver = 0;
-            if (sscanf(line + 7, "%d", &ver) != 1 || ver != 1) { st = BSA_ERR_LUT; break; }
+            if (sscanf(line + 7, "%d", &version) != 1 || (version != 1 && version != 2)) { st = BSA_ERR_LUT; break; }
             header = true;
+        } else if (!strncmp(line, "tree", 4)) {
+            TreeKey k;
+            memset(&k, 0, sizeof k);
+            int n = 0;
+            if (version != 2 || sscanf(line + 4, "%d %d %d %d", &k.B_Q, &k.B_KV, &k.d, &n) != 4 || n < 1 || n > kTreeMaxNodes ||
+                trees.count(k)) { st = BSA_ERR_LUT; break; }
+            cur_tree = &trees[k];
+            cur_tree->assign((size_t)n, TreeNode{-2, 0.0, -1, -1, {}});  // -2: not read yet
+            nodes_left = n;
+        } else if (!strncmp(line, "node", 4)) {
+            int idx = -1, used = 0;
+            if (!cur_tree || nodes_left <= 0 || sscanf(line + 4, "%d %n", &idx, &used) != 1 || idx < 0 ||
+                idx >= (int)cur_tree->size() || (*cur_tree)[idx].feature != -2) { st = BSA_ERR_LUT; break; }
+            TreeNode& nd = (*cur_tree)[idx];
+            const char* rest = line + 4 + used;
+            if (!strncmp(rest, "split", 5)) {
+                if (sscanf(rest + 5, "%d %lf %d %d", &nd.feature, &nd.threshold, &nd.left, &nd.right) != 4 || nd.feature < 0 ||
+                    nd.feature >= kTreeFeatures || nd.left <= idx || nd.right <= idx || nd.left >= (int)cur_tree->size() ||
+                    nd.right >= (int)cur_tree->size()) { st = BSA_ERR_LUT; break; }  // children after parents: no cycles
+            } else if (!strncmp(rest, "leaf", 4)) {
+                const char* colon = strchr(rest, ':');
+                nd.feature = -1;
+                if (!colon || !parse_ids(colon + 1, &nd.ranked)) { st = BSA_ERR_LUT; break; }
+            } else { st = BSA_ERR_LUT; break; }
+            --nodes_left;
         } else if (!strncmp(line, "catalog", 7)) {
             unsigned long long hsh = 0;
             if (sscanf(line + 7, "%llx", &hsh) != 1 || hsh != catalog_hash()) { st = BSA_ERR_LUT; break; }
@@ -234,16 +314,7 @@ bsa_status_t lut_load(const char* path) {
             if (sscanf(line + 6, "%d %d %d %d %d %d %d %d :%n", &k.B_Q, &k.B_KV, &k.d, &k.nb, &k.hb, &k.db, &k.sb, &k.rb,
                        &used) != 8 || used == 0) { st = BSA_ERR_LUT; break; }
             std::vector<int> ids;
-            const char* q = line + 6 + used;
-            char* end = nullptr;
-            while (true) {
-                long v = strtol(q, &end, 10);
-                if (end == q) break;
-                if (v < 0 || v >= kCatalogSize) { st = BSA_ERR_LUT; break; }
-                ids.push_back((int)v);
-                q = end;
-            }
-            if (st != BSA_OK || ids.empty()) { st = BSA_ERR_LUT; break; }
+            if (!parse_ids(line + 6 + used, &ids)) { st = BSA_ERR_LUT; break; }
             table[k] = ids;
         } else {
             st = BSA_ERR_LUT;
@@ -251,10 +322,11 @@ bsa_status_t lut_load(const char* path) {
         }
     }
     fclose(f);
-    if (st == BSA_OK && !(header && hash_ok)) st = BSA_ERR_LUT;
+    if (st == BSA_OK && (!(header && hash_ok) || nodes_left != 0)) st = BSA_ERR_LUT;
     if (st != BSA_OK) return st;
     std::lock_guard<std::mutex> lk(g_mu);
     g_table.swap(table);
+    g_trees.swap(trees);
     return BSA_OK;
 }
 
@@ -276,10 +348,25 @@ int lut_select(int B_Q, int B_KV, int64_t N, int heads, int d, double density, d
     bool hit = false;
     {
         std::lock_guard<std::mutex> lk(g_mu);
-        auto it = g_table.find(k);
-        if (it != g_table.end()) {
-            ranked = it->second;
-            hit = true;
+        TreeKey tk;
+        memset(&tk, 0, sizeof tk);
+        tk.B_Q = B_Q; tk.B_KV = B_KV; tk.d = d;
+        auto tt = g_trees.find(tk);
+        if (tt != g_trees.end()) {  // learned thresholds for this key: the leaf is the regime
+            const double f[kTreeFeatures] = {log2((double)(N > 0 ? N : 1)), (double)heads, density, skew, run_cov};
+            const int leaf = tree_leaf(tt->second, f);
+            if (leaf >= 0) {
+                ranked = tt->second[leaf].ranked;
+                hit = true;
+                if (buckets_out) buckets_out[3] = b[3] | ((leaf + 1) << 8);  // leaf index + 1 above the run-coverage bucket
+            }
+        }
+        if (!hit) {
+            auto it = g_table.find(k);
+            if (it != g_table.end()) {
+                ranked = it->second;
+                hit = true;
+            }
         }
     }
     if (!hit) ranked.push_back(base_plan(B_Q, B_KV, d));

@@ -237,9 +237,11 @@ __global__ void __launch_bounds__(256) mask_row_stats_packed_kernel(const uint32
 __global__ void __launch_bounds__(256) csr_fill_packed_kernel(const uint32_t* __restrict__ mask, long long stride_words,
                                                                int nrows, int nKb, const int32_t* __restrict__ row_ptr,
                                                                int32_t* __restrict__ col_idx) {
+    __shared__ int32_t stage[8][1024];  // a step of the packed format covers 32 x 32 block columns
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row = blockIdx.x * 8 + warp;
     if (row >= nrows) return;
+    int32_t* buf = stage[warp];
     const uint32_t* r = mask + (long long)row * stride_words;
     const int nwords = (nKb + 31) >> 5;
     int32_t out = row_ptr[row];
@@ -253,14 +255,19 @@ __global__ void __launch_bounds__(256) csr_fill_packed_kernel(const uint32_t* __
             const int x = __shfl_up_sync(kFull, incl, o);
             if (lane >= o) incl += x;
         }
-        int pos = out + incl - cnt;
+        const int total = __shfl_sync(kFull, incl, 31);
+        if (total == 0) continue;
+        int pos = incl - cnt;
         const int col0 = (w + lane) * 32;
         while (m) {
             const int b = __ffs(m) - 1;
-            col_idx[pos++] = col0 + b;
+            buf[pos++] = col0 + b;
             m &= m - 1;
         }
-        out += __shfl_sync(kFull, incl, 31);
+        __syncwarp();
+        for (int j = lane; j < total; j += 32) col_idx[out + j] = buf[j];  // consecutive lanes, coalesced
+        __syncwarp();
+        out += total;
     }
 }
 
@@ -319,104 +326,212 @@ __global__ void __launch_bounds__(1024) row_scan_kernel(const int32_t* __restric
 
 // ------------------------------------------------------------------------------------------
 // csr_fill: one warp per row; a warp scan over the lanes' popcounts keeps columns ascending.
+// The indices of a step (up to 512) are first put in order into a shared-memory buffer of the
+// warp and then written out by consecutive lanes, so the global stores are coalesced 128-byte
+// runs instead of one 4-byte store per active block scattered over the lanes.
 // ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void flush_step_indices(const int32_t* buf, int32_t* __restrict__ dst, int n, int lane) {
+    for (int j = lane; j < n; j += 32) dst[j] = buf[j];
+}
+
 __global__ void __launch_bounds__(256) csr_fill_kernel(const uint8_t* __restrict__ mask, int nrows, int nKb,
                                                         const int32_t* __restrict__ row_ptr,
                                                         int32_t* __restrict__ col_idx) {
+    __shared__ int32_t stage[8][512];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row = blockIdx.x * 8 + warp;
     if (row >= nrows) return;
+    int32_t* buf = stage[warp];
     const unsigned long long base = reinterpret_cast<unsigned long long>(mask);
     const uint4* words = reinterpret_cast<const uint4*>(base & ~15ull);
     const long long rb = (long long)(base & 15ull) + (long long)row * nKb, re = rb + nKb;
     const long long w0 = rb >> 4, w1 = (re + 15) >> 4;
     int32_t out = row_ptr[row];
+    // two steps' words are in flight ahead of the one being written out
     unsigned m_next = row_word_bits(words, w0 + lane, rb, re);
+    unsigned m_next2 = (w0 + 32 < w1) ? row_word_bits(words, w0 + 32 + lane, rb, re) : 0u;
     for (long long w = w0; w < w1; w += 32) {
-        unsigned m = m_next;  // the next step's words are loaded before this step's are written out
-        m_next = (w + 32 < w1) ? row_word_bits(words, w + 32 + lane, rb, re) : 0u;
+        unsigned m = m_next;
+        m_next = m_next2;
+        m_next2 = (w + 64 < w1) ? row_word_bits(words, w + 64 + lane, rb, re) : 0u;
         const int cnt = __popc(m);
         int incl = cnt;
         for (int o = 1; o < 32; o <<= 1) {
             const int x = __shfl_up_sync(kFull, incl, o);
             if (lane >= o) incl += x;
         }
-        int pos = out + incl - cnt;
+        const int total = __shfl_sync(kFull, incl, 31);
+        if (total == 0) continue;
+        int pos = incl - cnt;
         const int col0 = (int)((w + lane) * 16 - rb);  // column of this word's byte 0
         while (m) {
             const int b = __ffs(m) - 1;
-            col_idx[pos++] = col0 + b;
+            buf[pos++] = col0 + b;
             m &= m - 1;
         }
-        out += __shfl_sync(kFull, incl, 31);
+        __syncwarp();
+        flush_step_indices(buf, col_idx + out, total, lane);
+        __syncwarp();
+        out += total;
     }
 }
 
 // ------------------------------------------------------------------------------------------
-// tile_map: one CTA per physical Q tile row.  A shared-memory array holds one membership word
-// per KV tile column; the active blocks of the tile row's logical rows OR their bit into it
-// (Coarsened), or name `rk` finer tile columns each (Refined, column c -> c*rk .. c*rk+rk-1).
-// Non-zero words are then compacted in column order.  Output position of tile row t is a
-// capacity offset computed from the block-CSR alone, so no second scan is needed.
+// tile_map.  Output position of tile row t is a capacity offset computed from the block-CSR alone
+// (row_ptr of its first logical row times the refinement factors), so no second scan is needed.
+//
+// Two kernels.  Where no dimension is Coarsened (B_Q >= T_Q and B_KV >= T_KV: Direct or Refined),
+// the tile list of a tile row is the column list of its logical row, each column c expanded to
+// c*rk .. c*rk+rk-1: already sorted and unique, every membership word all-ones.  One WARP per
+// tile row streams it out (tile_map_expand_kernel).  Where a dimension is Coarsened, one CTA per
+// tile row ORs the activity bits of its logical rows into a shared-memory array with one
+// membership word per KV tile column and compacts the non-zero words in column order
+// (tile_map_bitmap_kernel).
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t* __restrict__ row_ptr,
-                                                        const int32_t* __restrict__ col_idx, int split_tau,
-                                                        int split_pmax, int32_t* __restrict__ tile_begin,
-                                                        int32_t* __restrict__ tile_cnt, int32_t* __restrict__ row_parts,
-                                                        int32_t* __restrict__ tile_col,
-                                                        uint64_t* __restrict__ tile_member,
-                                                        int32_t* __restrict__ head_counts, PlanCountersDev* counters) {
+__device__ __forceinline__ int32_t split_parts(int32_t cnt, int split_tau, int split_pmax) {
+    if (split_pmax > 1 && cnt > split_tau) return min(split_pmax, (cnt + split_tau - 1) / split_tau);
+    return 1;
+}
+
+__global__ void __launch_bounds__(256) tile_map_expand_kernel(MapGeom g, const int32_t* __restrict__ row_ptr,
+                                                               const int32_t* __restrict__ col_idx, int split_tau,
+                                                               int split_pmax, int32_t* __restrict__ tile_begin,
+                                                               int32_t* __restrict__ tile_cnt, int32_t* __restrict__ row_parts,
+                                                               int32_t* __restrict__ tile_col,
+                                                               uint64_t* __restrict__ tile_member,
+                                                               int32_t* __restrict__ head_counts, PlanCountersDev* counters) {
+    __shared__ int32_t w_head[8], w_parts[8], w_cnt[8];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // see organize_kernel
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int trow = blockIdx.x * 8 + warp;
+    const int nrows = g.H * g.nQt;
+    int32_t cnt = 0, P = 0, h = -1;
+    if (trow < nrows) {
+        h = trow / g.nQt;
+        const int t = trow % g.nQt;
+        const int r = t / g.rq, sub = t % g.rq;
+        const int32_t b = row_ptr[h * g.nQb + r], e = row_ptr[h * g.nQb + r + 1];
+        const int32_t len = e - b;
+        const int32_t cap_begin = (b * g.rq + sub * len) * g.rk;
+        // Only the row's last column can lose part of its rk tile columns (ragged N_kv), so positions have no holes.
+        for (int32_t i0 = 0; i0 < len; i0 += 128) {
+            int32_t c[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) c[u] = (i0 + u * 32 + lane < len) ? col_idx[b + i0 + u * 32 + lane] : -1;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (c[u] < 0) continue;
+                const int32_t pos = cap_begin + (i0 + u * 32 + lane) * g.rk;
+                for (int k = 0; k < g.rk; ++k) {
+                    const int tc = c[u] * g.rk + k;
+                    if (tc >= g.nKt) break;
+                    tile_col[pos + k] = tc;
+                    tile_member[(size_t)(pos + k) * g.slots] = 1ull;
+                    if (g.slots == 2) tile_member[(size_t)(pos + k) * 2 + 1] = 1ull;
+                }
+            }
+        }
+        if (lane == 0) {
+            cnt = len * g.rk;
+            if (len > 0) {
+                const int last = col_idx[e - 1];
+                const int lost = (last + 1) * g.rk - g.nKt;
+                if (lost > 0) cnt -= lost;
+            }
+            P = split_parts(cnt, split_tau, split_pmax);
+            tile_begin[trow] = cap_begin;
+            tile_cnt[trow] = cnt;
+            row_parts[trow] = P;
+        }
+    }
+    if (lane == 0) {
+        w_head[warp] = h;
+        w_parts[warp] = P;
+        w_cnt[warp] = cnt;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {  // one set of atomics per head that this CTA's eight tile rows touch (one or two heads)
+        unsigned long long tot = 0;
+        int w = 0;
+        while (w < 8 && w_head[w] >= 0) {
+            const int hh = w_head[w];
+            int32_t items = 0, nsplit = 0, slots = 0;
+            for (; w < 8 && w_head[w] == hh; ++w) {
+                items += w_parts[w];
+                if (w_parts[w] > 1) {
+                    ++nsplit;
+                    slots += w_parts[w];
+                }
+                tot += (unsigned long long)w_cnt[w];
+            }
+            atomicAdd(&head_counts[3 * hh + 0], items);
+            if (nsplit) {
+                atomicAdd(&head_counts[3 * hh + 1], nsplit);
+                atomicAdd(&head_counts[3 * hh + 2], slots);
+            }
+        }
+        if (tot) {
+            atomicAdd(&counters->ntiles, tot);
+            atomicAdd(&counters->nslot_tiles, tot * (unsigned long long)g.slots);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256) tile_map_bitmap_kernel(MapGeom g, const int32_t* __restrict__ row_ptr,
+                                                               const int32_t* __restrict__ col_idx, int split_tau,
+                                                               int split_pmax, int32_t* __restrict__ tile_begin,
+                                                               int32_t* __restrict__ tile_cnt, int32_t* __restrict__ row_parts,
+                                                               int32_t* __restrict__ tile_col,
+                                                               uint64_t* __restrict__ tile_member,
+                                                               int32_t* __restrict__ head_counts, PlanCountersDev* counters) {
     extern __shared__ unsigned long long bm[];  // [slots][nKt]: one membership word per 128-row slot
     __shared__ int32_t warp_cnt[8];
     __shared__ int32_t warp_slot_cnt[8];
+    __shared__ int32_t rp[20];  // CSR offsets of the tile row's logical rows (at most 16 of them, plus the end)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // see organize_kernel
     const int trow = blockIdx.x;
     const int h = trow / g.nQt, t = trow % g.nQt;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // the logical rows this tile row reads: sQ of them (Coarsened or Direct along Q), or one (Refined along Q)
+    const int r0 = (g.rq == 1) ? t * g.sQ : t / g.rq;
+    const int nr = (g.rq == 1) ? min(g.sQ, g.nQb - r0) : 1;
+    if (tid <= nr) rp[tid] = row_ptr[h * g.nQb + r0 + tid];
     for (int i = tid; i < g.nKt * g.slots; i += blockDim.x) bm[i] = 0ull;
     __syncthreads();
 
+    // All entries of the tile row are one contiguous range of the column-index array (its logical rows are adjacent
+    // in the block-CSR): one flat loop with four independent loads per thread in flight; the logical row of an entry
+    // is the number of row boundaries at or below its index.
+    const int32_t e0 = rp[0], e1 = rp[nr];
     int32_t cap_begin;
     if (g.rq == 1) {
-        const int r0 = t * g.sQ;
-        const int r1 = min(r0 + g.sQ, g.nQb);
-        const int32_t base = row_ptr[h * g.nQb + r0];
-        cap_begin = base * g.rk;
-        for (int r = r0; r < r1; ++r) {
-            const int a = r - r0;
+        cap_begin = e0 * g.rk;
+    } else {
+        cap_begin = (e0 * g.rq + (t % g.rq) * (e1 - e0)) * g.rk;
+    }
+    for (int32_t i0 = e0 + tid; i0 < e1; i0 += 4 * 256) {
+        int32_t c[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) c[u] = (i0 + u * 256 < e1) ? col_idx[i0 + u * 256] : -1;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (c[u] < 0) continue;
+            const int32_t i = i0 + u * 256;
+            int a = 0;
+            for (int k = 1; k < nr; ++k) a += (i >= rp[k]) ? 1 : 0;
             // which 128-row slot(s) the logical row feeds, and its sub-row inside the slot
             const int slot_lo = (g.B_Q >= g.T_Q) ? 0 : a / g.sQ128;
             const int slot_hi = (g.B_Q >= g.T_Q) ? g.slots - 1 : slot_lo;
-            const int arow = a % g.sQ128;
-            const int32_t b = row_ptr[h * g.nQb + r], e = row_ptr[h * g.nQb + r + 1];
-            for (int32_t i = b + tid; i < e; i += blockDim.x) {
-                const int c = col_idx[i];
-                for (int sl = slot_lo; sl <= slot_hi; ++sl) {
-                    unsigned long long* w = bm + (size_t)sl * g.nKt;
-                    if (g.rk == 1) {
-                        atomicOr(&w[c >> g.lgSK], 1ull << (arow * g.sK + (c & (g.sK - 1))));
-                    } else {
-                        for (int k = 0; k < g.rk; ++k) {
-                            const int tc = c * g.rk + k;
-                            if (tc < g.nKt) atomicOr(&w[tc], 1ull << arow);
-                        }
+            const int arow = (g.rq == 1) ? a % g.sQ128 : 0;
+            for (int sl = slot_lo; sl <= slot_hi; ++sl) {
+                unsigned long long* w = bm + (size_t)sl * g.nKt;
+                if (g.rk == 1) {
+                    atomicOr(&w[c[u] >> g.lgSK], 1ull << (arow * g.sK + (c[u] & (g.sK - 1))));
+                } else {
+                    for (int k = 0; k < g.rk; ++k) {
+                        const int tc = c[u] * g.rk + k;
+                        if (tc < g.nKt) atomicOr(&w[tc], 1ull << arow);
                     }
-                }
-            }
-        }
-    } else {
-        // Refined along Q (B_Q > T_Q): tile row t is the `sub`-th part of logical row r; one slot
-        const int r = t / g.rq, sub = t % g.rq;
-        const int32_t b = row_ptr[h * g.nQb + r], e = row_ptr[h * g.nQb + r + 1];
-        cap_begin = (b * g.rq + sub * (e - b)) * g.rk;
-        for (int32_t i = b + tid; i < e; i += blockDim.x) {
-            const int c = col_idx[i];
-            if (g.rk == 1) {
-                atomicOr(&bm[c >> g.lgSK], 1ull << (c & (g.sK - 1)));
-            } else {
-                for (int k = 0; k < g.rk; ++k) {
-                    const int tc = c * g.rk + k;
-                    if (tc < g.nKt) bm[tc] = 1ull;
                 }
             }
         }
@@ -466,8 +581,7 @@ __global__ void __launch_bounds__(256) tile_map_kernel(MapGeom g, const int32_t*
         const int32_t cnt = total;
         tile_begin[trow] = cap_begin;
         tile_cnt[trow] = cnt;
-        int32_t P = 1;
-        if (split_pmax > 1 && cnt > split_tau) P = min(split_pmax, (cnt + split_tau - 1) / split_tau);
+        const int32_t P = split_parts(cnt, split_tau, split_pmax);
         row_parts[trow] = P;
         atomicAdd(&head_counts[3 * h + 0], P);
         if (P > 1) {
@@ -778,14 +892,21 @@ cudaError_t launch_tile_map(const MapGeom& g, const int32_t* row_ptr, const int3
                             int split_pmax, int32_t* tile_begin, int32_t* tile_cnt, int32_t* row_parts,
                             int32_t* tile_col, uint64_t* tile_member, int32_t* head_counts, PlanCountersDev* counters,
                             cudaStream_t stream) {
+    if (g.sQ == 1 && g.sK == 1) {  // Direct or Refined in both dimensions: no membership bitmap needed
+        tile_map_expand_kernel<<<(g.H * g.nQt + 7) / 8, 256, 0, stream>>>(g, row_ptr, col_idx, split_tau, split_pmax,
+                                                                          tile_begin, tile_cnt, row_parts, tile_col,
+                                                                          tile_member, head_counts, counters);
+        count_launch();
+        return cudaGetLastError();
+    }
     const size_t smem = (size_t)g.nKt * g.slots * sizeof(unsigned long long);
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(tile_map_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (smem > 40 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(tile_map_bitmap_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    tile_map_kernel<<<g.H * g.nQt, 256, smem, stream>>>(g, row_ptr, col_idx, split_tau, split_pmax, tile_begin,
-                                                        tile_cnt, row_parts, tile_col, tile_member, head_counts,
-                                                        counters);
+    tile_map_bitmap_kernel<<<g.H * g.nQt, 256, smem, stream>>>(g, row_ptr, col_idx, split_tau, split_pmax, tile_begin,
+                                                               tile_cnt, row_parts, tile_col, tile_member, head_counts,
+                                                               counters);
     count_launch();
     return cudaGetLastError();
 }

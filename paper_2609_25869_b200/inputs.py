@@ -157,25 +157,26 @@ def config_tiny(seed: int = 0, H: int = 2, N: int = 2048, d: int = 64, B: int = 
     return Request("tiny", H, N, d, B, B, M, qkv_seed=seed, note=f"Bernoulli({p}) + diagonal")
 
 
-def config_mid(seed: int = 1, H: int = 8) -> Request:
+def config_mid(seed: int = 1, H: int = 8, extra: float = 0.02, win: Tuple[int, int, int] = (1, 1, 1)) -> Request:
     grid = (8, 4, 4)  # 16x32x32 latent in 2x8x8-token tiles -> 128 blocks of 128 tokens
     nb = 128
-    W = window_mask(grid, (1, 1, 1))
+    W = window_mask(grid, win)
     h, i, j = np.meshgrid(np.arange(H), np.arange(nb), np.arange(nb), indexing="ij")
-    M = (W[None] | bernoulli(0.02, seed, 2, h, i, j)).astype(np.uint8)
-    return Request("mid", H, 16384, 128, 128, 128, M, qkv_seed=seed, note="3-D window(1,1,1) + Bernoulli(0.02)")
+    M = (W[None] | bernoulli(extra, seed, 2, h, i, j)).astype(np.uint8)
+    return Request("mid", H, 16384, 128, 128, 128, M, qkv_seed=seed,
+                   note=f"3-D window({win[0]},{win[1]},{win[2]}) + Bernoulli({extra})")
 
 
-def config_hunyuan(seed: int = 2, H: int = 24) -> Request:
+def config_hunyuan(seed: int = 2, H: int = 24, extra: float = 0.03, win: Tuple[int, int, int] = (1, 1, 2)) -> Request:
     grid = (15, 6, 10)  # 30x48x80 latent in 2x8x8-token tiles -> 900 blocks of 128 tokens
     nb = 900
-    W = window_mask(grid, (1, 1, 2))
+    W = window_mask(grid, win)
     M = np.empty((H, nb, nb), dtype=np.uint8)
     i, j = np.meshgrid(np.arange(nb), np.arange(nb), indexing="ij")
     for h in range(H):
-        M[h] = W | bernoulli(0.03, seed * 1000 + h, 3, i, j)
+        M[h] = W | bernoulli(extra, seed * 1000 + h, 3, i, j)
     return Request("hunyuan", H, 115200, 128, 128, 128, M, qkv_seed=seed,
-                   note="3-D window(1,1,2) + per-head Bernoulli(0.03)")
+                   note=f"3-D window({win[0]},{win[1]},{win[2]}) + per-head Bernoulli({extra})")
 
 
 def _runs_row(nKb: int, target: int, seed: int, h: int, i: int) -> np.ndarray:
@@ -207,25 +208,25 @@ def _runs_row(nKb: int, target: int, seed: int, h: int, i: int) -> np.ndarray:
     return row
 
 
-def config_stress_a(seed: int = 3, H: int = 16, N: int = 32768) -> Request:
+def config_stress_a(seed: int = 3, H: int = 16, N: int = 32768, density: float = 0.15) -> Request:
     B_Q, B_KV = 16, 64
     nQb, nKb = cdiv(N, B_Q), cdiv(N, B_KV)
-    target = int(round(0.15 * nKb))
+    target = max(1, int(round(density * nKb)))
     M = np.zeros((H, nQb, nKb), dtype=np.uint8)
     for h in range(H):
         for i in range(nQb):
             M[h, i] = _runs_row(nKb, target, seed, h, i)
     return Request("stress_a", H, N, 64, B_Q, B_KV, M, qkv_seed=3,
-                   note="4-12 contiguous runs per row, geometric lengths rescaled to 15% density")
+                   note=f"4-12 contiguous runs per row, geometric lengths rescaled to {density:.0%} density")
 
 
-def config_stress_b(seed: int = 4, H: int = 16, N: int = 32768) -> Request:
+def config_stress_b(seed: int = 4, H: int = 16, N: int = 32768, p: float = 0.2) -> Request:
     B = 256
     nb = cdiv(N, B)
     h, i, j = np.meshgrid(np.arange(H), np.arange(nb), np.arange(nb), indexing="ij")
-    M = bernoulli(0.2, seed, 4, h, i, j).astype(np.uint8)
+    M = bernoulli(p, seed, 4, h, i, j).astype(np.uint8)
     M[:, np.arange(nb), np.arange(nb)] = 1
-    return Request("stress_b", H, N, 64, B, B, M, qkv_seed=3, note="Bernoulli(0.2) + diagonal")
+    return Request("stress_b", H, N, 64, B, B, M, qkv_seed=3, note=f"Bernoulli({p}) + diagonal")
 
 
 SWEEP_GEOMETRIES: List[Tuple[int, int]] = [(32, 32), (64, 128), (128, 64), (128, 128), (256, 256)]

@@ -3,8 +3,8 @@
 For every profiling case (a seeded synthetic mask with its request parameters) and every
 eligible catalog plan: run the plan, validate its output (Algorithm 1, lines 4-6), and record
 the median forward latency.  Validation has two parts.  (1) A masked-attention reference:
-``validator(req, plan_id, O, LSE) -> bool``, applied to every plan including the key's base
-plan.  The default, ``sampled_reference_validator``, recomputes seeded query blocks of every
+``validator(req, plan_id, O, LSE, qkv) -> bool`` (``qkv``: the CUDA tensors the plan ran on),
+applied to every plan including the key's base plan.  The default, ``sampled_reference_validator``, recomputes seeded query blocks of every
 head with plain fp32 torch operations on the expanded token-pair mask (dense scores, softmax,
 product with V) and compares O and LSE at the contract tolerances; a caller may pass its own
 (the tests pass one built on the CPU oracle).  (2) Agreement with the validated base plan's
@@ -62,10 +62,136 @@ def compile_table(cases: Sequence[Tuple[Hashable, Hashable]], latencies: Dict[Tu
     return table
 
 
-def write_table(path: str, table: Dict, catalog_hash: int, gpu_name: str, notes: Iterable[str] = ()):
-    """Regime line: ``regime B_Q B_KV d nb hb db sb rb : ranked plan ids``."""
+# --------------------------------------------------------------------------------------------
+# Second stage with learned thresholds (Section 5.1): a decision tree per request key over the
+# continuous request features; its leaves are the regimes.  Pure host logic (unit-tested on the CPU).
+# --------------------------------------------------------------------------------------------
+TREE_FEATURES = ("log2_N", "heads", "density", "skew", "run_coverage")  # indices as the runtime reads them
+
+
+def case_features(N: int, heads: int, density: float, skew: float, run_coverage: float) -> Tuple[float, ...]:
+    return (math.log2(max(1, N)), float(heads), float(density), float(skew), float(run_coverage))
+
+
+def _case_best(cid, lat) -> float:
+    ts = [t for (c, _), t in lat.items() if c == cid]
+    return min(ts) if ts else float("nan")
+
+
+def _ranking_and_loss(cids, lat, base: int):
+    """Ranking of a leaf as in Algorithm 1, lines 15-19 (plans valid on every case of the leaf by geometric-mean
+    latency, ties by id, base plan last) and the leaf's loss: the summed log-regret of its cases under the ranking's
+    head (a case the head has no latency for falls through the ranking like the runtime's ranked fallback; one that no
+    ranked plan serves is charged its slowest measured plan)."""
+    cand = None
+    for c in cids:
+        have = {p for (cc, p) in lat if cc == c}
+        cand = have if cand is None else cand & have
+    cand = cand or set()
+    gm = {p: math.exp(sum(math.log(lat[(c, p)]) for c in cids) / len(cids)) for p in cand}
+    ranked = sorted(cand, key=lambda p: (gm[p], p)) + [base]
+    return ranked, sum(case_log_regret(c, ranked, lat) for c in cids)
+
+
+def case_log_regret(cid, ranked, lat) -> float:
+    best = _case_best(cid, lat)
+    if not best == best:   # no measurement at all for this case
+        return 0.0
+    for p in ranked:
+        if (cid, p) in lat:
+            return math.log(lat[(cid, p)] / best)
+    return math.log(max(t for (c, _), t in lat.items() if c == cid) / best)
+
+
+def learn_tree(cids, feats, lat, base: int, min_leaf: int = 8, max_depth: int = 3):
+    """Greedy binary tree: at every node the (feature, threshold) whose two children have the smallest summed loss,
+    thresholds taken half-way between neighbouring distinct feature values, both children at least ``min_leaf`` cases;
+    a node stays a leaf when no split lowers its loss.  Returns nodes in pre-order (children after their parent):
+    ``{"feature": f, "threshold": t, "left": i, "right": j}`` or ``{"ranked": [...], "cases": n}``."""
+    nodes: List[dict] = []
+
+    def build(members, depth):
+        idx = len(nodes)
+        nodes.append({})
+        ranked, loss = _ranking_and_loss(members, lat, base)
+        best = None
+        if depth < max_depth and len(members) >= 2 * min_leaf:
+            for f in range(len(TREE_FEATURES)):
+                order = sorted(members, key=lambda c: (feats[c][f], str(c)))
+                vals = [feats[c][f] for c in order]
+                for k in range(min_leaf, len(order) - min_leaf + 1):
+                    if vals[k] == vals[k - 1]:
+                        continue
+                    thr = 0.5 * (vals[k] + vals[k - 1])
+                    lo, hi = order[:k], order[k:]
+                    total = _ranking_and_loss(lo, lat, base)[1] + _ranking_and_loss(hi, lat, base)[1]
+                    if best is None or total < best[0] - 1e-12:
+                        best = (total, f, thr, lo, hi)
+        if best is not None and best[0] < loss - 1e-9:
+            _, f, thr, lo, hi = best
+            nodes[idx] = {"feature": f, "threshold": thr}
+            nodes[idx]["left"] = build(lo, depth + 1)
+            nodes[idx]["right"] = build(hi, depth + 1)
+        else:
+            nodes[idx] = {"ranked": ranked, "cases": len(members)}
+        return idx
+
+    build(list(cids), 0)
+    return nodes
+
+
+def tree_leaf(nodes, feat) -> dict:
+    n = nodes[0]
+    while "ranked" not in n:
+        n = nodes[n["left"] if feat[n["feature"]] < n["threshold"] else n["right"]]
+    return n
+
+
+def choose_depth(cids, feats, groups, lat, base: int, min_leaf: int = 8, depths=(0, 1, 2, 3, 4), folds: int = 4):
+    """Tree depth by grouped cross-validation (Section 5.1: masks from the same source stay in one fold): the depth
+    with the smallest mean held-out log-regret, the smaller depth on ties.  Returns (depth, {depth: mean log-regret})."""
+    names = sorted({groups[c] for c in cids}, key=str)
+    fold_of = {g: i % folds for i, g in enumerate(names)}
+    score = {}
+    for D in depths:
+        tot, n = 0.0, 0
+        for f in range(min(folds, len(names))):
+            train = [c for c in cids if fold_of[groups[c]] != f]
+            held = [c for c in cids if fold_of[groups[c]] == f]
+            if not train or not held:
+                continue
+            tree = learn_tree(train, feats, lat, base, min_leaf, D)
+            for c in held:
+                tot += case_log_regret(c, tree_leaf(tree, feats[c])["ranked"], lat)
+                n += 1
+        score[D] = tot / max(1, n)
+    best = min(score, key=lambda D: (round(score[D], 9), D))
+    return best, score
+
+
+def compile_trees(cases, feats, groups, lat, base_plan, min_leaf: int = 8, max_depth: int = 4, folds: int = 4, log=None):
+    """One tree per request key that has at least ``2 * min_leaf`` cases; the others keep the fixed-edge regimes."""
+    by_key: Dict[Hashable, List[Hashable]] = {}
+    for cid, key in cases:
+        by_key.setdefault(key, []).append(cid)
+    trees = {}
+    for key, members in sorted(by_key.items()):
+        if len(members) < 2 * min_leaf:
+            continue
+        depth, score = choose_depth(members, feats, groups, lat, base_plan[key], min_leaf, tuple(range(max_depth + 1)), folds)
+        trees[key] = learn_tree(members, feats, lat, base_plan[key], min_leaf, depth)
+        if log:
+            log(f"tree {key}: {len(members)} cases, depth {depth} chosen from held-out regret "
+                + ", ".join(f"{D}: {math.exp(v):.4f}" for D, v in sorted(score.items()))
+                + f"; {sum(1 for n in trees[key] if 'ranked' in n)} leaves")
+    return trees
+
+
+def write_table(path: str, table: Dict, catalog_hash: int, gpu_name: str, notes: Iterable[str] = (), trees: Dict = None):
+    """Regime line: ``regime B_Q B_KV d nb hb db sb rb : ranked plan ids``; with ``trees`` the file is version 2 and
+    carries, per request key, ``tree B_Q B_KV d n`` followed by its ``node`` lines (pre-order, node 0 the root)."""
     with open(path, "w") as f:
-        f.write("BSA_LUT 1\n")
+        f.write(f"BSA_LUT {2 if trees else 1}\n")
         f.write(f"catalog {catalog_hash:x}\n")
         f.write(f"gpu {gpu_name}\n")
         for n in notes:
@@ -73,37 +199,87 @@ def write_table(path: str, table: Dict, catalog_hash: int, gpu_name: str, notes:
         for (key, bucket), ranked in sorted(table.items()):
             f.write("regime " + " ".join(str(x) for x in tuple(key) + tuple(bucket)) + " : " +
                     " ".join(str(p) for p in ranked) + "\n")
+        for key, nodes in sorted((trees or {}).items()):
+            f.write("tree " + " ".join(str(x) for x in key) + f" {len(nodes)}\n")
+            for i, n in enumerate(nodes):
+                if "ranked" in n:
+                    f.write(f"node {i} leaf : " + " ".join(str(p) for p in n["ranked"]) + "\n")
+                else:
+                    f.write(f"node {i} split {n['feature']} {n['threshold']!r} {n['left']} {n['right']}\n")
 
 
 # --------------------------------------------------------------------------------------------
 # profiling corpus
 # --------------------------------------------------------------------------------------------
-def corpus(scale: str = "full"):
-    """Seeded requests shaped like the five evaluation configurations (seeds >= 1000)."""
+def corpus_specs(scale: str = "full"):
+    """The profiling corpus as (generator name, keyword arguments, source group) triples: the five evaluation
+    generators with seeds >= 1000 and with head counts, token counts and densities spread over and BETWEEN the values
+    the evaluation configurations use, several cases per request key and regime.  ``source group`` names the mask
+    source for grouped cross-validation (cases that differ only in head count or seed offset share a source)."""
+    specs = []
+
+    def add(gen, group, **kw):
+        specs.append((gen, kw, group))
+
+    if scale == "quick":
+        for s in range(2):
+            add("tiny", f"tiny{s}", seed=1000 + s)
+        add("mid", "mid0", seed=1010)
+        add("stress_b", "sb0", seed=1030, H=4, N=8192)
+        return specs
+    # (64,64) d=64: Tiny's key
+    n = 0
+    for N in (1024, 2048, 4096, 8192):
+        for H, p in ((2, 0.25), (4, 0.1), (8, 0.4), (16, 0.05)):
+            add("tiny", f"tiny{n // 2}", seed=1000 + n, H=H, N=N, p=p)
+            n += 1
+    # (128,128) d=128: Mid and Hunyuan shapes, and the sweep's (128,128) requests
+    n = 0
+    for H in (1, 2, 4, 8, 16, 24):
+        for extra, win in ((0.02, (1, 1, 1)), (0.0, (1, 1, 1)), (0.1, (1, 1, 1)), (0.02, (2, 1, 1)), (0.3, (0, 0, 0))):
+            add("mid", f"mid{n // 2}", seed=1100 + n, H=H, extra=extra, win=win)
+            n += 1
+    n = 0
+    for H in (3, 6, 12, 24):
+        for extra, win in ((0.03, (1, 1, 2)), (0.0, (1, 1, 2)), (0.08, (1, 1, 1)), (0.01, (2, 2, 2))):
+            add("hunyuan", f"hy{n // 2}", seed=1200 + n, H=H, extra=extra, win=win)
+            n += 1
+    # (16,64) and (256,256) d=64: the two stress keys
+    n = 0
+    for N, H in ((8192, 16), (16384, 8), (32768, 16), (32768, 4)):
+        for dens in (0.05, 0.1, 0.15, 0.3):
+            add("stress_a", f"sa{n // 2}", seed=1300 + n, H=H, N=N, density=dens)
+            add("stress_b", f"sb{n // 2}", seed=1400 + n, H=H, N=N, p=min(0.6, dens * 1.4))
+            n += 1
+    # the sweep's five geometries (d=128, N=75600), densities on and between the sweep's targets
+    n = 0
+    for H in (6, 12, 24):  # head count outermost: the cases of one shape follow each other and share their tensors
+        for B in ((32, 32), (64, 128), (128, 64), (128, 128), (256, 256)):
+            for rho in (0.03, 0.05, 0.1, 0.17, 0.3, 0.45, 0.6):
+                add("sweep", f"sw{B[0]}x{B[1]}@{rho}", r=1000 + n, H=H, B=B, rho=rho)
+                n += 1
+    return specs
+
+
+def make_case(spec):
+    """One corpus case from its spec (host only; runs in the generation pool)."""
     from . import inputs as I
-    reqs = []
-    nseed = 1 if scale == "quick" else 2
-    for s in range(nseed):
-        reqs.append(I.config_tiny(seed=1000 + s))
-        reqs.append(I.config_mid(seed=1010 + s))
-        reqs.append(I.config_stress_b(seed=1030 + s))
-        r = I.config_stress_a(seed=1040 + s)
-        reqs.append(r)
-    reqs.append(I.config_hunyuan(seed=1020))
-    if scale != "quick":
-        # the same shapes with few heads (head bucket <= 4): what a head-sharded or head-pipelined request looks like
-        for n, h in enumerate((1, 2, 3, 4)):
-            reqs.append(I.config_mid(seed=1050 + n, H=h))
-        reqs.append(I.config_hunyuan(seed=1060, H=3))
-        k = 0
-        for B in I.SWEEP_GEOMETRIES:
-            for rho in I.SWEEP_DENSITIES:
-                reqs.append(I.config_sweep(1000 + k, B=B, rho=rho))
-                k += 1
-    for n, r in enumerate(reqs):
+    gen, kw, group = spec
+    fn = I.config_sweep if gen == "sweep" else I.CONFIGS[gen]
+    req = fn(**kw)
+    return req, group
+
+
+def corpus(scale: str = "full"):
+    """The corpus as requests (generated in this process): ``(requests, {case name: source group})``."""
+    reqs, groups = [], {}
+    for n, spec in enumerate(corpus_specs(scale)):
+        r, g = make_case(spec)
         r.name = f"{r.name}#{n}"
         r.qkv_seed = 5000 + n
-    return reqs
+        reqs.append(r)
+        groups[r.name] = g
+    return reqs, groups
 
 
 def head_bucket(heads: int) -> int:
@@ -146,7 +322,7 @@ def sampled_reference_validator(blocks_per_head: int = 2, seed: int = 4242):
         cache[key] = out
         return out
 
-    def validate(req, plan_id, O, LSE, qkv=None):
+    def validate(req, plan_id, O, LSE, qkv):
         q, k, v = qkv
         err_o, n_o, max_o, max_l = 0.0, 0, 0.0, 0.0
         for h, r0, r1, refO, refL in reference(req, q, k, v):
@@ -163,15 +339,17 @@ def sampled_reference_validator(blocks_per_head: int = 2, seed: int = 4242):
                 max_l = max(max_l, float((LSE[h, r0:r1][fin] - refL[fin]).abs().max()))
         return max_o <= O_TOL and err_o / max(1, n_o) <= O_MEAN_TOL and max_l <= LSE_TOL
 
-    validate.wants_qkv = True
     return validate
 
 
-def profile(reqs, plans=None, reps: int = 5, warmup: int = 3, log=print, validator=None):
+def profile(reqs, plans=None, reps: int = 5, warmup: int = 3, log=print, validator=None, features_out=None):
     """Algorithm 1, "Profiling": returns (cases, latencies, buckets, base plans).
 
-    ``validator(req, plan_id, O, LSE) -> bool`` is the masked-attention reference of lines 4-6 (default:
-    ``sampled_reference_validator()``); a plan it rejects gets no latency.  If it rejects the key's base plan, the
+    ``validator(req, plan_id, O, LSE, qkv) -> bool`` is the masked-attention reference of lines 4-6 (default:
+    ``sampled_reference_validator()``); ``qkv`` are the CUDA tensors the plan ran on (cases of one shape share
+    them).  A plan it rejects gets no latency.  ``features_out`` (a dict) receives the continuous request features of
+    every case (``case_features``), which the tree compiler partitions on.  ``reqs`` may be any iterable (a generator
+    that produces the cases while earlier ones are profiled).  If it rejects the key's base plan, the
     case has no trusted full-size output to compare the other plans with and every plan is judged by it alone."""
     import torch
     from . import bsa
@@ -184,9 +362,7 @@ def profile(reqs, plans=None, reps: int = 5, warmup: int = 3, log=print, validat
     qkv_cache = {}
 
     def passes(req, pid, O, L, qkv):
-        if getattr(validator, "wants_qkv", False):
-            return bool(validator(req, pid, O, L, qkv=qkv))
-        return bool(validator(req, pid, O, L))
+        return bool(validator(req, pid, O, L, qkv))
 
     for req in reqs:
         key = (req.B_Q, req.B_KV, req.d)
@@ -207,6 +383,8 @@ def profile(reqs, plans=None, reps: int = 5, warmup: int = 3, log=print, validat
             log(f"  base plan {bp} failed validation on {req.name}")
         bk = tuple(inf["regime_bucket"])
         bucket[req.name] = (bk[0], head_bucket(req.H), bk[1], bk[2], bk[3])
+        if features_out is not None:
+            features_out[req.name] = case_features(req.N, req.H, inf["density"], inf["skew"], inf["run_coverage"])
         cases.append((req.name, key))
         fin = torch.isfinite(refL)
         row = []
@@ -248,20 +426,49 @@ def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--out", default=DEFAULT_OUT)
     ap.add_argument("--scale", default="full", choices=["full", "quick"])
+    ap.add_argument("--min-leaf", type=int, default=6, help="fewest cases a tree leaf may hold (the paper, with a corpus "
+                    "of tens of thousands of cases, uses 32)")
+    ap.add_argument("--max-depth", type=int, default=4)
+    ap.add_argument("--no-trees", action="store_true", help="fixed-edge regimes only")
+    ap.add_argument("--latencies", default="", help="also write the measured latencies as JSON (for the regret report)")
     args = ap.parse_args(argv)
+    specs = corpus_specs(args.scale)
+    # masks are generated by worker processes (forked before CUDA is touched) while earlier cases are profiled
+    import multiprocessing as mp
+    pool = mp.get_context("fork").Pool(max(1, min(12, (os.cpu_count() or 2) - 2)))
+    stream = pool.imap(make_case, specs)
     import torch
     from . import bsa
     bsa.lut_clear()
     t0 = time.time()
-    reqs = corpus(args.scale)
-    print(f"corpus: {len(reqs)} cases ({time.time() - t0:.0f} s to generate)")
-    cases, lat, bucket, base = profile(reqs)
+    groups = {}
+
+    def cases_in_order():
+        for n, (req, group) in enumerate(stream):
+            req.name = f"{req.name}#{n}"
+            req.qkv_seed = 5000 + n
+            groups[req.name] = group
+            yield req
+
+    print(f"corpus: {len(specs)} cases")
+    feats = {}
+    cases, lat, bucket, base = profile(cases_in_order(), features_out=feats)
+    pool.terminate()
     table = compile_table(cases, lat, base, lambda cid: bucket[cid])
+    trees = {} if args.no_trees else compile_trees(cases, feats, groups, lat, base, min_leaf=args.min_leaf,
+                                                   max_depth=args.max_depth, log=print)
     write_table(args.out, table, int(bsa.lib().bsa_catalog_hash()), torch.cuda.get_device_name(0),
                 notes=[f"{len(cases)} profiling cases, seeds >= 1000, median of 5 forwards after 3 warm-ups, L2 flushed",
-                       "regime B_Q B_KV d floor(log2 N) head-bucket density-bucket skew-bucket runcov-bucket : ranked plans, base last"])
+                       "regime B_Q B_KV d floor(log2 N) head-bucket density-bucket skew-bucket runcov-bucket : ranked plans, base last",
+                       f"tree features: {' '.join(TREE_FEATURES)}; a key with a tree is looked up there, the others in the regimes"],
+                trees=trees)
+    if args.latencies:
+        import json
+        with open(args.latencies, "w") as f:
+            json.dump({"cases": [[c, list(k)] for c, k in cases], "lat": [[c, p, t] for (c, p), t in lat.items()],
+                       "features": feats, "groups": groups}, f)
     bsa.lut_load(args.out)
-    print(f"wrote {args.out}: {len(table)} regimes in {time.time() - t0:.0f} s")
+    print(f"wrote {args.out}: {len(table)} regimes, {len(trees)} trees in {time.time() - t0:.0f} s")
     return 0
 
 

@@ -117,9 +117,29 @@ def evaluate(reqs, log=print):
     return rows
 
 
+def off_grid_requests(n: int):
+    """Held-out requests drawn BETWEEN the corpus's grid points (seeds >= 2000: disjoint from the corpus and from the
+    evaluation configurations): geometry from the sweep's five, density log-uniform in [2 %, 70 %], 4-24 heads."""
+    import math as m
+    import numpy as np
+    from . import inputs as I
+    geoms = list(I.SWEEP_GEOMETRIES)
+    out = []
+    for i in range(n):
+        u = I.uniform01(2000 + i, 50, np.arange(3))
+        B = geoms[int(u[0] * len(geoms)) % len(geoms)]
+        rho = float(m.exp(m.log(0.02) + float(u[1]) * (m.log(0.7) - m.log(0.02))))
+        H = 4 * (1 + int(float(u[2]) * 6) % 6)
+        q = I.config_sweep(2000 + i, H=H, B=B, rho=round(rho, 4))
+        q.name = f"offgrid{i}"
+        out.append(q)
+    return out
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--sweep-requests", type=int, default=16)
+    ap.add_argument("--off-grid", type=int, default=16, help="held-out requests drawn between the corpus's grid points")
     ap.add_argument("--json", default="")
     args = ap.parse_args(argv)
     from . import inputs as I
@@ -128,9 +148,15 @@ def main(argv=None):
         q = I.config_sweep(r)
         q.name = f"sweep{r}"
         reqs.append(q)
+    reqs += off_grid_requests(args.off_grid)
     rows = evaluate(reqs)
     s = summarise(rows)
-    print(json.dumps(s))
+    print("all requests:", json.dumps(s))
+    for label, part in (("table hits", [r for r in rows if r["lut_hit"]]), ("table misses (base plan)", [r for r in rows if not r["lut_hit"]]),
+                        ("named configurations and sweep", [r for r in rows if not r["name"].startswith("offgrid")]),
+                        ("off-grid requests", [r for r in rows if r["name"].startswith("offgrid")])):
+        if part:
+            print(f"{label}:", json.dumps(summarise(part)))
     print("task organisation ablation:", json.dumps(organisation_ablation(rows)))
     cold = _gm([r["t_cold"] / r["t_selected"] for r in rows])
     a4 = _gm([r["t_a4"] / r["t_selected"] for r in rows])

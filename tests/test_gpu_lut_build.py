@@ -13,13 +13,14 @@ pytestmark = pytest.mark.gpu
 
 
 def _oracle_validator(corrupt=None):
-    """validator(req, plan_id, O, LSE): 8 seeded query blocks per head against the fp64 oracle at the contract
-    tolerances.  `corrupt` = (case name, plan id): that plan's output is damaged before it is validated."""
+    """validator(req, plan_id, O, LSE, qkv): 8 seeded query blocks per head against the fp64 oracle (on the tensors the
+    plan ran on) at the contract tolerances.  `corrupt` = (case name, plan id): that plan's output is damaged before
+    it is validated."""
     cache = {}
 
-    def validate(req, plan_id, O, LSE):
+    def validate(req, plan_id, O, LSE, qkv):
         if req.name not in cache:
-            Qb, Kb, Vb = (I.bf16_bits(t) for t in req.qkv())
+            Qb, Kb, Vb = (I.bf16_bits(t.cpu()) for t in qkv)
             smp = I.sample_query_blocks(5, req.H, req.nQb, min(8, req.nQb))
             sel = [(h, int(b)) for h in range(req.H) for b in smp[h]]
             cache[req.name] = (sel,) + tuple(oracle.attention_blocks(req.mask, req.B_Q, req.B_KV, req.N, req.d, Qb, Kb, Vb, sel)[:2])
@@ -110,12 +111,12 @@ def test_default_reference_of_the_validation_gate_accepts_a_plan_and_rejects_dam
         with bsa.plan_create(mask, req.B_Q, req.B_KV, req.N, req.H, req.d, plan_id=pid) as plan:
             O, L = plan.forward(q, k, v)
             torch.cuda.synchronize()
-        assert val(req, pid, O, L, qkv=(q, k, v))
+        assert val(req, pid, O, L, (q, k, v))
     row = int(np.flatnonzero(M[0].sum(axis=1) > 0)[0]) * 64
     O2 = O.clone(); O2[0, row] += 0.1
     L2 = L.clone(); L2[0, row] += 0.01
-    assert not val(req, 1, O2, L, qkv=(q, k, v)) and not val(req, 1, O, L2, qkv=(q, k, v))
+    assert not val(req, 1, O2, L, (q, k, v)) and not val(req, 1, O, L2, (q, k, v))
     empty = np.flatnonzero(M[1].sum(axis=1) == 0)
     assert len(empty)
     L3 = L.clone(); L3[1, int(empty[0]) * 64] = 0.0
-    assert not val(req, 1, O, L3, qkv=(q, k, v))
+    assert not val(req, 1, O, L3, (q, k, v))

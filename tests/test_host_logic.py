@@ -110,7 +110,7 @@ def test_plan_table_rejects_foreign_or_malformed_files(tmp_path):
     with pytest.raises(bsa.BsaError) as e:
         bsa.lut_load(p)
     assert e.value.status == 7 and bsa.lib().bsa_lut_num_regimes() == 0
-    _write_lut(p, good, version=2)                    # unknown version
+    _write_lut(p, good, version=3)                    # unknown version
     with pytest.raises(bsa.BsaError):
         bsa.lut_load(p)
     _write_lut(p, {(64, 64, 64, 11, 0, 5, 1, 0): [999]})  # unknown plan id
@@ -164,6 +164,60 @@ def test_offline_table_compilation_matches_algorithm_1(tmp_path):
     lut_build.write_table(path, got, int(bsa.lib().bsa_catalog_hash()), "test-gpu")
     bsa.lut_load(path)
     assert bsa.lib().bsa_lut_num_regimes() == len(got)
+    bsa.lut_clear()
+
+
+def test_decision_tree_regimes_hand_built_case(tmp_path):
+    """Second stage with learned thresholds (Section 5.1): on a hand-built corpus where plan 1 wins below 20 % density
+    and plan 3 above it, whatever the other features, the tree compiler finds one split on density between the two
+    clusters, cross-validation (folds by mask source) prefers depth 1 over depth 0, the leaves carry the rankings of
+    Algorithm 1 with the base plan last, and the runtime reads the file back and walks the same tree."""
+    from paper_2609_25869_b200 import lut_build as LB
+    key = (128, 128, 128)
+    cases, feats, groups, lat = [], {}, {}, {}
+    for n in range(24):
+        cid = f"c{n}"
+        low = n % 2 == 0
+        density = (0.04 + 0.01 * (n % 5)) if low else (0.35 + 0.02 * (n % 7))
+        cases.append((cid, key))
+        feats[cid] = LB.case_features(16384 if n % 3 else 65536, 8 + (n % 4), density, 1.0 + 0.1 * (n % 6), 0.5)
+        groups[cid] = f"source{n // 2}"            # a low and a high case per source
+        lat[(cid, 1)] = 1.0 if low else 2.0
+        lat[(cid, 3)] = 1.5 if low else 1.0
+        lat[(cid, 22)] = 3.0                        # the base plan: valid everywhere, never best
+        if n == 5:
+            del lat[(cid, 1)]                       # plan 1 failed validation on one high-density case
+    base = {key: 22}
+    depth, score = LB.choose_depth([c for c, _ in cases], feats, groups, lat, 22, min_leaf=4, depths=(0, 1, 2), folds=4)
+    assert depth == 1 and score[1] < score[0] - 0.1 and abs(score[1]) < 1e-12
+    trees = LB.compile_trees(cases, feats, groups, lat, base, min_leaf=4, max_depth=2, folds=4)
+    t = trees[key]
+    assert t[0]["feature"] == 2 and 0.08 < t[0]["threshold"] < 0.35 and len(t) == 3
+    lo, hi = t[t[0]["left"]], t[t[0]["right"]]
+    assert lo["ranked"] == [1, 3, 22, 22] and lo["cases"] == 12
+    assert hi["ranked"] == [3, 22, 22] and hi["cases"] == 12   # plan 1 is not valid on every high-density case
+    # with no split allowed the single leaf ranks by geometric mean over everything
+    flat = LB.learn_tree([c for c, _ in cases], feats, lat, 22, min_leaf=4, max_depth=0)
+    assert len(flat) == 1 and flat[0]["ranked"] == [3, 22, 22]
+    # too few cases for two leaves of min_leaf: no tree for the key
+    assert LB.compile_trees(cases[:6], feats, groups, lat, base, min_leaf=4) == {}
+    path = str(tmp_path / "tree.lut")
+    LB.write_table(path, {}, int(bsa.lib().bsa_catalog_hash()), "test", trees=trees)
+    bsa.lut_load(path)
+    assert bsa.lib().bsa_lut_num_trees() == 1 and bsa.lib().bsa_lut_num_regimes() == 0
+    assert bsa.lut_select(128, 128, 16384, 8, 128, 0.05, 0.5, 1.2) == (1, True)
+    assert bsa.lut_select(128, 128, 16384, 8, 128, 0.50, 0.5, 1.2) == (3, True)
+    assert bsa.lut_select(128, 128, 16384, 8, 128, t[0]["threshold"], 0.5, 1.2) == (3, True)   # feature < threshold goes left
+    assert bsa.lut_select(64, 64, 16384, 8, 128, 0.05, 0.5, 1.2) == (bsa.lib().bsa_base_plan(64, 64, 128), False)  # key without a tree
+    # malformed trees are rejected as a whole file
+    text = open(path).read()
+    for bad in (text.replace("BSA_LUT 2", "BSA_LUT 1"), text.replace("node 2 leaf", "node 1 leaf"),
+                text.replace("split 2", "split 9"), text.replace(" 3\nnode 0", " 4\nnode 0")):
+        with open(path, "w") as f:
+            f.write(bad)
+        with pytest.raises(bsa.BsaError):
+            bsa.lut_load(path)
+        assert bsa.lib().bsa_lut_num_trees() == 0
     bsa.lut_clear()
 
 
