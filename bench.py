@@ -37,7 +37,7 @@ NCU_TRAFFIC_BYTES = {
     "mid": (206.5e6, "one ncu capture of one launch of this workload"),
 }
 KERNEL_NAMES = {0: "bsa_attention_kernel<D,TK,false>", 1: "bsa_attention_pair_kernel<D,TK>", 2: "bsa_attention_cs_kernel<D,TK>",
-                3: "bsa_attention_kernel<D,TK,true>", 4: "bsa_attention_pp_kernel<D,TK,F16>"}
+                3: "bsa_attention_kernel<D,TK,true>", 4: "bsa_attention_pp_kernel<D,TK,F16>", 5: "bsa_attention_rb_kernel<D,CK>"}
 TENSOR_FLOP_PER_CLK_PER_SM = 8192  # dense bf16, fp32 accumulate
 
 

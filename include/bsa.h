@@ -3,7 +3,7 @@
  *
  * A request R = <A, M, B, x> (paper, Section 3 "Online request path" and Section 4.4) supplies a
  * logical block mask M with geometry B = (B_Q, B_KV) and the tensor properties x (here: bf16 or fp16,
- * head dim d in {64, 128}, layout [heads, N, d] or [N, heads, d]; bsa_options_t carries the non-default
+ * head dim d in {64, 128, 256}, layout [heads, N, d] or [N, heads, d]; bsa_options_t carries the non-default
  * ones, and N_kv when keys and queries differ in number).  The library computes masked attention
  * (Section 2.1, Eq. 1)
  *
@@ -40,7 +40,7 @@ typedef struct bsa_plan bsa_plan_t; /* opaque; owned by the library */
 typedef enum {
     BSA_OK = 0,
     BSA_ERR_INVALID_ARG = 1,      /* null pointer, N <= 0, heads <= 0, ... (GPU untouched)            */
-    BSA_ERR_UNSUPPORTED = 2,      /* d not in {64,128}; B_Q/B_KV not a power of two in [16,256]      */
+    BSA_ERR_UNSUPPORTED = 2,      /* d not in {64,128,256}; B_Q/B_KV not a power of two in [16,256]  */
     BSA_ERR_NO_ELIGIBLE_PLAN = 3, /* Algorithm 2, last line: no plan of the ranking is eligible      */
     BSA_ERR_OOM = 4,              /* device or host allocation failed                               */
     BSA_ERR_CUDA = 5,             /* a CUDA call failed; see bsa_last_cuda_error()                   */
@@ -143,7 +143,9 @@ typedef struct bsa_plan_info {
  *   N        : query tokens per head, N_q of Section 2.1; need not be a multiple of the block sizes.
  *              The key/value token count N_kv equals N unless options->N_kv says otherwise (_ex variants).
  *   heads    : independent (batch x head) problems.
- *   d        : head dimension, 64 or 128.  Scale is 1/sqrt(d); attention is non-causal.
+ *   d        : head dimension, 64, 128 or 256 (256: bf16 only, served by the single-tile kernels with 64-key
+ *              tiles, whose 256-column output accumulator fills half of tensor memory).  Scale is 1/sqrt(d);
+ *              attention is non-causal.
  *   out_plan : receives the plan; the plan owns its device buffers (CSR, tile lists, work items,
  *              Split-K workspace).  Reusable for any number of forwards with the same mask.
  *

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbsa.so")
-SOURCES = ["bsa_api.cu", "bsa_planner.cu", "bsa_attention.cu", "bsa_noalloc.cu", "bsa_lut.cpp"]
+SOURCES = ["bsa_api.cu", "bsa_planner.cu", "bsa_attention.cu", "bsa_attention_rb.cu", "bsa_noalloc.cu", "bsa_lut.cpp"]
 
 
 def _stale() -> bool:

@@ -126,7 +126,7 @@ struct bsa_plan_cache {
 static bsa_status_t validate(const void* mask, int B_Q, int B_KV, int64_t N, int heads, int d, void* out) {
     if (!mask || !out || N <= 0 || heads <= 0) return BSA_ERR_INVALID_ARG;
     auto p2 = [](int v) { return v >= 16 && v <= 256 && (v & (v - 1)) == 0; };
-    if (!(d == 64 || d == 128) || !p2(B_Q) || !p2(B_KV)) return BSA_ERR_UNSUPPORTED;
+    if (!(d == 64 || d == 128 || d == 256) || !p2(B_Q) || !p2(B_KV)) return BSA_ERR_UNSUPPORTED;
     if (N > (1ll << 30)) return BSA_ERR_UNSUPPORTED;
     return BSA_OK;
 }
@@ -404,6 +404,8 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     const size_t o_it0 = take(sizeof(WorkItem) * (size_t)p->max_items);
     const size_t o_it1 = take(sizeof(WorkItem) * (size_t)p->max_items);
     const size_t o_sr = take(sizeof(SplitRow) * (size_t)(pmax > 1 ? trows * g.slots : 1));
+    const size_t org_bytes = organize_scratch_bytes(g, p->desc.order, pmax);
+    const size_t o_org = take(org_bytes ? org_bytes : 4);
     if (p->arena2 && o > arena2_have) {  // the prediction was too small
         cudaFreeAsync(p->arena2, stream);
         p->arena2 = nullptr;
@@ -436,7 +438,8 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
                              p->row_parts, p->tile_col, p->tile_member, p->head_counts, p->counters, stream),
              "tile_map");
     BSA_CUDA(launch_organize(g, p->desc.order, pmax, p->tile_begin, p->tile_cnt, p->row_parts, p->head_counts,
-                             p->items_tmp, p->items, p->split_rows, p->counters, stream),
+                             p->items_tmp, p->items, p->split_rows, p->counters, stream,
+                             org_bytes ? reinterpret_cast<int32_t*>(p->arena2 + o_org) : nullptr),
              "organize");
     const double t4 = now_us();
     p->us_mask_state = (float)(t1 - t0);
@@ -713,7 +716,7 @@ extern "C" bsa_status_t bsa_plan_get_info(const bsa_plan_t* p, bsa_plan_info_t* 
     info->nitems = c.nitems;
     info->nsplit_rows = c.nsplit_rows;  // physical tile rows with more than one partition
     info->workspace_bytes = p->ws_bytes;
-    info->covered_pairs = (int64_t)c.nslot_tiles * kTQ * g.T_KV;
+    info->covered_pairs = (int64_t)c.nslot_tiles * (g.T_Q < kTQ ? g.T_Q : kTQ) * g.T_KV;
     info->us_mask_state = p->us_mask_state;
     info->us_stats_sync = p->us_stats_sync;
     info->us_lookup = p->us_lookup;

@@ -2115,13 +2115,13 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
     const int dev = (a.device >= 0 && a.device < kMaxDevices) ? a.device : 0;
     if (smem > attr_bytes_dev[dev].load(std::memory_order_relaxed)) {
         cudaError_t e;
-        if (KERNEL == 0)
+        if constexpr (KERNEL == 0)
             e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        else if (KERNEL == 3)
+        else if constexpr (KERNEL == 3)
             e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        else if (KERNEL == 1)
+        else if constexpr (KERNEL == 1)
             e = cudaFuncSetAttribute(bsa_attention_pair_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        else if (KERNEL == 2)
+        else if constexpr (KERNEL == 2)
             e = cudaFuncSetAttribute(bsa_attention_cs_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         else {
             e = cudaFuncSetAttribute(bsa_attention_pp_kernel<D, TK, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -2136,13 +2136,13 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
     }
     int grid = a.num_sms < a.max_items ? a.num_sms : a.max_items;
     if (grid < 1) grid = 1;
-    if (KERNEL == 0)
+    if constexpr (KERNEL == 0)
         bsa_attention_kernel<D, TK, false><<<grid, kThreads, smem, stream>>>(tq, tk, tv, p);
-    else if (KERNEL == 3)
+    else if constexpr (KERNEL == 3)
         bsa_attention_kernel<D, TK, true><<<grid, kThreads + 32, smem, stream>>>(tq, tk, tv, p);
-    else if (KERNEL == 1)
+    else if constexpr (KERNEL == 1)
         bsa_attention_pair_kernel<D, TK><<<grid, kPairThreads, smem, stream>>>(tq, tk, tv, p);
-    else if (KERNEL == 2)
+    else if constexpr (KERNEL == 2)
         bsa_attention_cs_kernel<D, TK><<<grid, kCsThreads, smem, stream>>>(tq, tk, tv, p);
     else {
         // The ping-pong kernel waits for its predecessor itself (grid_dependency_wait), so it may be scheduled while
@@ -2193,6 +2193,8 @@ static void split_stages(int total, int kernel, int* nk, int* nv) {
 }
 
 int attention_max_stages(int d, int T_KV, int kernel) {
+    if (kernel == kKernelRowBlock) return (d <= 128 && T_KV <= rb_max_chunk(d)) ? 2 : 0;  // one K and one V buffer per warp
+    if (d == 256 && !((kernel == 0 || kernel == 3) && T_KV == 64)) return 0;  // see launch_forward
     const int nb = kv_buffers_that_fit(d, T_KV, kernel);
     if (kernel == 1 || kernel == 4) return nb > 2 * kMaxStages ? 2 * kMaxStages : nb;  // total K + V buffers
     const int s = nb / 2;
@@ -2250,6 +2252,7 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     if (a.kernel == 1 || a.kernel == 4) split_stages(a.stages, a.kernel, &p.stages, &p.stages_v);
     p.scale_log2 = (float)(1.4426950408889634 / sqrt((double)a.d));
     cudaError_t e;
+    if (a.kernel == kKernelRowBlock) return launch_forward_rb(a, stream, err_detail);
     const int key = a.kernel * 1000 + a.d + a.g.T_KV / 64;  // kernel, d, T_KV
     if (key == 128 + 2) e = launch_attn<128, 128, 0>(a, p, stream, err_detail);
     else if (key == 128 + 1) e = launch_attn<128, 64, 0>(a, p, stream, err_detail);
@@ -2267,6 +2270,10 @@ cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char
     else if (key == 3000 + 128 + 1) e = launch_attn<128, 64, 3>(a, p, stream, err_detail);
     else if (key == 3000 + 64 + 2) e = launch_attn<64, 128, 3>(a, p, stream, err_detail);
     else if (key == 3000 + 64 + 1) e = launch_attn<64, 64, 3>(a, p, stream, err_detail);
+    // d = 256: the output accumulator takes 256 of the 512 tensor-memory columns, which leaves room for the two score
+    // buffers only where P is written in place over S (the single-tile kernels), with 64-key tiles
+    else if (key == 256 + 1) e = launch_attn<256, 64, 0>(a, p, stream, err_detail);
+    else if (key == 3000 + 256 + 1) e = launch_attn<256, 64, 3>(a, p, stream, err_detail);
     else if (key == 4000 + 128 + 2) e = launch_attn<128, 128, 4>(a, p, stream, err_detail);
     else if (key == 4000 + 128 + 1) e = launch_attn<128, 64, 4>(a, p, stream, err_detail);
     else if (key == 4000 + 64 + 2) e = launch_attn<64, 128, 4>(a, p, stream, err_detail);
@@ -2288,7 +2295,10 @@ cudaError_t launch_merge(const ForwardArgs& a, cudaStream_t stream) {
     const long long want = (long long)a.max_split_rows * (kTQ * (a.d / 8) / 256);
     int grid = want < 8ll * a.num_sms ? (int)want : 8 * a.num_sms;
     if (grid < 1) grid = 1;
-    if (a.d == 128)
+    if (a.d == 256)
+        bsa_merge_kernel<256><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
+                                                        reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16, o_head, o_row);
+    else if (a.d == 128)
         bsa_merge_kernel<128><<<grid, 256, 0, stream>>>(a.split_rows, a.counters, a.ws_O, a.ws_LSE,
                                                         reinterpret_cast<__nv_bfloat16*>(a.O), a.LSE, (int)a.g.N, a.f16, o_head, o_row);
     else

@@ -8,7 +8,7 @@
 namespace bsa {
 
 constexpr int kMaxDevices = 64;  // per-device host state (accumulators, kernel attributes) is kept for this many GPUs
-constexpr int kTQ = 128;  // physical Q tile height of every catalog kernel (one MMA M=128 per CTA)
+constexpr int kTQ = 128;  // rows of one tcgen05 MMA (one 128-row slot); the row-block kernel's tiles are smaller
 
 // One unit of work for a persistent CTA: one Q tile row of one head, restricted to the KV tiles
 // [tile_begin, tile_end) of the plan's tile arrays (a Split-K partition when nparts > 1).
@@ -87,10 +87,13 @@ cudaError_t launch_tile_map(const MapGeom& g, const int32_t* row_ptr, const int3
                             int split_pmax, int32_t* tile_begin, int32_t* tile_cnt, int32_t* row_parts,
                             int32_t* tile_col, uint64_t* tile_member, int32_t* head_counts /* [3*H] */,
                             PlanCountersDev* counters, cudaStream_t stream);
+// `scratch` (may be null): organize_scratch_bytes() bytes in the plan's arena for the long-list path.
 cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const int32_t* tile_begin,
                             const int32_t* tile_cnt, const int32_t* row_parts, const int32_t* head_counts, WorkItem* items_tmp,
-                            WorkItem* items, SplitRow* split_rows, PlanCountersDev* counters, cudaStream_t stream);
+                            WorkItem* items, SplitRow* split_rows, PlanCountersDev* counters, cudaStream_t stream,
+                            int32_t* scratch = nullptr);
 size_t organize_smem_bytes(const MapGeom& g, int order, int split_pmax);
+size_t organize_scratch_bytes(const MapGeom& g, int order, int split_pmax);
 
 // ---- attention + merge (bsa_attention.cu) ----------------------------------------------------
 struct ForwardArgs {
@@ -120,6 +123,10 @@ struct ForwardArgs {
 };
 cudaError_t launch_forward(const ForwardArgs& a, cudaStream_t stream, const char** err_detail);
 cudaError_t launch_merge(const ForwardArgs& a, cudaStream_t stream);  // the Split-K reduction kernel alone
+// Row-block kernel (bsa_attention_rb.cu): 16-row physical Q tiles on the register-level tensor instruction.
+constexpr int kKernelRowBlock = 5;
+cudaError_t launch_forward_rb(const ForwardArgs& a, cudaStream_t stream, const char** err_detail);
+int rb_max_chunk(int d);  // largest T_KV (keys per staged chunk) for head dimension d
 // `stages` counts K buffers plus V buffers for the paired kernel (kernel 1), K = V ring depth for kernel 0
 int attention_max_stages(int d, int T_KV, int kernel);
 int attention_smem_bytes(int d, int T_KV, int stages, int kernel);

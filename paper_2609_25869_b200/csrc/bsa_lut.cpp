@@ -60,6 +60,13 @@ static const bsa_plan_desc_t kCatalog[] = {
     {31, 128, 128, 0, 0, 1, BSA_ORDER_GLOBAL_BUCKETS, 4, "q128k128_pp_gb"},
     {32, 128, 64, 0, 0, 1, BSA_ORDER_NATURAL, 4, "q128k64_pp_natural"},
     {33, 128, 64, 0, 0, 1, BSA_ORDER_GLOBAL_BUCKETS, 4, "q128k64_pp_gb"},
+    // 16-row Q tiles, one warp each, on the register-level tensor instruction (mma.sync): logical blocks of up to 64
+    // rows keep their own KV lists instead of being Coarsened onto 128 rows
+    {34, 16, 64, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 5, "q16k64_rb"},
+    {35, 16, 32, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 5, "q16k32_rb"},
+    {36, 16, 16, 0, 0, 1, BSA_ORDER_HEAD_MAJOR_LPT, 5, "q16k16_rb"},
+    {37, 16, 64, 0, 0, 1, BSA_ORDER_NATURAL, 5, "q16k64_rb_natural"},
+    {38, 16, 32, 0, 0, 1, BSA_ORDER_NATURAL, 5, "q16k32_rb_natural"},
 };
 static const int kCatalogSize = (int)(sizeof(kCatalog) / sizeof(kCatalog[0]));
 static const int64_t kDefaultWorkspace = 2ll << 30;
@@ -86,8 +93,8 @@ bool make_geom(const bsa_plan_desc_t& P, int B_Q, int B_KV, int64_t N, int64_t N
     g->B_KV = B_KV;
     g->T_Q = P.T_Q;
     g->T_KV = P.T_KV;
-    g->slots = P.T_Q / kTQ;
-    g->sQ128 = B_Q < kTQ ? kTQ / B_Q : 1;
+    g->slots = P.T_Q >= kTQ ? P.T_Q / kTQ : 1;                 // 128-row MMA slots (one for the 16-row tiles)
+    g->sQ128 = (B_Q < kTQ && P.T_Q >= kTQ) ? kTQ / B_Q : 1;    // logical rows per slot where the slot is Coarsened
     g->nQb = (int)((N + B_Q - 1) / B_Q);
     g->nKb = (int)((N_kv + B_KV - 1) / B_KV);
     g->nQt = (int)((N + P.T_Q - 1) / P.T_Q);
@@ -115,7 +122,13 @@ bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, 
     if (!P) return false;
     if (dtype != BSA_DTYPE_BF16 && dtype != BSA_DTYPE_FP16) return false;
     if (dtype == BSA_DTYPE_FP16 && P->kernel != 4) return false;  // tensor property: only the ping-pong kernel takes half
-    if (!(d == 64 || d == 128)) return false;
+    if (P->kernel == kKernelRowBlock) {
+        // 16-row tiles: for logical blocks of up to 64 rows (on larger ones the 128-row tile wastes nothing that this
+        // kernel could win back), KV tiles no wider than the logical block (no membership masks in this kernel) and
+        // no larger than a warp's staging buffer, no Split-K
+        if (B_Q > 64 || B_KV < P->T_KV || P->T_KV > rb_max_chunk(d) || P->split_pmax > 1) return false;
+    }
+    if (!(d == 64 || d == 128 || d == 256)) return false;
     if (!pow2_in(B_Q, 16, 256) || !pow2_in(B_KV, 16, 256)) return false;
     if (N <= 0 || heads <= 0 || N > (1ll << 30)) return false;
     MapGeom g;
@@ -138,7 +151,7 @@ bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, 
 int base_plan(int B_Q, int B_KV, int d) {
     (void)B_Q;
     (void)B_KV;
-    (void)d;
+    if (d == 256) return 19;  // q128k64_di: the kernels with P in place over S are the ones that hold a 256-column O
     return 22;  // q128k128_pp: eligible for every supported geometry (membership <= 64 bits), no workspace
 }
 

@@ -117,12 +117,17 @@ __global__ void __launch_bounds__(256) mask_row_stats_kernel(const uint8_t* __re
         // byte of a step does not know its right neighbour yet: if its left neighbour is inactive it is counted one
         // step later, by lane 0, once that neighbour (bit 0 of the next step) is known.
         unsigned carry = 0;  // bits 1:0 = the previous step's last two bytes (bit 1 = the last one)
-        unsigned m_next = row_word_bits(words, w0 + lane, rb, re);
+        // three steps' words are in flight ahead of the one being counted (a row of a few KB is then read almost at once)
+        unsigned m_q0 = row_word_bits(words, w0 + lane, rb, re);
+        unsigned m_q1 = (w0 + 32 < w1) ? row_word_bits(words, w0 + 32 + lane, rb, re) : 0u;
+        unsigned m_q2 = (w0 + 64 < w1) ? row_word_bits(words, w0 + 64 + lane, rb, re) : 0u;
         MaskHash hash;
         for (long long w = w0; w < w1; w += 32) {
-            const unsigned m = m_next;
+            const unsigned m = m_q0;
             if (HASH) hash.add(m, row, w - w0 + lane);
-            m_next = (w + 32 < w1) ? row_word_bits(words, w + 32 + lane, rb, re) : 0u;
+            m_q0 = m_q1;
+            m_q1 = m_q2;
+            m_q2 = (w + 96 < w1) ? row_word_bits(words, w + 96 + lane, rb, re) : 0u;
             // neighbours across lanes: previous lane's bit 15, next lane's bit 0
             unsigned prev15 = __shfl_up_sync(kFull, m >> 15, 1);
             unsigned next0 = __shfl_down_sync(kFull, m & 1u, 1);
@@ -347,13 +352,15 @@ __global__ void __launch_bounds__(256) csr_fill_kernel(const uint8_t* __restrict
     const long long rb = (long long)(base & 15ull) + (long long)row * nKb, re = rb + nKb;
     const long long w0 = rb >> 4, w1 = (re + 15) >> 4;
     int32_t out = row_ptr[row];
-    // two steps' words are in flight ahead of the one being written out
+    // three steps' words are in flight ahead of the one being written out
     unsigned m_next = row_word_bits(words, w0 + lane, rb, re);
     unsigned m_next2 = (w0 + 32 < w1) ? row_word_bits(words, w0 + 32 + lane, rb, re) : 0u;
+    unsigned m_next3 = (w0 + 64 < w1) ? row_word_bits(words, w0 + 64 + lane, rb, re) : 0u;
     for (long long w = w0; w < w1; w += 32) {
         unsigned m = m_next;
         m_next = m_next2;
-        m_next2 = (w + 64 < w1) ? row_word_bits(words, w + 64 + lane, rb, re) : 0u;
+        m_next2 = m_next3;
+        m_next3 = (w + 96 < w1) ? row_word_bits(words, w + 96 + lane, rb, re) : 0u;
         const int cnt = __popc(m);
         int incl = cnt;
         for (int o = 1; o < 32; o <<= 1) {
@@ -843,7 +850,125 @@ __global__ void __launch_bounds__(1024) organize_kernel(MapGeom g, int order, in
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// organize, long lists: the global orders over many thousands of Q tile rows (one item per row:
+// plans that never split) as a stable counting sort spread over many CTAs, three launches:
+//   1. every CTA histograms the sort keys of its 512 consecutive rows;
+//   2. one CTA turns the histograms into start positions: bins longest first, and inside a bin
+//      the CTAs' shares in row order (so equal keys keep (head, q_tile) order);
+//   3. every CTA ranks its rows in order (one warp, 32 rows per step, equal keys found with
+//      shuffles) and writes each item straight to its final place.
+// ------------------------------------------------------------------------------------------
+constexpr int kOrgChunk = 512;  // rows per CTA
+
+__device__ __forceinline__ int32_t organize_key(int32_t ntiles, bool bucketed) {
+    return bucketed ? length_bucket(ntiles) : ntiles;
+}
+
+__global__ void __launch_bounds__(256) organize_hist_kernel(int nrows, int nbins, int bucketed,
+                                                             const int32_t* __restrict__ tile_cnt,
+                                                             int32_t* __restrict__ hist /* [chunks][nbins] */) {
+    extern __shared__ int32_t sh[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // launched behind the tile map with programmatic serialisation
+    for (int b = threadIdx.x; b < nbins; b += blockDim.x) sh[b] = 0;
+    __syncthreads();
+    const int r0 = blockIdx.x * kOrgChunk;
+    for (int i = threadIdx.x; i < kOrgChunk && r0 + i < nrows; i += blockDim.x)
+        atomicAdd(&sh[organize_key(tile_cnt[r0 + i], bucketed != 0)], 1);
+    __syncthreads();
+    for (int b = threadIdx.x; b < nbins; b += blockDim.x) hist[(size_t)blockIdx.x * nbins + b] = sh[b];
+}
+
+__global__ void __launch_bounds__(1024) organize_scan_kernel(int nrows, int nbins, int nchunks, int32_t* __restrict__ hist,
+                                                              int32_t* __restrict__ bin_start /* [nbins] scratch */,
+                                                              PlanCountersDev* counters) {
+    __shared__ int32_t carry_s;
+    // per bin: exclusive prefix over the chunks (in place), total into bin_start
+    for (int b = threadIdx.x; b < nbins; b += blockDim.x) {
+        int32_t run = 0;
+        for (int c = 0; c < nchunks; ++c) {
+            const int32_t v = hist[(size_t)c * nbins + b];
+            hist[(size_t)c * nbins + b] = run;
+            run += v;
+        }
+        bin_start[b] = run;
+    }
+    __syncthreads();
+    // bin starts, longest first (warp 0 walks the bins from the top, 32 at a time)
+    if (threadIdx.x < 32) {
+        int32_t carry = 0;
+        for (int hi = nbins - 1; hi >= 0; hi -= 32) {
+            const int b = hi - (int)threadIdx.x;
+            const int32_t c = (b >= 0) ? bin_start[b] : 0;
+            int32_t incl = c;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t x = __shfl_up_sync(kFull, incl, o);
+                if ((int)threadIdx.x >= o) incl += x;
+            }
+            if (b >= 0) bin_start[b] = carry + incl - c;
+            carry += __shfl_sync(kFull, incl, 31);
+        }
+        if (threadIdx.x == 0) carry_s = carry;
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < nbins; b += blockDim.x) {
+        const int32_t st = bin_start[b];
+        for (int c = 0; c < nchunks; ++c) hist[(size_t)c * nbins + b] += st;
+    }
+    if (threadIdx.x == 0) {
+        counters->nitems = nrows;  // one item per row
+        counters->nsplit_rows = 0;
+        counters->nslots = 0;
+        (void)carry_s;
+    }
+}
+
+__global__ void __launch_bounds__(256) organize_scatter_kernel(MapGeom g, int nrows, int nbins, int bucketed,
+                                                                const int32_t* __restrict__ tile_begin,
+                                                                const int32_t* __restrict__ tile_cnt,
+                                                                const int32_t* __restrict__ hist, WorkItem* __restrict__ items) {
+    extern __shared__ int32_t sh[];   // [nbins] next free position per key for this CTA's rows, then [kOrgChunk] ranks
+    int32_t* next = sh;
+    int32_t* rank = sh + nbins;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    for (int b = threadIdx.x; b < nbins; b += blockDim.x) next[b] = hist[(size_t)blockIdx.x * nbins + b];
+    __syncthreads();
+    const int r0 = blockIdx.x * kOrgChunk;
+    const int n = min(kOrgChunk, nrows - r0);
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        for (int i0 = 0; i0 < n; i0 += 32) {
+            const int i = i0 + lane;
+            const bool valid = i < n;
+            const int32_t k = valid ? organize_key(tile_cnt[r0 + i], bucketed != 0) : -1 - lane;  // invalid lanes: unique keys
+            const unsigned peers = warp_peers(k);
+            if (valid) rank[i] = next[k] + __popc(peers & ((1u << lane) - 1u));
+            __syncwarp();
+            if (valid && (peers >> lane) <= 1u) next[k] += __popc(peers);  // highest lane of the peer set
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const int r = r0 + i;
+        const int32_t tb = tile_begin[r], cnt = tile_cnt[r];
+        int4* dst = reinterpret_cast<int4*>(items + rank[i]);
+        dst[0] = make_int4(r / g.nQt, r % g.nQt, tb, tb + cnt);   // head, q_tile, tile_begin, tile_end
+        dst[1] = make_int4(0, 1, -1, cnt);                         // part, nparts, ws_slot, ntiles
+    }
+}
+
 }  // namespace
+
+// Scratch (bytes) the long-list organisation needs in the plan's arena; 0 when the single-kernel path serves.
+size_t organize_scratch_bytes(const MapGeom& g, int order, int split_pmax) {
+    const bool global_group = (order == BSA_ORDER_GLOBAL_LPT || order == BSA_ORDER_GLOBAL_BUCKETS);
+    const long long rows = (long long)g.H * g.nQt;
+    if (!global_group || split_pmax > 1 || rows < 4096) return 0;
+    const size_t chunks = (size_t)((rows + kOrgChunk - 1) / kOrgChunk);
+    return (chunks + 1) * (size_t)organize_bins(g) * sizeof(int32_t);
+}
 
 cudaError_t launch_mask_row_stats(const uint8_t* mask, int nrows, int nKb, int32_t* row_nnz, MaskStatsDev* stats,
                                   cudaStream_t stream, MaskStatsHost* post, unsigned seq, bool with_hash) {
@@ -925,7 +1050,38 @@ size_t organize_smem_bytes(const MapGeom& g, int order, int split_pmax) {
 cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const int32_t* tile_begin,
                             const int32_t* tile_cnt, const int32_t* row_parts, const int32_t* head_counts,
                             WorkItem* items_tmp, WorkItem* items, SplitRow* split_rows, PlanCountersDev* counters,
-                            cudaStream_t stream) {
+                            cudaStream_t stream, int32_t* scratch) {
+    if (scratch && organize_scratch_bytes(g, order, split_pmax) > 0) {
+        const int nrows = g.H * g.nQt, nbins = organize_bins(g);
+        const int nchunks = (nrows + kOrgChunk - 1) / kOrgChunk;
+        const int bucketed = (order == BSA_ORDER_GLOBAL_BUCKETS) ? 1 : 0;
+        int32_t* hist = scratch;
+        int32_t* bin_start = scratch + (size_t)nchunks * nbins;
+        const size_t sm1 = (size_t)nbins * sizeof(int32_t), sm3 = (size_t)(nbins + kOrgChunk) * sizeof(int32_t);
+        if (sm3 > 40 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(organize_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(organize_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm3);
+            if (e != cudaSuccess) return e;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)nchunks);
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = sm1;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, organize_hist_kernel, nrows, nbins, bucketed, tile_cnt, hist);
+        count_launch();
+        if (e != cudaSuccess) return e;
+        organize_scan_kernel<<<1, 1024, 0, stream>>>(nrows, nbins, nchunks, hist, bin_start, counters);
+        count_launch();
+        organize_scatter_kernel<<<nchunks, 256, sm3, stream>>>(g, nrows, nbins, bucketed, tile_begin, tile_cnt, hist, items);
+        count_launch();
+        return cudaGetLastError();
+    }
     // the caller checked organize_smem_bytes() against the device limit when it chose `order`; whatever shared
     // memory is left up to 200 KB holds per-warp histograms for the parallel ranking (up to one per warp)
     const size_t base = organize_smem_bytes(g, order, split_pmax);

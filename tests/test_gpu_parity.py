@@ -19,7 +19,7 @@ def _sample(req, per_head, seed=77, heads=None):
 
 
 # ---------------------------------------------------------------- the five configurations
-@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29, 30, 31, 32, 33])
+@pytest.mark.parametrize("plan_id", [-1, 0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 18, 19, 20, 21, 22, 23, 24, 25, 26, 27, 28, 29, 30, 31, 32, 33, 34, 35, 36, 37, 38])
 def test_tiny_full_oracle_every_plan(plan_id):
     res = Hh.run_request(I.config_tiny(), plan_id=plan_id)
     assert res["pairs"] == res["info"]["nnz_blocks"] * 64 * 64
@@ -41,7 +41,22 @@ def test_hunyuan_shaped_sampled_oracle():
 def test_stress_a_coarsened(plan_id):
     req = I.config_stress_a()
     res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64), heads=[0, 15])
-    assert res["info"]["map_q"] == 1  # Coarsened along Q: 8 logical rows of 16 per 128-row tile
+    if bsa.catalog()[res["info"]["plan"]["plan_id"]]["kernel"] != 5:
+        assert res["info"]["map_q"] == 1  # Coarsened along Q: 8 logical rows of 16 per 128-row tile
+
+
+@pytest.mark.parametrize("plan_id", [34, 35, 37])
+def test_stress_a_on_16_row_tiles(plan_id):
+    """The same request on the row-block kernel: every 16-row logical block is its own physical tile (Direct along Q,
+    Direct or Refined along KV), so the plan covers exactly the active pairs."""
+    req = I.config_stress_a()
+    res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64), heads=[3])
+    inf = res["info"]
+    assert inf["map_q"] == 0 and inf["plan"]["T_Q"] == 16 and inf["covered_pairs"] == res_pairs(req)
+
+
+def res_pairs(req):
+    return oracle.active_pairs(req.mask, req.B_Q, req.B_KV, req.N, req.n_kv)
 
 
 @pytest.mark.parametrize("plan_id", [-1, 0, 1, 10, 11, 14, 15, 18, 19, 22, 23, 25])
@@ -61,6 +76,16 @@ def test_sweep_requests_ragged_n(r, B, rho):
     the full 24 heads are in the next test."""
     req = I.config_sweep(r, H=6, B=B, rho=rho)
     Hh.run_request(req, plan_id=-1, sel=_sample(req, 64), row_step=4 if rho >= 0.3 else 1, heads=[0, 5])
+
+
+@pytest.mark.parametrize("plan_id,rho", [(35, 0.03), (38, 0.10), (36, 0.03)])
+def test_sweep_32x32_request_on_16_row_tiles(plan_id, rho):
+    """A (32,32) sweep request (d = 128, ragged N) on the row-block kernel: two 16-row tiles per logical row block
+    (Refined along Q), 32- or 16-key tiles, no pair outside E(M) computed."""
+    req = I.config_sweep(1, H=6, B=(32, 32), rho=rho)
+    res = Hh.run_request(req, plan_id=plan_id, sel=_sample(req, 64), heads=[5])
+    inf = res["info"]
+    assert inf["map_q"] == 2 and inf["covered_pairs"] == inf["nnz_blocks"] * 32 * 32   # whole blocks: the ragged edge counts in full
 
 
 @pytest.mark.parametrize("r,B,rho,row_step", [(7, (32, 32), 0.30, 4), (8, (128, 128), 0.10, 1)])
@@ -89,6 +114,8 @@ def test_sweep_requests_at_all_24_heads(r, B, rho, row_step):
     (16, 16, 1000, 64, 22), (32, 64, 777, 128, 23), (64, 32, 1300, 128, 22), (128, 256, 2100, 64, 23),
     (256, 128, 2100, 128, 22), (256, 16, 900, 64, 24), (16, 256, 900, 128, 24), (128, 128, 127, 128, 25),
     (64, 64, 130, 64, 22), (128, 128, 1, 64, 23), (128, 128, 129, 128, 22), (32, 32, 3000, 64, 25),
+    (16, 16, 1000, 64, 36), (32, 64, 777, 128, 35), (64, 32, 1300, 128, 35), (16, 256, 900, 128, 38), (16, 64, 1000, 64, 34),
+    (32, 32, 3000, 64, 35), (64, 128, 2100, 64, 37), (64, 64, 130, 64, 34), (16, 16, 1, 128, 36), (32, 256, 1111, 64, 34),
 ])
 def test_geometries_with_ragged_tail(B_Q, B_KV, N, d, plan_id):
     H = 3
@@ -110,7 +137,7 @@ def test_degenerate_masks(kind):
     elif kind == "empty_head":
         M[0] = I.random_mask(1, 1, nb, nb, 0.5)[0]
     req = I.Request(kind, H, N, d, B, B, M, qkv_seed=3)
-    for plan_id in (0, 3, 10, 12, 14, 16, 18, 20, 22, 24):
+    for plan_id in (0, 3, 10, 12, 14, 16, 18, 20, 22, 24, 34, 36):
         Hh.run_request(req, plan_id=plan_id)
 
 
@@ -119,7 +146,8 @@ def test_degenerate_masks(kind):
                                                   (16, 64, 1000, 64, 10), (64, 32, 700, 128, 11), (256, 256, 1100, 128, 12),
                                                   (16, 64, 1000, 64, 14), (64, 32, 700, 128, 15), (256, 256, 1100, 128, 16),
                                                   (16, 64, 1000, 64, 18), (64, 32, 700, 128, 19), (256, 256, 1100, 128, 20),
-                                                  (16, 64, 1000, 64, 22), (64, 32, 700, 128, 23), (256, 256, 1100, 128, 24)])
+                                                  (16, 64, 1000, 64, 22), (64, 32, 700, 128, 23), (256, 256, 1100, 128, 24),
+                                                  (16, 64, 1000, 64, 34), (64, 32, 700, 128, 35), (32, 16, 900, 128, 36)])
 def test_zero_keys_give_log_count_and_mean_value(B_Q, B_KV, N, d, plan_id):
     """K = 0: every score is 0, so LSE = ln(#reachable keys) exactly and O = mean of reachable V.
     Catches any off-by-one in ragged-edge or membership masking (one key off moves LSE by ~1/count)."""
@@ -180,7 +208,7 @@ def test_growing_scores_force_a_rescale_at_every_tile(plan_id):
 
 
 @pytest.mark.parametrize("name,plan_id", [("stress_b", 22), ("stress_b", 23), ("stress_b", 18), ("mid", 22), ("mid", 24),
-                                          ("stress_a", 23), ("tiny", 27)])
+                                          ("stress_a", 23), ("tiny", 27), ("stress_a", 34), ("tiny", 36)])
 def test_repeated_runs_are_bitwise_identical(name, plan_id):
     """No atomics and a fixed accumulation order: six forwards of one plan give the same bits.  Long work items
     (Stress-B has about a hundred tiles per item) give a timing-dependent hand-off the most chances to show."""
@@ -324,7 +352,8 @@ def test_bit_packed_mask_gives_the_same_plan_and_output(B_Q, B_KV, N, d, plan_id
     (16, 32, 900, 2500, 64, 25), (32, 16, 2500, 900, 128, 0), (128, 64, 130, 4000, 128, 2),
     (256, 128, 1500, 520, 64, 1), (64, 256, 600, 2050, 128, 10), (128, 128, 4096, 128, 128, 23),
     (16, 16, 300, 1111, 64, 14), (64, 64, 1000, 3000, 128, 24), (32, 32, 3000, 1000, 64, 18),
-    (128, 128, 1, 777, 128, -1), (64, 64, 777, 1, 64, -1)])
+    (128, 128, 1, 777, 128, -1), (64, 64, 777, 1, 64, -1), (16, 64, 900, 2500, 64, 34), (32, 32, 2500, 900, 128, 35),
+    (64, 16, 777, 1, 64, 36)])
 def test_rectangular_requests_match_the_oracle(B_Q, B_KV, N_q, N_kv, d, plan_id):
     """More (or fewer) key tokens than query tokens: ragged last blocks on both sides, every kernel family,
     Direct / Coarsened / Refined mappings, Split-K plans; all rows compared, tile plan == E(M)."""
@@ -414,6 +443,26 @@ def test_half_precision_mid_and_ineligible_plans():
         assert not torch.equal(Oh.view(torch.int16), Ob.view(torch.int16))
 
 
+# ---------------------------------------------------------------- head dimension 256 (a tensor property of the request)
+@pytest.mark.parametrize("B_Q,B_KV,N,N_kv,plan_id", [(128, 128, 2100, 0, -1), (64, 64, 1000, 0, 19), (16, 32, 900, 1500, 1),
+                                                      (256, 256, 1500, 0, 3), (128, 64, 3000, 0, 5), (32, 16, 700, 0, 9)])
+def test_head_dim_256_matches_the_oracle(B_Q, B_KV, N, N_kv, plan_id):
+    """d = 256: the output accumulator takes half of tensor memory, so the request is served by the single-tile kernels
+    (P in place over S) with 64-key tiles, Split-K included; every other plan is ineligible and the base plan of the
+    key is one of those kernels.  All rows against the oracle, tile plan == E(M)."""
+    H, d = 2, 256
+    M = I.random_mask(91, H, I.cdiv(N, B_Q), I.cdiv(N_kv or N, B_KV), 0.35, diag=True, empty_rows=0.1)
+    req = I.Request("d256", H, N, d, B_Q, B_KV, M, qkv_seed=37, N_kv=N_kv)
+    res = Hh.run_request(req, plan_id=plan_id, guards=False)
+    cat = bsa.catalog()[res["info"]["plan"]["plan_id"]]
+    assert cat["kernel"] in (0, 3) and cat["T_KV"] == 64 and res["info"]["d"] == 256
+    mask = torch.from_numpy(M).cuda()
+    for bad in (22, 18, 10, 14, 36):     # ping-pong, 128-key tiles, paired, column-split, row-block
+        with pytest.raises(bsa.BsaError) as e:
+            bsa.plan_create(mask, B_Q, B_KV, N, H, d, plan_id=bad, N_kv=N_kv)
+        assert e.value.status == 3
+
+
 # ---------------------------------------------------------------- token-major layout [N, heads, d]
 @pytest.mark.parametrize("B_Q,B_KV,N,N_kv,d,dtype", [(64, 64, 2048, 0, 64, "bf16"), (128, 128, 3000, 0, 128, "bf16"),
                                                       (32, 64, 1500, 2600, 128, "bf16"), (128, 128, 2500, 0, 128, "fp16")])
@@ -427,12 +476,12 @@ def test_token_major_layout_gives_the_same_output(B_Q, B_KV, N, N_kv, d, dtype):
     qt, kt, vt = (t.permute(1, 0, 2).contiguous() for t in (q, k, v))
     cat = bsa.catalog()
     plans = []
-    for kern in (4, 0, 1, 2, 3):
+    for kern in (4, 0, 1, 2, 3, 5):
         ids = [c["plan_id"] for c in cat if c["kernel"] == kern and c["split_pmax"] == 1 and
-               (dtype == "bf16" or kern == 4) and bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d)]
+               bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d, N_kv=N_kv, dtype=dtype)]
         plans += ids[:1]
-    plans += [c["plan_id"] for c in cat if c["split_pmax"] > 1 and (dtype == "bf16" or c["kernel"] == 4) and
-              bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d)][:1]
+    plans += [c["plan_id"] for c in cat if c["split_pmax"] > 1 and
+              bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d, N_kv=N_kv, dtype=dtype)][:1]
     assert len(plans) >= (6 if dtype == "bf16" else 2)
     for n, pid in enumerate(plans):
         with bsa.plan_create(mask, B_Q, B_KV, N, H, d, plan_id=pid, N_kv=N_kv, dtype=dtype) as pa, \
@@ -596,8 +645,7 @@ def _random_request(n):
                     a = int(r.randint(0, nKb))
                     M[h, q, a:a + int(r.randint(1, 9))] = 1
     cat = bsa.catalog()
-    ok = [c["plan_id"] for c in cat if (dtype == "bf16" or c["kernel"] == 4) and
-          bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d)]
+    ok = [c["plan_id"] for c in cat if bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d, N_kv=N_kv, dtype=dtype)]
     plan_id = -1 if r.rand() < 0.3 else int(r.choice(ok))
     return I.Request(f"random{n}", H, N, d, B_Q, B_KV, M, qkv_seed=300 + n, N_kv=N_kv, dtype=dtype), plan_id
 

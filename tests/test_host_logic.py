@@ -40,14 +40,14 @@ def test_catalog_and_eligibility():
     cat = bsa.catalog()
     assert len(cat) >= 6 and [c["plan_id"] for c in cat] == list(range(len(cat)))
     assert len(set(c["name"] for c in cat)) == len(cat)
-    assert {c["T_KV"] for c in cat} == {64, 128} and {c["T_Q"] for c in cat} == {128, 256}
-    assert {c["kernel"] for c in cat} == {0, 1, 2, 3, 4}
+    assert {c["T_KV"] for c in cat} == {16, 32, 64, 128} and {c["T_Q"] for c in cat} == {16, 128, 256}
+    assert {c["kernel"] for c in cat} == {0, 1, 2, 3, 4, 5}
     base = bsa.lib().bsa_base_plan(128, 128, 128)
     # the base plan is eligible for every supported request key
     for B_Q in (16, 32, 64, 128, 256):
         for B_KV in (16, 32, 64, 128, 256):
-            for d in (64, 128):
-                assert bsa.plan_eligible(base, B_Q, B_KV, 75600, 24, d)
+            for d in (64, 128, 256):
+                assert bsa.plan_eligible(bsa.lib().bsa_base_plan(B_Q, B_KV, d), B_Q, B_KV, 75600, 24, d)
     assert not bsa.plan_eligible(base, 8, 64, 1024, 1, 64)       # block size below 16
     assert not bsa.plan_eligible(base, 64, 64, 1024, 1, 96)      # head dim outside the catalog
     assert not bsa.plan_eligible(len(cat), 64, 64, 1024, 1, 64)  # unknown plan
@@ -55,6 +55,14 @@ def test_catalog_and_eligibility():
     assert bsa.plan_eligible(split["plan_id"], 64, 64, 2048, 2, 64)
     assert not bsa.plan_eligible(split["plan_id"], 64, 64, 2048, 2, 64, max_workspace_bytes=4096)  # workspace
     assert not bsa.plan_eligible(split["plan_id"], 128, 128, 115200, 24, 128)  # default workspace limit
+    # the 16-row-tile kernel: logical blocks of up to 64 rows, KV tiles no wider than the block or the staging buffer, bf16
+    rb = {c["name"]: c["plan_id"] for c in cat if c["kernel"] == 5}
+    assert bsa.plan_eligible(rb["q16k64_rb"], 16, 64, 32768, 16, 64) and bsa.plan_eligible(rb["q16k32_rb"], 32, 32, 75600, 24, 128)
+    assert not bsa.plan_eligible(rb["q16k64_rb"], 16, 64, 32768, 16, 128)     # 64 keys x 128 x 2 bytes > 8 KB staging
+    assert not bsa.plan_eligible(rb["q16k64_rb"], 16, 32, 32768, 16, 64)      # would need membership masks
+    assert not bsa.plan_eligible(rb["q16k32_rb"], 128, 128, 16384, 8, 128)    # nothing to win on 128-row blocks
+    assert not bsa.plan_eligible(rb["q16k32_rb"], 32, 32, 75600, 24, 128, dtype="fp16")
+    assert bsa.plan_eligible(22, 128, 128, 4096, 2, 128, N_kv=999, dtype="fp16") and not bsa.plan_eligible(0, 128, 128, 4096, 2, 128, dtype="fp16")
 
 
 def test_feature_schema_buckets():
