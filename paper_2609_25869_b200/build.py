@@ -28,6 +28,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--threads", "4"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("BSA_NVCC_FLAGS", "").split()  # e.g. -DBSA_TRACE for the timeline-tracing debug build
     cmd += ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:
