@@ -142,12 +142,15 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons), "source": "nvidia-smi"}
 
 
-def make_request(workload: str, rank: int):
+def make_request(workload: str, rank: int, heads: int = 0):
+    """The named workload; `heads` > 0 overrides its head count (a reduced copy of the same shape, e.g. for a profiler
+    capture that must stay small)."""
     from paper_2609_25869_b200 import inputs as I
+    kw = {"H": heads} if heads > 0 else {}
     if workload.startswith("sweep"):
-        req = I.config_sweep(int(workload[5:] or 0) + 50 * rank)
+        req = I.config_sweep(int(workload[5:] or 0) + 50 * rank, **kw)
     else:
-        req = I.CONFIGS[workload]()
+        req = I.CONFIGS[workload](**kw)
     if rank:
         req.qkv_seed += 7919 * rank
     return req
@@ -185,7 +188,7 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     from oracle import oracle
-    req = make_request(args.workload, 0)
+    req = make_request(args.workload, 0, args.heads)
     qkv = req.qkv()
     nblocks = args.ref_blocks
     oracle_sample(req, qkv, min(nblocks, 8))  # builds/loads the library
@@ -222,8 +225,9 @@ def start_sweep_generation(n_requests: int, heads: int):
     """Generates the sweep's masks in worker processes (forked BEFORE this process touches CUDA) while the main
     benchmarks run; returns (pool, ordered result iterator)."""
     import multiprocessing as mp
-    workers = max(1, min(12, (os.cpu_count() or 2) - 2, n_requests))
-    pool = mp.get_context("fork").Pool(workers)
+    # at most half of the cores, at low priority: the timed host path (statistics poll, launches) must not wait for a core
+    workers = max(1, min(8, (os.cpu_count() or 2) // 2, n_requests))
+    pool = mp.get_context("fork").Pool(workers, initializer=os.nice, initargs=(15,))
     return pool, pool.imap(_gen_sweep_request, [(r, heads) for r in range(n_requests)])
 
 
@@ -375,6 +379,7 @@ def main():
     ap.add_argument("--workload", default="hunyuan",
                     help="hunyuan (default: the largest single-GPU configuration), mid, tiny, stress_a, stress_b, sweepN, sweep")
     ap.add_argument("--plan", type=int, default=-1, help="force a catalog plan id (-1: Algorithm 2)")
+    ap.add_argument("--heads", type=int, default=0, help="override the workload's head count (reduced copies for profiler captures)")
     ap.add_argument("--lut", default="", help="plan table to load instead of the packaged one")
     ap.add_argument("--ref-blocks", type=int, default=256, help="query blocks per reference step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -423,7 +428,7 @@ def main():
         torch.cuda.synchronize()
 
     def bench_workload(name, steps, warmup, primary):
-        req = make_request(name, 0 if args.shard_heads else rank)
+        req = make_request(name, 0 if args.shard_heads else rank, args.heads if primary else 0)
         q, k, v = req.qkv()
         if args.shard_heads:  # every rank builds the same request and keeps its own contiguous range of heads
             import dataclasses
@@ -504,7 +509,7 @@ def main():
         k_ms = [a.elapsed_time(b) for a, b in kev]
         res = {"req": req, "pairs": pairs, "flops": flops, "step_ms": sum(step_ms) / len(step_ms),
                "step_ms_median": statistics.median(step_ms), "host_us": statistics.median(host_us),
-               "planning_ms": sum(plan_ms) / len(plan_ms),
+               "planning_ms": statistics.median(plan_ms), "planning_ms_all": [round(x, 4) for x in plan_ms],
                "destroy_us": statistics.median(destroy_us) if destroy_us else None,
                "kernel_ms": sum(k_ms) / len(k_ms), "kernel_ms_median": statistics.median(k_ms), "info": info,
                "launches": launches, "clocks": clocks, "qkv": (q, k, v)}
@@ -641,7 +646,8 @@ def main():
                     "us_plan_create_host": inf["us_total"], "us_plan_destroy_host": r["destroy_us"],
                     "us_mask_state": inf["us_mask_state"], "us_stats_sync": inf["us_stats_sync"],
                     "us_lookup": inf["us_lookup"], "us_launch_prep": inf["us_launch_prep"],
-                    "us_planning_gpu": r["planning_ms"] * 1e3, "planning_fraction": r["planning_ms"] / r["step_ms"],
+                    "us_planning_gpu": r["planning_ms"] * 1e3, "us_planning_gpu_samples": [x * 1e3 for x in r["planning_ms_all"]],
+                    "planning_fraction": r["planning_ms"] / r["step_ms"],
                     "plan": inf["plan"]["name"], "lut_hit": inf["lut_hit"], "lut_regimes": lut_regimes,
                     "ntiles": inf["ntiles"],
                     "nitems": inf["nitems"], "active_pairs": r["pairs"], "covered_pairs": inf["covered_pairs"],

@@ -360,9 +360,10 @@ BSA_API bsa_status_t bsa_lut_load(const char* path);
 BSA_API void bsa_lut_clear(void);
 BSA_API int bsa_lut_num_regimes(void);
 /* Request keys for which the loaded table holds a learned second-stage partition (Section 5.1: thresholds learned by
- * a decision tree over log2 N, heads, density, skew and run coverage; its leaves are the regimes).  Such a key is
- * looked up in its tree; the other keys use the regimes of the fixed bucket edges.  In bsa_plan_info_t a tree lookup
- * shows as lut_hit = 1 with (leaf index + 1) << 8 added to regime_bucket[3]. */
+ * a decision tree over log2 N, heads, density, skew and run coverage; its leaves are regimes too).  A request is
+ * looked up in the regimes of the fixed bucket edges first; if the table has no such regime, in its key's tree; if the
+ * key has no tree either, the base plan is used.  In bsa_plan_info_t a tree lookup shows as lut_hit = 1 with
+ * (leaf index + 1) << 8 added to regime_bucket[3]. */
 BSA_API int bsa_lut_num_trees(void);
 /* Regime lookup + ranked fallback only (no GPU): returns the plan id Algorithm 2 selects for these
  * request scalars, or -1 for no-eligible-plan.  *hit_out (optional) = 1 if the regime was found. */

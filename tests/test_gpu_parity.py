@@ -622,7 +622,7 @@ def test_head_sharded_forward_equals_the_unsharded_one():
 # ---------------------------------------------------------------- seeded random requests
 def _random_request(n):
     """Request n of a seeded family: geometry, token counts (ragged, N_q != N_kv in a third of the cases), head
-    dimension, element type, mask structure (Bernoulli, runs, banded, with empty rows) and plan all follow from n."""
+    dimension (64, 128 and now and then 256), element type, mask structure (Bernoulli, runs, banded, with empty rows) and plan all follow from n."""
     r = np.random.RandomState(1000 + n)
     B_Q, B_KV = (int(2 ** r.randint(4, 9)) for _ in range(2))
     d = int(r.choice([64, 128]))
@@ -646,6 +646,8 @@ def _random_request(n):
                 for _ in range(int(r.randint(0, 4))):
                     a = int(r.randint(0, nKb))
                     M[h, q, a:a + int(r.randint(1, 9))] = 1
+    if dtype == "bf16" and r.rand() < 0.12:
+        d = 256     # served by the single-tile kernels only
     cat = bsa.catalog()
     ok = [c["plan_id"] for c in cat if bsa.plan_eligible(c["plan_id"], B_Q, B_KV, N, H, d, N_kv=N_kv, dtype=dtype)]
     plan_id = -1 if r.rand() < 0.3 else int(r.choice(ok))

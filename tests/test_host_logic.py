@@ -217,6 +217,13 @@ def test_decision_tree_regimes_hand_built_case(tmp_path):
     assert bsa.lut_select(128, 128, 16384, 8, 128, 0.50, 0.5, 1.2) == (3, True)
     assert bsa.lut_select(128, 128, 16384, 8, 128, t[0]["threshold"], 0.5, 1.2) == (3, True)   # feature < threshold goes left
     assert bsa.lut_select(64, 64, 16384, 8, 128, 0.05, 0.5, 1.2) == (bsa.lib().bsa_base_plan(64, 64, 128), False)  # key without a tree
+    # a fixed-edge regime of the same key takes precedence where it exists; everywhere else the tree answers
+    b = bsa.lut_buckets(16384, 0.05, 1.2, 0.5)
+    LB.write_table(path, {(key, (b[0], 1, b[1], b[2], b[3])): [7, 22]}, int(bsa.lib().bsa_catalog_hash()), "test", trees=trees)
+    bsa.lut_load(path)
+    assert bsa.lut_select(128, 128, 16384, 8, 128, 0.05, 0.5, 1.2) == (7, True)
+    assert bsa.lut_select(128, 128, 16384, 8, 128, 0.50, 0.5, 1.2) == (3, True)
+    LB.write_table(path, {}, int(bsa.lib().bsa_catalog_hash()), "test", trees=trees)
     # malformed trees are rejected as a whole file
     text = open(path).read()
     for bad in (text.replace("BSA_LUT 2", "BSA_LUT 1"), text.replace("node 2 leaf", "node 1 leaf"),
