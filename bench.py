@@ -34,7 +34,9 @@ METRIC = "effective TFLOP/s on active blocks (4*d flops per active token pair)"
 # whole under the pool's size rule; its figure is a 4-head capture of the same shape scaled by heads (the plan keeps
 # heads apart in the queue, so traffic grows in proportion to them).
 NCU_TRAFFIC_BYTES = {
+    "hunyuan": (6 * 798.2e6, "ncu capture of one launch of the same shape at 4 heads (682.3 MB read + 116.0 MB written), x 24/4"),
     "mid": (206.5e6, "one ncu capture of one launch of this workload"),
+    "stress_a": (266.9e6, "one ncu capture of one launch of this workload (row-block kernel)"),
 }
 KERNEL_NAMES = {0: "bsa_attention_kernel<D,TK,false>", 1: "bsa_attention_pair_kernel<D,TK>", 2: "bsa_attention_cs_kernel<D,TK>",
                 3: "bsa_attention_kernel<D,TK,true>", 4: "bsa_attention_pp_kernel<D,TK,F16>", 5: "bsa_attention_rb_kernel<D,CK>"}

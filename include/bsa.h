@@ -74,7 +74,8 @@ typedef struct bsa_plan_desc {
 
 /* Element type of Q, K, V and O (a tensor property x of the request, Section 4.4).  Scores, softmax state and the
  * output accumulator are fp32 either way; P is rounded to the same 16-bit type for the second product.  Half inputs
- * are served by the plans of the ping-pong kernel only (the others are not eligible for such a request). */
+ * are served by the single-tile, ping-pong and row-block kernels; the plans of the paired and of the column-split
+ * kernel are not eligible for such a request. */
 enum { BSA_DTYPE_BF16 = 0, BSA_DTYPE_FP16 = 1 };
 /* Storage layout of Q, K, V and O (another tensor property of the request, Section 3 / Section 4.4):
  * [heads][N][d] (head-major, the default) or [N][heads][d] (token-major, what a fused QKV projection of a
@@ -143,8 +144,8 @@ typedef struct bsa_plan_info {
  *   N        : query tokens per head, N_q of Section 2.1; need not be a multiple of the block sizes.
  *              The key/value token count N_kv equals N unless options->N_kv says otherwise (_ex variants).
  *   heads    : independent (batch x head) problems.
- *   d        : head dimension, 64, 128 or 256 (256: bf16 only, served by the single-tile kernels with 64-key
- *              tiles, whose 256-column output accumulator fills half of tensor memory).  Scale is 1/sqrt(d);
+ *   d        : head dimension, 64, 128 or 256 (256: served by the single-tile kernels with 64-key tiles, whose
+ *              256-column output accumulator fills half of tensor memory).  Scale is 1/sqrt(d);
  *              attention is non-causal.
  *   out_plan : receives the plan; the plan owns its device buffers (CSR, tile lists, work items,
  *              Split-K workspace).  Reusable for any number of forwards with the same mask.

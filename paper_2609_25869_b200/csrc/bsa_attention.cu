@@ -88,7 +88,7 @@ struct __align__(8) Barriers {
 // P = exp2(s * c2 - m_ref) rounded to bf16 and written to t_p (over S in place when t_p == t_s), running sum.
 // The reference maximum moves only when the tile maximum exceeds it by kRescaleThreshold (log2
 // units), so P stays below 2^8 and the running output needs rescaling (by `alpha`) only then.
-template <int TK>
+template <int TK, bool F16 = false>
 __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, bool need_mask, uint32_t row_bits, int lgBKV, int n_valid,
                                              float c2, bool not_first, float& m_ref, float& l, float& alpha,
                                              bool& rescale) {
@@ -139,8 +139,8 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, bool ne
         const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
         sum01 = add_f32x2(sum01, pack_f32x2(p0, p1));
         sum23 = add_f32x2(sum23, pack_f32x2(p2, p3));
-        r[i / 2] = pack_bf16x2(p0, p1);
-        r[i / 2 + 1] = pack_bf16x2(p2, p3);
+        r[i / 2] = pack_16x2<F16>(p0, p1);
+        r[i / 2 + 1] = pack_16x2<F16>(p2, p3);
     }
     float s0, s1, s2, s3;
     unpack_f32x2(sum01, s0, s1);
@@ -156,7 +156,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t t_s, uint32_t t_p, bool ne
 // DUAL = true adds a seventh warp so that Q K^T and P V are issued by two different threads: the
 // Q K^T issuer runs up to two tiles ahead (S is double-buffered) instead of stalling behind the wait
 // for the softmax of the previous tile; ordering between the two issuers is carried by mbarriers only.
-template <int D, int TK, bool DUAL>
+template <int D, int TK, bool DUAL, bool F16>
 __global__ void __launch_bounds__(DUAL ? kThreads + 32 : kThreads, 1)
 bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
@@ -261,8 +261,8 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     } else if (warp == 5 && !DUAL) {
         // =========================== MMA issuer ===========================
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
-            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            constexpr uint32_t idesc_qk = make_idesc_f32(kTQ, TK, 0, 0, F16);
+            constexpr uint32_t idesc_pv = make_idesc_f32(kTQ, D, 0, 1, F16);
             const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
             const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
             const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
@@ -330,7 +330,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     } else if (warp == 5) {
         // =========================== Q K^T issuer (DUAL) ===========================
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = make_idesc_bf16_f32(kTQ, TK, 0, 0);
+            constexpr uint32_t idesc_qk = make_idesc_f32(kTQ, TK, 0, 0, F16);
             const uint64_t descQ = make_smem_desc_sw128(smem_u32(sQ), 16, 1024);
             const uint64_t descK = make_smem_desc_sw128(smem_u32(sK), 16, 1024);
             uint32_t itq = 0, g = 0;
@@ -376,7 +376,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     } else if (warp == 6) {
         // =========================== P V issuer (DUAL) ===========================
         if (lane == 0) {
-            constexpr uint32_t idesc_pv = make_idesc_bf16_f32(kTQ, D, 0, 1);
+            constexpr uint32_t idesc_pv = make_idesc_f32(kTQ, D, 0, 1, F16);
             const uint64_t descV = make_smem_desc_sw128(smem_u32(sV), KV_SUB, 1024);
             uint32_t itq = 0, g = 0;
             bool ok = true;
@@ -455,7 +455,7 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 const uint32_t t_s = tmem + lane_base + (sb ? kColS1 : kColS0);
                 float alpha;
                 bool rescale;
-                softmax_tile<TK>(t_s, t_s, need_mask, row_bits, p.lgBKV, n_valid, c2, j > 0, m_ref, l, alpha, rescale);
+                softmax_tile<TK, F16>(t_s, t_s, need_mask, row_bits, p.lgBKV, n_valid, c2, j > 0, m_ref, l, alpha, rescale);
 #ifdef BSA_TRACE
                 if (lane == 0 && blockIdx.x == 0 && tn + 3 < 4096) {
                     g_trace[2 + warp][tn++] = (g_trace_aux[warp][0] << 8) | 11;
@@ -507,10 +507,10 @@ bsa_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 uint4 v;
-                                v.x = pack_bf16x2(__uint_as_float(r[q * 8 + 0]) * inv_l, __uint_as_float(r[q * 8 + 1]) * inv_l);
-                                v.y = pack_bf16x2(__uint_as_float(r[q * 8 + 2]) * inv_l, __uint_as_float(r[q * 8 + 3]) * inv_l);
-                                v.z = pack_bf16x2(__uint_as_float(r[q * 8 + 4]) * inv_l, __uint_as_float(r[q * 8 + 5]) * inv_l);
-                                v.w = pack_bf16x2(__uint_as_float(r[q * 8 + 6]) * inv_l, __uint_as_float(r[q * 8 + 7]) * inv_l);
+                                v.x = pack_16x2<F16>(__uint_as_float(r[q * 8 + 0]) * inv_l, __uint_as_float(r[q * 8 + 1]) * inv_l);
+                                v.y = pack_16x2<F16>(__uint_as_float(r[q * 8 + 2]) * inv_l, __uint_as_float(r[q * 8 + 3]) * inv_l);
+                                v.z = pack_16x2<F16>(__uint_as_float(r[q * 8 + 4]) * inv_l, __uint_as_float(r[q * 8 + 5]) * inv_l);
+                                v.w = pack_16x2<F16>(__uint_as_float(r[q * 8 + 6]) * inv_l, __uint_as_float(r[q * 8 + 7]) * inv_l);
                                 *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = v;
                             }
                         }
@@ -2055,7 +2055,7 @@ EncodeTiledFn get_encode_fn() {
 
 // bf16 [heads][N][d] viewed as a 3-D tensor {d, N, heads}; box = {64, rows, 1}; rows beyond N read as zero.
 // `nhd`: the tensor is stored [N][heads][d] instead (token-major); only the two byte strides change.
-bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows, bool nhd) {
+bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, int box_rows, bool f16, bool nhd) {
     EncodeTiledFn enc = get_encode_fn();
     if (!enc) return false;
     cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)heads};
@@ -2066,7 +2066,8 @@ bool encode_map(CUtensorMap* m, const void* base, int64_t N, int heads, int d, i
     }
     cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
     cuuint32_t es[3] = {1, 1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+    return enc(m, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims,
+               strides, box, es,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -2097,16 +2098,16 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
                              ? (encode_map4(&tq, a.Q, a.g.N, a.g.H, D, kTQ, a.f16, a.nhd) &&
                                 encode_map4(&tk, a.K, a.g.N_kv, a.g.H, D, TK, a.f16, a.nhd) &&
                                 encode_map4(&tv, a.V, a.g.N_kv, a.g.H, D, TK, a.f16, a.nhd))
-                             : (encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ, a.nhd) &&
-                                encode_map(&tk, a.K, a.g.N_kv, a.g.H, D, TK, a.nhd) &&
-                                encode_map(&tv, a.V, a.g.N_kv, a.g.H, D, TK, a.nhd));
+                             : (encode_map(&tq, a.Q, a.g.N, a.g.H, D, kTQ, a.f16, a.nhd) &&
+                                encode_map(&tk, a.K, a.g.N_kv, a.g.H, D, TK, a.f16, a.nhd) &&
+                                encode_map(&tv, a.V, a.g.N_kv, a.g.H, D, TK, a.f16, a.nhd));
     if (!ok_maps) {
         *err = "cuTensorMapEncodeTiled failed";
         return cudaErrorInvalidValue;
     }
     const int smem = attention_smem_bytes(D, TK, a.stages, KERNEL);
-    if (a.f16 && KERNEL != 4) {  // only the ping-pong kernel is instantiated for half inputs (eligibility says so too)
-        *err = "fp16 inputs need a ping-pong-kernel plan";
+    if (a.f16 && (KERNEL == 1 || KERNEL == 2)) {  // not instantiated for half inputs (eligibility says so too)
+        *err = "fp16 inputs need a single-tile, ping-pong or row-block plan";
         return cudaErrorInvalidValue;
     }
     // largest size already allowed, per instantiation and per device (the attribute belongs to the device's copy of
@@ -2115,10 +2116,11 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
     const int dev = (a.device >= 0 && a.device < kMaxDevices) ? a.device : 0;
     if (smem > attr_bytes_dev[dev].load(std::memory_order_relaxed)) {
         cudaError_t e;
-        if constexpr (KERNEL == 0)
-            e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        else if constexpr (KERNEL == 3)
-            e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if constexpr (KERNEL == 0 || KERNEL == 3) {
+            e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, KERNEL == 3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(bsa_attention_kernel<D, TK, KERNEL == 3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        }
         else if constexpr (KERNEL == 1)
             e = cudaFuncSetAttribute(bsa_attention_pair_kernel<D, TK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         else if constexpr (KERNEL == 2)
@@ -2136,10 +2138,13 @@ cudaError_t launch_attn(const ForwardArgs& a, const AttnParams& p, cudaStream_t 
     }
     int grid = a.num_sms < a.max_items ? a.num_sms : a.max_items;
     if (grid < 1) grid = 1;
-    if constexpr (KERNEL == 0)
-        bsa_attention_kernel<D, TK, false><<<grid, kThreads, smem, stream>>>(tq, tk, tv, p);
-    else if constexpr (KERNEL == 3)
-        bsa_attention_kernel<D, TK, true><<<grid, kThreads + 32, smem, stream>>>(tq, tk, tv, p);
+    if constexpr (KERNEL == 0 || KERNEL == 3) {
+        constexpr int threads = KERNEL == 3 ? kThreads + 32 : kThreads;
+        if (a.f16)
+            bsa_attention_kernel<D, TK, KERNEL == 3, true><<<grid, threads, smem, stream>>>(tq, tk, tv, p);
+        else
+            bsa_attention_kernel<D, TK, KERNEL == 3, false><<<grid, threads, smem, stream>>>(tq, tk, tv, p);
+    }
     else if constexpr (KERNEL == 1)
         bsa_attention_pair_kernel<D, TK><<<grid, kPairThreads, smem, stream>>>(tq, tk, tv, p);
     else if constexpr (KERNEL == 2)

@@ -6,7 +6,7 @@
 // active pairs on masks whose neighbouring row blocks select different columns).  This kernel keeps such masks at
 // their own granularity instead: one WARP owns a 16-row fragment of a logical row block (a 16-row physical tile,
 // Refined along Q for B_Q > 16) and walks that block's own KV tile list with the register-level tensor instruction
-// mma.sync.m16n8k16 (bf16 in, fp32 accumulate), FlashAttention-2 style:
+// mma.sync.m16n8k16 (bf16 or fp16 in, fp32 accumulate), FlashAttention-2 style:
 //   * K and V chunks of T_KV keys (8 KB each at most) are gathered with cp.async into a 16 KB staging area private to
 //     the warp (128-byte-row XOR swizzle), K read back with ldmatrix, V with ldmatrix.trans; the next K chunk is in
 //     flight during the softmax and P V of the current one, the next V chunk during the next Q K^T;
@@ -65,21 +65,32 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, u
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                  : "r"(addr));
 }
-// D (16x8, fp32) += A (16x16, bf16, row-major) * B (16x8, bf16, column-major)
+// D (16x8, fp32) += A (16x16, row-major) * B (16x8, column-major); A and B bf16, or IEEE half with F16
+template <bool F16>
 __device__ __forceinline__ void mma_16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    if (F16)
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+template <bool F16>
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {  // two fp32 -> the kernel's 16-bit element type
     uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    if (F16)
+        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    else
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
 
@@ -108,7 +119,7 @@ __device__ __forceinline__ void stage_chunk(uint32_t dst, const __nv_bfloat16* _
     }
 }
 
-template <int D, int CK>
+template <int D, int CK, bool F16>
 __global__ void __launch_bounds__(kRbWarps * 32, 1) bsa_attention_rb_kernel(const RbParams p) {
     static_assert(CK * D * 2 <= kRbStageBytes, "a chunk must fit its staging buffer");
     static_assert(CK % 16 == 0 && D % 16 == 0, "whole MMA steps");
@@ -197,8 +208,8 @@ __global__ void __launch_bounds__(kRbWarps * 32, 1) bsa_attention_rb_kernel(cons
                     const int chunk = ks * 2 + ((lane >> 3) & 1);
                     uint32_t b0, b1, b2, b3;
                     ldmatrix_x4(sK + swz<D * 2>(key, chunk), b0, b1, b2, b3);
-                    mma_16816(s[2 * np], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
-                    mma_16816(s[2 * np + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
+                    mma_16816<F16>(s[2 * np], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+                    mma_16816<F16>(s[2 * np + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
                 }
             }
             __syncwarp();  // every lane has read the K buffer
@@ -237,8 +248,8 @@ __global__ void __launch_bounds__(kRbWarps * 32, 1) bsa_attention_rb_kernel(cons
                 const float p2 = ex2(fmaf(s[n][2], c2, nm_hi)), p3 = ex2(fmaf(s[n][3], c2, nm_hi));
                 sum_lo += p0 + p1;
                 sum_hi += p2 + p3;
-                pa[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
-                pa[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+                pa[n >> 1][(n & 1) * 2 + 0] = pack_bf16<F16>(p0, p1);
+                pa[n >> 1][(n & 1) * 2 + 1] = pack_bf16<F16>(p2, p3);
             }
             l_lo = fmaf(l_lo, a_lo, sum_lo);
             l_hi = fmaf(l_hi, a_hi, sum_hi);
@@ -263,8 +274,8 @@ __global__ void __launch_bounds__(kRbWarps * 32, 1) bsa_attention_rb_kernel(cons
                     const int chunk = nd * 2 + (lane >> 4);
                     uint32_t b0, b1, b2, b3;
                     ldmatrix_x4_trans(sV + swz<D * 2>(key, chunk), b0, b1, b2, b3);
-                    mma_16816(o[2 * nd], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b0, b1);
-                    mma_16816(o[2 * nd + 1], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b2, b3);
+                    mma_16816<F16>(o[2 * nd], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b0, b1);
+                    mma_16816<F16>(o[2 * nd + 1], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b2, b3);
                 }
             }
             __syncwarp();  // every lane has read the V buffer
@@ -281,8 +292,8 @@ __global__ void __launch_bounds__(kRbWarps * 32, 1) bsa_attention_rb_kernel(cons
         const float inv_lo = (l_lo > 0.f) ? 1.f / l_lo : 0.f, inv_hi = (l_hi > 0.f) ? 1.f / l_hi : 0.f;
 #pragma unroll
         for (int n = 0; n < NT_O; ++n) {
-            if (r_lo < p.N) *reinterpret_cast<uint32_t*>(o_lo + n * 8 + 2 * t) = pack_bf16(o[n][0] * inv_lo, o[n][1] * inv_lo);
-            if (r_hi < p.N) *reinterpret_cast<uint32_t*>(o_hi + n * 8 + 2 * t) = pack_bf16(o[n][2] * inv_hi, o[n][3] * inv_hi);
+            if (r_lo < p.N) *reinterpret_cast<uint32_t*>(o_lo + n * 8 + 2 * t) = pack_bf16<F16>(o[n][0] * inv_lo, o[n][1] * inv_lo);
+            if (r_hi < p.N) *reinterpret_cast<uint32_t*>(o_hi + n * 8 + 2 * t) = pack_bf16<F16>(o[n][2] * inv_hi, o[n][3] * inv_hi);
         }
         if (t == 0) {
             if (r_lo < p.N)
@@ -293,13 +304,13 @@ __global__ void __launch_bounds__(kRbWarps * 32, 1) bsa_attention_rb_kernel(cons
     }
 }
 
-template <int D, int CK>
-cudaError_t launch_rb(const ForwardArgs& a, const RbParams& p, cudaStream_t stream, const char** err) {
+template <int D, int CK, bool F16>
+cudaError_t launch_rb_t(const ForwardArgs& a, const RbParams& p, cudaStream_t stream, const char** err) {
     constexpr int smem = kRbWarps * 2 * kRbStageBytes;
     static std::atomic<int> attr_set_dev[kMaxDevices];
     const int dev = (a.device >= 0 && a.device < kMaxDevices) ? a.device : 0;
     if (!attr_set_dev[dev].load(std::memory_order_relaxed)) {
-        cudaError_t e = cudaFuncSetAttribute(bsa_attention_rb_kernel<D, CK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(bsa_attention_rb_kernel<D, CK, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) {
             *err = "cudaFuncSetAttribute(max dynamic shared memory)";
             return e;
@@ -309,9 +320,13 @@ cudaError_t launch_rb(const ForwardArgs& a, const RbParams& p, cudaStream_t stre
     long long want = ((long long)a.max_items + kRbWarps - 1) / kRbWarps;
     int grid = want < a.num_sms ? (int)want : a.num_sms;
     if (grid < 1) grid = 1;
-    bsa_attention_rb_kernel<D, CK><<<grid, kRbWarps * 32, smem, stream>>>(p);
+    bsa_attention_rb_kernel<D, CK, F16><<<grid, kRbWarps * 32, smem, stream>>>(p);
     count_launch();
     return cudaGetLastError();
+}
+template <int D, int CK>
+cudaError_t launch_rb(const ForwardArgs& a, const RbParams& p, cudaStream_t stream, const char** err) {
+    return a.f16 ? launch_rb_t<D, CK, true>(a, p, stream, err) : launch_rb_t<D, CK, false>(a, p, stream, err);
 }
 
 }  // namespace
@@ -320,10 +335,6 @@ cudaError_t launch_rb(const ForwardArgs& a, const RbParams& p, cudaStream_t stre
 int rb_max_chunk(int d) { return kRbStageBytes / (d * 2); }
 
 cudaError_t launch_forward_rb(const ForwardArgs& a, cudaStream_t stream, const char** err_detail) {
-    if (a.f16) {
-        *err_detail = "the row-block kernel takes bf16 tensors only";
-        return cudaErrorInvalidValue;
-    }
     RbParams p;
     p.Q = reinterpret_cast<const __nv_bfloat16*>(a.Q);
     p.K = reinterpret_cast<const __nv_bfloat16*>(a.K);

@@ -121,7 +121,8 @@ bool plan_eligible(int plan_id, int B_Q, int B_KV, int64_t N, int heads, int d, 
     const bsa_plan_desc_t* P = catalog_entry(plan_id);
     if (!P) return false;
     if (dtype != BSA_DTYPE_BF16 && dtype != BSA_DTYPE_FP16) return false;
-    if (dtype == BSA_DTYPE_FP16 && P->kernel != 4) return false;  // tensor property: only the ping-pong kernel takes half
+    // tensor property: the paired and the column-split kernels are not instantiated for half tensors
+    if (dtype == BSA_DTYPE_FP16 && (P->kernel == 1 || P->kernel == 2)) return false;
     if (P->kernel == kKernelRowBlock) {
         // 16-row tiles: for logical blocks of up to 64 rows (on larger ones the 128-row tile wastes nothing that this
         // kernel could win back), KV tiles no wider than the logical block (no membership masks in this kernel) and

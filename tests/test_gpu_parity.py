@@ -409,29 +409,33 @@ def test_rectangular_request_from_host_buffers_packed_mask_and_cache():
 # ---------------------------------------------------------------- fp16 tensors (request property x, Section 4.4)
 @pytest.mark.parametrize("B_Q,B_KV,N,N_kv,d,plan_id", [
     (128, 128, 4096, 0, 128, -1), (64, 64, 3000, 0, 64, -1), (128, 128, 2100, 0, 128, 23), (16, 32, 1500, 0, 64, 25),
-    (128, 64, 2000, 0, 128, 26), (64, 64, 2048, 0, 64, 24), (32, 32, 1000, 2500, 128, 29), (128, 128, 4096, 0, 64, 33)])
+    (128, 64, 2000, 0, 128, 26), (64, 64, 2048, 0, 64, 24), (32, 32, 1000, 2500, 128, 29), (128, 128, 4096, 0, 64, 33),
+    (128, 128, 2100, 0, 128, 0), (64, 32, 1300, 0, 64, 3), (16, 64, 1500, 0, 128, 18), (256, 256, 1500, 0, 64, 19),
+    (16, 64, 1000, 0, 64, 34), (32, 32, 900, 1700, 128, 35), (64, 16, 700, 0, 64, 36),
+    (128, 128, 1500, 0, 256, -1), (32, 64, 900, 0, 256, 3)])
 def test_half_precision_requests_match_the_oracle(B_Q, B_KV, N, N_kv, d, plan_id):
-    """Q, K, V, O in IEEE half: the ping-pong kernel's fp16 instantiation (both head dims and tile widths, Direct /
-    Coarsened / Refined mappings, Split-K with the merge kernel's half output), all rows against the oracle reading
-    the same half bit patterns."""
+    """Q, K, V, O in IEEE half: the fp16 instantiations of the ping-pong kernel (both head dims and tile widths,
+    Direct / Coarsened / Refined mappings, Split-K with the merge kernel's half output), of the single-tile kernels
+    (one and two issuers, Split-K, d = 256) and of the row-block kernel, all rows against the oracle reading the same
+    half bit patterns."""
     H = 3
     M = I.random_mask(61, H, I.cdiv(N, B_Q), I.cdiv(N_kv or N, B_KV), 0.35, empty_rows=0.1)
     req = I.Request("half", H, N, d, B_Q, B_KV, M, qkv_seed=23, N_kv=N_kv, dtype="fp16")
     res = Hh.run_request(req, plan_id=plan_id)
     assert res["info"]["dtype"] == 1
-    assert bsa.catalog()[res["info"]["plan"]["plan_id"]]["kernel"] == 4
+    assert bsa.catalog()[res["info"]["plan"]["plan_id"]]["kernel"] in (0, 3, 4, 5)
 
 
 def test_half_precision_mid_and_ineligible_plans():
-    """The bench workload's shape in half; plans of the other kernel families are not eligible for a half request
-    (forced: no eligible plan; looked up: the ranking falls through to a ping-pong plan)."""
+    """The Mid shape in half; plans of the paired and column-split kernels are not eligible for a half request (forced:
+    no eligible plan; looked up: the ranking falls through to the next plan that is)."""
     req = I.config_mid()
     req.dtype = "fp16"
     Hh.run_request(req, plan_id=-1, sel=_sample(req, 16))
     mask, q, k, v, _ = Hh.to_dev(I.config_tiny())
     t = I.config_tiny()
     with pytest.raises(bsa.BsaError) as e:
-        bsa.plan_create(mask, t.B_Q, t.B_KV, t.N, t.H, t.d, plan_id=0, dtype="fp16")
+        bsa.plan_create(mask, t.B_Q, t.B_KV, t.N, t.H, t.d, plan_id=14, dtype="fp16")
     assert e.value.status == 3
     # the same bits through a bf16 plan and a half plan differ: the plan's dtype is what the kernel reads
     th = I.config_tiny()

@@ -61,8 +61,11 @@ def test_catalog_and_eligibility():
     assert not bsa.plan_eligible(rb["q16k64_rb"], 16, 64, 32768, 16, 128)     # 64 keys x 128 x 2 bytes > 8 KB staging
     assert not bsa.plan_eligible(rb["q16k64_rb"], 16, 32, 32768, 16, 64)      # would need membership masks
     assert not bsa.plan_eligible(rb["q16k32_rb"], 128, 128, 16384, 8, 128)    # nothing to win on 128-row blocks
-    assert not bsa.plan_eligible(rb["q16k32_rb"], 32, 32, 75600, 24, 128, dtype="fp16")
-    assert bsa.plan_eligible(22, 128, 128, 4096, 2, 128, N_kv=999, dtype="fp16") and not bsa.plan_eligible(0, 128, 128, 4096, 2, 128, dtype="fp16")
+    # half tensors: every kernel family but the paired (ids 10-13) and the column-split one (14-17)
+    assert bsa.plan_eligible(rb["q16k32_rb"], 32, 32, 75600, 24, 128, dtype="fp16")
+    assert bsa.plan_eligible(22, 128, 128, 4096, 2, 128, N_kv=999, dtype="fp16") and bsa.plan_eligible(0, 128, 128, 4096, 2, 128, dtype="fp16")
+    assert not bsa.plan_eligible(10, 128, 128, 4096, 2, 128, dtype="fp16") and not bsa.plan_eligible(14, 128, 128, 4096, 2, 128, dtype="fp16")
+    assert bsa.plan_eligible(19, 128, 128, 4096, 2, 256, dtype="fp16") and not bsa.plan_eligible(22, 128, 128, 4096, 2, 256, dtype="fp16")
 
 
 def test_feature_schema_buckets():
