@@ -515,27 +515,6 @@ def main():
                "destroy_us": statistics.median(destroy_us) if destroy_us else None,
                "kernel_ms": sum(k_ms) / len(k_ms), "kernel_ms_median": statistics.median(k_ms), "info": info,
                "launches": launches, "clocks": clocks, "qkv": (q, k, v)}
-        # Back-to-back forwards (no flush) for at least 250 ms with the clock sampled underneath: the fraction of the
-        # tensor pipe's issue capacity at the clock the kernel actually ran at, whatever the power state.
-        kern_s = res["kernel_ms"] * 1e-3
-        reps = max(3, min(20000, int(0.25 / max(kern_s, 1e-6)) + 1))
-        cs = ClockSampler(local_rank)
-        torch.cuda.synchronize()
-        cs.start()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for _ in range(reps):
-            plan.forward(qd, kd, vd, O, LSE)
-        b.record(stream)
-        b.synchronize()
-        cl = cs.stop()
-        bb_ms = a.elapsed_time(b) / reps
-        res["back_to_back"] = {"launch_ms": bb_ms, "launches": reps, "sm_mhz": cl.get("sm_mhz"),
-                               "sm_min_mhz": cl.get("sm_min_mhz"), "power_w_max": cl.get("power_w_max"),
-                               "reasons": cl.get("reasons"), "tflops": flops / (bb_ms * 1e-3) / 1e12}
-        if cl.get("sm_mhz"):
-            res["back_to_back"]["frac_of_tensor_issue_at_clock"] = flops / (
-                bb_ms * 1e-3 * cl["sm_mhz"] * 1e6 * num_sms * TENSOR_FLOP_PER_CLK_PER_SM)
         if info["plan"]["split_pmax"] > 1 and info["nsplit_rows"] > 0:
             # the Split-K reduction kernel alone (HBM-bound), over the partials the forwards above left behind
             mev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
@@ -577,6 +556,28 @@ def main():
             cache.destroy()
             w_ms = [a.elapsed_time(b) for a, b in wev]
             res["warm_ms"] = sum(w_ms) / len(w_ms)
+        # Last, because it heats the GPU into its power cap: back-to-back forwards (no flush) for at least 250 ms with the
+        # clock sampled underneath, for the fraction of the tensor pipe's issue capacity at the clock the kernel actually
+        # ran at, whatever the power state.
+        kern_s = res["kernel_ms"] * 1e-3
+        reps = max(3, min(20000, int(0.25 / max(kern_s, 1e-6)) + 1))
+        cs = ClockSampler(local_rank)
+        torch.cuda.synchronize()
+        cs.start()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            plan.forward(qd, kd, vd, O, LSE)
+        b.record(stream)
+        b.synchronize()
+        cl = cs.stop()
+        bb_ms = a.elapsed_time(b) / reps
+        res["back_to_back"] = {"launch_ms": bb_ms, "launches": reps, "sm_mhz": cl.get("sm_mhz"),
+                               "sm_min_mhz": cl.get("sm_min_mhz"), "power_w_max": cl.get("power_w_max"),
+                               "reasons": cl.get("reasons"), "tflops": flops / (bb_ms * 1e-3) / 1e12}
+        if cl.get("sm_mhz"):
+            res["back_to_back"]["frac_of_tensor_issue_at_clock"] = flops / (
+                bb_ms * 1e-3 * cl["sm_mhz"] * 1e6 * num_sms * TENSOR_FLOP_PER_CLK_PER_SM)
         info2 = plan.info()
         assert info2["device_status"] == 0, "a bounded device wait expired during the bench"
         plan.destroy()
@@ -620,7 +621,7 @@ def main():
     # runs under the 1 kW power cap like the seconds-long GEMM loop behind the "sustained" figure, which is given too.
     peak_key = "bf16_tflops"
     base_name = args.workload.rstrip("0123456789") if args.workload.startswith("sweep") else args.workload
-    traffic = NCU_TRAFFIC_BYTES.get(base_name)
+    traffic = NCU_TRAFFIC_BYTES.get(base_name) if not args.heads and args.plan < 0 else None  # the captured launch only
     line = {
         "metric": METRIC,
         "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -208,7 +208,7 @@ static std::mutex g_mu;
 // An inner node sends a request left when feature < threshold; a leaf holds a ranking.  Lookup order: the request's
 // fixed-edge regime if the table has it, else the leaf of its key's tree, else the key's base plan.  (Leaving each
 // mask source out of the corpus in turn, this order gave a geometric-mean regret of 1.026 against 1.030 for the trees
-// alone and 1.27 for the regimes alone, whose buckets a request from an unseen source hits only 22 % of the time.)
+// alone and 1.29 for the regimes alone, whose buckets a request from an unseen source hits only 22 % of the time.)
 struct TreeNode {
     int feature;        // -1: leaf
     double threshold;
