@@ -92,7 +92,15 @@ typedef struct bsa_options {
                                      The mask then has ceil(N_kv / B_KV) block columns, K and V are
                                      [heads, N_kv, d]; Q, O and LSE keep N rows.                      */
     int32_t layout;               /* BSA_LAYOUT_*                                                     */
-    int32_t reserved2;
+    int32_t batch;                /* explicit batch size (the paper's batch is a request dimension, Section 5.1); 0 or 1:
+                                     none.  `heads` still counts all independent problems, batch x heads-per-element
+                                     (mask [heads, nQb, nKb], LSE [heads, N]), and must be a multiple of it.  With
+                                     BSA_LAYOUT_HND the tensors are [batch][heads/batch][N][d], which is [heads][N][d]:
+                                     nothing changes.  With BSA_LAYOUT_NHD they are [batch][N][heads/batch][d]: the
+                                     plan is then one token-major plan per batch element (each selects its own
+                                     catalog plan) and bsa_forward runs them one after the other on the stream;
+                                     bsa_plan_get_info sums them, bsa_plan_export_* and the plan cache answer
+                                     BSA_ERR_UNSUPPORTED for such a plan.                              */
 } bsa_options_t;
 
 /* Scalar mask statistics s_A(M) (Section 5.1) and what launch preparation produced. */

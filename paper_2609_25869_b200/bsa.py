@@ -35,7 +35,7 @@ LAYOUTS = {"hnd": 0, "nhd": 1}   # BSA_LAYOUT_*: [heads, N, d] or [N, heads, d]
 class Options(ctypes.Structure):
     _fields_ = [("force_plan_id", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("max_workspace_bytes", ctypes.c_int64), ("N_kv", ctypes.c_int64),
-                ("layout", ctypes.c_int32), ("reserved2", ctypes.c_int32)]
+                ("layout", ctypes.c_int32), ("batch", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -157,6 +157,15 @@ def _stream_ptr(stream) -> Optional[int]:
     return getattr(stream, "cuda_stream", stream) or None
 
 
+def _lse_shape(Q, layout: str):
+    """[heads, N] for Q stored [heads, N, d], [N, heads, d] or, batched and token-major, [batch, N, heads/batch, d]."""
+    if layout == "hnd":
+        return (Q.shape[0], Q.shape[1]) if Q.dim() == 3 else (Q.shape[0] * Q.shape[1], Q.shape[2])
+    if Q.dim() == 4:
+        return (Q.shape[0] * Q.shape[2], Q.shape[1])
+    return (Q.shape[1], Q.shape[0])
+
+
 class Plan:
     """Handle of a prepared plan (``bsa_plan_create`` ... ``bsa_plan_destroy``)."""
 
@@ -172,8 +181,7 @@ class Plan:
         if O is None:
             O = torch.empty_like(Q)
         if LSE is None:  # [heads, N] whatever the layout of Q
-            hn = Q.shape[:2] if self.layout == "hnd" else (Q.shape[1], Q.shape[0])
-            LSE = torch.empty(hn, dtype=torch.float32, device=Q.device)
+            LSE = torch.empty(_lse_shape(Q, self.layout), dtype=torch.float32, device=Q.device)
         _check(lib().bsa_forward(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(),
                                  _stream_ptr(stream)), "bsa_forward")
         return O, LSE
@@ -229,13 +237,14 @@ class Plan:
 
 def plan_create(mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, plan_id: int = -1,
                 max_workspace_bytes: int = 0, stream=None, N_kv: int = 0, dtype: str = "bf16",
-                layout: str = "hnd") -> Plan:
+                layout: str = "hnd", batch: int = 0) -> Plan:
     """``bsa_plan_create_ex``: ``mask`` is a uint8/bool CUDA tensor ``[heads, nQb, nKb]``; ``N_kv`` > 0 gives K and V
-    that many tokens per head (Q, O, LSE keep ``N``); ``dtype`` "fp16" prepares the plan for half tensors."""
+    that many tokens per head (Q, O, LSE keep ``N``); ``dtype`` "fp16" prepares the plan for half tensors; ``batch`` > 1
+    with ``layout="nhd"`` makes the tensors ``[batch, N, heads / batch, d]`` (``heads`` counts all problems)."""
     import torch
     assert mask.is_cuda and mask.is_contiguous() and mask.dtype in (torch.uint8, torch.bool)
     h = ctypes.c_void_p()
-    opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv, LAYOUTS[layout], 0)
+    opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv, LAYOUTS[layout], batch)
     _check(lib().bsa_plan_create_ex(mask.data_ptr(), B_Q, B_KV, N, heads, d, ctypes.byref(opt), _stream_ptr(stream),
                                     ctypes.byref(h)), "bsa_plan_create")
     return Plan(h.value, layout)
@@ -250,8 +259,7 @@ def request(mask, B_Q: int, B_KV: int, N: int, heads: int, d: int, Q, K, V, O=No
     if O is None:
         O = torch.empty_like(Q)
     if LSE is None:
-        hn = Q.shape[:2] if layout == "hnd" else (Q.shape[1], Q.shape[0])
-        LSE = torch.empty(hn, dtype=torch.float32, device=Q.device)
+        LSE = torch.empty(_lse_shape(Q, layout), dtype=torch.float32, device=Q.device)
     h = ctypes.c_void_p()
     opt = Options(plan_id, DTYPES[dtype], max_workspace_bytes, N_kv, LAYOUTS[layout], 0)
     _check(lib().bsa_request_device(mask.data_ptr(), row_stride, B_Q, B_KV, N, heads, d, Q.data_ptr(), K.data_ptr(),
@@ -343,12 +351,12 @@ class PlanCache:
 
 
 def request_host(mask: np.ndarray, B_Q: int, B_KV: int, N: int, heads: int, d: int, Q, K, V, O, LSE,
-                 plan_id: int = -1, N_kv: int = 0, dtype: str = "bf16", layout: str = "hnd") -> Dict:
+                 plan_id: int = -1, N_kv: int = 0, dtype: str = "bf16", layout: str = "hnd", batch: int = 0) -> Dict:
     """``bsa_request_host``: all arguments are HOST buffers (torch CPU tensors or numpy arrays)."""
     def ptr(x):
         return x.data_ptr() if hasattr(x, "data_ptr") else x.ctypes.data
     inf = PlanInfo()
-    opt = Options(plan_id, DTYPES[dtype], 0, N_kv, LAYOUTS[layout], 0)
+    opt = Options(plan_id, DTYPES[dtype], 0, N_kv, LAYOUTS[layout], batch)
     _check(lib().bsa_request_host(ptr(mask), B_Q, B_KV, N, heads, d, ptr(Q), ptr(K), ptr(V), ptr(O), ptr(LSE),
                                   ctypes.byref(opt), ctypes.byref(inf)), "bsa_request_host")
     return inf.as_dict()

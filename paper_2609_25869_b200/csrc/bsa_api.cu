@@ -100,6 +100,10 @@ struct bsa_plan {
     // such forward): the plan's buffers go back to the pool in the create stream's order, so that stream waits for
     // this event first.  Forwards on one plan are stream-ordered among themselves, so the latest record covers all.
     std::atomic<cudaEvent_t> last_use;
+    // Batched token-major request (options->batch > 1 with BSA_LAYOUT_NHD): the plan is a list of per-batch-element
+    // plans (each an ordinary token-major request over heads / batch heads) and owns nothing else on the device.
+    bsa_plan** kids;
+    int nkids;
 };
 
 // ---- plan cache (warm path of Section 5.2: a prepared plan is reused while the mask stays the same) ----
@@ -135,8 +139,14 @@ static int64_t request_n_kv(const bsa_options_t* options, int64_t N) {
     return (options && options->N_kv > 0) ? options->N_kv : N;
 }
 
+static bool release_plan(bsa_plan* p);
 static void free_plan(bsa_plan* p) {
     if (!p) return;
+    if (p->kids) {
+        for (int b = 0; b < p->nkids; ++b)
+            if (p->kids[b]) release_plan(p->kids[b]);
+        delete[] p->kids;
+    }
     if (p->ready) cudaEventDestroy(p->ready);
     if (cudaEvent_t lu = p->last_use.load(std::memory_order_acquire)) {
         // a forward on another stream may still be reading the arenas and the workspace
@@ -179,6 +189,46 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
     if (dtype != BSA_DTYPE_BF16 && dtype != BSA_DTYPE_FP16) return BSA_ERR_UNSUPPORTED;
     const int layout = options ? options->layout : BSA_LAYOUT_HND;
     if (layout != BSA_LAYOUT_HND && layout != BSA_LAYOUT_NHD) return BSA_ERR_UNSUPPORTED;
+    const int batch = (options && options->batch > 1) ? options->batch : 1;
+    if (options && options->batch < 0) return BSA_ERR_INVALID_ARG;
+    if (batch > 1 && heads % batch != 0) return BSA_ERR_INVALID_ARG;
+    if (batch > 1 && layout == BSA_LAYOUT_NHD) {
+        // [batch][N][heads / batch][d] tensors: one ordinary token-major plan per batch element (in the head-major
+        // layout the batch folds into `heads` exactly and nothing has to be done)
+        if (cache) return BSA_ERR_UNSUPPORTED;
+        *out_plan = nullptr;
+        bsa_plan* parent = new (std::nothrow) bsa_plan();
+        if (!parent) return BSA_ERR_OOM;
+        memset(static_cast<void*>(parent), 0, sizeof *parent);
+        parent->refs.store(1, std::memory_order_relaxed);
+        parent->last_use.store(nullptr, std::memory_order_relaxed);
+        parent->stream = reinterpret_cast<cudaStream_t>(stream_v);
+        parent->d = d;
+        parent->dtype = dtype;
+        parent->layout = layout;
+        parent->kids = new (std::nothrow) bsa_plan*[batch]();
+        if (!parent->kids) { delete parent; return BSA_ERR_OOM; }
+        parent->nkids = batch;
+        const int hb = heads / batch;
+        const int64_t nQb64 = (N + B_Q - 1) / B_Q, nKb64 = (N_kv + B_KV - 1) / B_KV;
+        const int64_t mask_step = packed_stride > 0 ? (int64_t)hb * nQb64 * packed_stride : (int64_t)hb * nQb64 * nKb64;
+        bsa_options_t kid_opt = *options;
+        kid_opt.batch = 0;
+        for (int b = 0; b < batch; ++b) {
+            bsa_status_t st = create_impl(mask_dev + (size_t)b * mask_step, packed_stride, B_Q, B_KV, N, hb, d, &kid_opt, stream_v,
+                                          &parent->kids[b]);
+            if (st != BSA_OK) {
+                free_plan(parent);
+                return st;
+            }
+        }
+        MapGeom& pg = parent->g;  // enough of the geometry for bsa_forward's pointer steps and bsa_plan_get_info
+        pg = parent->kids[0]->g;
+        pg.H = heads;
+        parent->desc = parent->kids[0]->desc;
+        *out_plan = parent;
+        return BSA_OK;
+    }
     if (packed_stride > 0) {
         const int64_t nKb64 = (N_kv + B_KV - 1) / B_KV;
         if (packed_stride % 4 != 0 || packed_stride * 8 < nKb64 || (reinterpret_cast<uintptr_t>(mask_dev) & 3u))
@@ -594,7 +644,7 @@ static void fill_forward_args(const bsa_plan_t* p, const void* Q, const void* K,
 
 extern "C" bsa_status_t bsa_debug_merge_only(const bsa_plan_t* p, void* O, float* LSE, void* stream_v) {
     if (!p || !O || !LSE) return BSA_ERR_INVALID_ARG;
-    if (p->desc.split_pmax <= 1) return BSA_ERR_UNSUPPORTED;
+    if (p->kids || p->desc.split_pmax <= 1) return BSA_ERR_UNSUPPORTED;
     ForwardArgs a;
     fill_forward_args(p, nullptr, nullptr, nullptr, O, LSE, a);
     cudaError_t e = launch_merge(a, reinterpret_cast<cudaStream_t>(stream_v));
@@ -612,6 +662,17 @@ extern "C" bsa_status_t bsa_forward(const bsa_plan_t* p, const void* Q, const vo
          reinterpret_cast<uintptr_t>(O)) & 15)
         return BSA_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(LSE) & 3) return BSA_ERR_INVALID_ARG;
+    if (p->kids) {  // batched token-major request: element b's tensors start b * N * (heads / batch) * d elements further
+        const int hb = p->g.H / p->nkids;
+        const size_t q_step = (size_t)p->g.N * hb * p->d * 2, kv_step = (size_t)p->g.N_kv * hb * p->d * 2;
+        for (int b = 0; b < p->nkids; ++b) {
+            bsa_status_t st = bsa_forward(p->kids[b], static_cast<const uint8_t*>(Q) + b * q_step,
+                                          static_cast<const uint8_t*>(K) + b * kv_step, static_cast<const uint8_t*>(V) + b * kv_step,
+                                          static_cast<uint8_t*>(O) + b * q_step, LSE + (size_t)b * hb * p->g.N, stream_v);
+            if (st != BSA_OK) return st;
+        }
+        return BSA_OK;
+    }
     ForwardArgs a;
     fill_forward_args(p, Q, K, V, O, LSE, a);
     const char* detail = "launch";
@@ -684,8 +745,44 @@ extern "C" bsa_status_t bsa_plan_destroy(bsa_plan_t* p) {
     return BSA_OK;
 }
 
+// counts and times of `info` added to `tot` (the request's info over several sub-plans)
+static void add_info(bsa_plan_info_t& tot, const bsa_plan_info_t& info) {
+    tot.heads += info.heads;
+    tot.nnz_blocks += info.nnz_blocks;
+    tot.blocks_in_runs += info.blocks_in_runs;
+    if (info.max_row_nnz > tot.max_row_nnz) tot.max_row_nnz = info.max_row_nnz;
+    tot.ntiles += info.ntiles;
+    tot.nitems += info.nitems;
+    tot.nsplit_rows += info.nsplit_rows;
+    tot.workspace_bytes += info.workspace_bytes;
+    tot.covered_pairs += info.covered_pairs;
+    tot.us_mask_state += info.us_mask_state;
+    tot.us_stats_sync += info.us_stats_sync;
+    tot.us_lookup += info.us_lookup;
+    tot.us_launch_prep += info.us_launch_prep;
+    tot.us_total += info.us_total;
+    tot.device_status |= info.device_status;
+}
+static void finish_info(bsa_plan_info_t& tot) {
+    const double rows = (double)tot.heads * (double)tot.nQb, nnz = (double)tot.nnz_blocks;
+    tot.density = rows > 0 ? nnz / (rows * (double)tot.nKb) : 0.0;
+    tot.run_coverage = nnz > 0 ? (double)tot.blocks_in_runs / nnz : 0.0;
+    tot.skew = nnz > 0 ? (double)tot.max_row_nnz / (nnz / rows) : 0.0;
+}
+
 extern "C" bsa_status_t bsa_plan_get_info(const bsa_plan_t* p, bsa_plan_info_t* info) {
     if (!p || !info) return BSA_ERR_INVALID_ARG;
+    if (p->kids) {  // statistics of the whole mask, sums over the batch elements, the first element's plan
+        for (int b = 0; b < p->nkids; ++b) {
+            bsa_plan_info_t one;
+            bsa_status_t st = bsa_plan_get_info(p->kids[b], &one);
+            if (st != BSA_OK) return st;
+            if (b == 0) *info = one;
+            else add_info(*info, one);
+        }
+        finish_info(*info);
+        return BSA_OK;
+    }
     cudaError_t e = cudaDeviceSynchronize();
     PlanCountersDev c;
     if (e == cudaSuccess) e = cudaMemcpy(&c, p->counters, sizeof c, cudaMemcpyDeviceToHost);
@@ -728,6 +825,7 @@ extern "C" bsa_status_t bsa_plan_get_info(const bsa_plan_t* p, bsa_plan_info_t* 
 
 extern "C" bsa_status_t bsa_plan_export_csr(const bsa_plan_t* p, int32_t* row_ptr_host, int32_t* col_idx_host) {
     if (!p) return BSA_ERR_INVALID_ARG;
+    if (p->kids) return BSA_ERR_UNSUPPORTED;  // ask the per-element plans of a batched token-major request
     cudaError_t e = cudaDeviceSynchronize();
     const size_t nrows = (size_t)p->g.H * p->g.nQb;
     if (e == cudaSuccess && row_ptr_host)
@@ -745,6 +843,7 @@ extern "C" bsa_status_t bsa_plan_export_tiles(const bsa_plan_t* p, int head, int
                                               int32_t* tile_col_host, uint64_t* tile_member_host, int64_t cap,
                                               int64_t* ntiles_out) {
     if (!p || head < 0 || head >= p->g.H || !ntiles_out) return BSA_ERR_INVALID_ARG;
+    if (p->kids) return BSA_ERR_UNSUPPORTED;
     cudaError_t e = cudaDeviceSynchronize();
     const int nQt = p->g.nQt;
     int32_t* tb = new (std::nothrow) int32_t[2 * (size_t)nQt];
@@ -788,6 +887,7 @@ extern "C" bsa_status_t bsa_plan_export_tiles(const bsa_plan_t* p, int head, int
 extern "C" bsa_status_t bsa_plan_export_items(const bsa_plan_t* p, int32_t* items_host, int64_t cap,
                                               int64_t* nitems_out) {
     if (!p || !nitems_out) return BSA_ERR_INVALID_ARG;
+    if (p->kids) return BSA_ERR_UNSUPPORTED;
     cudaError_t e = cudaDeviceSynchronize();
     PlanCountersDev c;
     if (e == cudaSuccess) e = cudaMemcpy(&c, p->counters, sizeof c, cudaMemcpyDeviceToHost);
@@ -904,28 +1004,9 @@ extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int 
                 tot = info;
                 continue;
             }
-            tot.heads += info.heads;
-            tot.nnz_blocks += info.nnz_blocks;
-            tot.blocks_in_runs += info.blocks_in_runs;
-            if (info.max_row_nnz > tot.max_row_nnz) tot.max_row_nnz = info.max_row_nnz;
-            tot.ntiles += info.ntiles;
-            tot.nitems += info.nitems;
-            tot.nsplit_rows += info.nsplit_rows;
-            tot.workspace_bytes += info.workspace_bytes;
-            tot.covered_pairs += info.covered_pairs;
-            tot.us_mask_state += info.us_mask_state;
-            tot.us_stats_sync += info.us_stats_sync;
-            tot.us_lookup += info.us_lookup;
-            tot.us_launch_prep += info.us_launch_prep;
-            tot.us_total += info.us_total;
-            tot.device_status |= info.device_status;
+            add_info(tot, info);
         }
-        if (G > 1) {
-            const double rows = (double)tot.heads * (double)tot.nQb, nnz = (double)tot.nnz_blocks;
-            tot.density = rows > 0 ? nnz / (rows * (double)tot.nKb) : 0.0;
-            tot.run_coverage = nnz > 0 ? (double)tot.blocks_in_runs / nnz : 0.0;
-            tot.skew = nnz > 0 ? (double)tot.max_row_nnz / (nnz / rows) : 0.0;
-        }
+        if (G > 1) finish_info(tot);
         if (info_out) *info_out = tot;
     }
     for (int g = 0; g < G; ++g)

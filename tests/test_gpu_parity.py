@@ -502,6 +502,47 @@ def test_token_major_layout_gives_the_same_output(B_Q, B_KV, N, N_kv, d, dtype):
                 Hh.compare_with_oracle(req, Ob.permute(1, 0, 2).contiguous(), Lb, qkv_cpu)
 
 
+@pytest.mark.parametrize("B_Q,B_KV,N,N_kv,d,dtype,plan_id", [(64, 64, 1000, 0, 64, "bf16", -1), (128, 128, 1500, 2100, 128, "bf16", 22),
+                                                              (32, 64, 900, 0, 128, "fp16", -1), (16, 64, 700, 0, 64, "bf16", 34)])
+def test_batched_token_major_request(B_Q, B_KV, N, N_kv, d, dtype, plan_id):
+    """Explicit batch (a request dimension): tensors stored [batch, N, heads, d] with `heads` counting batch x heads
+    problems.  The output equals, problem by problem, the head-major run of the folded request (bit for bit) and the
+    oracle; the info sums the batch elements; exports and the plan cache refuse such a plan; with the head-major
+    layout the batch option changes nothing."""
+    Bt, Hb = 3, 2
+    H = Bt * Hb
+    M = I.random_mask(97, H, I.cdiv(N, B_Q), I.cdiv(N_kv or N, B_KV), 0.3, empty_rows=0.1)
+    req = I.Request("batched", H, N, d, B_Q, B_KV, M, qkv_seed=41, N_kv=N_kv, dtype=dtype)
+    mask, q, k, v, qkv_cpu = Hh.to_dev(req)
+    args = (B_Q, B_KV, N, H, d)
+    kw = dict(plan_id=plan_id, N_kv=N_kv, dtype=dtype)
+
+    def to_bnhd(t):   # [B*Hb, n, d] -> [B, n, Hb, d]
+        return t.view(Bt, Hb, t.shape[1], d).permute(0, 2, 1, 3).contiguous()
+
+    with bsa.plan_create(mask, *args, **kw) as plain, bsa.plan_create(mask, *args, layout="nhd", batch=Bt, **kw) as batched, \
+            bsa.plan_create(mask, *args, batch=Bt, **kw) as folded:
+        O, L = plain.forward(q, k, v)
+        Ob, Lb = batched.forward(to_bnhd(q), to_bnhd(k), to_bnhd(v))
+        Of, Lf = folded.forward(q, k, v)
+        torch.cuda.synchronize()
+        assert Ob.shape == (Bt, N, Hb, d) and Lb.shape == (H, N)
+        if plan_id >= 0:   # the same catalog plan everywhere: the same bits (a lookup may choose per batch element)
+            assert torch.equal(Ob.permute(0, 2, 1, 3).reshape(H, N, d), O) and torch.equal(Lb, L)
+        assert torch.equal(Of, O) and torch.equal(Lf, L)
+        Hh.compare_with_oracle(req, Ob.permute(0, 2, 1, 3).reshape(H, N, d).contiguous(), Lb, qkv_cpu, guards=False)
+        ia, ib = plain.info(), batched.info()
+        for key in ("heads", "nnz_blocks", "blocks_in_runs", "max_row_nnz") + (("covered_pairs",) if plan_id >= 0 else ()):
+            assert ia[key] == ib[key], key
+        assert abs(ia["density"] - ib["density"]) < 1e-12 and ib["device_status"] == 0 and ib["layout"] == 1
+        with pytest.raises(bsa.BsaError) as e:
+            batched.export_csr()
+        assert e.value.status == 2
+    with pytest.raises(bsa.BsaError) as e:       # heads must be a multiple of the batch size
+        bsa.plan_create(mask, *args, layout="nhd", batch=4, **kw)
+    assert e.value.status == 1
+
+
 def test_token_major_layout_from_host_buffers_and_cache_key():
     req = I.config_tiny()
     mask, q, k, v, qkv_cpu = Hh.to_dev(req)
