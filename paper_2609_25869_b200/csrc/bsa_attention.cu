@@ -28,10 +28,12 @@ using namespace ptx;
 
 // Optional timeline tracing (compile with -DBSA_TRACE): CTA 0 records clock64() at barrier events of the
 // single-tile kernel, per role, into a device buffer that bsa_debug_trace_copy() reads back.
-#ifdef BSA_TRACE
+#if defined(BSA_TRACE) || defined(BSA_PHASES)
 __device__ long long g_trace[12][4096];  // producer, Q K^T (or single) issuer, softmax warps 0-7, P V issuer (role 6 in the 7-warp kernel)
 __device__ long long g_trace_aux[12][4];  // last tile's stamps inside softmax_tile, per warp
 __device__ long long g_cta_times[2][4096];  // %globaltimer at entry and exit of every CTA of the ping-pong kernel
+#endif
+#ifdef BSA_TRACE
 #define BSA_TRACE_DECL(n) int n = 0
 #define BSA_TRACE_POINT(role, n, tag)                                              \
     do {                                                                           \
@@ -40,6 +42,18 @@ __device__ long long g_cta_times[2][4096];  // %globaltimer at entry and exit of
 #else
 #define BSA_TRACE_DECL(n)
 #define BSA_TRACE_POINT(role, n, tag)
+#endif
+
+// Optional phase accounting (compile with -DBSA_PHASES): every softmax warp of the ping-pong kernel adds up the clocks it
+// spends between fixed points of its tile loop; CTA 1 writes the sums out at its end (bsa_debug_trace_copy, roles 2-9).
+#ifdef BSA_PHASES
+#define BSA_PH_DECL uint32_t ph_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, ph_n = 0, ph_t = (uint32_t)clock()
+#define BSA_PH(k) do { const uint32_t now_ = (uint32_t)clock(); ph_acc[k] += now_ - ph_t; ph_t = now_; } while (0)
+#define BSA_STAMP(role, tile, k) do { if (blockIdx.x == 1 && (tile) >= 40 && (tile) < 240) g_trace[role][16 + 4 * ((tile) - 40) + (k)] = clock64(); } while (0)
+#else
+#define BSA_PH_DECL
+#define BSA_PH(k)
+#define BSA_STAMP(role, tile, k)
 #endif
 
 // Test hook (bsa_debug_withhold_arrival): while non-zero, the V producer of the ping-pong kernel leaves out the copy
@@ -1652,6 +1666,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             uint32_t itq = 0, g = 0;
             bool ok = true;
             BSA_TRACE_DECL(tn);
+            BSA_PH_DECL;
             int n_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items).ntiles;
             for (int kr = 0; kr < n_rounds && ok; ++kr) {
                 const int n = n_next;
@@ -1671,6 +1686,8 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     else
                         ok = mbar_wait(smem_u32(&bars.k_full[stage]), ph, abortp);
                     if (!ok) break;
+                    BSA_PH(0);
+                    BSA_STAMP(0, gs, 0);
                     BSA_TRACE_POINT(1, tn, 6);
                     tc_fence_after();
                     const uint32_t d_s = tmem + (sb ? kColS1 : kColS0);
@@ -1682,12 +1699,20 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     }
                     mma_commit(smem_u32(&bars.k_empty[stage]));
                     mma_commit(smem_u32(&bars.s_full[sb]));
+                    BSA_PH(1);
+                    BSA_STAMP(0, gs, 1);
+#ifdef BSA_PHASES
+                    ++ph_n;
+#endif
                     BSA_TRACE_POINT(1, tn, 2);
                     if (j == n - 1) mma_commit(smem_u32(&bars.q_empty[qb]));
                 }
                 g += n;
                 ++itq;
             }
+#ifdef BSA_PHASES
+            if (blockIdx.x == 1) { g_trace[0][0] = ph_acc[0]; g_trace[0][1] = ph_acc[1]; g_trace[0][8] = ph_n; }
+#endif
         } else if (warp == 10 && lane == 0) {
             // =========================== P V issuer ===========================
             constexpr uint32_t idesc_pv = make_idesc_f32(kTQ, D, 0, 1, F16);
@@ -1696,6 +1721,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
             uint32_t itq = 0, g = 0;
             bool ok = true;
             BSA_TRACE_DECL(tn);
+            BSA_PH_DECL;
             int n_next = load_item(p.items, cta_item_index(0, blockIdx.x, gridDim.x), n_items).ntiles;
             for (int kr = 0; kr < n_rounds && ok; ++kr) {
                 const int n = n_next;
@@ -1713,6 +1739,8 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     }
                     ok = mbar_wait2(smem_u32(&bars.v_full[stage]), ph, smem_u32(&bars.p_ready[sb]), (gp >> 1) & 1, abortp);
                     if (!ok) break;
+                    BSA_PH(0);
+                    BSA_STAMP(1, gp, 0);
                     BSA_TRACE_POINT(10, tn, 3);
 
                     tc_fence_after();
@@ -1725,11 +1753,19 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     mma_commit(smem_u32(&bars.v_empty[stage]));
                     mma_commit(smem_u32(&bars.pv_done[sb]));
                     if (j == n - 1) mma_commit(smem_u32(&bars.o_full));
+                    BSA_PH(1);
+                    BSA_STAMP(1, gp, 1);
+#ifdef BSA_PHASES
+                    ++ph_n;
+#endif
                     BSA_TRACE_POINT(10, tn, 5);
                 }
                 g += n;
                 ++itq;
             }
+#ifdef BSA_PHASES
+            if (blockIdx.x == 1) { g_trace[1][0] = ph_acc[0]; g_trace[1][1] = ph_acc[1]; g_trace[1][8] = ph_n; }
+#endif
         }
     } else {
         // =========================== softmax warpgroup x ===========================
@@ -1746,6 +1782,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
         BSA_TRACE_DECL(tn);
         const float c2 = p.scale_log2;
         const unsigned long long sub_mask = (p.sK >= 64) ? ~0ull : ((1ull << p.sK) - 1ull);
+        BSA_PH_DECL;
         // The reference after global tile t (taken by the other warpgroup), given a word read earlier from its slot:
         // if that word already carries the publish's tag it is used, else the slot is polled (bounded).
         auto take_reference = [&](uint32_t t, uint32_t word, float& m_out) -> bool {
@@ -1815,14 +1852,18 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 const uint32_t row_bits = (uint32_t)((member >> ((tw >> p.lgBQ) * p.sK)) & sub_mask);
                 const int n_valid = p.Nkv - kv0;
                 if (lane == 0 && j == j0) BSA_TRACE_POINT(2 + warp, tn, 35);
+                BSA_PH(7);
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), (gs >> 1) & 1, abortp));
                 if (!ok) break;
+                BSA_PH(0);
+                if (lane == 0) BSA_STAMP(2 + warp, gs, 0);
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 10);
                 tc_fence_after();
                 uint32_t r[TK];
 #pragma unroll
                 for (int c = 0; c < TK / 32; ++c) tmem_ld32(t_s + c * 32, &r[c * 32]);
                 tc_wait_ld();
+                BSA_PH(1);
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.s_free[x]));  // S[x] is in registers: the next Q K^T into it may start
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 11);
@@ -1861,6 +1902,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     if (!ok) break;
                     if (j > 0) m_prev = m_taken;  // the previous tile belongs to this item
                 }
+#ifdef BSA_PHASES
+                asm volatile("" ::"f"(mx2), "f"(m_prev));
+#endif
+                BSA_PH(2);
 #ifdef BSA_TRACE
                 if (lane == 0 && m_prev != 12345.f) BSA_TRACE_POINT(2 + warp, tn, 18);
 #endif
@@ -1880,6 +1925,7 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 }
                 // publish: the next tile's warpgroup may take its decision
                 *reinterpret_cast<volatile uint32_t*>(&mref[x][tw]) = __float_as_uint(m_know) | (((gs >> 1) + 1) & 3u);
+                BSA_PH(3);
                 const float neg_m = (m_know == -INFINITY) ? 0.f : -m_know;
                 const uint64_t c22 = pack_f32x2(c2, c2), nm2 = pack_f32x2(neg_m, neg_m);
                 uint64_t sum01 = pack_f32x2(0.f, 0.f), sum23 = sum01;
@@ -1908,12 +1954,19 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 unpack_f32x2(sum01, s0, s1);
                 unpack_f32x2(sum23, s2, s3);
                 l += (s0 + s1) + (s2 + s3);
+#ifdef BSA_PHASES
+                asm volatile("" ::"f"(l), "r"(r[TK / 2 - 1]));
+#endif
+                BSA_PH(4);
+                if (lane == 0) BSA_STAMP(2 + warp, gs, 1);
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 14);
                 if (!kStoreInLoop) {
                     if (gs >= 2) {
                         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.pv_done[x]), ((gs >> 1) - 1) & 1, abortp));
                         if (!ok) break;
                     }
+                    BSA_PH(5);
+                    if (lane == 0) BSA_STAMP(2 + warp, gs, 2);
 #pragma unroll
                     for (int c = 0; c < TK / 32; ++c) tmem_st16(t_p + c * 16, &r[c * 16]);
                 }
@@ -1936,6 +1989,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.p_ready[x]));
+                BSA_PH(6);
+                if (lane == 0) BSA_STAMP(2 + warp, gs, 3);
+#ifdef BSA_PHASES
+                ++ph_n;
+#endif
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 16);
             }
             if (!ok) break;
@@ -1960,7 +2018,14 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 if (lane == 0) BSA_TRACE_POINT(2 + warp, tn, 30);
             }
             g += n;
+            BSA_PH(7);  // item boundary: sums handed over, next item's first tile not yet waited for
         }
+#ifdef BSA_PHASES
+        if (blockIdx.x == 1 && lane == 0) {
+            for (int k = 0; k < 8; ++k) g_trace[2 + warp][k] = ph_acc[k];
+            g_trace[2 + warp][8] = ph_n;
+        }
+#endif
     }
 
     tc_fence_before();
@@ -2215,7 +2280,7 @@ int attention_smem_bytes(int d, int T_KV, int stages, int kernel) {
     return need;
 }
 
-#ifdef BSA_TRACE
+#if defined(BSA_TRACE) || defined(BSA_PHASES)
 extern "C" __attribute__((visibility("default"))) int bsa_debug_trace_copy(long long* host, int role) {
     if (role >= 100)  // 100 / 101: CTA entry / exit times
         return (int)cudaMemcpyFromSymbol(host, g_cta_times, sizeof(long long) * 4096, sizeof(long long) * 4096 * (role - 100));
