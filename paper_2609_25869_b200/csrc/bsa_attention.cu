@@ -1903,7 +1903,10 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                     if (j > 0) m_prev = m_taken;  // the previous tile belongs to this item
                 }
 #ifdef BSA_PHASES
-                asm volatile("" ::"f"(mx2), "f"(m_prev));
+                {
+                    float f0_ = mx2, f1_ = m_prev;  // real instructions that read the values: the clock is read after them
+                    asm volatile("mov.b32 %0, %0;\n\tmov.b32 %1, %1;" : "+f"(f0_), "+f"(f1_));
+                }
 #endif
                 BSA_PH(2);
 #ifdef BSA_TRACE
@@ -1955,7 +1958,11 @@ bsa_attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_co
                 unpack_f32x2(sum23, s2, s3);
                 l += (s0 + s1) + (s2 + s3);
 #ifdef BSA_PHASES
-                asm volatile("" ::"f"(l), "r"(r[TK / 2 - 1]));
+                {
+                    float f0_ = l;
+                    uint32_t u0_ = r[TK / 2 - 1];
+                    asm volatile("mov.b32 %0, %0;\n\tmov.b32 %1, %1;" : "+f"(f0_), "+r"(u0_));
+                }
 #endif
                 BSA_PH(4);
                 if (lane == 0) BSA_STAMP(2 + warp, gs, 1);
