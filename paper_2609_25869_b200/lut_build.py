@@ -227,16 +227,19 @@ def corpus_specs(scale: str = "full"):
         add("mid", "mid0", seed=1010)
         add("stress_b", "sb0", seed=1030, H=4, N=8192)
         return specs
+    # Every request key gets at least 64 cases, so that a tree with the paper's 32 cases per leaf can split it.
     # (64,64) d=64: Tiny's key
     n = 0
     for N in (1024, 2048, 4096, 8192):
         for H, p in ((2, 0.25), (4, 0.1), (8, 0.4), (16, 0.05)):
-            add("tiny", f"tiny{n // 2}", seed=1000 + n, H=H, N=N, p=p)
-            n += 1
+            for rep in range(4):
+                add("tiny", f"tiny{n // 2}", seed=1000 + n, H=H, N=N, p=p * (1.0 + 0.15 * rep))
+                n += 1
     # (128,128) d=128: Mid and Hunyuan shapes, and the sweep's (128,128) requests
     n = 0
     for H in (1, 2, 4, 8, 16, 24):
-        for extra, win in ((0.02, (1, 1, 1)), (0.0, (1, 1, 1)), (0.1, (1, 1, 1)), (0.02, (2, 1, 1)), (0.3, (0, 0, 0))):
+        for extra, win in ((0.02, (1, 1, 1)), (0.0, (1, 1, 1)), (0.1, (1, 1, 1)), (0.02, (2, 1, 1)), (0.3, (0, 0, 0)),
+                           (0.05, (1, 1, 1)), (0.01, (1, 2, 2)), (0.2, (1, 0, 0)), (0.5, (0, 0, 0)), (0.0, (2, 2, 2))):
             add("mid", f"mid{n // 2}", seed=1100 + n, H=H, extra=extra, win=win)
             n += 1
     n = 0
@@ -247,17 +250,19 @@ def corpus_specs(scale: str = "full"):
     # (16,64) and (256,256) d=64: the two stress keys
     n = 0
     for N, H in ((8192, 16), (16384, 8), (32768, 16), (32768, 4)):
-        for dens in (0.05, 0.1, 0.15, 0.3):
-            add("stress_a", f"sa{n // 2}", seed=1300 + n, H=H, N=N, density=dens)
-            add("stress_b", f"sb{n // 2}", seed=1400 + n, H=H, N=N, p=min(0.6, dens * 1.4))
-            n += 1
+        for dens in (0.03, 0.05, 0.07, 0.1, 0.15, 0.2, 0.3, 0.4):
+            for rep in range(2):
+                add("stress_a", f"sa{n // 2}", seed=1300 + n, H=H, N=N, density=dens)
+                add("stress_b", f"sb{n // 2}", seed=1400 + n, H=H, N=N, p=min(0.6, dens * 1.4))
+                n += 1
     # the sweep's five geometries (d=128, N=75600), densities on and between the sweep's targets
     n = 0
-    for H in (6, 12, 24):  # head count outermost: the cases of one shape follow each other and share their tensors
+    for H in (3, 6, 12, 24):  # head count outermost: the cases of one shape follow each other and share their tensors
         for B in ((32, 32), (64, 128), (128, 64), (128, 128), (256, 256)):
-            for rho in (0.03, 0.05, 0.1, 0.17, 0.3, 0.45, 0.6):
-                add("sweep", f"sw{B[0]}x{B[1]}@{rho}", r=1000 + n, H=H, B=B, rho=rho)
-                n += 1
+            for rho in (0.03, 0.05, 0.08, 0.1, 0.17, 0.3, 0.45, 0.6):
+                for rep in range(2):
+                    add("sweep", f"sw{B[0]}x{B[1]}@{rho}#{rep}", r=1000 + n, H=H, B=B, rho=rho)
+                    n += 1
     return specs
 
 
@@ -422,16 +427,74 @@ def profile(reqs, plans=None, reps: int = 5, warmup: int = 3, log=print, validat
     return cases, lat, bucket, base
 
 
+def leave_source_out(path: str, min_leaf: int = 32, max_depth: int = 4, log=print) -> Dict[str, dict]:
+    """Offline check of how the table generalises, from a latencies file written by ``--latencies``: every mask source
+    in turn is left out of the corpus, regimes and trees are compiled from the rest, and each left-out case is looked
+    up in them in three ways (regimes then trees then base plan, as the runtime does; trees alone; regimes alone).
+    Returns per way the geometric-mean regret, the share within 3 % and the share of cases that found a regime or leaf.
+    Needs the library only for the fixed-edge bucket function and the base plans (no GPU)."""
+    import ctypes
+    import json
+    from . import bsa
+    with open(path) as f:
+        d = json.load(f)
+    cases = [(c, tuple(k)) for c, k in d["cases"]]
+    lat = {(c, int(pid)): t for c, pid, t in d["lat"]}
+    feats = {c: tuple(v) for c, v in d["features"].items()}
+    groups = d["groups"]
+    lib = bsa.lib()
+    lib.bsa_lut_buckets.argtypes = [ctypes.c_int64, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                    ctypes.POINTER(ctypes.c_int32)]
+    lib.bsa_lut_buckets.restype = None
+    bucket, base = {}, {}
+    for c, key in cases:
+        lg, heads, dens, skew, rc = feats[c]
+        out = (ctypes.c_int32 * 4)()
+        lib.bsa_lut_buckets(int(round(2.0 ** lg)), dens, skew, rc, out)
+        bucket[c] = (out[0], head_bucket(int(heads)), out[1], out[2], out[3])
+        base[key] = int(lib.bsa_base_plan(key[0], key[1], key[2]))
+    sources = sorted(set(groups.values()))
+    acc = {w: {"log": 0.0, "n": 0, "within": 0, "found": 0} for w in ("regime_tree_base", "tree_base", "regime_base")}
+    for src in sources:
+        held = [(c, k) for c, k in cases if groups[c] == src]
+        keys = {k for _, k in held}  # only the tables of the left-out cases' own request keys matter
+        train = [(c, k) for c, k in cases if groups[c] != src and k in keys]
+        table = compile_table(train, lat, base, lambda cid: bucket[cid])
+        trees = compile_trees(train, feats, groups, lat, base, min_leaf=min_leaf, max_depth=max_depth)
+        for c, key in held:
+            reg = table.get((key, bucket[c]))
+            leaf = tree_leaf(trees[key], feats[c])["ranked"] if key in trees else None
+            for way, ranked in (("regime_tree_base", reg or leaf), ("tree_base", leaf), ("regime_base", reg)):
+                a = acc[way]
+                lr = case_log_regret(c, ranked if ranked else [base[key]], lat)
+                a["log"] += lr
+                a["n"] += 1
+                a["within"] += 1 if lr <= math.log(1.03) else 0
+                a["found"] += 1 if ranked else 0
+    res = {}
+    for way, a in acc.items():
+        res[way] = {"cases": a["n"], "regret_gm": math.exp(a["log"] / max(a["n"], 1)),
+                    "within_3pct": a["within"] / max(a["n"], 1), "found": a["found"] / max(a["n"], 1)}
+        if log:
+            log(f"{way}: {res[way]}")
+    return res
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--leave-source-out", default="", metavar="LATENCIES.json",
+                    help="no profiling: leave every mask source out of the recorded corpus in turn and report the regret "
+                    "of the left-out cases (host only)")
     ap.add_argument("--out", default=DEFAULT_OUT)
     ap.add_argument("--scale", default="full", choices=["full", "quick"])
-    ap.add_argument("--min-leaf", type=int, default=6, help="fewest cases a tree leaf may hold (the paper, with a corpus "
-                    "of tens of thousands of cases, uses 32)")
+    ap.add_argument("--min-leaf", type=int, default=32, help="fewest cases a tree leaf may hold (Section 5.1: 32)")
     ap.add_argument("--max-depth", type=int, default=4)
     ap.add_argument("--no-trees", action="store_true", help="fixed-edge regimes only")
     ap.add_argument("--latencies", default="", help="also write the measured latencies as JSON (for the regret report)")
     args = ap.parse_args(argv)
+    if args.leave_source_out:
+        leave_source_out(args.leave_source_out, args.min_leaf, args.max_depth)
+        return 0
     specs = corpus_specs(args.scale)
     # masks are generated by worker processes (forked before CUDA is touched) while earlier cases are profiled
     import multiprocessing as mp
