@@ -37,6 +37,21 @@ O_TOL, O_MEAN_TOL, LSE_TOL = 2e-2, 2e-3, 1e-3  # validation gate (the contract t
 # --------------------------------------------------------------------------------------------
 # Algorithm 1, "Regimes and rankings" (pure host logic; unit-tested on the CPU)
 # --------------------------------------------------------------------------------------------
+_INDEX: Dict[int, Tuple[int, Dict]] = {}
+
+
+def _by_case(lat: Dict[Tuple[Hashable, int], float]) -> Dict[Hashable, Dict[int, float]]:
+    """``lat`` regrouped as {case id: {plan id: latency}}; built once per dictionary (and again if it has grown)."""
+    hit = _INDEX.get(id(lat))
+    if hit is None or hit[0] != len(lat):
+        idx: Dict[Hashable, Dict[int, float]] = {}
+        for (c, p), t in lat.items():
+            idx.setdefault(c, {})[p] = t
+        _INDEX.clear()  # one table is compiled at a time
+        _INDEX[id(lat)] = hit = (len(lat), idx)
+    return hit[1]
+
+
 def compile_table(cases: Sequence[Tuple[Hashable, Hashable]], latencies: Dict[Tuple[Hashable, int], float],
                   base_plan: Dict[Hashable, int], bucket_of: Callable[[Hashable], Hashable]) -> Dict:
     """``cases``: (case id, request key); ``latencies[(case id, plan id)]``: validated median latency
@@ -51,8 +66,9 @@ def compile_table(cases: Sequence[Tuple[Hashable, Hashable]], latencies: Dict[Tu
             buckets.setdefault(bucket_of(cid), []).append(cid)
         for b, cids in buckets.items():
             candidates = None
+            per_case = _by_case(latencies)
             for cid in cids:
-                have = {p for (c, p) in latencies if c == cid}
+                have = set(per_case.get(cid, ()))
                 candidates = have if candidates is None else candidates & have
             if not candidates:
                 continue
@@ -74,8 +90,8 @@ def case_features(N: int, heads: int, density: float, skew: float, run_coverage:
 
 
 def _case_best(cid, lat) -> float:
-    ts = [t for (c, _), t in lat.items() if c == cid]
-    return min(ts) if ts else float("nan")
+    ts = _by_case(lat).get(cid)
+    return min(ts.values()) if ts else float("nan")
 
 
 def _ranking_and_loss(cids, lat, base: int):
@@ -84,8 +100,9 @@ def _ranking_and_loss(cids, lat, base: int):
     head (a case the head has no latency for falls through the ranking like the runtime's ranked fallback; one that no
     ranked plan serves is charged its slowest measured plan)."""
     cand = None
+    per_case = _by_case(lat)
     for c in cids:
-        have = {p for (cc, p) in lat if cc == c}
+        have = set(per_case.get(c, ()))
         cand = have if cand is None else cand & have
     cand = cand or set()
     gm = {p: math.exp(sum(math.log(lat[(c, p)]) for c in cids) / len(cids)) for p in cand}
@@ -100,7 +117,7 @@ def case_log_regret(cid, ranked, lat) -> float:
     for p in ranked:
         if (cid, p) in lat:
             return math.log(lat[(cid, p)] / best)
-    return math.log(max(t for (c, _), t in lat.items() if c == cid) / best)
+    return math.log(max(_by_case(lat)[cid].values()) / best)
 
 
 def learn_tree(cids, feats, lat, base: int, min_leaf: int = 8, max_depth: int = 3):
@@ -170,13 +187,14 @@ def choose_depth(cids, feats, groups, lat, base: int, min_leaf: int = 8, depths=
 
 
 def compile_trees(cases, feats, groups, lat, base_plan, min_leaf: int = 8, max_depth: int = 4, folds: int = 4, log=None):
-    """One tree per request key that has at least ``2 * min_leaf`` cases; the others keep the fixed-edge regimes."""
+    """One tree per request key that has at least ``min_leaf`` cases (a single leaf, i.e. one ranking for the key, unless
+    it has the ``2 * min_leaf`` a split needs); the other keys keep the fixed-edge regimes alone."""
     by_key: Dict[Hashable, List[Hashable]] = {}
     for cid, key in cases:
         by_key.setdefault(key, []).append(cid)
     trees = {}
     for key, members in sorted(by_key.items()):
-        if len(members) < 2 * min_leaf:
+        if len(members) < min_leaf:
             continue
         depth, score = choose_depth(members, feats, groups, lat, base_plan[key], min_leaf, tuple(range(max_depth + 1)), folds)
         trees[key] = learn_tree(members, feats, lat, base_plan[key], min_leaf, depth)

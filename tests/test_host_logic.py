@@ -210,8 +210,10 @@ def test_decision_tree_regimes_hand_built_case(tmp_path):
     # with no split allowed the single leaf ranks by geometric mean over everything
     flat = LB.learn_tree([c for c, _ in cases], feats, lat, 22, min_leaf=4, max_depth=0)
     assert len(flat) == 1 and flat[0]["ranked"] == [3, 22, 22]
-    # too few cases for two leaves of min_leaf: no tree for the key
-    assert LB.compile_trees(cases[:6], feats, groups, lat, base, min_leaf=4) == {}
+    # too few cases for two leaves of min_leaf: a single leaf (one ranking for the key); fewer than one leaf's worth: no tree
+    single = LB.compile_trees(cases[:6], feats, groups, lat, base, min_leaf=4)
+    assert len(single[key]) == 1 and single[key][0]["cases"] == 6 and single[key][0]["ranked"][-1] == 22
+    assert LB.compile_trees(cases[:3], feats, groups, lat, base, min_leaf=4) == {}
     path = str(tmp_path / "tree.lut")
     LB.write_table(path, {}, int(bsa.lib().bsa_catalog_hash()), "test", trees=trees)
     bsa.lut_load(path)
