@@ -924,16 +924,33 @@ extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int 
     const size_t o_m = 0, o_q = align_up(mbytes), o_k = o_q + align_up(tbytes), o_v = o_k + align_up(kbytes),
                  o_o = o_v + align_up(kbytes), o_l = o_o + align_up(tbytes), total = o_l + align_up(lbytes);
     // Heads are independent, and with the head-major layout a range of heads is a contiguous slice of every tensor:
-    // the request is cut into up to 8 groups of heads (at least 32 MB of Q, K, V each: with smaller groups the
+    // the request is cut into up to 8 groups of heads (more than 32 MB of Q, K, V each: with smaller groups the
     // copies themselves got slower, 43 instead of 53 GB/s) and pipelined over three streams kept per host thread --
     // inputs of group g+1 travel (s2) while group g is planned and computed (s) and the output of group g-1 travels
     // back (s3; the link is full duplex).  What is left after the last input byte is one group's forward and its
     // output copy.  The token-major layout is not cut.
     const size_t head_in = ((size_t)N + 2 * (size_t)N_kv) * d * 2;
-    int hc = (int)(((size_t)32 << 20) / (head_in ? head_in : 1)) + 1;  // heads per group
+    const int hmin = (int)(((size_t)32 << 20) / (head_in ? head_in : 1)) + 1;  // fewest heads a group may have
+    int hc = hmin;                                                             // heads per group
     if (hc < (heads + 7) / 8) hc = (heads + 7) / 8;
     if (hc > heads || (options && options->layout == BSA_LAYOUT_NHD)) hc = heads;
     const int G = (heads + hc - 1) / hc;
+    // Group boundaries.  Where the smallest allowed group is well below the even share, the last two groups are made
+    // small (hmin and 2 hmin heads) and the others share the rest: the tail after the last input byte is then the
+    // forward and the output copy of hmin heads instead of hc (24 heads of the Hunyuan-shaped request: 4 4 4 3 3 3 2 1).
+    int hb[9];
+    for (int g = 0; g <= G; ++g) hb[g] = g * hc < heads ? g * hc : heads;
+    if (G >= 4 && 3 * hmin < hc + (heads - (G - 1) * hc)) {
+        const int rest = heads - 3 * hmin, ng = G - 2;
+        int at = 0;
+        for (int g = 0; g < ng; ++g) {
+            hb[g] = at;
+            at += rest / ng + (g < rest % ng ? 1 : 0);
+        }
+        hb[G - 2] = at;
+        hb[G - 1] = at + 2 * hmin;
+        hb[G] = heads;
+    }
     static thread_local cudaStream_t s = nullptr, s2 = nullptr, s3 = nullptr;
     static thread_local cudaEvent_t buf_ready = nullptr, in_ready[8] = {}, out_ready[8] = {};
     cudaError_t e = cudaSuccess;
@@ -958,7 +975,7 @@ extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int 
     if (e == cudaSuccess) e = cudaStreamWaitEvent(s3, buf_ready, 0);
     const size_t q_head = (size_t)N * d * 2, k_head = (size_t)N_kv * d * 2, l_head = (size_t)N * 4;
     for (int g = 0; g < G && e == cudaSuccess; ++g) {  // all input copies are queued first, in group order
-        const size_t h0 = (size_t)g * hc, nh = (size_t)((g + 1) * hc <= heads ? hc : heads - g * hc);
+        const size_t h0 = (size_t)hb[g], nh = (size_t)(hb[g + 1] - hb[g]);
         e = cudaMemcpyAsync(buf + o_q + h0 * q_head, static_cast<const uint8_t*>(Q_host) + h0 * q_head, nh * q_head,
                             cudaMemcpyHostToDevice, s2);
         if (e == cudaSuccess)
@@ -970,8 +987,8 @@ extern "C" bsa_status_t bsa_request_host(const uint8_t* mask_host, int B_Q, int 
         if (e == cudaSuccess) e = cudaEventRecord(in_ready[g], s2);
     }
     for (int g = 0; g < G && e == cudaSuccess && st == BSA_OK; ++g) {
-        const size_t h0 = (size_t)g * hc;
-        const int nh = (g + 1) * hc <= heads ? hc : heads - g * hc;
+        const size_t h0 = (size_t)hb[g];
+        const int nh = hb[g + 1] - hb[g];
         st = bsa_plan_create_ex(buf + o_m + h0 * nQb * nKb, B_Q, B_KV, N, nh, d, options, s, &plans[g]);
         if (st != BSA_OK) break;
         e = cudaStreamWaitEvent(s, in_ready[g], 0);

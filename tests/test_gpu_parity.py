@@ -293,6 +293,28 @@ def test_pipelined_request_from_pinned_host_buffers():
         assert abs(inf[key] - w[key]) < 1e-9, key
 
 
+def test_host_request_with_tapered_head_groups():
+    """With more than 32 MB of Q, K, V per head a group may be a single head, and bsa_request_host then tapers the
+    groups towards the end (12 heads: 3 2 2 2 2 1) so that little work is left after the last input byte.  Every head
+    lands in the right place: outputs against the oracle on sampled query blocks of every head, no row left unwritten,
+    and the aggregated counts equal those of one plan over the whole mask."""
+    req = I.config_tiny(seed=31, H=12, N=49152, d=128, B=128, p=0.01)   # 37.7 MB of Q, K, V per head
+    q, k, v = req.qkv()
+    qp, kp, vp = (t.pin_memory() for t in (q, k, v))
+    O = torch.empty_like(q).pin_memory()
+    LSE = torch.empty((req.H, req.N), dtype=torch.float32).pin_memory()
+    O.fill_(float("nan"))
+    LSE.fill_(float("nan"))
+    inf = bsa.request_host(torch.from_numpy(req.mask).pin_memory(), req.B_Q, req.B_KV, req.N, req.H, req.d, qp, kp, vp, O, LSE)
+    assert inf["device_status"] == 0 and inf["heads"] == req.H
+    assert not torch.isnan(O.float()).any() and not torch.isnan(LSE).any()
+    Hh.compare_with_oracle(req, O, LSE, (q, k, v), sel=_sample(req, 4))
+    with bsa.plan_create(torch.from_numpy(req.mask).cuda(), req.B_Q, req.B_KV, req.N, req.H, req.d) as whole:
+        w = whole.info()
+    for key in ("nnz_blocks", "blocks_in_runs", "max_row_nnz", "ntiles", "nitems", "covered_pairs"):
+        assert inf[key] == w[key], key
+
+
 @pytest.mark.parametrize("plan_id", [22, 27])
 def test_forward_replays_from_a_cuda_graph(plan_id):
     """bsa_forward only launches kernels (no allocation, no synchronisation): it can be captured into a CUDA graph
