@@ -485,7 +485,7 @@ static bsa_status_t create_impl(const uint8_t* mask_dev, int64_t packed_stride, 
         BSA_CUDA(launch_csr_fill(mask_dev, nrows, nKb, p->row_ptr, p->col_idx, stream), "csr_fill");
     }
     BSA_CUDA(launch_tile_map(g, p->row_ptr, p->col_idx, p->desc.split_tau, pmax, p->tile_begin, p->tile_cnt,
-                             p->row_parts, p->tile_col, p->tile_member, p->head_counts, p->counters, stream),
+                             p->row_parts, p->tile_col, p->tile_member, p->head_counts, p->counters, stream, nnz_i),
              "tile_map");
     BSA_CUDA(launch_organize(g, p->desc.order, pmax, p->tile_begin, p->tile_cnt, p->row_parts, p->head_counts,
                              p->items_tmp, p->items, p->split_rows, p->counters, stream,

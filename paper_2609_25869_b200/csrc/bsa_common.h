@@ -86,7 +86,7 @@ cudaError_t launch_csr_fill(const uint8_t* mask, int nrows, int nKb, const int32
 cudaError_t launch_tile_map(const MapGeom& g, const int32_t* row_ptr, const int32_t* col_idx, int split_tau,
                             int split_pmax, int32_t* tile_begin, int32_t* tile_cnt, int32_t* row_parts,
                             int32_t* tile_col, uint64_t* tile_member, int32_t* head_counts /* [3*H] */,
-                            PlanCountersDev* counters, cudaStream_t stream);
+                            PlanCountersDev* counters, cudaStream_t stream, int64_t nnz = 0);
 // `scratch` (may be null): organize_scratch_bytes() bytes in the plan's arena for the long-list path.
 cudaError_t launch_organize(const MapGeom& g, int order, int split_pmax, const int32_t* tile_begin,
                             const int32_t* tile_cnt, const int32_t* row_parts, const int32_t* head_counts, WorkItem* items_tmp,

@@ -293,6 +293,17 @@ def test_pipelined_request_from_pinned_host_buffers():
         assert abs(inf[key] - w[key]) < 1e-9, key
 
 
+def test_dense_coarsened_mask_takes_the_bit_plane_tile_map():
+    """From 1536 active blocks per tile row on, a Coarsened mask with a small membership word is mapped by the
+    bit-plane kernel (one bitmap per membership bit instead of one word per tile column): (32,32) blocks at 50 %
+    density, N = 32768, on 128x64 tiles has 2048 per tile row.  Tile lists and membership words against the oracle bit
+    for bit, outputs on sampled query blocks; the same plan on a sparse mask of the same shape takes the other kernel."""
+    for p_active in (0.5, 0.05):
+        req = I.config_tiny(seed=41, H=2, N=32768, d=128, B=32, p=p_active)
+        pid = next(i for i, c in enumerate(bsa.catalog()) if c["name"] == "q128k64_pp_gb")
+        Hh.run_request(req, plan_id=pid, sel=_sample(req, 2), guards=False)
+
+
 def test_host_request_with_tapered_head_groups():
     """With more than 32 MB of Q, K, V per head a group may be a single head, and bsa_request_host then tapers the
     groups towards the end (12 heads: 3 2 2 2 2 1) so that little work is left after the last input byte.  Every head
