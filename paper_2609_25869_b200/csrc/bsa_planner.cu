@@ -547,6 +547,29 @@ __global__ void __launch_bounds__(kTmThreads) tile_map_bitmap_kernel(MapGeom g, 
     const int lgSQ128 = 31 - __clz(g.sQ128), lgRK = 31 - __clz(g.rk);
     const bool whole_tile_rows = g.B_Q >= g.T_Q;  // one logical row feeds every slot of the tile row
     unsigned* bm32 = reinterpret_cast<unsigned*>(bm);
+    if (g.rq == 1 && g.rk == 1 && nr >= kTmThreads / 32) {
+        // At least one logical row per warp: a warp walks whole rows, so the row of an entry (and with it the slot and the
+        // sub-row bits) is known without the search below; two loads per lane in flight.
+        for (int a = warp; a < nr; a += kTmThreads / 32) {
+            const int slot_lo = whole_tile_rows ? 0 : a >> lgSQ128;
+            const int slot_hi = whole_tile_rows ? g.slots - 1 : slot_lo;
+            const int bit0 = (a & (g.sQ128 - 1)) << g.lgSK;
+            const int32_t r1 = rp[a + 1];
+            for (int32_t i = rp[a] + lane; i < r1; i += 64) {
+                const int32_t ca = col_idx[i];
+                const int32_t cb = (i + 32 < r1) ? col_idx[i + 32] : -1;
+                for (int sl = slot_lo; sl <= slot_hi; ++sl) {
+                    const int wbase = sl * g.nKt;
+                    const int ba = bit0 + (ca & (g.sK - 1));
+                    atomicOr(&bm32[2 * (wbase + (ca >> g.lgSK)) + (ba >> 5)], 1u << (ba & 31));
+                    if (cb >= 0) {
+                        const int bb = bit0 + (cb & (g.sK - 1));
+                        atomicOr(&bm32[2 * (wbase + (cb >> g.lgSK)) + (bb >> 5)], 1u << (bb & 31));
+                    }
+                }
+            }
+        }
+    } else
     for (int32_t i0 = e0 + tid; i0 < e1; i0 += 4 * kTmThreads) {
         int32_t c[4];
 #pragma unroll
