@@ -271,10 +271,12 @@ BSA_API bsa_status_t bsa_plan_cache_destroy(bsa_plan_cache_t* cache);
  * bsa_request_host -- one complete request from HOST buffers: copies mask, Q, K, V to the device,
  * creates the plan, runs the forward, copies O and LSE back, frees everything.  Same results as
  * the three calls above; used to measure end-to-end request cost including transfers.  Heads are
- * independent, so with the head-major layout the request is cut into up to 8 groups of heads (of at
- * least 32 MB of Q, K and V) that are pipelined: a group's inputs travel while the previous group is planned and computed and the
- * one before travels back (pinned host buffers are needed for the copies to overlap).  Each group
- * selects its own plan from its own part of the mask.
+ * independent, so with the head-major layout the request is cut into up to 8 groups of heads (of
+ * more than 32 MB of Q, K and V; smaller towards the end of the request where a single head already
+ * has that much, so that little is left to do after the last input byte) that are pipelined: a
+ * group's inputs travel while the previous group is planned and computed and the one before travels
+ * back (pinned host buffers are needed for the copies to overlap).  Each group selects its own plan
+ * from its own part of the mask.
  *   info_out (optional) receives the request's info: counts and times summed over the groups,
  *   statistics of the whole mask, the first group's plan.
  */
